@@ -1,0 +1,167 @@
+/*
+ * vq.h — C-ABI boundary of the B200 VQ-decode linear-layer library.
+ *
+ * The library implements the decode-phase linear layer of GPTVQ (arXiv 2402.15319):
+ * weights live in HBM vector-quantized, are expanded through small per-block
+ * look-up tables and multiplied by the token activations on the fly.
+ *
+ * Representation (paper Sec. 2.1 and Sec. 3.1): a weight matrix W (N out-features x
+ * K in-features, row-major) is split into blocks of block_rows x block_cols weights.
+ * Each block is stored as the tuple
+ *   (1) packed VQ indices, (2) its codebook / LUT, (3) an optional scale factor.
+ * One index of `index_bits` bits selects one of k = 2^index_bits codebook entries;
+ * an entry holds `vq_dim` values which are `vq_dim` ADJACENT COLUMNS of one row
+ * (Sec. 4, "we quantize d columns at a time").  Bits per value follow the paper's
+ * formula  log2(k)/d + k*d*b_c/l  (Sec. 4, "Total bits per value").
+ *
+ * Memory layout fixed by this library (the paper only says "packed tightly"):
+ *   indices : N rows; row n is a little-endian bitstream: index j (covering columns
+ *             j*d .. j*d+d-1) occupies bits [j*b, (j+1)*b) where bit t of the stream is
+ *             bit (t mod 8) of byte (t div 8).  Rows start at n*row_stride_bytes;
+ *             row_stride_bytes = ceil(K/d*b/8) rounded up to a multiple of 16.
+ *             Padding bits/bytes are ignored.
+ *   codebook: cb[blk][entry][t], t < d; blk = (n / block_rows)*(K / block_cols) + (k / block_cols).
+ *             VQ_CB_FP16: IEEE binary16.  VQ_CB_INT8_SCALED: signed 8-bit.
+ *   scale   : VQ_CB_INT8_SCALED only: one binary16 per block, w = scale * int8.
+ *   x / X   : activations, binary16, X[batch][K] row-major.
+ *   y / Y   : outputs, binary16, Y[batch][N] row-major; accumulated in fp32, rounded once.
+ *
+ * Conventions for every entry point:
+ *   - `extern "C"`, plain pointers and sizes.  Pointers named d_* are DEVICE pointers,
+ *     h_* are HOST pointers; `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *   - The caller owns all buffers.  Inputs are read-only.  The library allocates nothing,
+ *     frees nothing, never synchronises: work is enqueued on `stream` and the call returns.
+ *   - All argument checks run on the host before any launch; on error nothing is launched.
+ *   - Same inputs give bit-identical outputs (no floating-point atomics).
+ */
+#ifndef VQ_B200_H
+#define VQ_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  VQ_OK = 0,
+  VQ_ERR_NULL = 1,        /* required pointer is NULL, or scale pointer presence does not match cb_type */
+  VQ_ERR_FORMAT = 2,      /* vq_dim not in {1,2,4}, index_bits not in 1..8, unknown cb_type            */
+  VQ_ERR_SHAPE = 3,       /* N % block_rows, K % block_cols, block_cols % vq_dim, sizes <= 0            */
+  VQ_ERR_ALIGN = 4,       /* a device pointer is not 16-byte aligned                                    */
+  VQ_ERR_WORKSPACE = 5,   /* workspace smaller than vq_workspace_bytes() or NULL when needed            */
+  VQ_ERR_BATCH = 6,       /* batch outside 1..16                                                        */
+  VQ_ERR_UNSUPPORTED = 7, /* valid format but the requested kernel variant does not cover it            */
+  VQ_ERR_CUDA = 8         /* a CUDA runtime call or the launch itself reported an error                 */
+} vq_status;
+
+typedef enum { VQ_CB_FP16 = 0, VQ_CB_INT8_SCALED = 1 } vq_cb_type;
+
+/* Kernel selection for the *_impl entry points.  VQ_IMPL_AUTO is what the plain entry points use. */
+typedef enum {
+  VQ_IMPL_AUTO = 0,     /* tuned kernel when one covers the format/shape, else the generic one   */
+  VQ_IMPL_GENERIC = 1,  /* format-generic fp32-FMA kernel (any valid format)                     */
+  VQ_IMPL_TUNED = 2     /* tuned kernel only; VQ_ERR_UNSUPPORTED if none covers the format/shape */
+} vq_impl;
+
+/* Caller-filled description of one VQ-compressed matrix (paper Sec. 2.1 notation in comments). */
+typedef struct {
+  int32_t n_rows;      /* N, out features (rows of W)                         */
+  int32_t k_cols;      /* K, in features (columns of W)                       */
+  int32_t vq_dim;      /* d in {1,2,4}: values per codebook entry             */
+  int32_t index_bits;  /* b = log2(k) in 1..8: bits per index                 */
+  int32_t block_rows;  /* rows of the block sharing one codebook              */
+  int32_t block_cols;  /* columns of that block (multiple of d); l = rows*cols */
+  int32_t cb_type;     /* vq_cb_type                                          */
+} vq_format;
+
+/* Library-filled sizes for a format. */
+typedef struct {
+  int32_t entries;                  /* k = 2^b                                              */
+  int32_t codebook_bits;            /* b_c: 16 (fp16) or 8 (int8)                           */
+  int64_t indices_per_row;          /* K/d                                                  */
+  int64_t row_stride_bytes;         /* bytes between consecutive rows of the index stream   */
+  int64_t index_bytes;              /* N * row_stride_bytes                                 */
+  int64_t n_blocks;                 /* (N/block_rows) * (K/block_cols)                      */
+  int64_t codebook_bytes_per_block; /* k * d * b_c/8                                        */
+  int64_t codebook_bytes;           /* n_blocks * codebook_bytes_per_block                  */
+  int64_t scale_bytes;              /* 2*n_blocks for INT8_SCALED, else 0                   */
+  int64_t total_bytes;              /* index + codebook + scale bytes                       */
+  double bpv_paper;                 /* log2(k)/d + k*d*b_c/l  (no scale term)               */
+  double bpv_stored;                /* 8*total_bytes/(N*K), everything stored               */
+} vq_pack_info_t;
+
+/* Sizes and bits-per-value of a format (paper Sec. 4 "Total bits per value"; Sec. 3.1 tuple).
+ * Host only, no CUDA call.  Errors: NULL, FORMAT, SHAPE. */
+vq_status vq_pack_info(const vq_format* fmt, vq_pack_info_t* out);
+
+/* Bytes of device scratch the GEMV/GEMM entry points need for (fmt, batch): room for the
+ * fp32 split-K partial sums (Sec. 3.2 mat-vec; the split is this library's).  Host only.
+ * Returns 0 for an invalid format or batch. */
+size_t vq_workspace_bytes(const vq_format* fmt, int batch);
+
+/* Materialise W: unpack every index and look its entry up (paper App. A: "Q is constructed by
+ * looking up values of C"; Sec. 3.2 decode step; App. B transfer+decode experiment).
+ *   d_idx, d_cb, d_scale : device, layouts above; d_scale NULL iff cb_type == VQ_CB_FP16.
+ *   d_W   : device, binary16 [N][K] row-major, written completely.
+ * FP16 codebooks are copied bit-exactly; INT8_SCALED values are fp32(scale)*int8 rounded once
+ * to binary16 (round-to-nearest-even).  Errors: NULL, FORMAT, SHAPE, ALIGN, CUDA. */
+vq_status vq_decode_weights(const vq_format* fmt, const void* d_idx, const void* d_cb,
+                            const void* d_scale, void* d_W, void* stream);
+
+/* y = W x for one token (paper Sec. 3.2: indices -> LUT -> values -> matrix-vector product).
+ *   d_x : device binary16 [K];  d_y : device binary16 [N], written completely.
+ *   d_ws / ws_bytes : device scratch of at least vq_workspace_bytes(fmt, 1) bytes, 16-byte
+ *                     aligned; contents on entry are ignored, contents on exit unspecified.
+ * Errors: NULL, FORMAT, SHAPE, ALIGN, WORKSPACE, CUDA. */
+vq_status vq_gemv(const vq_format* fmt, const void* d_idx, const void* d_cb, const void* d_scale,
+                  const void* d_x, void* d_y, void* d_ws, size_t ws_bytes, void* stream);
+
+/* Y[m][n] = sum_k W[n][k] X[m][k] for batch = 1..16 token rows (same passage as vq_gemv).
+ *   d_X : device binary16 [batch][K];  d_Y : device binary16 [batch][N].
+ *   workspace of at least vq_workspace_bytes(fmt, batch) bytes.
+ * Errors: as vq_gemv plus BATCH. */
+vq_status vq_gemm_small_batch(const vq_format* fmt, const void* d_idx, const void* d_cb,
+                              const void* d_scale, const void* d_X, void* d_Y, int batch,
+                              void* d_ws, size_t ws_bytes, void* stream);
+
+/* Same computation as vq_gemm_small_batch with the kernel family chosen by the caller
+ * (vq_impl); used by the tests to exercise every kernel against the oracle.
+ * Errors: as vq_gemm_small_batch plus UNSUPPORTED. */
+vq_status vq_gemm_small_batch_impl(const vq_format* fmt, const void* d_idx, const void* d_cb,
+                                   const void* d_scale, const void* d_X, void* d_Y, int batch,
+                                   void* d_ws, size_t ws_bytes, void* stream, int impl);
+
+/* Same computation with HOST activations and outputs: copies h_X (binary16 [batch][K]) to the
+ * device, runs vq_gemm_small_batch, copies Y back into h_Y (binary16 [batch][N]); all three
+ * steps are enqueued on `stream` and the call returns without synchronising, so the caller
+ * must synchronise the stream before reading h_Y.  Pinned host memory keeps the copies
+ * asynchronous.  The compressed weights stay resident on the device (paper Sec. 1: every
+ * weight is read once per generated token; only activations cross the host boundary).
+ *   d_ws must hold vq_workspace_bytes(fmt, batch) + 2*batch*(K+N) bytes rounded up to 256:
+ *   use vq_workspace_bytes_host(fmt, batch).
+ * Errors: as vq_gemm_small_batch. */
+vq_status vq_gemm_small_batch_host(const vq_format* fmt, const void* d_idx, const void* d_cb,
+                                   const void* d_scale, const void* h_X, void* h_Y, int batch,
+                                   void* d_ws, size_t ws_bytes, void* stream);
+size_t vq_workspace_bytes_host(const vq_format* fmt, int batch);
+
+/* Uniform INT4 group-128 reference GEMV used as the bandwidth yard-stick beside the VQ
+ * kernels (paper Sec. 2.1 symmetric uniform quantiser x ~ s*x_int; Sec. 5 "INT4 g128", 4.125 bpv).
+ *   d_q     : device, N rows of K/2 bytes; column k of row n is nibble (k mod 2) of byte k/2
+ *             (low nibble first); stored value q in 0..15 means integer q-8.
+ *   d_scale : device binary16 [N][K/128];  w[n][k] = scale[n][k/128] * (q-8).
+ *   d_X binary16 [batch][K], d_Y binary16 [batch][N], batch 1..16.  K % 128 == 0, K/2 % 16 == 0.
+ * Errors: NULL, SHAPE, ALIGN, BATCH, CUDA. */
+vq_status vq_int4g128_gemm_small_batch(int32_t n_rows, int32_t k_cols, const void* d_q,
+                                       const void* d_scale, const void* d_X, void* d_Y,
+                                       int batch, void* stream);
+
+/* Human-readable name of a status code; never NULL. */
+const char* vq_status_string(vq_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VQ_B200_H */

@@ -1,0 +1,202 @@
+"""ctypes front-end of the CPU oracle (oracle/vq_oracle.cpp).
+
+TEST INFRASTRUCTURE ONLY: the parity reference and the timed CPU baseline.  Nothing in the
+product package imports this module, and this module imports nothing from the product.
+
+All arrays are numpy; binary16 data travels as uint16 bit patterns or np.float16 views.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "vq_oracle.cpp")
+_LIB = os.path.join(_HERE, "libvq_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (no CUDA involved)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(
+            ["g++", "-O2", "-std=c++17", "-shared", "-fPIC", "-pthread", "-o", _LIB, _SRC]
+        )
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        L = ctypes.CDLL(_LIB)
+        c_ll, c_i, c_d, c_p = ctypes.c_longlong, ctypes.c_int, ctypes.c_double, ctypes.c_void_p
+        L.ref_bpv.restype = c_d
+        L.ref_bpv.argtypes = [c_i, c_i, c_i, c_ll]
+        L.ref_bpv_uniform.restype = c_d
+        L.ref_bpv_uniform.argtypes = [c_i, c_i, c_i]
+        L.ref_row_stride_bytes.restype = c_ll
+        L.ref_row_stride_bytes.argtypes = [c_i, c_i, c_i]
+        L.ref_f64_to_f16.restype = ctypes.c_uint16
+        L.ref_f64_to_f16.argtypes = [c_d]
+        L.ref_f16_to_f64.restype = c_d
+        L.ref_f16_to_f64.argtypes = [ctypes.c_uint16]
+        L.ref_pack.restype = None
+        L.ref_pack.argtypes = [c_i, c_i, c_i, c_i, c_p, c_p, c_ll]
+        L.ref_unpack.restype = None
+        L.ref_unpack.argtypes = [c_i, c_i, c_i, c_i, c_p, c_ll, c_p]
+        L.ref_decode.restype = None
+        L.ref_decode.argtypes = [c_i] * 7 + [c_p, c_ll, c_p, c_p, c_p, c_p]
+        L.ref_gemm.restype = None
+        L.ref_gemm.argtypes = [c_i] * 7 + [c_p, c_ll, c_p, c_p, c_p, c_i, c_p, c_ll, c_p, c_p, c_i]
+        L.ref_dense_gemm.restype = None
+        L.ref_dense_gemm.argtypes = [c_i, c_i, c_p, c_p, c_i, c_p]
+        L.ref_int4g128_gemm.restype = None
+        L.ref_int4g128_gemm.argtypes = [c_i, c_i, c_p, c_p, c_p, c_i, c_p, c_p, c_i]
+        L.ref_hardware_threads.restype = c_i
+        L.ref_hardware_threads.argtypes = []
+        _lib = L
+    return _lib
+
+
+@dataclass(frozen=True)
+class Fmt:
+    """One VQ-compressed matrix: N x K weights, VQ dim d, b index bits, Br x Bc blocks."""
+
+    N: int
+    K: int
+    d: int
+    b: int
+    Br: int
+    Bc: int
+    int8: bool
+
+    @property
+    def entries(self) -> int:
+        return 1 << self.b
+
+    @property
+    def n_blocks(self) -> int:
+        return (self.N // self.Br) * (self.K // self.Bc)
+
+    @property
+    def stride(self) -> int:
+        return row_stride_bytes(self.K, self.d, self.b)
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _u16(a):
+    a = np.ascontiguousarray(a)
+    return a.view(np.uint16) if a.dtype == np.float16 else a.astype(np.uint16, copy=False)
+
+
+def bpv(k: int, d: int, b_c: int, l: int) -> float:
+    return _load().ref_bpv(k, d, b_c, l)
+
+
+def bpv_uniform(bits: int, scale_bits: int, group: int) -> float:
+    return _load().ref_bpv_uniform(bits, scale_bits, group)
+
+
+def row_stride_bytes(K: int, d: int, b: int) -> int:
+    return _load().ref_row_stride_bytes(K, d, b)
+
+
+def f64_to_f16_bits(x: float) -> int:
+    return _load().ref_f64_to_f16(float(x))
+
+
+def f16_bits_to_f64(h: int) -> float:
+    return _load().ref_f16_to_f64(int(h))
+
+
+def pack(f: Fmt, I: np.ndarray, fill: np.ndarray | None = None) -> np.ndarray:
+    """Indices I[N][K/d] (uint8) -> packed rows uint8[N][stride]; `fill` pre-sets padding."""
+    I = np.ascontiguousarray(I, dtype=np.uint8)
+    assert I.shape == (f.N, f.K // f.d)
+    out = np.zeros((f.N, f.stride), np.uint8) if fill is None else np.array(fill, dtype=np.uint8, copy=True)
+    assert out.shape == (f.N, f.stride) and out.flags.c_contiguous
+    _load().ref_pack(f.N, f.K, f.d, f.b, _p(I), _p(out), f.stride)
+    return out
+
+
+def unpack(f: Fmt, idx: np.ndarray) -> np.ndarray:
+    idx = np.ascontiguousarray(idx, dtype=np.uint8)
+    assert idx.size == f.N * f.stride
+    I = np.empty((f.N, f.K // f.d), np.uint8)
+    _load().ref_unpack(f.N, f.K, f.d, f.b, _p(idx), f.stride, _p(I))
+    return I
+
+
+def _check_layer(f: Fmt, idx, cb, scale):
+    idx = np.ascontiguousarray(idx, dtype=np.uint8)
+    assert idx.size == f.N * f.stride
+    if f.int8:
+        cb = np.ascontiguousarray(cb, dtype=np.int8)
+        scale = _u16(scale)
+        assert scale.size == f.n_blocks
+    else:
+        cb = _u16(cb)
+        scale = None
+    assert cb.size == f.n_blocks * f.entries * f.d
+    return idx, cb, scale
+
+
+def decode(f: Fmt, idx, cb, scale=None, exact: bool = True, half: bool = True):
+    """Returns (W_exact float64 [N][K] or None, W16 uint16 [N][K] or None)."""
+    idx, cb, scale = _check_layer(f, idx, cb, scale)
+    We = np.empty((f.N, f.K), np.float64) if exact else None
+    Wh = np.empty((f.N, f.K), np.uint16) if half else None
+    _load().ref_decode(f.N, f.K, f.d, f.b, f.Br, f.Bc, int(f.int8), _p(idx), f.stride, _p(cb),
+                       _p(scale), _p(We), _p(Wh))
+    return We, Wh
+
+
+def gemm(f: Fmt, idx, cb, scale, X, rows=None, threads: int = 1):
+    """Y[m][r], A[m][r] in float64 for X[batch][K] (float16).  rows: optional row subset."""
+    idx, cb, scale = _check_layer(f, idx, cb, scale)
+    X = _u16(np.atleast_2d(X))
+    batch = X.shape[0]
+    assert X.shape[1] == f.K
+    if rows is not None:
+        rows = np.ascontiguousarray(rows, dtype=np.int32)
+        n_out = rows.size
+    else:
+        n_out = f.N
+    Y = np.empty((batch, n_out), np.float64)
+    A = np.empty((batch, n_out), np.float64)
+    _load().ref_gemm(f.N, f.K, f.d, f.b, f.Br, f.Bc, int(f.int8), _p(idx), f.stride, _p(cb),
+                     _p(scale), _p(X), batch, _p(rows), n_out, _p(Y), _p(A), int(threads))
+    return Y, A
+
+
+def dense_gemm(W: np.ndarray, X) -> np.ndarray:
+    W = np.ascontiguousarray(W, dtype=np.float64)
+    X = _u16(np.atleast_2d(X))
+    N, K = W.shape
+    Y = np.empty((X.shape[0], N), np.float64)
+    _load().ref_dense_gemm(N, K, _p(W), _p(X), X.shape[0], _p(Y))
+    return Y
+
+
+def int4g128_gemm(q: np.ndarray, scale, X, threads: int = 1):
+    q = np.ascontiguousarray(q, dtype=np.uint8)
+    N, K = q.shape[0], q.shape[1] * 2
+    scale = _u16(scale)
+    assert scale.size == N * (K // 128)
+    X = _u16(np.atleast_2d(X))
+    Y = np.empty((X.shape[0], N), np.float64)
+    A = np.empty((X.shape[0], N), np.float64)
+    _load().ref_int4g128_gemm(N, K, _p(q), _p(scale), _p(X), X.shape[0], _p(Y), _p(A), int(threads))
+    return Y, A
+
+
+def hardware_threads() -> int:
+    return _load().ref_hardware_threads()

@@ -1,0 +1,414 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests compares the oracle with itself or with the CUDA path: expected values are
+the paper's printed numbers (tests/golden/*.txt, each with its citation), hand-written
+matrices, an independent big-integer / exact-rational brute force, numpy's float16, or
+algebraic invariants.
+"""
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import vq_synth
+from oracle import vq_oracle as orc
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rows(name):
+    out = []
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                out.append(line)
+    return out
+
+
+# --------------------------------------------------------------------------------------
+# P1 / P2: bits per value, Sec. 4 "Total bits per value", against rows the paper prints
+# --------------------------------------------------------------------------------------
+def test_bpv_matches_paper_rows():
+    rows = _rows("bpv_rows.txt")
+    assert len(rows) >= 15
+    for r in rows:
+        k, d, b_c, l, printed = r.split()[:5]
+        assert orc.bpv(int(k), int(d), int(b_c), int(l)) == pytest.approx(float(printed), abs=1e-12), r
+
+
+def test_bpv_uniform_rows():
+    for r in _rows("uniform_bpv_rows.txt"):
+        bits, sb, g, printed = r.split()[:4]
+        assert orc.bpv_uniform(int(bits), int(sb), int(g)) == pytest.approx(float(printed), abs=1e-12)
+
+
+def test_relative_footprint_column():
+    # App. B table prints bpv/4 to two decimals
+    for r in _rows("rel_footprint_rows.txt"):
+        bpv, printed = r.split()[:2]
+        rel = float(bpv) / 4.0
+        assert abs(rel - float(printed)) <= 0.005 + 1e-12, r
+    # and the VQ rows of that table are reachable by the closed form
+    assert orc.bpv(16, 2, 8, 2048) / 4 == pytest.approx(0.53125)
+    assert orc.bpv(64, 2, 8, 8192) / 4 == pytest.approx(0.78125)
+
+
+def test_bpv_of_benchmark_formats():
+    # 2-D, 6-bit indices, fp16 codebook per 128x128 block -> 3.125; 4-D 8-bit per 256x512 -> 2.125
+    assert orc.bpv(64, 2, 16, 128 * 128) == pytest.approx(3.125)
+    assert orc.bpv(256, 4, 16, 256 * 512) == pytest.approx(2.125)
+    assert orc.bpv(16, 2, 16, 1024) == pytest.approx(2.5)
+    # Sec. 2.1: 3 bits per value in pairs -> 2^6 = 64 centroids
+    assert 2 ** (3 * 2) == 64
+
+
+# --------------------------------------------------------------------------------------
+# binary16 conversions against numpy (an independent implementation)
+# --------------------------------------------------------------------------------------
+def test_f16_to_f64_all_patterns():
+    bits = np.arange(65536, dtype=np.uint16)
+    want = bits.view(np.float16).astype(np.float64)
+    got = np.array([orc.f16_bits_to_f64(int(b)) for b in bits])
+    fin = np.isfinite(want)
+    assert np.array_equal(got[fin], want[fin])
+    assert np.array_equal(np.isnan(got), np.isnan(want))
+    assert np.array_equal(np.isinf(got), np.isinf(want))
+    assert np.array_equal(np.signbit(got[fin]), np.signbit(want[fin]))
+
+
+def test_f64_to_f16_rounding():
+    rng = np.random.default_rng(0)
+    xs = np.concatenate([
+        rng.normal(size=20000), rng.normal(size=5000) * 1e-5, rng.normal(size=5000) * 1e-7,
+        rng.normal(size=2000) * 3e4, rng.normal(size=200) * 1e5,
+        np.array([0.0, -0.0, 65504.0, 65519.99, 65520.0, 2.0 ** -24, 2.0 ** -25, 3 * 2.0 ** -25,
+                  2.0 ** -14, 1.0 + 2.0 ** -11, 1.0 + 3 * 2.0 ** -11, 1.0 + 2.0 ** -11 + 2.0 ** -30]),
+    ])
+    # exact ties between neighbouring halves
+    h = rng.integers(0, 0x7BFF, size=4000).astype(np.uint16)
+    lo = h.view(np.float16).astype(np.float64)
+    hi = (h + 1).astype(np.uint16).view(np.float16).astype(np.float64)
+    xs = np.concatenate([xs, (lo + hi) / 2, -(lo + hi) / 2])
+    with np.errstate(over="ignore"):
+        want = xs.astype(np.float16).view(np.uint16)
+    got = np.array([orc.f64_to_f16_bits(float(x)) for x in xs], dtype=np.uint16)
+    assert np.array_equal(got, want)
+
+
+# --------------------------------------------------------------------------------------
+# P5: packing — hand-derived bytes, identity
+# --------------------------------------------------------------------------------------
+def test_pack_golden_bytes():
+    for r in _rows("pack_bytes.txt"):
+        b_s, idx_s, bytes_s = [p.strip() for p in r.split("|")]
+        b = int(b_s)
+        I = np.array([int(v) for v in idx_s.split()], dtype=np.uint8)[None, :]
+        want = bytes(int(v, 16) for v in bytes_s.split())
+        f = orc.Fmt(N=1, K=I.shape[1], d=1, b=b, Br=1, Bc=I.shape[1], int8=False)
+        packed = orc.pack(f, I)
+        assert packed.shape == (1, 16)  # stride is rounded up to 16 bytes
+        assert bytes(packed[0, : len(want)]) == want, r
+        assert not packed[0, len(want):].any()
+        assert np.array_equal(orc.unpack(f, packed), I)
+
+
+def test_row_stride_rule():
+    # ceil(K/d*b/8) rounded up to 16; values for the benchmark shapes
+    assert orc.row_stride_bytes(4096, 2, 4) == 1024
+    assert orc.row_stride_bytes(4096, 1, 4) == 2048
+    assert orc.row_stride_bytes(4096, 2, 6) == 1536
+    assert orc.row_stride_bytes(11008, 2, 6) == 4128
+    assert orc.row_stride_bytes(5120, 4, 8) == 1280
+    assert orc.row_stride_bytes(13824, 4, 8) == 3456
+    assert orc.row_stride_bytes(8192, 2, 4) == 2048
+    assert orc.row_stride_bytes(28672, 2, 4) == 7168
+    assert orc.row_stride_bytes(16, 1, 1) == 16
+    assert orc.row_stride_bytes(136, 1, 1) == 32
+
+
+@pytest.mark.parametrize("b", range(1, 9))
+@pytest.mark.parametrize("d", [1, 2, 4])
+def test_pack_unpack_identity_and_padding_ignored(b, d):
+    rng = np.random.default_rng(100 * b + d)
+    N, K = 5, 24 * d
+    f = orc.Fmt(N, K, d, b, 1, K, False)
+    I = rng.integers(0, 1 << b, size=(N, K // d)).astype(np.uint8)
+    zero_pad = orc.pack(f, I)
+    junk = rng.integers(0, 256, size=(N, f.stride)).astype(np.uint8)
+    junk_pad = orc.pack(f, I, fill=junk)
+    assert np.array_equal(orc.unpack(f, zero_pad), I)
+    assert np.array_equal(orc.unpack(f, junk_pad), I)
+    used_bits = (K // d) * b
+    # bytes wholly inside the used range are identical whatever the padding was
+    assert np.array_equal(zero_pad[:, : used_bits // 8], junk_pad[:, : used_bits // 8])
+
+
+# --------------------------------------------------------------------------------------
+# P4: brute force — big-integer bit reader + exact rationals, no code shared with the oracle
+# --------------------------------------------------------------------------------------
+def _brute_index(row_bytes: bytes, j: int, b: int) -> int:
+    big = int.from_bytes(row_bytes, "little")
+    return (big // (2 ** (j * b))) % (2 ** b)
+
+
+def _frac_half(v) -> Fraction:
+    return Fraction(float(np.float16(v)))
+
+
+def _brute_layer(f, idx, cb, scale, X):
+    """W as exact Fractions and Y = W X exactly, straight from the definition."""
+    W = [[None] * f.K for _ in range(f.N)]
+    for n in range(f.N):
+        rb = bytes(idx[n])
+        for k in range(f.K):
+            e = _brute_index(rb, k // f.d, f.b)
+            blk = (n // f.Br) * (f.K // f.Bc) + (k // f.Bc)
+            c = cb[blk][e][k % f.d]
+            W[n][k] = Fraction(int(c)) * _frac_half(scale[blk]) if f.int8 else _frac_half(c)
+    Y = [[sum(W[n][k] * _frac_half(X[m][k]) for k in range(f.K)) for n in range(f.N)] for m in range(X.shape[0])]
+    A = [[sum(abs(W[n][k] * _frac_half(X[m][k])) for k in range(f.K)) for n in range(f.N)] for m in range(X.shape[0])]
+    return W, Y, A
+
+
+BLOCKS_8x16 = [(1, 16), (1, 8), (8, 16), (2, 4), (4, 8), (8, 4)]
+
+
+@pytest.mark.parametrize("int8", [False, True])
+@pytest.mark.parametrize("b", range(1, 9))
+@pytest.mark.parametrize("d", [1, 2, 4])
+def test_bruteforce_8x16(d, b, int8):
+    N, K = 8, 16
+    Br, Bc = BLOCKS_8x16[(b + d) % len(BLOCKS_8x16)]
+    spec = vq_synth.LayerSpec("t", N, K, d, b, Br, Bc, int8)
+    f = orc.Fmt(N, K, d, b, Br, Bc, int8)
+    L = vq_synth.make_layer(spec, f.stride, seed=1000 + 31 * b + d)
+    X = vq_synth.make_x(spec, seed=7, batch=3)
+    Wb, Yb, Ab = _brute_layer(f, L.idx, L.cb, L.scale, X)
+
+    I = orc.unpack(f, L.idx)
+    for n in range(N):
+        for j in range(K // d):
+            assert I[n, j] == _brute_index(bytes(L.idx[n]), j, b)
+
+    We, Wh = orc.decode(f, L.idx, L.cb, L.scale)
+    for n in range(N):
+        for k in range(K):
+            assert Fraction(We[n, k]) == Wb[n][k]          # exact in fp64
+            want_half = np.float16(float(Wb[n][k]))         # numpy RN-even from the exact value
+            assert Wh[n, k] == want_half.view(np.uint16)
+    Y, A = orc.gemm(f, L.idx, L.cb, L.scale, X)
+    for m in range(3):
+        for n in range(N):
+            tol = 1e-13 * float(Ab[m][n]) + 1e-300
+            assert abs(Y[m, n] - float(Yb[m][n])) <= tol
+            assert abs(A[m, n] - float(Ab[m][n])) <= tol
+
+
+# --------------------------------------------------------------------------------------
+# P3: exact decode on a hand-built codebook — expected matrix written out by hand
+# --------------------------------------------------------------------------------------
+def test_decode_hand_built_fp16():
+    # N=2, K=8, d=2, b=2 (4 entries), blocks 1x4 -> 4 blocks: (row0,c0-3) (row0,c4-7) (row1,..) (row1,..)
+    f = orc.Fmt(2, 8, 2, 2, 1, 4, False)
+    cb = np.zeros((4, 4, 2), np.float16)
+    for blk in range(4):
+        for e in range(4):
+            cb[blk, e] = [blk * 10 + e, -(blk * 10 + e) - 0.5]
+    # row 0 indices (per pair of columns): 0 1 | 2 3 ; row 1: 3 3 | 0 2
+    I = np.array([[0, 1, 2, 3], [3, 3, 0, 2]], np.uint8)
+    idx = orc.pack(f, I)
+    assert idx[0, 0] == 0b11100100 and idx[1, 0] == 0b10001111
+    want = np.array([
+        [0, -0.5, 1, -1.5, 12, -12.5, 13, -13.5],
+        [23, -23.5, 23, -23.5, 30, -30.5, 32, -32.5],
+    ], np.float64)
+    We, Wh = orc.decode(f, idx, cb)
+    assert np.array_equal(We, want)
+    assert np.array_equal(Wh, want.astype(np.float16).view(np.uint16))
+
+
+def test_decode_hand_built_int8_block_rows():
+    # N=4, K=4, d=1, b=1 (2 entries), blocks 2x2 -> blk = (n//2)*2 + k//2
+    f = orc.Fmt(4, 4, 1, 1, 2, 2, True)
+    cb = np.array([[[-3], [5]], [[7], [-127]], [[0], [1]], [[100], [-100]]], np.int8)
+    scale = np.array([0.5, 2.0, 0.25, 1.0], np.float16)
+    I = np.array([[0, 1, 1, 0], [1, 1, 0, 0], [1, 0, 0, 1], [0, 0, 1, 1]], np.uint8)
+    idx = orc.pack(f, I)
+    want = np.array([
+        [-1.5, 2.5, -254.0, 14.0],
+        [2.5, 2.5, 14.0, 14.0],
+        [0.25, 0.0, 100.0, -100.0],
+        [0.0, 0.0, -100.0, -100.0],
+    ])
+    We, _ = orc.decode(f, idx, cb, scale)
+    assert np.array_equal(We, want)
+    # y = W x with x = (1, 2, 3, 4), by hand
+    x = np.array([[1, 2, 3, 4]], np.float16)
+    Y, A = orc.gemm(f, idx, cb, scale, x)
+    assert np.array_equal(Y[0], [-1.5 + 5 - 762 + 56, 2.5 + 5 + 42 + 56, 0.25 + 0 + 300 - 400, -300 - 400])
+    assert np.array_equal(A[0], [1.5 + 5 + 762 + 56, 105.5, 700.25, 700])
+
+
+# --------------------------------------------------------------------------------------
+# P6 / P7: invariants
+# --------------------------------------------------------------------------------------
+def _rand_layer(seed, N=12, K=48, d=2, b=6, Br=4, Bc=16, int8=False):
+    spec = vq_synth.LayerSpec("t", N, K, d, b, Br, Bc, int8)
+    f = orc.Fmt(N, K, d, b, Br, Bc, int8)
+    return f, spec, vq_synth.make_layer(spec, f.stride, seed)
+
+
+@pytest.mark.parametrize("int8", [False, True])
+def test_unit_vector_returns_decoded_column(int8):
+    f, spec, L = _rand_layer(11, int8=int8)
+    We, _ = orc.decode(f, L.idx, L.cb, L.scale)
+    X = np.eye(f.K, dtype=np.float16)[:16]
+    Y, A = orc.gemm(f, L.idx, L.cb, L.scale, X)
+    for k in range(16):
+        assert np.array_equal(Y[k], We[:, k])
+        assert np.array_equal(A[k], np.abs(We[:, k]))
+
+
+@pytest.mark.parametrize("d,b,int8", [(1, 4, True), (2, 4, False), (4, 8, False), (2, 5, True), (1, 3, False)])
+def test_fused_equals_decode_then_dense(d, b, int8):
+    f, spec, L = _rand_layer(5, N=8, K=32 * d, d=d, b=b, Br=2, Bc=8 * d, int8=int8)
+    X = vq_synth.make_x(spec, 3, batch=4)
+    We, _ = orc.decode(f, L.idx, L.cb, L.scale)
+    Y, A = orc.gemm(f, L.idx, L.cb, L.scale, X)
+    assert np.array_equal(Y, orc.dense_gemm(We, X))  # same summation order -> same bits
+    # and against numpy's own matmul (different order -> tolerance)
+    ref = X.astype(np.float64) @ We.T
+    assert np.allclose(Y, ref, rtol=0, atol=1e-12 * A.max())
+    assert np.allclose(A, np.abs(X.astype(np.float64)) @ np.abs(We).T, rtol=1e-12)
+
+
+def test_linearity_in_x():
+    f, spec, L = _rand_layer(21)
+    # small integers: sums are exact in fp64 so linearity holds exactly
+    rng = np.random.default_rng(3)
+    x1 = rng.integers(-8, 9, size=(1, f.K)).astype(np.float16)
+    x2 = rng.integers(-8, 9, size=(1, f.K)).astype(np.float16)
+    cb = (rng.integers(-64, 65, size=L.cb.shape) / 64.0).astype(np.float16)
+    y1, _ = orc.gemm(f, L.idx, cb, None, x1)
+    y2, _ = orc.gemm(f, L.idx, cb, None, x2)
+    y12, _ = orc.gemm(f, L.idx, cb, None, (x1 + 2 * x2).astype(np.float16))
+    assert np.array_equal(y12, y1 + 2 * y2)
+
+
+def test_all_indices_equal_closed_form():
+    # every index = e  =>  y[n] = sum_j <cb[blk(n,j)][e], x_j>
+    N, K, d, b, Br, Bc = 6, 32, 2, 3, 3, 8
+    f = orc.Fmt(N, K, d, b, Br, Bc, False)
+    rng = np.random.default_rng(5)
+    cb = (rng.integers(-32, 33, size=(f.n_blocks, 8, d)) / 8.0).astype(np.float16)
+    x = rng.integers(-4, 5, size=(1, K)).astype(np.float16)
+    for e in (0, 5, 7):
+        idx = orc.pack(f, np.full((N, K // d), e, np.uint8))
+        Y, _ = orc.gemm(f, idx, cb, None, x)
+        for n in range(N):
+            want = 0.0
+            for cbk in range(K // Bc):
+                blk = (n // Br) * (K // Bc) + cbk
+                seg = x[0, cbk * Bc:(cbk + 1) * Bc].astype(np.float64).reshape(-1, d)
+                want += float((seg * cb[blk, e].astype(np.float64)).sum())
+            assert Y[0, n] == want
+
+
+def test_codebook_permutation_invariance():
+    # App. "Codebook compression": sorting a codebook and re-assigning indices leaves the tensor unchanged
+    f, spec, L = _rand_layer(33, d=2, b=4, Br=4, Bc=16)
+    X = vq_synth.make_x(spec, 1, batch=2)
+    I = orc.unpack(f, L.idx)
+    rng = np.random.default_rng(9)
+    cb2 = L.cb.copy()
+    I2 = I.copy()
+    for blk in range(f.n_blocks):
+        perm = rng.permutation(f.entries)           # new position p holds old entry perm[p]
+        inv = np.argsort(perm)
+        cb2[blk] = L.cb[blk][perm]
+        r0 = (blk // (f.K // f.Bc)) * f.Br
+        c0 = (blk % (f.K // f.Bc)) * f.Bc // f.d
+        sub = I[r0:r0 + f.Br, c0:c0 + f.Bc // f.d]
+        I2[r0:r0 + f.Br, c0:c0 + f.Bc // f.d] = inv[sub]
+    idx2 = orc.pack(f, I2)
+    W1, H1 = orc.decode(f, L.idx, L.cb)
+    W2, H2 = orc.decode(f, idx2, cb2)
+    assert np.array_equal(W1, W2) and np.array_equal(H1, H2)
+    assert np.array_equal(orc.gemm(f, L.idx, L.cb, None, X)[0], orc.gemm(f, idx2, cb2, None, X)[0])
+
+
+def test_gemm_row_equals_gemv_and_row_subset():
+    f, spec, L = _rand_layer(44, int8=True)
+    X = vq_synth.make_x(spec, 2, batch=5)
+    Y, A = orc.gemm(f, L.idx, L.cb, L.scale, X)
+    for m in range(5):
+        y, a = orc.gemm(f, L.idx, L.cb, L.scale, X[m])
+        assert np.array_equal(y[0], Y[m]) and np.array_equal(a[0], A[m])
+    rows = np.array([7, 0, 11, 3], np.int32)
+    Ys, As = orc.gemm(f, L.idx, L.cb, L.scale, X, rows=rows)
+    assert np.array_equal(Ys, Y[:, rows]) and np.array_equal(As, A[:, rows])
+    Yt, At = orc.gemm(f, L.idx, L.cb, L.scale, X, threads=3)
+    assert np.array_equal(Yt, Y) and np.array_equal(At, A)
+
+
+def test_int8_unit_scale_integer_inputs_exact():
+    f, spec, L = _rand_layer(55, int8=True, d=2, b=4)
+    scale = np.ones(f.n_blocks, np.float16)
+    rng = np.random.default_rng(1)
+    x = rng.integers(-16, 17, size=(1, f.K)).astype(np.float16)
+    Y, _ = orc.gemm(f, L.idx, L.cb, scale, x)
+    I = orc.unpack(f, L.idx)
+    for n in range(f.N):
+        want = 0
+        for k in range(f.K):
+            blk = (n // f.Br) * (f.K // f.Bc) + k // f.Bc
+            want += int(L.cb[blk, I[n, k // f.d], k % f.d]) * int(x[0, k])
+        assert Y[0, n] == want
+
+
+def test_int4g128_bruteforce():
+    N, K = 3, 256
+    q, s = vq_synth.make_int4g128(N, K, seed=2)
+    spec = vq_synth.LayerSpec("t", N, K, 1, 4, 1, 128, True)
+    X = vq_synth.make_x(spec, 5, batch=2)
+    Y, A = orc.int4g128_gemm(q, s, X)
+    for m in range(2):
+        for n in range(N):
+            acc = Fraction(0)
+            for k in range(K):
+                byte = int(q[n, k // 2])
+                nib = (byte // 16) if k % 2 else (byte % 16)
+                acc += Fraction(nib - 8) * _frac_half(s[n, k // 128]) * _frac_half(X[m, k])
+            assert abs(Y[m, n] - float(acc)) <= 1e-13 * A[m, n]
+    # hand case: all nibbles 0x9 -> +1, scale 2 -> y = 2*sum(x)
+    q1 = np.full((1, 64), 0x99, np.uint8)
+    s1 = np.full((1, 1), 2.0, np.float16)
+    x1 = np.arange(128, dtype=np.float16)[None, :]
+    Y1, A1 = orc.int4g128_gemm(q1, s1, x1)
+    assert Y1[0, 0] == 2 * (127 * 128 // 2) and A1[0, 0] == Y1[0, 0]
+    # low nibble first: byte 0x1f -> column 0 holds 15-8 = 7, column 1 holds 1-8 = -7
+    q2 = np.zeros((1, 64), np.uint8) + 0x88
+    q2[0, 0] = 0x1F
+    x2 = np.zeros((1, 128), np.float16)
+    x2[0, 0] = 1
+    assert orc.int4g128_gemm(q2, np.ones((1, 1), np.float16), x2)[0][0, 0] == 7
+    x2[0, 0], x2[0, 1] = 0, 1
+    assert orc.int4g128_gemm(q2, np.ones((1, 1), np.float16), x2)[0][0, 0] == -7
+
+
+def test_synth_is_deterministic_and_distributed():
+    a = vq_synth.normal(3, 1, 200001)
+    b = vq_synth.normal(3, 1, 200001)
+    assert np.array_equal(a, b)
+    assert abs(a.mean()) < 0.01 and abs(a.std() - 1) < 0.01
+    u = vq_synth.uniform01(3, 2, 100000)
+    assert 0 <= u.min() and u.max() < 1 and abs(u.mean() - 0.5) < 0.01
+    by = vq_synth.random_bytes(1, 1, 100003)
+    assert by.size == 100003 and abs(by.mean() - 127.5) < 1.5
+    spec = vq_synth.CONFIGS["cfg2"]["layers"][0]
+    L = vq_synth.make_layer(vq_synth.LayerSpec("s", 64, 4096, 1, 4, 1, 2048, True), 2048, 1)
+    assert L.cb.min() >= -127 and L.cb.max() <= 127
+    assert 0.0005 <= float(L.scale.min()) and float(L.scale.max()) <= 0.002
+    assert spec.N == 4096 and spec.K == 4096
