@@ -1,0 +1,10 @@
+"""B200-native VQ-decode linear layer (GPTVQ storage format): thin Python binding over the
+C-ABI library libvq_b200.so.  Importing the package loads nothing; the first call loads the
+shared library and raises if it has not been built."""
+from .binding import (  # noqa: F401
+    VQ_CB_FP16, VQ_CB_INT8_SCALED, VQ_IMPL_AUTO, VQ_IMPL_GENERIC, VQ_IMPL_TUNED,
+    VQError, VQFormat, PackInfo, lib_path, load, exported_symbols,
+    vq_pack_info, vq_workspace_bytes, vq_workspace_bytes_host, vq_decode_weights, vq_gemv,
+    vq_gemm_small_batch, vq_gemm_small_batch_impl, vq_gemm_small_batch_host,
+    vq_int4g128_gemm_small_batch, vq_status_string,
+)

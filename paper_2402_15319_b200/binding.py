@@ -1,0 +1,181 @@
+"""ctypes binding with the same names as include/vq.h.  Argument marshalling only: every step
+of the computation runs in the CUDA library.  Tensors are torch CUDA tensors (device memory and
+streams are torch's); there is no CPU fallback — a missing library is an error."""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+VQ_CB_FP16, VQ_CB_INT8_SCALED = 0, 1
+VQ_IMPL_AUTO, VQ_IMPL_GENERIC, VQ_IMPL_TUNED = 0, 1, 2
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libvq_b200.so")
+_lib = None
+
+
+class VQError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {vq_status_string(code)}")
+
+
+class _CFormat(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("n_rows", "k_cols", "vq_dim", "index_bits", "block_rows", "block_cols", "cb_type")]
+
+
+class _CPackInfo(ctypes.Structure):
+    _fields_ = [("entries", ctypes.c_int32), ("codebook_bits", ctypes.c_int32),
+                ("indices_per_row", ctypes.c_int64), ("row_stride_bytes", ctypes.c_int64),
+                ("index_bytes", ctypes.c_int64), ("n_blocks", ctypes.c_int64),
+                ("codebook_bytes_per_block", ctypes.c_int64), ("codebook_bytes", ctypes.c_int64),
+                ("scale_bytes", ctypes.c_int64), ("total_bytes", ctypes.c_int64),
+                ("bpv_paper", ctypes.c_double), ("bpv_stored", ctypes.c_double)]
+
+
+@dataclass(frozen=True)
+class VQFormat:
+    n_rows: int
+    k_cols: int
+    vq_dim: int
+    index_bits: int
+    block_rows: int
+    block_cols: int
+    cb_type: int
+
+    def c(self) -> _CFormat:
+        return _CFormat(self.n_rows, self.k_cols, self.vq_dim, self.index_bits, self.block_rows,
+                        self.block_cols, self.cb_type)
+
+
+@dataclass(frozen=True)
+class PackInfo:
+    entries: int
+    codebook_bits: int
+    indices_per_row: int
+    row_stride_bytes: int
+    index_bytes: int
+    n_blocks: int
+    codebook_bytes_per_block: int
+    codebook_bytes: int
+    scale_bytes: int
+    total_bytes: int
+    bpv_paper: float
+    bpv_stored: float
+
+
+_SIGNATURES = {
+    "vq_pack_info": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
+    "vq_workspace_bytes": (ctypes.c_size_t, [ctypes.c_void_p, ctypes.c_int]),
+    "vq_workspace_bytes_host": (ctypes.c_size_t, [ctypes.c_void_p, ctypes.c_int]),
+    "vq_decode_weights": (ctypes.c_int, [ctypes.c_void_p] * 6),
+    "vq_gemv": (ctypes.c_int, [ctypes.c_void_p] * 7 + [ctypes.c_size_t, ctypes.c_void_p]),
+    "vq_gemm_small_batch": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
+    "vq_gemm_small_batch_impl": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_int]),
+    "vq_gemm_small_batch_host": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
+    "vq_int4g128_gemm_small_batch": (ctypes.c_int, [ctypes.c_int32, ctypes.c_int32] + [ctypes.c_void_p] * 4 + [ctypes.c_int, ctypes.c_void_p]),
+    "vq_status_string": (ctypes.c_char_p, [ctypes.c_int]),
+}
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def exported_symbols():
+    return sorted(_SIGNATURES)
+
+
+def load():
+    """Load libvq_b200.so; raises if it has not been built (there is no fallback path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2402_15319_b200.build`")
+        lib = ctypes.CDLL(_LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def vq_status_string(code: int) -> str:
+    return load().vq_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise VQError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def vq_pack_info(fmt: VQFormat) -> PackInfo:
+    c, out = fmt.c(), _CPackInfo()
+    _check(load().vq_pack_info(ctypes.byref(c), ctypes.byref(out)), "vq_pack_info")
+    return PackInfo(*[getattr(out, n) for n, _ in _CPackInfo._fields_])
+
+
+def vq_workspace_bytes(fmt: VQFormat, batch: int) -> int:
+    c = fmt.c()
+    return load().vq_workspace_bytes(ctypes.byref(c), int(batch))
+
+
+def vq_workspace_bytes_host(fmt: VQFormat, batch: int) -> int:
+    c = fmt.c()
+    return load().vq_workspace_bytes_host(ctypes.byref(c), int(batch))
+
+
+def vq_decode_weights(fmt: VQFormat, d_idx, d_cb, d_scale, d_W, stream=None) -> None:
+    c = fmt.c()
+    _check(load().vq_decode_weights(ctypes.byref(c), _ptr(d_idx), _ptr(d_cb), _ptr(d_scale), _ptr(d_W),
+                                    _stream(stream)), "vq_decode_weights")
+
+
+def vq_gemv(fmt: VQFormat, d_idx, d_cb, d_scale, d_x, d_y, d_ws, stream=None) -> None:
+    c = fmt.c()
+    _check(load().vq_gemv(ctypes.byref(c), _ptr(d_idx), _ptr(d_cb), _ptr(d_scale), _ptr(d_x), _ptr(d_y),
+                          _ptr(d_ws), d_ws.numel() * d_ws.element_size(), _stream(stream)), "vq_gemv")
+
+
+def vq_gemm_small_batch(fmt: VQFormat, d_idx, d_cb, d_scale, d_X, d_Y, batch: int, d_ws, stream=None) -> None:
+    c = fmt.c()
+    _check(load().vq_gemm_small_batch(ctypes.byref(c), _ptr(d_idx), _ptr(d_cb), _ptr(d_scale), _ptr(d_X),
+                                      _ptr(d_Y), int(batch), _ptr(d_ws), d_ws.numel() * d_ws.element_size(),
+                                      _stream(stream)), "vq_gemm_small_batch")
+
+
+def vq_gemm_small_batch_impl(fmt: VQFormat, d_idx, d_cb, d_scale, d_X, d_Y, batch: int, d_ws, impl: int,
+                             stream=None) -> None:
+    c = fmt.c()
+    _check(load().vq_gemm_small_batch_impl(ctypes.byref(c), _ptr(d_idx), _ptr(d_cb), _ptr(d_scale), _ptr(d_X),
+                                           _ptr(d_Y), int(batch), _ptr(d_ws),
+                                           d_ws.numel() * d_ws.element_size(), _stream(stream), int(impl)),
+           "vq_gemm_small_batch_impl")
+
+
+def vq_gemm_small_batch_host(fmt: VQFormat, d_idx, d_cb, d_scale, h_X, h_Y, batch: int, d_ws, stream=None) -> None:
+    """h_X / h_Y are host tensors (pinned for asynchronous copies); synchronise before reading h_Y."""
+    c = fmt.c()
+    _check(load().vq_gemm_small_batch_host(ctypes.byref(c), _ptr(d_idx), _ptr(d_cb), _ptr(d_scale), _ptr(h_X),
+                                           _ptr(h_Y), int(batch), _ptr(d_ws),
+                                           d_ws.numel() * d_ws.element_size(), _stream(stream)),
+           "vq_gemm_small_batch_host")
+
+
+def vq_int4g128_gemm_small_batch(n_rows: int, k_cols: int, d_q, d_scale, d_X, d_Y, batch: int, stream=None) -> None:
+    _check(load().vq_int4g128_gemm_small_batch(int(n_rows), int(k_cols), _ptr(d_q), _ptr(d_scale), _ptr(d_X),
+                                               _ptr(d_Y), int(batch), _stream(stream)),
+           "vq_int4g128_gemm_small_batch")

@@ -1,0 +1,187 @@
+// C-ABI entry points: host-side validation and kernel dispatch.  No kernel lives here.
+#include <math.h>
+
+#include "vq_common.cuh"
+
+namespace vq {
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static vq_status check_format(const vq_format* f) {
+  if (!f) return VQ_ERR_NULL;
+  if (!(f->vq_dim == 1 || f->vq_dim == 2 || f->vq_dim == 4)) return VQ_ERR_FORMAT;
+  if (f->index_bits < 1 || f->index_bits > 8) return VQ_ERR_FORMAT;
+  if (!(f->cb_type == VQ_CB_FP16 || f->cb_type == VQ_CB_INT8_SCALED)) return VQ_ERR_FORMAT;
+  if (f->n_rows <= 0 || f->k_cols <= 0 || f->block_rows <= 0 || f->block_cols <= 0) return VQ_ERR_SHAPE;
+  if (f->n_rows % f->block_rows || f->k_cols % f->block_cols || f->block_cols % f->vq_dim) return VQ_ERR_SHAPE;
+  return VQ_OK;
+}
+
+static long long row_stride(const vq_format* f) {
+  const long long bits = static_cast<long long>(f->k_cols / f->vq_dim) * f->index_bits;
+  return ((bits + 7) / 8 + 15) / 16 * 16;
+}
+
+vq_status make_geometry(const vq_format* f, Geometry* g) {
+  vq_status st = check_format(f);
+  if (st != VQ_OK) return st;
+  g->N = f->n_rows;
+  g->K = f->k_cols;
+  g->d = f->vq_dim;
+  g->b = f->index_bits;
+  g->Br = f->block_rows;
+  g->Bc = f->block_cols;
+  g->cb_int8 = f->cb_type == VQ_CB_INT8_SCALED;
+  g->entries = 1 << f->index_bits;
+  g->J = f->k_cols / f->vq_dim;
+  g->blocks_per_row = f->k_cols / f->block_cols;
+  g->stride = row_stride(f);
+  return VQ_OK;
+}
+
+static size_t round256(size_t v) { return (v + 255) / 256 * 256; }
+
+static vq_status check_layer(const vq_format* fmt, const void* d_idx, const void* d_cb,
+                             const void* d_scale, Geometry* g, LayerPtrs* p) {
+  vq_status st = make_geometry(fmt, g);
+  if (st != VQ_OK) return st;
+  if (!d_idx || !d_cb) return VQ_ERR_NULL;
+  if (g->cb_int8 ? d_scale == nullptr : d_scale != nullptr) return VQ_ERR_NULL;
+  if (!aligned16(d_idx) || !aligned16(d_cb) || !aligned16(d_scale)) return VQ_ERR_ALIGN;
+  p->idx = static_cast<const uint8_t*>(d_idx);
+  p->cb = d_cb;
+  p->scale = static_cast<const __half*>(d_scale);
+  return VQ_OK;
+}
+
+}  // namespace vq
+
+using namespace vq;
+
+extern "C" {
+
+vq_status vq_pack_info(const vq_format* fmt, vq_pack_info_t* out) {
+  if (!out) return VQ_ERR_NULL;
+  vq_status st = check_format(fmt);
+  if (st != VQ_OK) return st;
+  const long long N = fmt->n_rows, K = fmt->k_cols, d = fmt->vq_dim;
+  const long long k = 1LL << fmt->index_bits;
+  const int b_c = fmt->cb_type == VQ_CB_INT8_SCALED ? 8 : 16;
+  const long long l = static_cast<long long>(fmt->block_rows) * fmt->block_cols;
+  out->entries = static_cast<int32_t>(k);
+  out->codebook_bits = b_c;
+  out->indices_per_row = K / d;
+  out->row_stride_bytes = row_stride(fmt);
+  out->index_bytes = N * out->row_stride_bytes;
+  out->n_blocks = (N / fmt->block_rows) * (K / fmt->block_cols);
+  out->codebook_bytes_per_block = k * d * b_c / 8;
+  out->codebook_bytes = out->n_blocks * out->codebook_bytes_per_block;
+  out->scale_bytes = fmt->cb_type == VQ_CB_INT8_SCALED ? 2 * out->n_blocks : 0;
+  out->total_bytes = out->index_bytes + out->codebook_bytes + out->scale_bytes;
+  out->bpv_paper = static_cast<double>(fmt->index_bits) / d + static_cast<double>(k * d * b_c) / static_cast<double>(l);
+  out->bpv_stored = 8.0 * static_cast<double>(out->total_bytes) / static_cast<double>(N * K);
+  return VQ_OK;
+}
+
+size_t vq_workspace_bytes(const vq_format* fmt, int batch) {
+  if (check_format(fmt) != VQ_OK || batch < 1 || batch > 16) return 0;
+  // fp32 partial sums of every K-split: [kMaxSplits][batch][N]
+  return round256(static_cast<size_t>(kMaxSplits) * batch * fmt->n_rows * sizeof(float));
+}
+
+size_t vq_workspace_bytes_host(const vq_format* fmt, int batch) {
+  const size_t base = vq_workspace_bytes(fmt, batch);
+  if (!base) return 0;
+  return base + round256(static_cast<size_t>(batch) * fmt->k_cols * 2) + round256(static_cast<size_t>(batch) * fmt->n_rows * 2);
+}
+
+vq_status vq_decode_weights(const vq_format* fmt, const void* d_idx, const void* d_cb,
+                            const void* d_scale, void* d_W, void* stream) {
+  Geometry g;
+  LayerPtrs p;
+  vq_status st = check_layer(fmt, d_idx, d_cb, d_scale, &g, &p);
+  if (st != VQ_OK) return st;
+  if (!d_W) return VQ_ERR_NULL;
+  if (!aligned16(d_W)) return VQ_ERR_ALIGN;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = launch_decode_tuned(g, p, static_cast<__half*>(d_W), s);
+  if (st == VQ_ERR_UNSUPPORTED) st = launch_decode_generic(g, p, static_cast<__half*>(d_W), s);
+  return st;
+}
+
+vq_status vq_gemm_small_batch_impl(const vq_format* fmt, const void* d_idx, const void* d_cb,
+                                   const void* d_scale, const void* d_X, void* d_Y, int batch,
+                                   void* d_ws, size_t ws_bytes, void* stream, int impl) {
+  Geometry g;
+  LayerPtrs p;
+  vq_status st = check_layer(fmt, d_idx, d_cb, d_scale, &g, &p);
+  if (st != VQ_OK) return st;
+  if (batch < 1 || batch > 16) return VQ_ERR_BATCH;
+  if (!d_X || !d_Y) return VQ_ERR_NULL;
+  if (!aligned16(d_X) || !aligned16(d_Y)) return VQ_ERR_ALIGN;
+  if (!d_ws || ws_bytes < vq_workspace_bytes(fmt, batch)) return VQ_ERR_WORKSPACE;
+  if (!aligned16(d_ws)) return VQ_ERR_ALIGN;
+  if (impl != VQ_IMPL_AUTO && impl != VQ_IMPL_GENERIC && impl != VQ_IMPL_TUNED) return VQ_ERR_UNSUPPORTED;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const __half* X = static_cast<const __half*>(d_X);
+  __half* Y = static_cast<__half*>(d_Y);
+  if (impl != VQ_IMPL_GENERIC) {
+    st = launch_gemm_tuned(g, p, X, Y, batch, static_cast<float*>(d_ws), s);
+    if (st != VQ_ERR_UNSUPPORTED || impl == VQ_IMPL_TUNED) return st;
+  }
+  return launch_gemm_generic(g, p, X, Y, batch, s);
+}
+
+vq_status vq_gemm_small_batch(const vq_format* fmt, const void* d_idx, const void* d_cb,
+                              const void* d_scale, const void* d_X, void* d_Y, int batch,
+                              void* d_ws, size_t ws_bytes, void* stream) {
+  return vq_gemm_small_batch_impl(fmt, d_idx, d_cb, d_scale, d_X, d_Y, batch, d_ws, ws_bytes, stream, VQ_IMPL_AUTO);
+}
+
+vq_status vq_gemv(const vq_format* fmt, const void* d_idx, const void* d_cb, const void* d_scale,
+                  const void* d_x, void* d_y, void* d_ws, size_t ws_bytes, void* stream) {
+  return vq_gemm_small_batch_impl(fmt, d_idx, d_cb, d_scale, d_x, d_y, 1, d_ws, ws_bytes, stream, VQ_IMPL_AUTO);
+}
+
+vq_status vq_gemm_small_batch_host(const vq_format* fmt, const void* d_idx, const void* d_cb,
+                                   const void* d_scale, const void* h_X, void* h_Y, int batch,
+                                   void* d_ws, size_t ws_bytes, void* stream) {
+  if (!h_X || !h_Y) return VQ_ERR_NULL;
+  if (batch < 1 || batch > 16) return VQ_ERR_BATCH;
+  Geometry g;
+  LayerPtrs p;
+  vq_status st = check_layer(fmt, d_idx, d_cb, d_scale, &g, &p);
+  if (st != VQ_OK) return st;
+  const size_t need = vq_workspace_bytes_host(fmt, batch);
+  if (!d_ws || ws_bytes < need) return VQ_ERR_WORKSPACE;
+  if (!aligned16(d_ws)) return VQ_ERR_ALIGN;
+  const size_t base = vq_workspace_bytes(fmt, batch);
+  const size_t x_bytes = static_cast<size_t>(batch) * fmt->k_cols * 2;
+  const size_t y_bytes = static_cast<size_t>(batch) * fmt->n_rows * 2;
+  char* ws = static_cast<char*>(d_ws);
+  void* d_X = ws + base;
+  void* d_Y = ws + base + round256(x_bytes);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(d_X, h_X, x_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return VQ_ERR_CUDA;
+  st = vq_gemm_small_batch(fmt, d_idx, d_cb, d_scale, d_X, d_Y, batch, d_ws, base, stream);
+  if (st != VQ_OK) return st;
+  if (cudaMemcpyAsync(h_Y, d_Y, y_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return VQ_ERR_CUDA;
+  return VQ_OK;
+}
+
+const char* vq_status_string(vq_status s) {
+  switch (s) {
+    case VQ_OK: return "VQ_OK";
+    case VQ_ERR_NULL: return "VQ_ERR_NULL: missing pointer or scale pointer does not match cb_type";
+    case VQ_ERR_FORMAT: return "VQ_ERR_FORMAT: vq_dim/index_bits/cb_type out of range";
+    case VQ_ERR_SHAPE: return "VQ_ERR_SHAPE: sizes not positive or not divisible by the block shape";
+    case VQ_ERR_ALIGN: return "VQ_ERR_ALIGN: device pointer not 16-byte aligned";
+    case VQ_ERR_WORKSPACE: return "VQ_ERR_WORKSPACE: workspace missing or too small";
+    case VQ_ERR_BATCH: return "VQ_ERR_BATCH: batch outside 1..16";
+    case VQ_ERR_UNSUPPORTED: return "VQ_ERR_UNSUPPORTED: requested kernel variant does not cover this format";
+    case VQ_ERR_CUDA: return "VQ_ERR_CUDA: CUDA runtime reported an error";
+  }
+  return "unknown vq_status";
+}
+
+}  // extern "C"

@@ -1,0 +1,46 @@
+// Shared declarations of the CUDA side of the VQ-decode library (sm_100a).
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "vq.h"
+
+namespace vq {
+
+// Format with derived quantities, passed by value to kernels.
+struct Geometry {
+  int N, K, d, b, Br, Bc;
+  int cb_int8;            // 0: fp16 codebook, 1: int8 codebook + fp16 block scale
+  int entries;            // 2^b
+  int J;                  // indices per row = K/d
+  int blocks_per_row;     // K/Bc
+  long long stride;       // bytes between index rows
+};
+
+struct LayerPtrs {
+  const uint8_t* idx;
+  const void* cb;
+  const __half* scale;
+};
+
+// Maximum number of K-splits any kernel uses; fixes the workspace size.
+constexpr int kMaxSplits = 8;
+
+vq_status make_geometry(const vq_format* fmt, Geometry* g);
+
+// Kernel launchers.  Each returns VQ_OK, VQ_ERR_UNSUPPORTED (format/shape not covered by this
+// family) or VQ_ERR_CUDA.
+vq_status launch_decode_generic(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s);
+vq_status launch_gemm_generic(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y,
+                              int batch, cudaStream_t s);
+vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y,
+                            int batch, float* ws, cudaStream_t s);
+vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s);
+
+inline vq_status check_launch() {
+  return cudaGetLastError() == cudaSuccess ? VQ_OK : VQ_ERR_CUDA;
+}
+
+}  // namespace vq

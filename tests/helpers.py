@@ -1,0 +1,73 @@
+"""Shared test plumbing: draw a synthetic layer, describe it to the oracle and to the library."""
+from __future__ import annotations
+
+import numpy as np
+
+import vq_synth
+from oracle import vq_oracle as orc
+
+TOL = 1e-3  # |y_gpu - y_ref| <= TOL * sum_k |W_nk x_k| per output element
+
+
+def oracle_fmt(spec: vq_synth.LayerSpec) -> orc.Fmt:
+    return orc.Fmt(spec.N, spec.K, spec.d, spec.b, spec.Br, spec.Bc, spec.int8)
+
+
+def lib_fmt(spec: vq_synth.LayerSpec):
+    import paper_2402_15319_b200 as vq
+    return vq.VQFormat(spec.N, spec.K, spec.d, spec.b, spec.Br, spec.Bc,
+                       vq.VQ_CB_INT8_SCALED if spec.int8 else vq.VQ_CB_FP16)
+
+
+def draw(spec: vq_synth.LayerSpec, seed: int, layer_id: int = 0) -> vq_synth.Layer:
+    return vq_synth.make_layer(spec, oracle_fmt(spec).stride, seed, layer_id)
+
+
+class DeviceLayer:
+    """Device copies of one layer + workspace, made with torch (memory plumbing only)."""
+
+    def __init__(self, spec, layer, max_batch=16, device="cuda:0"):
+        import torch
+        import paper_2402_15319_b200 as vq
+        self.spec, self.fmt = spec, lib_fmt(spec)
+        self.idx = torch.from_numpy(layer.idx).to(device)
+        self.cb = torch.from_numpy(layer.cb).to(device)
+        self.scale = None if layer.scale is None else torch.from_numpy(layer.scale).to(device)
+        self.ws = torch.empty(vq.vq_workspace_bytes(self.fmt, max_batch), dtype=torch.uint8, device=device)
+        self.device = device
+
+    def gemm(self, X: np.ndarray, impl=None):
+        import torch
+        import paper_2402_15319_b200 as vq
+        X = np.ascontiguousarray(np.atleast_2d(X))
+        batch = X.shape[0]
+        dX = torch.from_numpy(X).to(self.device)
+        dY = torch.full((batch, self.spec.N), float("nan"), dtype=torch.float16, device=self.device)
+        if impl is None:
+            vq.vq_gemm_small_batch(self.fmt, self.idx, self.cb, self.scale, dX, dY, batch, self.ws)
+        else:
+            vq.vq_gemm_small_batch_impl(self.fmt, self.idx, self.cb, self.scale, dX, dY, batch, self.ws, impl)
+        torch.cuda.synchronize()
+        return dY.cpu().numpy()
+
+    def decode(self):
+        import torch
+        import paper_2402_15319_b200 as vq
+        dW = torch.full((self.spec.N, self.spec.K), float("nan"), dtype=torch.float16, device=self.device)
+        vq.vq_decode_weights(self.fmt, self.idx, self.cb, self.scale, dW)
+        torch.cuda.synchronize()
+        return dW.cpu().numpy()
+
+
+def assert_outputs_close(Y_gpu: np.ndarray, Y_ref: np.ndarray, A_ref: np.ndarray, what=""):
+    """The acceptance bound: per element |y_gpu - y_ref| <= 1e-3 * sum_k |W x|."""
+    assert Y_gpu.shape == Y_ref.shape, (Y_gpu.shape, Y_ref.shape)
+    assert np.isfinite(Y_gpu.astype(np.float64)).all(), f"{what}: non-finite output"
+    err = np.abs(Y_gpu.astype(np.float64) - Y_ref)
+    bound = TOL * A_ref
+    bad = err > bound
+    if bad.any():
+        i = np.unravel_index(np.argmax(err - bound), err.shape)
+        raise AssertionError(f"{what}: {bad.sum()} outputs beyond tolerance; worst at {i}: "
+                             f"gpu={Y_gpu[i]} ref={Y_ref[i]} err={err[i]:.3e} bound={bound[i]:.3e}")
+    return float((err / np.maximum(bound, 1e-300)).max())

@@ -1,0 +1,215 @@
+"""GPU parity: the CUDA library, called through the C-ABI, against the CPU oracle on the same
+seeded inputs.  Unpack/decode must be bit-exact; GEMV/GEMM outputs must satisfy
+|y_gpu - y_ref| <= 1e-3 * sum_k |W_nk x_k| per element."""
+import numpy as np
+import pytest
+
+import vq_synth
+from oracle import vq_oracle as orc
+from tests.helpers import DeviceLayer, assert_outputs_close, draw, oracle_fmt
+
+pytestmark = pytest.mark.gpu
+
+import paper_2402_15319_b200 as vq  # noqa: E402
+
+IMPLS = [vq.VQ_IMPL_GENERIC, vq.VQ_IMPL_AUTO]
+
+
+def _check_layer(spec, seed, batches, impls=IMPLS, decode=True, rows=None, layer_id=0):
+    f = oracle_fmt(spec)
+    L = draw(spec, seed, layer_id)
+    dev = DeviceLayer(spec, L)
+    if decode:
+        _, W16 = orc.decode(f, L.idx, L.cb, L.scale, exact=False)
+        W_gpu = dev.decode().view(np.uint16)
+        assert np.array_equal(W_gpu, W16), f"{spec.name}: decode not bit-exact"
+    worst = 0.0
+    for batch in batches:
+        X = vq_synth.make_x(spec, seed + 17, batch, layer_id)
+        Y, A = orc.gemm(f, L.idx, L.cb, L.scale, X, rows=rows, threads=8)
+        for impl in impls:
+            Yg = dev.gemm(X, impl)
+            if rows is not None:
+                Yg = Yg[:, rows]
+            worst = max(worst, assert_outputs_close(Yg, Y, A, f"{spec.name} batch={batch} impl={impl}"))
+    return worst
+
+
+# ---- every (d, b, codebook type) on small ragged shapes --------------------------------------
+@pytest.mark.parametrize("int8", [False, True])
+@pytest.mark.parametrize("b", range(1, 9))
+@pytest.mark.parametrize("d", [1, 2, 4])
+def test_all_formats_small(d, b, int8):
+    # K/d = 104 indices: not a multiple of 8*anything nice, 13 groups of 8; 37 rows: ragged vs 8/16-row tiles
+    spec = vq_synth.LayerSpec(f"small_d{d}b{b}", N=37, K=104 * d, d=d, b=b, Br=1, Bc=52 * d, int8=int8)
+    _check_layer(spec, seed=10 * b + d, batches=(1, 3))
+    # tall blocks, several block rows, K/d = 9 -> a ragged last group of indices
+    spec = vq_synth.LayerSpec(f"tall_d{d}b{b}", N=48, K=9 * d, d=d, b=b, Br=16, Bc=3 * d, int8=int8)
+    _check_layer(spec, seed=20 * b + d, batches=(2,))
+
+
+@pytest.mark.parametrize("batch", range(1, 17))
+def test_every_batch(batch):
+    spec = vq_synth.LayerSpec("b", N=200, K=512, d=2, b=6, Br=8, Bc=128, int8=False)
+    _check_layer(spec, seed=batch, batches=(batch,), decode=False)
+    spec = vq_synth.LayerSpec("b8", N=96, K=1024, d=2, b=4, Br=1, Bc=512, int8=True)
+    _check_layer(spec, seed=batch + 50, batches=(batch,), decode=False)
+
+
+def test_degenerate_shapes():
+    _check_layer(vq_synth.LayerSpec("one", N=1, K=4, d=4, b=8, Br=1, Bc=4, int8=False), 1, (1, 16))
+    _check_layer(vq_synth.LayerSpec("one_idx", N=3, K=1, d=1, b=1, Br=3, Bc=1, int8=True), 2, (1,))
+    _check_layer(vq_synth.LayerSpec("wide", N=2, K=16384, d=2, b=5, Br=2, Bc=8192, int8=False), 3, (1, 2))
+    _check_layer(vq_synth.LayerSpec("tall", N=5000, K=8, d=2, b=3, Br=1000, Bc=8, int8=True), 4, (1,))
+
+
+# ---- tile-aligned shapes of the benchmark format families, several tiles + row tails ----------
+FAMILY = [
+    vq_synth.LayerSpec("fam1", N=272, K=2048, d=2, b=4, Br=1, Bc=1024, int8=False),
+    vq_synth.LayerSpec("fam2", N=144, K=4096, d=1, b=4, Br=1, Bc=2048, int8=True),
+    vq_synth.LayerSpec("fam3", N=384, K=1024, d=2, b=6, Br=128, Bc=128, int8=False),
+    vq_synth.LayerSpec("fam3w", N=128, K=11008, d=2, b=6, Br=128, Bc=128, int8=False),
+    vq_synth.LayerSpec("fam4", N=512, K=1024, d=4, b=8, Br=256, Bc=512, int8=False, cb_sigma=0.015),
+    vq_synth.LayerSpec("fam5", N=208, K=4096, d=2, b=4, Br=1, Bc=2048, int8=True),
+]
+
+
+@pytest.mark.parametrize("spec", FAMILY, ids=lambda s: s.name)
+def test_benchmark_families_medium(spec):
+    _check_layer(spec, seed=77, batches=(1, 2, 4, 8, 16))
+
+
+# ---- properties that hold at any size ---------------------------------------------------------
+def test_unit_vectors_return_decoded_columns():
+    spec = vq_synth.LayerSpec("unit", N=256, K=256, d=2, b=6, Br=128, Bc=128, int8=False)
+    L = draw(spec, 5)
+    dev = DeviceLayer(spec, L)
+    W = dev.decode()
+    for k0 in (0, 1, 127, 128, 255):
+        X = np.zeros((1, spec.K), np.float16)
+        X[0, k0] = 1.0
+        for impl in IMPLS:
+            assert np.array_equal(dev.gemm(X, impl)[0].view(np.uint16), W[:, k0].view(np.uint16))
+
+
+def test_int8_unit_scale_integer_inputs_exact_and_deterministic():
+    spec = vq_synth.LayerSpec("int", N=64, K=4096, d=2, b=4, Br=1, Bc=2048, int8=True)
+    L = draw(spec, 6)
+    L.scale[:] = 1.0
+    rng = np.random.default_rng(0)
+    X = rng.integers(-2, 3, size=(2, spec.K)).astype(np.float16)
+    Y, _ = orc.gemm(oracle_fmt(spec), L.idx, L.cb, L.scale, X)
+    assert np.abs(Y).max() < 2048 * 8  # integers exactly representable after fp32 accumulation
+    dev = DeviceLayer(spec, L)
+    for impl in IMPLS:
+        Yg = dev.gemm(X, impl)
+        assert np.array_equal(Yg.astype(np.float64), Y.astype(np.float16).astype(np.float64))
+        assert np.array_equal(dev.gemm(X, impl).view(np.uint16), Yg.view(np.uint16))  # run-to-run identical
+
+
+def test_zero_codebook_gives_exact_zero():
+    spec = vq_synth.LayerSpec("zero", N=64, K=2048, d=2, b=4, Br=1, Bc=1024, int8=False)
+    L = draw(spec, 8)
+    L.cb[:] = 0
+    dev = DeviceLayer(spec, L)
+    X = vq_synth.make_x(spec, 1, 4)
+    for impl in IMPLS:
+        assert not dev.gemm(X, impl).any()
+
+
+# ---- the five benchmark configurations at full size -------------------------------------------
+def _sample_rows(N, Br, n=192, seed=0):
+    rng = np.random.default_rng(seed)
+    rows = set(rng.integers(0, N, size=n).tolist()) | {0, 1, N - 1, N - 2, min(N - 1, Br), max(0, N - Br - 1)}
+    return np.array(sorted(rows), np.int32)
+
+
+def _decode_slab_check(spec, L, dev_W, block_row):
+    """Bit-exact decode of one block-row (Br rows) of a full-size layer."""
+    r0 = block_row * spec.Br
+    bpr = spec.K // spec.Bc
+    sub = orc.Fmt(spec.Br, spec.K, spec.d, spec.b, spec.Br, spec.Bc, spec.int8)
+    cb = L.cb[block_row * bpr:(block_row + 1) * bpr]
+    sc = None if L.scale is None else L.scale[block_row * bpr:(block_row + 1) * bpr]
+    _, W16 = orc.decode(sub, L.idx[r0:r0 + spec.Br], cb, sc, exact=False)
+    assert np.array_equal(dev_W[r0:r0 + spec.Br].view(np.uint16), W16), f"{spec.name}: decode rows {r0}.."
+
+
+@pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+def test_benchmark_configs_full_size(cfg):
+    conf = vq_synth.CONFIGS[cfg]
+    seen = set()
+    for layer_id, spec in enumerate(conf["layers"]):
+        if (spec.N, spec.K) in seen:       # q/k/v/o share a shape: one of each shape is enough
+            continue
+        seen.add((spec.N, spec.K))
+        f = oracle_fmt(spec)
+        L = draw(spec, conf["seed"], layer_id)
+        dev = DeviceLayer(spec, L)
+        W = dev.decode()
+        n_block_rows = spec.N // spec.Br
+        slabs = {0, n_block_rows - 1, n_block_rows // 2} if spec.Br > 1 else set(range(0, spec.N, max(1, spec.N // 24))) | {spec.N - 1}
+        for br in sorted(slabs):
+            _decode_slab_check(spec, L, W, br)
+        del W
+        rows = _sample_rows(spec.N, spec.Br, seed=layer_id)
+        for batch in conf["batches"]:
+            X = vq_synth.make_x(spec, conf["seed"], batch, layer_id)
+            Y, A = orc.gemm(f, L.idx, L.cb, L.scale, X, rows=rows, threads=8)
+            Yg = dev.gemm(X)
+            assert np.isfinite(Yg.astype(np.float64)).all()
+            assert_outputs_close(Yg[:, rows], Y, A, f"{spec.name} batch={batch}")
+            if batch == 1:
+                Yg2 = dev.gemm(X, vq.VQ_IMPL_GENERIC)
+                assert_outputs_close(Yg2[:, rows], Y, A, f"{spec.name} generic")
+
+
+# ---- INT4 g128 yard-stick ---------------------------------------------------------------------
+@pytest.mark.parametrize("N,K", [(100, 256), (64, 4096), (37, 11008 - 11008 % 128)])
+def test_int4g128(N, K):
+    import torch
+    q, s = vq_synth.make_int4g128(N, K, seed=3)
+    spec = vq_synth.LayerSpec("i4", N, K, 1, 4, 1, 128, True)
+    for batch in (1, 5, 16):
+        X = vq_synth.make_x(spec, 9, batch)
+        Y, A = orc.int4g128_gemm(q, s, X, threads=4)
+        dq, ds, dX = (torch.from_numpy(a).cuda() for a in (q, s, X))
+        dY = torch.full((batch, N), float("nan"), dtype=torch.float16, device="cuda")
+        vq.vq_int4g128_gemm_small_batch(N, K, dq, ds, dX, dY, batch)
+        torch.cuda.synchronize()
+        assert_outputs_close(dY.cpu().numpy(), Y, A, f"int4 {N}x{K} b{batch}")
+
+
+def test_host_buffer_entry_point():
+    import torch
+    spec = vq_synth.LayerSpec("host", N=256, K=1024, d=2, b=6, Br=128, Bc=128, int8=False)
+    L = draw(spec, 12)
+    dev = DeviceLayer(spec, L)
+    batch = 4
+    X = vq_synth.make_x(spec, 2, batch)
+    hX = torch.from_numpy(X).pin_memory()
+    hY = torch.zeros((batch, spec.N), dtype=torch.float16).pin_memory()
+    ws = torch.empty(vq.vq_workspace_bytes_host(dev.fmt, batch), dtype=torch.uint8, device="cuda")
+    vq.vq_gemm_small_batch_host(dev.fmt, dev.idx, dev.cb, dev.scale, hX, hY, batch, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(hY.numpy().view(np.uint16), dev.gemm(X).view(np.uint16))
+
+
+def test_runtime_argument_errors_on_device_pointers():
+    import torch
+    spec = vq_synth.LayerSpec("err", N=16, K=64, d=2, b=4, Br=1, Bc=64, int8=False)
+    L = draw(spec, 1)
+    dev = DeviceLayer(spec, L)
+    X = torch.zeros((1, 64), dtype=torch.float16, device="cuda")
+    Y = torch.zeros((1, 16), dtype=torch.float16, device="cuda")
+    small = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(vq.VQError) as e:
+        vq.vq_gemm_small_batch(dev.fmt, dev.idx, dev.cb, None, X, Y, 1, small)
+    assert e.value.code == 5
+    with pytest.raises(vq.VQError) as e:
+        buf = torch.zeros(256, dtype=torch.uint8, device="cuda")
+        vq.vq_gemm_small_batch(dev.fmt, dev.idx, dev.cb, None, buf[2:130].view(torch.float16), Y, 1, dev.ws)
+    assert e.value.code == 4
+    with pytest.raises(vq.VQError) as e:
+        vq.vq_gemm_small_batch_impl(dev.fmt, dev.idx, dev.cb, None, X, Y, 1, dev.ws, 9)
+    assert e.value.code == 7

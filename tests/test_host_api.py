@@ -1,0 +1,147 @@
+"""CPU-only checks of the C-ABI library: it loads, exports what include/vq.h declares, sizes and
+bits-per-value agree with the paper's printed rows, and every argument error is caught on the
+host before any CUDA call (fake non-null pointers are never dereferenced)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2402_15319_b200 as vq
+from paper_2402_15319_b200 import build as vq_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+GOLD = os.path.join(ROOT, "tests", "golden")
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    vq_build.build()
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "vq.h")).read()
+    declared = set(re.findall(r"\b(vq_[a-z0-9_]+)\s*\(", header))
+    assert {"vq_pack_info", "vq_decode_weights", "vq_gemv", "vq_gemm_small_batch"} <= declared
+    lib = ctypes.CDLL(vq.lib_path())
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert declared == set(vq.exported_symbols())
+
+
+def test_pack_info_matches_paper_bpv_rows():
+    # rows of the paper's tables that are expressible as a block of l weights: take 1 x l blocks
+    for line in open(os.path.join(GOLD, "bpv_rows.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        k, d, b_c, l, printed = line.split()[:5]
+        k, d, b_c, l = int(k), int(d), int(b_c), int(l)
+        b = k.bit_length() - 1
+        f = vq.VQFormat(4, l * 2, d, b, 1, l, vq.VQ_CB_FP16 if b_c == 16 else vq.VQ_CB_INT8_SCALED)
+        assert vq.vq_pack_info(f).bpv_paper == pytest.approx(float(printed), abs=1e-12), line
+
+
+def test_pack_info_benchmark_sizes():
+    # compressed bytes of the benchmark layers (index + codebook + scale)
+    f1 = vq.VQFormat(4096, 4096, 2, 4, 1, 1024, vq.VQ_CB_FP16)
+    i1 = vq.vq_pack_info(f1)
+    assert (i1.index_bytes, i1.codebook_bytes, i1.scale_bytes, i1.total_bytes) == (4194304, 1048576, 0, 5242880)
+    assert i1.bpv_paper == 2.5 and i1.bpv_stored == 2.5 and i1.row_stride_bytes == 1024
+    f2 = vq.VQFormat(4096, 4096, 1, 4, 1, 2048, vq.VQ_CB_INT8_SCALED)
+    i2 = vq.vq_pack_info(f2)
+    assert (i2.index_bytes, i2.codebook_bytes, i2.scale_bytes) == (8388608, 131072, 16384)
+    assert i2.bpv_paper == 4.0625 and i2.bpv_stored == pytest.approx(4.0703125)
+    f3 = vq.VQFormat(11008, 4096, 2, 6, 128, 128, vq.VQ_CB_FP16)
+    i3 = vq.vq_pack_info(f3)
+    assert i3.bpv_paper == 3.125 and i3.row_stride_bytes == 1536 and i3.entries == 64
+    assert vq.vq_pack_info(vq.VQFormat(4096, 11008, 2, 6, 128, 128, 0)).row_stride_bytes == 4128
+    f4 = vq.VQFormat(5120, 13824, 4, 8, 256, 512, vq.VQ_CB_FP16)
+    i4 = vq.vq_pack_info(f4)
+    assert i4.bpv_paper == 2.125 and i4.codebook_bytes_per_block == 2048 and i4.row_stride_bytes == 3456
+    f5 = vq.VQFormat(28672, 8192, 2, 4, 1, 2048, vq.VQ_CB_INT8_SCALED)
+    i5 = vq.vq_pack_info(f5)
+    assert i5.bpv_paper == 2.125 and i5.bpv_stored == pytest.approx(2.1328125)
+    # ragged stride: 3 indices of 5 bits -> 2 bytes -> padded to 16
+    assert vq.vq_pack_info(vq.VQFormat(2, 3, 1, 5, 1, 3, 0)).row_stride_bytes == 16
+
+
+GOOD = vq.VQFormat(8, 16, 2, 4, 1, 16, vq.VQ_CB_FP16)
+FAKE = ctypes.c_void_p(0x10000)       # aligned, never dereferenced: every call below fails validation first
+ODD = ctypes.c_void_p(0x10008)
+
+
+def _call_gemm(fmt, idx=FAKE, cb=FAKE, scale=None, X=FAKE, Y=FAKE, batch=1, ws=FAKE, ws_bytes=1 << 30):
+    c = fmt.c()
+    return vq.load().vq_gemm_small_batch(ctypes.byref(c), idx, cb, scale, X, Y, batch, ws, ws_bytes, None)
+
+
+def _replace(fmt, **kw):
+    d = dict(fmt.__dict__)
+    d.update(kw)
+    return vq.VQFormat(**d)
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(vq_dim=3), 2), (dict(vq_dim=0), 2), (dict(index_bits=0), 2), (dict(index_bits=9), 2),
+    (dict(cb_type=2), 2), (dict(n_rows=0), 3), (dict(k_cols=-4), 3), (dict(block_rows=3), 3),
+    (dict(block_cols=5), 3), (dict(block_cols=0), 3), (dict(vq_dim=4, block_cols=2, k_cols=16), 3),
+])
+def test_bad_formats_rejected(kw, code):
+    f = _replace(GOOD, **kw)
+    with pytest.raises(vq.VQError) as e:
+        vq.vq_pack_info(f)
+    assert e.value.code == code
+    assert vq.vq_workspace_bytes(f, 1) == 0
+    assert _call_gemm(f) == code
+
+
+def test_argument_errors_before_any_launch():
+    lib = vq.load()
+    c = GOOD.c()
+    assert lib.vq_pack_info(None, None) == 1
+    assert lib.vq_pack_info(ctypes.byref(c), None) == 1
+    assert _call_gemm(GOOD, idx=None) == 1
+    assert _call_gemm(GOOD, cb=None) == 1
+    assert _call_gemm(GOOD, X=None) == 1
+    assert _call_gemm(GOOD, Y=None) == 1
+    assert _call_gemm(GOOD, scale=FAKE) == 1                      # fp16 codebook must not carry a scale
+    assert _call_gemm(_replace(GOOD, cb_type=1), scale=None) == 1  # int8 codebook needs one
+    for k in ("idx", "cb", "X", "Y", "ws"):
+        assert _call_gemm(GOOD, **{k: ODD}) == 4
+    assert _call_gemm(_replace(GOOD, cb_type=1), scale=ODD) == 4
+    assert _call_gemm(GOOD, batch=0) == 6
+    assert _call_gemm(GOOD, batch=17) == 6
+    assert _call_gemm(GOOD, ws=None) == 5
+    assert _call_gemm(GOOD, ws_bytes=vq.vq_workspace_bytes(GOOD, 1) - 1) == 5
+    assert vq.vq_workspace_bytes(GOOD, 0) == 0 and vq.vq_workspace_bytes(GOOD, 17) == 0
+    assert vq.vq_workspace_bytes(GOOD, 16) >= vq.vq_workspace_bytes(GOOD, 1) > 0
+    assert vq.vq_workspace_bytes_host(GOOD, 2) > vq.vq_workspace_bytes(GOOD, 2)
+    # decode
+    assert lib.vq_decode_weights(ctypes.byref(c), FAKE, FAKE, None, None, None) == 1
+    assert lib.vq_decode_weights(ctypes.byref(c), FAKE, FAKE, None, ODD, None) == 4
+    assert lib.vq_decode_weights(ctypes.byref(c), None, FAKE, None, FAKE, None) == 1
+    # impl selector out of range
+    assert lib.vq_gemm_small_batch_impl(ctypes.byref(c), FAKE, FAKE, None, FAKE, FAKE, 1, FAKE, 1 << 30, None, 9) == 7
+    # host-buffer variant
+    assert lib.vq_gemm_small_batch_host(ctypes.byref(c), FAKE, FAKE, None, None, FAKE, 1, FAKE, 1 << 30, None) == 1
+    assert lib.vq_gemm_small_batch_host(ctypes.byref(c), FAKE, FAKE, None, FAKE, FAKE, 1, FAKE, 16, None) == 5
+    # INT4 yard-stick
+    assert lib.vq_int4g128_gemm_small_batch(8, 100, FAKE, FAKE, FAKE, FAKE, 1, None) == 3
+    assert lib.vq_int4g128_gemm_small_batch(8, 256, None, FAKE, FAKE, FAKE, 1, None) == 1
+    assert lib.vq_int4g128_gemm_small_batch(8, 256, FAKE, FAKE, ODD, FAKE, 1, None) == 4
+    assert lib.vq_int4g128_gemm_small_batch(8, 256, FAKE, FAKE, FAKE, FAKE, 0, None) == 6
+
+
+def test_status_strings():
+    names = [vq.vq_status_string(i) for i in range(9)]
+    assert names[0] == "VQ_OK" and len(set(names)) == 9
+    assert "unknown" in vq.vq_status_string(99)
+
+
+def test_missing_library_is_an_error(monkeypatch, tmp_path):
+    from paper_2402_15319_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "_LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="missing"):
+        binding.load()
