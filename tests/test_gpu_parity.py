@@ -99,7 +99,7 @@ def test_int8_unit_scale_integer_inputs_exact_and_deterministic():
     rng = np.random.default_rng(0)
     X = rng.integers(-2, 3, size=(2, spec.K)).astype(np.float16)
     Y, _ = orc.gemm(oracle_fmt(spec), L.idx, L.cb, L.scale, X)
-    assert np.abs(Y).max() < 2048 * 8  # integers exactly representable after fp32 accumulation
+    assert np.abs(Y).max() < 60000  # partial sums are integers < 2^24: exact in fp32, finite in fp16
     dev = DeviceLayer(spec, L)
     for impl in IMPLS:
         Yg = dev.gemm(X, impl)
