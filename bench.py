@@ -1,0 +1,427 @@
+#!/usr/bin/env python
+"""Benchmark of the VQ-decode linear-layer hot path on B200.
+
+A step = one pass of the whole hot path (stream indices, stage codebooks, unpack, look up,
+multiply-accumulate, reduce + store) over one batch of synthetic activations for every layer
+of one benchmark configuration (default: the Llama-2-7B-shaped layer set, 2-D VQ with 6-bit
+indices, batch 1).  Metric: compressed bytes (indices + codebooks + scales + activations +
+outputs) moved per second, i.e. achieved HBM bandwidth on the compressed representation.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import vq_synth  # noqa: E402
+
+METRIC = "vq_decode_gemv_compressed_byte_hbm_bandwidth"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def layer_bytes(spec: vq_synth.LayerSpec, stride: int, batch: int) -> int:
+    """Algorithmic bytes of one layer call: everything stored for W plus activations and outputs."""
+    idx = spec.N * stride
+    cb = spec.n_blocks * spec.entries * spec.d * (1 if spec.int8 else 2)
+    sc = spec.n_blocks * 2 if spec.int8 else 0
+    return idx + cb + sc + 2 * batch * (spec.K + spec.N)
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Polls NVML for SM clock and throttle reasons while the timed region runs."""
+
+    BAD = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20}
+    NOTE = {"sw_power_cap": 0x4}
+
+    def __init__(self, uuid: str):
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _poll(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h) if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons") \
+                    else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for name, bit in {**self.BAD, **self.NOTE}.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self.nv:
+            self._stop.clear()
+            self._thread = threading.Thread(target=self._poll, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread:
+            self._stop.set()
+            self._thread.join()
+            self._thread = None
+
+    def summary(self, source: str):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0, "source": "nvml unavailable"}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples), "source": source}
+
+
+# ------------------------------------------------------------------------------------------
+# the CUDA arm
+# ------------------------------------------------------------------------------------------
+class DeviceSet:
+    """R distinct device copies of every layer of a configuration, so that a layer's bytes have
+    been evicted from L2 by the time its copy is read again."""
+
+    def __init__(self, cfg_name: str, batch: int, device, max_copies=None):
+        import torch
+        import paper_2402_15319_b200 as vq
+        self.vq, self.torch = vq, torch
+        conf = vq_synth.CONFIGS[cfg_name]
+        self.cfg_name, self.batch, self.device = cfg_name, batch, device
+        self.specs = conf["layers"]
+        self.fmts, self.host, self.bytes_per_layer = [], [], []
+        for lid, spec in enumerate(self.specs):
+            fmt = vq.VQFormat(spec.N, spec.K, spec.d, spec.b, spec.Br, spec.Bc, int(spec.int8))
+            info = vq.vq_pack_info(fmt)
+            L = vq_synth.make_layer(spec, info.row_stride_bytes, conf["seed"], lid)
+            X = vq_synth.make_x(spec, conf["seed"], batch, lid)
+            self.fmts.append(fmt)
+            self.host.append((L, X))
+            self.bytes_per_layer.append(layer_bytes(spec, info.row_stride_bytes, batch))
+        self.step_bytes = int(sum(self.bytes_per_layer))
+        self.n_weights = sum(s.n_weights for s in self.specs)
+        self.copies = max(2, -(-2 * L2_BYTES // self.step_bytes))
+        if max_copies:
+            self.copies = min(self.copies, max_copies)
+        self.dev = []  # [copy][layer] -> (idx, cb, scale)
+        base = []
+        for (L, X) in self.host:
+            base.append((torch.from_numpy(L.idx).to(device), torch.from_numpy(L.cb).to(device),
+                         None if L.scale is None else torch.from_numpy(L.scale).to(device)))
+        self.dev.append(base)
+        for _ in range(1, self.copies):
+            self.dev.append([tuple(None if t is None else t.clone() for t in lay) for lay in base])
+        self.X = [torch.from_numpy(X).to(device) for (_, X) in self.host]
+        self.Y = [torch.empty((batch, s.N), dtype=torch.float16, device=device) for s in self.specs]
+        self.ws = [torch.empty(vq.vq_workspace_bytes(f, batch), dtype=torch.uint8, device=device) for f in self.fmts]
+        # host side of the end-to-end path
+        self.hX = [torch.from_numpy(X).pin_memory() for (_, X) in self.host]
+        self.hY = [torch.empty((batch, s.N), dtype=torch.float16).pin_memory() for s in self.specs]
+        self.ws_host = [torch.empty(vq.vq_workspace_bytes_host(f, batch), dtype=torch.uint8, device=device) for f in self.fmts]
+        self.h2d = sum(int(x.numel()) * 2 for x in self.hX)
+        self.d2h = sum(int(y.numel()) * 2 for y in self.hY)
+
+    def step(self, copy: int):
+        vq = self.vq
+        for i, fmt in enumerate(self.fmts):
+            idx, cb, sc = self.dev[copy][i]
+            vq.vq_gemm_small_batch(fmt, idx, cb, sc, self.X[i], self.Y[i], self.batch, self.ws[i])
+
+    def step_host(self, copy: int):
+        vq = self.vq
+        for i, fmt in enumerate(self.fmts):
+            idx, cb, sc = self.dev[copy][i]
+            vq.vq_gemm_small_batch_host(fmt, idx, cb, sc, self.hX[i], self.hY[i], self.batch, self.ws_host[i])
+        self.torch.cuda.synchronize()
+
+    def launches_per_step(self) -> int:
+        return len(self.fmts) * self.vq.vq_kernel_launches() if hasattr(self.vq, "vq_kernel_launches") else len(self.fmts)
+
+    def graph(self, n_steps: int, first_copy: int = 0):
+        torch = self.torch
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for s in range(n_steps):
+                self.step((first_copy + s) % self.copies)
+        return g
+
+
+def time_steps(ds: DeviceSet, steps: int, warmup: int, barrier=None):
+    """Times exactly `steps` steps as CUDA-graph replays (one graph = one round over all copies)."""
+    torch = ds.torch
+    chunk = ds.copies
+    ds.step(0)
+    torch.cuda.synchronize()
+    g_full = ds.graph(chunk)
+    rem = steps % chunk
+    g_rem = ds.graph(rem) if rem else None
+    for _ in range(max(1, -(-warmup // chunk))):
+        g_full.replay()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps // chunk):
+        g_full.replay()
+    if g_rem:
+        g_rem.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    return e0.elapsed_time(e1)  # ms
+
+
+def time_e2e(ds: DeviceSet, steps: int, warmup: int):
+    torch = ds.torch
+    for s in range(max(3, min(warmup, 10))):
+        ds.step_host(s % ds.copies)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for s in range(steps):
+        ds.step_host(s % ds.copies)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1)
+
+
+class OracleWork:
+    """Host copies of a configuration for the CPU oracle; a pass covers the first rows of each layer."""
+
+    def __init__(self, cfg_name: str, batch: int):
+        from oracle import vq_oracle as orc
+        self.orc = orc
+        conf = vq_synth.CONFIGS[cfg_name]
+        self.cfg_name, self.batch = cfg_name, batch
+        self.total_w = sum(s.n_weights for s in conf["layers"])
+        self.work = []
+        for lid, spec in enumerate(conf["layers"]):
+            f = orc.Fmt(spec.N, spec.K, spec.d, spec.b, spec.Br, spec.Bc, spec.int8)
+            L = vq_synth.make_layer(spec, f.stride, conf["seed"], lid)
+            X = vq_synth.make_x(spec, conf["seed"], batch, lid)
+            self.work.append((f, L, X, spec))
+
+    def run(self, max_weights: float, threads: int):
+        """One bounded pass; returns (seconds, algorithmic bytes covered, description)."""
+        frac = min(1.0, max_weights / self.total_w)
+        t0 = time.perf_counter()
+        nbytes = 0.0
+        for f, L, X, spec in self.work:
+            n_rows = max(1, int(round(spec.N * frac)))
+            rows = None if n_rows >= spec.N else np.arange(n_rows, dtype=np.int32)
+            self.orc.gemm(f, L.idx, L.cb, L.scale, X, rows=rows, threads=threads)
+            nbytes += layer_bytes(spec, f.stride, self.batch) * n_rows / spec.N
+        dt = time.perf_counter() - t0
+        desc = (f"{self.cfg_name} batch {self.batch}: first {frac * 100:.2f}% of the rows of every layer "
+                f"(about {int(self.total_w * frac)} of {self.total_w} weights) per pass, fp64 oracle as it stands")
+        return dt, nbytes, desc
+
+
+ORACLE_WEIGHTS_PER_SEC_PER_THREAD = 15e6  # sizing guess only; the timing itself is measured
+
+
+def run_reference(args):
+    from oracle import vq_oracle as orc
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    orc.build()
+    threads = orc.hardware_threads() or os.cpu_count() or 1
+    # bounded sample per step so that the whole run ends within a few minutes
+    per_step_s = min(3.0, max(0.02, 150.0 / (args.steps + args.warmup)))
+    max_w = per_step_s * ORACLE_WEIGHTS_PER_SEC_PER_THREAD * threads
+    ow = OracleWork(args.config, args.batch)
+    for _ in range(args.warmup):
+        ow.run(max_w, threads)
+    t, nbytes, desc = 0.0, 0.0, ""
+    for _ in range(args.steps):
+        dt, nb, desc = ow.run(max_w, threads)
+        t += dt
+        nbytes += nb
+    val = nbytes / t / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{args.config} batch {args.batch}", "sample_per_step": desc},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def dram_traffic_note(cfg_name: str):
+    """Per-launch DRAM traffic of the dominant kernel from the committed ncu summary, if any."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
+            return json.load(f).get(cfg_name)
+    except Exception:
+        return None
+
+
+def run_ours(args):
+    import torch
+    import paper_2402_15319_b200 as vq
+    vq.load()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU fallback"
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    peak, peak_src = measured_peaks()
+    ds = DeviceSet(args.config, args.batch, dev)
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
+    sampler.start()
+    ms = time_steps(ds, args.steps, args.warmup, barrier)
+    sampler.stop()
+    clock_src = "polled during the timed region"
+    if len(sampler.samples) < 3:  # region shorter than a few polls: repeat the identical loop for the clock record
+        sampler.start()
+        t_end = time.time() + 0.5
+        while time.time() < t_end:
+            time_steps(ds, args.steps, 0)
+        sampler.stop()
+        clock_src = "timed region too short to poll; polled during immediate repeats of the same loop"
+    if dist:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * ds.step_bytes / (ms_per_step * 1e-3) / 1e9
+
+    e2e_steps = max(5, min(args.steps, 200))
+    ms_e2e = time_e2e(ds, e2e_steps, args.warmup)
+    if dist:
+        t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    e2e_val = world * ds.step_bytes / (ms_e2e / e2e_steps * 1e-3) / 1e9
+
+    launches = len(ds.fmts) * args.steps
+    per_launch_gbs = ds.step_bytes / (ms_per_step * 1e-3) / 1e9  # one GPU's kernels
+    traffic = dram_traffic_note(args.config)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {
+            "workload": f"{args.config}: {ds.specs[0].name.split('.')[0]} layer set ({len(ds.specs)} layers, "
+                        f"{ds.n_weights} weights), d={ds.specs[0].d}, {ds.specs[0].b}-bit indices, "
+                        f"{'int8+scale' if ds.specs[0].int8 else 'fp16'} codebook per "
+                        f"{ds.specs[0].Br}x{ds.specs[0].Bc} block, batch {args.batch}",
+            "bytes_per_step": ds.step_bytes, "us_per_layer_set": ms_per_step * 1e3,
+            "cold_cache": f"{ds.copies} distinct device copies of every layer visited round-robin "
+                          f"({ds.copies * ds.step_bytes / 2**20:.0f} MiB > 2 x L2); inputs larger than L2, no flush",
+            "launch": "CUDA graph of one round over all copies, replayed",
+            "pct_of_nominal_8TBps": 100 * per_launch_gbs / NOMINAL_HBM_GBS,
+            "parallelism": "replicas only (one GPU per process, no collective)" if world > 1 else "single GPU",
+        },
+        "clocks": sampler.summary(clock_src),
+        "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": ds.h2d, "d2h_bytes_per_step": ds.d2h,
+                "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps,
+                "what": "vq_gemm_small_batch_host per layer: pinned-host activations copied in, kernel, outputs copied back, stream synchronised every step; compressed weights resident in HBM"},
+        "gpu_launches": launches,
+        "roofline": {
+            "bound": "hbm", "kernel": "vq gemm kernel (one launch per layer)", "achieved": per_launch_gbs, "peak": peak,
+            "unit": "GB/s", "frac": per_launch_gbs / peak, "peak_source": peak_src,
+            "algorithmic_bytes_per_launch": ds.step_bytes / len(ds.fmts),
+            "avg_launch_us": ms_per_step * 1e3 / len(ds.fmts), "traffic": traffic,
+        },
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import vq_oracle as orc
+        orc.build()
+        threads = orc.hardware_threads() or os.cpu_count() or 1
+        dt, nbytes, desc = OracleWork(args.config, args.batch).run(12.0 * ORACLE_WEIGHTS_PER_SEC_PER_THREAD * threads, threads)
+        line["cpu_baseline"] = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": desc, "seconds": dt}
+    if rank == 0 and args.all_configs and world == 1:
+        per = {}
+        del ds
+        torch.cuda.empty_cache()
+        for cfg in vq_synth.CONFIGS:
+            for b in vq_synth.CONFIGS[cfg]["batches"]:
+                d2 = DeviceSet(cfg, b, dev)
+                st = max(d2.copies * 20, 200)
+                m = time_steps(d2, st, d2.copies * 3) / st
+                g = d2.step_bytes / (m * 1e-3) / 1e9
+                per[f"{cfg}.b{b}"] = {"us_per_step": m * 1e3, "GBps": g, "frac_of_measured": g / peak,
+                                      "pct_of_nominal_8TBps": 100 * g / NOMINAL_HBM_GBS, "bytes": d2.step_bytes}
+                del d2
+                torch.cuda.empty_cache()
+        line["per_config"] = per
+    if rank == 0:
+        print(json.dumps(line))
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=4000)
+    ap.add_argument("--warmup", type=int, default=40)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="cfg3", choices=sorted(vq_synth.CONFIGS))
+    ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--all-configs", action="store_true", help="also time every configuration and batch (adds per_config)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
