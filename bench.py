@@ -337,7 +337,7 @@ def run_ours(args):
     value = world * ds.step_bytes / (ms_per_step * 1e-3) / 1e9
 
     e2e_steps = max(5, min(args.steps, 200))
-    ms_e2e = time_e2e(ds, e2e_steps, args.warmup)
+    ms_e2e = time_e2e(ds, e2e_steps, args.warmup) if not args.no_e2e else float("nan")
     if dist:
         t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -414,6 +414,7 @@ def main():
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--all-configs", action="store_true", help="also time every configuration and batch (adds per_config)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end loop (profiling runs)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -37,6 +37,8 @@ vq_status launch_gemm_generic(const Geometry& g, const LayerPtrs& p, const __hal
                               int batch, cudaStream_t s);
 vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y,
                             int batch, float* ws, cudaStream_t s);
+vq_status launch_gemm_blockcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
+                              cudaStream_t s);
 vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s);
 
 inline vq_status check_launch() {
