@@ -27,6 +27,8 @@ struct LayerPtrs {
 
 // Maximum number of K-splits any kernel uses; fixes the workspace size.
 constexpr int kMaxSplits = 8;
+// Devices per process the launchers keep per-device set-up state for.
+constexpr int kMaxDevices = 64;
 
 vq_status make_geometry(const vq_format* fmt, Geometry* g);
 
@@ -39,6 +41,8 @@ vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half*
                             int batch, float* ws, cudaStream_t s);
 vq_status launch_gemm_blockcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
                               cudaStream_t s);
+vq_status launch_gemm_rowcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
+                            cudaStream_t s);
 vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s);
 
 inline vq_status check_launch() {
