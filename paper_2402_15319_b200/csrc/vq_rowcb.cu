@@ -2,26 +2,35 @@
 // are indexed by 4-bit indices: the "mobile LUT" layouts (16-entry int8 codebook + fp16 scale per
 // row segment) and the 16-entry fp16 2-D codebooks.
 //
-// Work decomposition.  A warp owns a tile of 16 rows and walks a range of columns in steps of
-// STEP_COLS columns.  Lane (g = lane/4, t = lane%4) streams, with one 128-bit load per row and
-// step, the 32 indices of rows g and g+8 that cover its quarter of the step, one step ahead of
-// their use.  The indices are expanded to fp16 weights in registers and fed, as the A fragment,
-// to mma.sync m16n8k16; the activations are the B fragment (batch row = g), accumulation is fp32.
+// Work decomposition.  A CTA owns WR tiles of 16 rows and a column range; warp (wr, wk) walks part
+// wk of that range for tile wr in steps of STEP_COLS columns.  Lane (g = lane/4, t = lane%4)
+// streams, with one 128-bit load per row and step, the 32 indices of rows g and g+8 that cover
+// its quarter of the step, a few steps ahead of their use.  The indices are expanded to fp16
+// weights in registers and fed, as the A fragment, to mma.sync m16n8k16; the activations are the
+// B fragment (batch row = g), staged once per CTA in shared memory in the order the lanes
+// consume them and read only by the lanes whose batch row exists; accumulation is fp32.
 // Two ways of expanding an index:
-//   * PrmtI8: the row's 16 int8 entries live in 4 registers per VQ dimension and are looked up
+//   * PrmtI8 (1-D int8 codebooks): the row's 16 entries live in 4 registers and are looked up
 //     with byte permutes - the register-file analogue of the paper's LUT instruction (Sec. 3.2:
 //     index -> 8-bit value).  The bytes become fp16 by the 0x6400 exponent trick, exactly.
-//   * LdsTbl: the rows' entries are expanded once per block into lane-private fp16 tables in
-//     shared memory (bank = lane: conflict-free for any index pattern) and gathered with ld.shared.
-// Which weight column sits in which reduction slot of the mma is free; the activations of the
-// CTA's column range are staged once in shared memory in exactly the order the lanes consume them.
+//   * LdsTbl (2-D codebooks, fp16 or int8): the rows' entries are expanded once per block into
+//     lane-private fp16 tables in shared memory (bank = lane: conflict-free for any index
+//     pattern) and gathered with ld.shared; index bits and the lane's address bits are merged by
+//     one logic operation.
 // int8 codebooks: the block scale multiplies the block's fp32 partial sum (Sec. 3.1 scale factor).
-// The K dimension is split over the warps of a CTA and over the CTAs of a thread block cluster;
-// partial sums meet in the shared memory of cluster rank 0 and are added in a fixed order.
+// Partial sums of the K parts (warps of the CTA, CTAs of a thread block cluster) meet in the
+// shared memory of cluster rank 0 and are added in a fixed order.
 #include <cstdlib>
 
 #include "vq_common.cuh"
 #include "vq_device.cuh"
+
+#ifndef VQ_ROW_MIN_CTAS
+#define VQ_ROW_MIN_CTAS 1   // resident 256-thread CTAs per SM the register budget allows
+#endif
+#ifndef VQ_ROW_PREFETCH
+#define VQ_ROW_PREFETCH 2   // steps of the index stream a lane keeps in flight
+#endif
 
 namespace vq {
 namespace {
@@ -49,6 +58,7 @@ struct RowArgs {
 constexpr uint32_t kMagic = 0x64646464u;      // high byte of fp16 1024.0
 constexpr uint32_t kBias2 = 0x64806480u;      // fp16 pair (1152, 1152) = 1024 + 128
 
+// (1024 + u) - 1152 = u - 128, exact in fp16
 __device__ __forceinline__ uint32_t sub_bias(uint32_t h) {
   uint32_t r;
   asm("sub.f16x2 %0, %1, %2;" : "=r"(r) : "r"(h), "r"(kBias2));
@@ -56,34 +66,23 @@ __device__ __forceinline__ uint32_t sub_bias(uint32_t h) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// PrmtI8<D>: 16 int8 entries of D dims per (row, block); register LUT.
+// PrmtI8: 16 int8 entries of 1 dim per (row, block); register LUT.
 // ---------------------------------------------------------------------------------------------
-template <int D_>
 struct PrmtI8 {
-  static constexpr int D = D_;
-  static constexpr int STEP_COLS = 128 * D;   // 4 lanes x 32 indices x D
-  static constexpr int CHUNKS = 4 * D;        // 8-column activation chunks per lane and step
+  static constexpr int D = 1;
+  static constexpr int STEP_COLS = 128;       // 4 lanes x 32 indices
+  static constexpr int WORD_CHUNKS = 1;       // 8-column activation chunks per index word
   static constexpr bool SCALED = true;
   static constexpr int TABLE_BYTES_PER_WARP = 0;
-  static constexpr int CB_ROW_BYTES = 16 * D;
-
-  // order in which a lane consumes the 8 activations of a chunk
-  static __device__ __forceinline__ uint4 permute_x(uint4 in) {
-    if constexpr (D == 1) {
-      return in;
-    } else {
-      return make_uint4(prmt(in.x, in.z, 0x5410), prmt(in.y, in.w, 0x5410), prmt(in.x, in.z, 0x7632),
-                        prmt(in.y, in.w, 0x7632));
-    }
-  }
+  static constexpr int CB_ROW_BYTES = 16;
 
   struct State {
-    uint32_t T[2][D][4];   // [row g / g+8][plane][entries 4q..4q+3], biased by +128
+    uint32_t T[2][4];   // [row g / g+8][entries 4q..4q+3], biased by +128
     const uint8_t* cb_row[2];
     const __half* sc_row[2];
     float sc[2];
 
-    __device__ __forceinline__ void init(const RowArgs& a, int rl, int rh, int, uint32_t) {
+    __device__ __forceinline__ void init(const RowArgs& a, int, int rl, int rh, int, uint32_t) {
       cb_row[0] = a.cb + static_cast<long long>(rl) * a.blocks_per_row * CB_ROW_BYTES;
       cb_row[1] = a.cb + static_cast<long long>(rh) * a.blocks_per_row * CB_ROW_BYTES;
       sc_row[0] = a.scale + static_cast<long long>(rl) * a.blocks_per_row;
@@ -93,57 +92,29 @@ struct PrmtI8 {
     __device__ __forceinline__ void load_block(int blk) {
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
-        const uint8_t* p = cb_row[h] + static_cast<long long>(blk) * CB_ROW_BYTES;
-        if constexpr (D == 1) {
-          const uint4 v = ldg128_nc(p);
-          T[h][0][0] = v.x ^ 0x80808080u; T[h][0][1] = v.y ^ 0x80808080u;
-          T[h][0][2] = v.z ^ 0x80808080u; T[h][0][3] = v.w ^ 0x80808080u;
-        } else {
-          const uint4 v0 = ldg128_nc(p), v1 = ldg128_nc(p + 16);
-          const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            T[h][0][q] = prmt(w[2 * q], w[2 * q + 1], 0x6420) ^ 0x80808080u;
-            T[h][1][q] = prmt(w[2 * q], w[2 * q + 1], 0x7531) ^ 0x80808080u;
-          }
-        }
+        const uint4 v = ldg128_nc(cb_row[h] + static_cast<long long>(blk) * CB_ROW_BYTES);
+        T[h][0] = v.x ^ 0x80808080u; T[h][1] = v.y ^ 0x80808080u;
+        T[h][2] = v.z ^ 0x80808080u; T[h][3] = v.w ^ 0x80808080u;
         sc[h] = __half2float(__ldg(sc_row[h] + blk));
       }
     }
 
-    // 4 looked-up bytes (indices i0..i0+3 of the word, plane p) of row h
-    __device__ __forceinline__ uint32_t look4(int h, int p, uint32_t sel, uint32_t pick) const {
-      const uint32_t lo = prmt(T[h][p][0], T[h][p][1], sel);
-      const uint32_t hi = prmt(T[h][p][2], T[h][p][3], sel);
-      return prmt(lo, hi, pick);
-    }
-
-    // One index word of each row (8 indices = 8*D columns) -> A fragments of 2*D mma steps.
+    // One index word of each row (8 indices = 8 columns) -> A fragments of 2 mma steps.
     // a[c][q][.]: chunk c of the word, mma q of the chunk, registers a0..a3.
-    __device__ __forceinline__ void decode(uint32_t wl, uint32_t wh, uint32_t (&a)[D][2][4]) const {
+    __device__ __forceinline__ void decode(uint32_t wl, uint32_t wh, uint32_t (&a)[1][2][4]) const {
       const uint32_t w[2] = {wl, wh};
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
+        // byte permute: selector nibble = entry mod 8 (bit 3 would mean "replicate sign"), looked
+        // up in entries 0..7 and 8..15; a second permute picks per index by the index's bit 3
         const uint32_t sel = w[h] & 0x77777777u;
         const uint32_t pick = ((w[h] >> 1) & 0x44444444u) | 0x32103210u;
-        const uint32_t selH = sel >> 16, pickH = pick >> 16;
-        if constexpr (D == 1) {
-          const uint32_t rL = look4(h, 0, sel, pick), rH = look4(h, 0, selH, pickH);
-          a[0][0][h] = sub_bias(prmt(rL, kMagic, 0x4140));
-          a[0][0][h + 2] = sub_bias(prmt(rL, kMagic, 0x4342));
-          a[0][1][h] = sub_bias(prmt(rH, kMagic, 0x4140));
-          a[0][1][h + 2] = sub_bias(prmt(rH, kMagic, 0x4342));
-        } else {
-#pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            const uint32_t r0 = look4(h, 0, c ? selH : sel, c ? pickH : pick);
-            const uint32_t r1 = look4(h, 1, c ? selH : sel, c ? pickH : pick);
-            a[c][0][h] = sub_bias((r0 & 0x00FF00FFu) | 0x64006400u);   // columns 0,4 of the chunk
-            a[c][0][h + 2] = sub_bias(prmt(r0, kMagic, 0x4341));         // columns 2,6
-            a[c][1][h] = sub_bias((r1 & 0x00FF00FFu) | 0x64006400u);   // columns 1,5
-            a[c][1][h + 2] = sub_bias(prmt(r1, kMagic, 0x4341));         // columns 3,7
-          }
-        }
+        const uint32_t rL = prmt(prmt(T[h][0], T[h][1], sel), prmt(T[h][2], T[h][3], sel), pick);
+        const uint32_t rH = prmt(prmt(T[h][0], T[h][1], sel >> 16), prmt(T[h][2], T[h][3], sel >> 16), pick >> 16);
+        a[0][0][h] = sub_bias(prmt(rL, kMagic, 0x4140));       // columns 0,1
+        a[0][0][h + 2] = sub_bias(prmt(rL, kMagic, 0x4342));   // columns 2,3
+        a[0][1][h] = sub_bias(prmt(rH, kMagic, 0x4140));       // columns 4,5
+        a[0][1][h + 2] = sub_bias(prmt(rH, kMagic, 0x4342));   // columns 6,7
       }
     }
   };
@@ -151,18 +122,17 @@ struct PrmtI8 {
 
 // ---------------------------------------------------------------------------------------------
 // LdsTbl<INT8>: 16 entries of 2 dims per (row, block), fp16 or int8; lane-private fp16 tables in
-// shared memory: word (half, entry, lane) at half*2048 + entry*128 + lane*4.
+// shared memory, 4096-byte aligned per warp: word (half, entry, lane) at half*2048 + entry*128 +
+// lane*4, so the entry index occupies address bits 7..10 and never carries.
 // ---------------------------------------------------------------------------------------------
 template <bool INT8>
 struct LdsTbl {
   static constexpr int D = 2;
   static constexpr int STEP_COLS = 256;
-  static constexpr int CHUNKS = 8;
+  static constexpr int WORD_CHUNKS = 2;
   static constexpr bool SCALED = INT8;
   static constexpr int TABLE_BYTES_PER_WARP = 4096;
   static constexpr int CB_ROW_BYTES = INT8 ? 32 : 64;
-
-  static __device__ __forceinline__ uint4 permute_x(uint4 in) { return in; }
 
   struct State {
     const uint8_t* cb_row[2];
@@ -171,84 +141,80 @@ struct LdsTbl {
     uint32_t tbl;   // shared address of this lane's column of the table
     uint32_t fill;  // shared address this lane writes when building the table
 
-    __device__ __forceinline__ void init(const RowArgs& a, int rl, int rh, int lane, uint32_t warp_tbl) {
-      const int t = lane & 3, g = lane >> 2;
-      cb_row[0] = a.cb + static_cast<long long>(rl) * a.blocks_per_row * CB_ROW_BYTES + t * (CB_ROW_BYTES / 4);
-      cb_row[1] = a.cb + static_cast<long long>(rh) * a.blocks_per_row * CB_ROW_BYTES + t * (CB_ROW_BYTES / 4);
+    // The table is BUILT with a different lane mapping than it is read with: lane l fetches
+    // entries 4*(l/8)..+3 of rows l%8 and l%8+8, so that the 8 lanes of a quarter warp write 8
+    // different 16-byte bank groups (conflict-free 128-bit stores).
+    __device__ __forceinline__ void init(const RowArgs& a, int row0, int rl, int rh, int lane, uint32_t warp_tbl) {
+      const int gb = lane & 7, tb = lane >> 3;
+      const int b_lo = min(row0 + gb, a.N - 1), b_hi = min(row0 + gb + 8, a.N - 1);
+      cb_row[0] = a.cb + static_cast<long long>(b_lo) * a.blocks_per_row * CB_ROW_BYTES + tb * (CB_ROW_BYTES / 4);
+      cb_row[1] = a.cb + static_cast<long long>(b_hi) * a.blocks_per_row * CB_ROW_BYTES + tb * (CB_ROW_BYTES / 4);
       if constexpr (INT8) {
         sc_row[0] = a.scale + static_cast<long long>(rl) * a.blocks_per_row;
         sc_row[1] = a.scale + static_cast<long long>(rh) * a.blocks_per_row;
       }
       tbl = warp_tbl + lane * 4;
-      fill = warp_tbl + (4 * t) * 128 + g * 16;   // entries 4t..4t+3, the 4 copies of row g
+      fill = warp_tbl + (4 * tb) * 128 + gb * 16;   // entries 4tb..4tb+3, the 4 copies of row gb
     }
 
-    // Lane (g, t) fetches entries 4t..4t+3 of rows g and g+8 and writes each 4 times (one copy
-    // per lane of the row's quad).
+    // Each fetched entry is written 4 times (one copy per lane of the row's quad).
     __device__ __forceinline__ void load_block(int blk) {
-      __syncwarp();   // every lane is done with the previous block's table
+      uint32_t e[2][4];
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         const uint8_t* p = cb_row[h] + static_cast<long long>(blk) * CB_ROW_BYTES;
-        uint32_t e[4];
         if constexpr (INT8) {
           const uint2 v = ldg64_nc(p);   // 4 entries x (c0, c1)
-          e[0] = sub_bias(prmt(v.x ^ 0x80808080u, kMagic, 0x4140));
-          e[1] = sub_bias(prmt(v.x ^ 0x80808080u, kMagic, 0x4342));
-          e[2] = sub_bias(prmt(v.y ^ 0x80808080u, kMagic, 0x4140));
-          e[3] = sub_bias(prmt(v.y ^ 0x80808080u, kMagic, 0x4342));
+          e[h][0] = sub_bias(prmt(v.x ^ 0x80808080u, kMagic, 0x4140));
+          e[h][1] = sub_bias(prmt(v.x ^ 0x80808080u, kMagic, 0x4342));
+          e[h][2] = sub_bias(prmt(v.y ^ 0x80808080u, kMagic, 0x4140));
+          e[h][3] = sub_bias(prmt(v.y ^ 0x80808080u, kMagic, 0x4342));
           sc[h] = __half2float(__ldg(sc_row[h] + blk));
         } else {
           const uint4 v = ldg128_nc(p);
-          e[0] = v.x; e[1] = v.y; e[2] = v.z; e[3] = v.w;
+          e[h][0] = v.x; e[h][1] = v.y; e[h][2] = v.z; e[h][3] = v.w;
         }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) sts128(fill + h * 2048 + i * 128, make_uint4(e[i], e[i], e[i], e[i]));
       }
+      __syncwarp();   // every lane is done with the previous block's table
+#pragma unroll
+      for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) sts128(fill + h * 2048 + i * 128, make_uint4(e[h][i], e[h][i], e[h][i], e[h][i]));
       __syncwarp();
+      fence_value(tbl);   // gathers of the new block stay behind the rewrite
     }
 
-    // shared address of entry (index I of word w) in this lane's column: the 4 index bits are
-    // moved to bits 7..10 and merged with the lane's constant address bits by one logic op
-    template <int I>
-    __device__ __forceinline__ uint32_t entry_addr(uint32_t w, uint32_t base) const {
+    template <int I, int HALF>
+    __device__ __forceinline__ uint32_t gather(uint32_t w) const {
       constexpr int p = 4 * I;
-      uint32_t x;
-      if constexpr (p < 7) {
-        x = w << (7 - p);
-      } else {
-#ifdef VQ_SHIFT_VIA_MULHI
-        asm("mul.hi.u32 %0, %1, %2;" : "=r"(x) : "r"(w), "n"(1u << (32 - (p - 7))));
-#else
-        x = w >> (p - 7);
-#endif
-      }
-      return (x & 0x780u) | base;
+      const uint32_t x = p < 7 ? w << (7 - p) : w >> (p - 7);
+      return lds32_off<HALF * 2048>((x & 0x780u) | tbl);
     }
 
     __device__ __forceinline__ void decode(uint32_t wl, uint32_t wh, uint32_t (&a)[2][2][4]) const {
       // chunk c = indices 4c..4c+3; mma q of the chunk = indices 4c+2q, 4c+2q+1
-      const uint32_t lo = tbl, hi = tbl + 2048;
-      a[0][0][0] = lds32(entry_addr<0>(wl, lo));        a[0][0][1] = lds32(entry_addr<0>(wh, hi));
-      a[0][0][2] = lds32(entry_addr<1>(wl, lo));        a[0][0][3] = lds32(entry_addr<1>(wh, hi));
-      a[0][1][0] = lds32(entry_addr<2>(wl, lo));        a[0][1][1] = lds32(entry_addr<2>(wh, hi));
-      a[0][1][2] = lds32(entry_addr<3>(wl, lo));        a[0][1][3] = lds32(entry_addr<3>(wh, hi));
-      a[1][0][0] = lds32(entry_addr<4>(wl, lo));        a[1][0][1] = lds32(entry_addr<4>(wh, hi));
-      a[1][0][2] = lds32(entry_addr<5>(wl, lo));        a[1][0][3] = lds32(entry_addr<5>(wh, hi));
-      a[1][1][0] = lds32(entry_addr<6>(wl, lo));        a[1][1][1] = lds32(entry_addr<6>(wh, hi));
-      a[1][1][2] = lds32(entry_addr<7>(wl, lo));        a[1][1][3] = lds32(entry_addr<7>(wh, hi));
+      a[0][0][0] = gather<0, 0>(wl); a[0][0][1] = gather<0, 1>(wh); a[0][0][2] = gather<1, 0>(wl); a[0][0][3] = gather<1, 1>(wh);
+      a[0][1][0] = gather<2, 0>(wl); a[0][1][1] = gather<2, 1>(wh); a[0][1][2] = gather<3, 0>(wl); a[0][1][3] = gather<3, 1>(wh);
+      a[1][0][0] = gather<4, 0>(wl); a[1][0][1] = gather<4, 1>(wh); a[1][0][2] = gather<5, 0>(wl); a[1][0][3] = gather<5, 1>(wh);
+      a[1][1][0] = gather<6, 0>(wl); a[1][1][1] = gather<6, 1>(wh); a[1][1][2] = gather<7, 0>(wl); a[1][1][3] = gather<7, 1>(wh);
     }
   };
 };
 
 // ---------------------------------------------------------------------------------------------
 // The kernel.  Grid (S, ceil(N / (16*WR))), cluster (S, 1, 1); CTA = WR*WK warps.
+// Activations in shared memory: 16-byte chunk (step, chunk c of the lane's columns, batch row m,
+// lane quarter t) at index ((step*CHUNKS + c)*batch + m)*4 + t, so that the lanes of a warp that
+// read (those with g < batch) touch consecutive chunks.
 // ---------------------------------------------------------------------------------------------
 template <class P, int NB>
-__global__ void __launch_bounds__(256) rowcb_kernel(const RowArgs a) {
-  constexpr int D = P::D;
+__global__ void __launch_bounds__(256, VQ_ROW_MIN_CTAS) rowcb_kernel(const RowArgs a) {
+  constexpr int PF = VQ_ROW_PREFETCH;
+  constexpr int WC = P::WORD_CHUNKS;
+  constexpr int CHUNKS = 4 * WC;                 // chunks of a lane per step
+  constexpr int LANE_COLS = P::STEP_COLS / 4;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  // the tables' address bits 7..11 must be free for the index and the row half
+  // the tables' address bits 7..11 must be free for the entry index and the row half
   const uint32_t smem_base = (smem_u32(smem_raw) + 4095u) & ~4095u;
   unsigned char* smem = smem_raw + (smem_base - smem_u32(smem_raw));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -264,28 +230,30 @@ __global__ void __launch_bounds__(256) rowcb_kernel(const RowArgs a) {
   const int cta_s1 = a.n_steps * ((rank + 1) * a.WK) / T;
   const int s0 = a.n_steps * part / T, s1 = a.n_steps * (part + 1) / T;
 
-  const int tile = blockIdx.y * a.WR + wr;
-  const int r_lo = tile * 16 + g, r_hi = r_lo + 8;
+  const int row0 = (blockIdx.y * a.WR + wr) * 16;
+  const int r_lo = row0 + g, r_hi = r_lo + 8;
   const int rl = min(r_lo, a.N - 1), rh = min(r_hi, a.N - 1);   // tail rows load a valid row, store nothing
-  const uint8_t* pl = a.idx + rl * a.stride + t * 16;
-  const uint8_t* ph = a.idx + rh * a.stride + t * 16;
+  const uint8_t* pl = a.idx + rl * a.stride + t * 16 + static_cast<long long>(s0) * 64;
+  const uint8_t* ph = a.idx + rh * a.stride + t * 16 + static_cast<long long>(s0) * 64;
 
   typename P::State st;
-  st.init(a, rl, rh, lane, smem_base + warp * P::TABLE_BYTES_PER_WARP);
+  st.init(a, row0, rl, rh, lane, smem_base + warp * P::TABLE_BYTES_PER_WARP);
 
-  // indices of the first step and the first block's tables: weights do not depend on the
-  // previous kernel, so they are requested before the dependency wait
-  uint4 nl = make_uint4(0, 0, 0, 0), nh = nl;
-  pl += static_cast<long long>(s0) * 64;
-  ph += static_cast<long long>(s0) * 64;
-  if (s0 < s1) {
-    nl = ldg128_stream(pl);
-    nh = ldg128_stream(ph);
-    st.load_block(s0 / a.steps_per_block);
+  // Indices of the first PF steps and the first block's tables: weights do not depend on the
+  // previous kernel of the stream, so they are requested before the dependency wait.
+  uint4 ql[PF], qh[PF];
+#pragma unroll
+  for (int u = 0; u < PF; ++u) {
+    ql[u] = qh[u] = make_uint4(0, 0, 0, 0);
+    if (s0 + u < s1) {
+      ql[u] = ldg128_stream(pl + u * 64);
+      qh[u] = ldg128_stream(ph + u * 64);
+    }
   }
+  if (s0 < s1) st.load_block(s0 / a.steps_per_block);
 
-  // ---- activations of the CTA's column range, in consumption order ----
-  pdl_wait();
+  // ---- activations of the CTA's column range ----
+  pdl_wait();   // the activations (and Y) belong to the previous kernel until here
   {
     const int col0 = cta_s0 * P::STEP_COLS;
     const int n8 = (cta_s1 - cta_s0) * (P::STEP_COLS / 8);
@@ -295,8 +263,8 @@ __global__ void __launch_bounds__(256) rowcb_kernel(const RowArgs a) {
       for (int c8 = tid; c8 < n8; c8 += blockDim.x) {
         const int col = c8 * 8;
         const int step = col / P::STEP_COLS, within = col % P::STEP_COLS;
-        const int tt = within / (P::STEP_COLS / 4), chunk = (within % (P::STEP_COLS / 4)) / 8;
-        xs[((step * P::CHUNKS + chunk) * a.batch + m) * 4 + tt] = P::permute_x(__ldg(src + c8));
+        const int tt = within / LANE_COLS, chunk = (within % LANE_COLS) / 8;
+        xs[((step * CHUNKS + chunk) * a.batch + m) * 4 + tt] = __ldg(src + c8);
       }
     }
   }
@@ -308,58 +276,70 @@ __global__ void __launch_bounds__(256) rowcb_kernel(const RowArgs a) {
 #pragma unroll
     for (int e = 0; e < 4; ++e) acc[nb][e] = total[nb][e] = 0.f;
 
+  // B fragments: two register sets used alternately; lanes without a batch row keep zeros
   bool on[NB];
   uint32_t xaddr[NB];
+  uint4 xb[2][NB][WC];
 #pragma unroll
   for (int nb = 0; nb < NB; ++nb) {
     on[nb] = nb * 8 + g < a.batch;
-    xaddr[nb] = smem_base + a.x_offset + (((s0 - cta_s0) * P::CHUNKS * a.batch + nb * 8 + g) * 4 + t) * 16;
+    xaddr[nb] = smem_base + a.x_offset + (((s0 - cta_s0) * CHUNKS * a.batch + nb * 8 + g) * 4 + t) * 16;
+#pragma unroll
+    for (int c = 0; c < WC; ++c) xb[0][nb][c] = xb[1][nb][c] = make_uint4(0, 0, 0, 0);
   }
   const uint32_t xstride = a.batch * 64;   // bytes between consecutive chunks
 
   int in_blk = s0 % a.steps_per_block, blk = s0 / a.steps_per_block;
-  for (int s = s0; s < s1; ++s) {
-    const uint4 cl = nl, ch = nh;
-    pl += 64;
-    ph += 64;
-    if (s + 1 < s1) {
-      nl = ldg128_stream(pl);
-      nh = ldg128_stream(ph);
-    }
-    const uint32_t wl[4] = {cl.x, cl.y, cl.z, cl.w}, wh[4] = {ch.x, ch.y, ch.z, ch.w};
+  for (int sb = s0; sb < s1; sb += PF) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      uint32_t af[D][2][4];
-      st.decode(wl[j], wh[j], af);
+    for (int u = 0; u < PF; ++u) {
+      const int s = sb + u;
+      if (s >= s1) break;
+      const uint4 cl = ql[u], ch = qh[u];
+      if (s + PF < s1) {
+        ql[u] = ldg128_stream(pl + PF * 64);
+        qh[u] = ldg128_stream(ph + PF * 64);
+      }
+      pl += 64;
+      ph += 64;
+      const uint32_t wl[4] = {cl.x, cl.y, cl.z, cl.w}, wh[4] = {ch.x, ch.y, ch.z, ch.w};
 #pragma unroll
-      for (int c = 0; c < D; ++c) {
+      for (int j = 0; j < 4; ++j) {
 #pragma unroll
-        for (int nb = 0; nb < NB; ++nb) {
-          uint4 xb = make_uint4(0, 0, 0, 0);
-          if (on[nb]) xb = lds128(xaddr[nb] + (j * D + c) * xstride);
-          mma16816(acc[nb], af[c][0][0], af[c][0][1], af[c][0][2], af[c][0][3], xb.x, xb.y);
-          mma16816(acc[nb], af[c][1][0], af[c][1][1], af[c][1][2], af[c][1][3], xb.z, xb.w);
+        for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+          for (int c = 0; c < WC; ++c) lds128_if(xb[j & 1][nb][c], xaddr[nb] + (j * WC + c) * xstride, on[nb]);
+        uint32_t af[WC][2][4];
+        st.decode(wl[j], wh[j], af);
+#pragma unroll
+        for (int c = 0; c < WC; ++c) {
+#pragma unroll
+          for (int nb = 0; nb < NB; ++nb) {
+            const uint4 b = xb[j & 1][nb][c];
+            mma16816(acc[nb], af[c][0][0], af[c][0][1], af[c][0][2], af[c][0][3], b.x, b.y);
+            mma16816(acc[nb], af[c][1][0], af[c][1][1], af[c][1][2], af[c][1][3], b.z, b.w);
+          }
         }
       }
-    }
 #pragma unroll
-    for (int nb = 0; nb < NB; ++nb) xaddr[nb] += P::CHUNKS * xstride;
-    if (++in_blk == a.steps_per_block || s + 1 == s1) {
-      // end of a codebook block: apply its scale to the block's partial sums
-#pragma unroll
-      for (int nb = 0; nb < NB; ++nb) {
+      for (int nb = 0; nb < NB; ++nb) xaddr[nb] += CHUNKS * xstride;
+      if (++in_blk == a.steps_per_block || s + 1 == s1) {
+        // end of a codebook block: apply its scale to the block's partial sums
         if constexpr (P::SCALED) {
-          total[nb][0] = fmaf(st.sc[0], acc[nb][0], total[nb][0]);
-          total[nb][1] = fmaf(st.sc[0], acc[nb][1], total[nb][1]);
-          total[nb][2] = fmaf(st.sc[1], acc[nb][2], total[nb][2]);
-          total[nb][3] = fmaf(st.sc[1], acc[nb][3], total[nb][3]);
 #pragma unroll
-          for (int e = 0; e < 4; ++e) acc[nb][e] = 0.f;
+          for (int nb = 0; nb < NB; ++nb) {
+            total[nb][0] = fmaf(st.sc[0], acc[nb][0], total[nb][0]);
+            total[nb][1] = fmaf(st.sc[0], acc[nb][1], total[nb][1]);
+            total[nb][2] = fmaf(st.sc[1], acc[nb][2], total[nb][2]);
+            total[nb][3] = fmaf(st.sc[1], acc[nb][3], total[nb][3]);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[nb][e] = 0.f;
+          }
         }
+        in_blk = 0;
+        ++blk;
+        if (s + 1 < s1) st.load_block(blk);
       }
-      in_blk = 0;
-      ++blk;
-      if (s + 1 < s1) st.load_block(blk);
     }
   }
   if constexpr (!P::SCALED) {
@@ -381,24 +361,24 @@ __global__ void __launch_bounds__(256) rowcb_kernel(const RowArgs a) {
       }
     return;
   }
-  // red[part][wr][row 0..15][n 0..8*NB-1] in the shared memory of cluster rank 0
+  // red[K part][tile wr][row 0..15][batch row 0..8*NB-1] in the shared memory of cluster rank 0
+  constexpr int NBT = 8 * NB;
   const uint32_t red_local = smem_base + a.red_offset;
-  const uint32_t mine = red_local + (((part * a.WR + wr) * 16 + g) * (8 * NB) + 2 * t) * 4;
+  const uint32_t mine = red_local + (((part * a.WR + wr) * 16 + g) * NBT + 2 * t) * 4;
   if (S > 1) {
     cluster_wait_acquire();   // every CTA of the cluster has started: rank 0's shared memory exists
     const uint32_t dst = map_to_rank(mine, 0);
 #pragma unroll
     for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-      for (int e = 0; e < 4; ++e)
-        st_cluster_f32(dst + (((e >> 1) * 8 * (8 * NB)) + nb * 8 + (e & 1)) * 4, total[nb][e]);
+      for (int e = 0; e < 4; ++e) st_cluster_f32(dst + ((e >> 1) * 8 * NBT + nb * 8 + (e & 1)) * 4, total[nb][e]);
     cluster_arrive_release();
     cluster_wait_acquire();
   } else {
 #pragma unroll
     for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) sts32f(mine + (((e >> 1) * 8 * (8 * NB)) + nb * 8 + (e & 1)) * 4, total[nb][e]);
+      for (int e = 0; e < 4; ++e) sts32f(mine + ((e >> 1) * 8 * NBT + nb * 8 + (e & 1)) * 4, total[nb][e]);
     __syncthreads();
   }
   if (rank != 0) return;
@@ -410,7 +390,7 @@ __global__ void __launch_bounds__(256) rowcb_kernel(const RowArgs a) {
     const int r = row_base + rr;
     if (r >= a.N) continue;
     float sum = 0.f;
-    for (int p = 0; p < T; ++p) sum += red[((p * a.WR) * 16 + rr) * (8 * NB) + n];
+    for (int p = 0; p < T; ++p) sum += red[(p * cta_rows + rr) * NBT + n];
     a.Y[static_cast<long long>(n) * a.N + r] = __float2half_rn(sum);
   }
 }
@@ -431,29 +411,40 @@ int env_int(const char* name, int dflt) {
   return dflt;
 }
 
-// Choose the CTA shape and the K split.  Targets: about 16 resident warps per SM, at least two
-// steps per warp, many more CTAs than SMs for large layers (the hardware balances them).
-Plan make_plan(int N, int n_steps, int sms) {
+// Choose the CTA shape (WR row tiles x WK column parts, at most 8 warps) and the cluster size S.
+// Model: an SM works through ceil(CTAs / SMs) CTAs; a warp costs its steps plus a fixed overhead
+// (prologue, table set-up, reduction; more with a cluster) plus its share of staging the CTA's
+// activations; the SM runs at full rate from about 24 resident warps on.  x_budget: bytes of
+// shared memory the activations of one CTA may take.
+Plan make_plan(int N, int n_steps, int step_cols, int batch, int sms, size_t x_budget) {
   const int row_tiles = (N + 15) / 16;
-  const long long want_warps = static_cast<long long>(sms) * 16;
-  int T = static_cast<int>((want_warps + row_tiles - 1) / row_tiles);
-  int max_T = n_steps / 2;
-  if (max_T < 1) max_T = 1;
-  if (T > max_T) T = max_T;
-  if (T > 64) T = 64;
-  // round down to a power of two
-  int p = 1;
-  while (2 * p <= T) p *= 2;
-  T = p;
-  Plan pl;
-  pl.WK = T < 8 ? T : 8;
-  pl.S = T / pl.WK;
-  pl.WR = 8 / pl.WK;
-  if (T == 1) pl.WR = 4;   // large layers: 64-row CTAs
-  pl.WK = env_int("VQ_WK", pl.WK);
-  pl.WR = env_int("VQ_WR", pl.WR);
-  pl.S = env_int("VQ_S", pl.S);
-  return pl;
+  Plan best = {0, 0, 0};
+  double best_cost = -1.0;
+  for (int S = 1; S <= 8; S *= 2)
+    for (int WK = 1; WK <= 8; WK *= 2)
+      for (int WR = 1; WR * WK <= 8; WR *= 2) {
+        const int T = S * WK;
+        if (T > n_steps || (T > 1 && 2 * T > n_steps)) continue;   // at least two steps per warp
+        const double cta_steps = static_cast<double>(n_steps) / S;
+        if ((cta_steps + 1.0) * step_cols * 2.0 * batch > static_cast<double>(x_budget)) continue;
+        const long long ctas = static_cast<long long>((row_tiles + WR - 1) / WR) * S;
+        const double per_sm = static_cast<double>((ctas + sms - 1) / sms);
+        const int W = WR * WK;
+        const double steps = static_cast<double>(n_steps) / T;
+        const double ovh = (S > 1 ? 4.0 : (WK > 1 ? 2.5 : 2.0)) + 0.25 * cta_steps * batch / W;
+        double resident = per_sm * W;
+        if (resident > 32.0) resident = 32.0;
+        const double rate = resident >= 24.0 ? 1.0 : resident / 24.0;
+        const double cost = per_sm * W * (steps + ovh) / rate;
+        if (best_cost < 0.0 || cost < best_cost) {
+          best_cost = cost;
+          best = {WR, WK, S};
+        }
+      }
+  best.WR = env_int("VQ_WR", best.WR);
+  best.WK = env_int("VQ_WK", best.WK);
+  best.S = env_int("VQ_S", best.S);
+  return best;
 }
 
 template <class P, int NB>
@@ -467,10 +458,9 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
   if (sms_of[dev] == 0) {
     int n = 0;
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return VQ_ERR_CUDA;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) return VQ_ERR_CUDA;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024) != cudaSuccess) return VQ_ERR_CUDA;
     sms_of[dev] = n;
   }
-  const int sms = sms_of[dev];
   RowArgs a;
   a.idx = p.idx;
   a.cb = static_cast<const uint8_t*>(p.cb);
@@ -484,32 +474,27 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
   a.n_steps = g.K / P::STEP_COLS;
   a.steps_per_block = g.Bc / P::STEP_COLS;
   a.blocks_per_row = g.blocks_per_row;
-  Plan pl = make_plan(g.N, a.n_steps, sms);
-  // activations of a CTA's column range must fit in shared memory: split K further if not
-  size_t x_bytes, red_bytes, tbl_bytes;
-  for (;;) {
-    const int T = pl.S * pl.WK;
-    int cta_steps = 0;
-    for (int r = 0; r < pl.S; ++r) {
-      const int c = a.n_steps * ((r + 1) * pl.WK) / T - a.n_steps * (r * pl.WK) / T;
-      if (c > cta_steps) cta_steps = c;
-    }
-    x_bytes = static_cast<size_t>(cta_steps) * P::STEP_COLS * 2 * batch;
-    red_bytes = T > 1 ? static_cast<size_t>(T) * pl.WR * 16 * 8 * NB * sizeof(float) : 0;
-    tbl_bytes = static_cast<size_t>(P::TABLE_BYTES_PER_WARP) * pl.WR * pl.WK;
-    if (x_bytes + red_bytes + tbl_bytes <= 160 * 1024) break;
-    if (pl.S >= 8 || pl.S * 2 * pl.WK > a.n_steps) return VQ_ERR_UNSUPPORTED;
-    pl.S *= 2;
-  }
-  if (pl.S * pl.WK > a.n_steps) return VQ_ERR_UNSUPPORTED;
+  constexpr size_t kXBudget = 128 * 1024;
+  const Plan pl = make_plan(g.N, a.n_steps, P::STEP_COLS, batch, sms_of[dev], kXBudget);
+  const int T = pl.S * pl.WK;
+  if (pl.WR < 1 || pl.WK < 1 || pl.WR * pl.WK > 8 || pl.S < 1 || pl.S > 8 || T > a.n_steps) return VQ_ERR_UNSUPPORTED;
   a.WR = pl.WR;
   a.WK = pl.WK;
+  int cta_steps = 0;   // longest column range of a CTA of the cluster
+  for (int r = 0; r < pl.S; ++r) {
+    const int c = a.n_steps * ((r + 1) * pl.WK) / T - a.n_steps * (r * pl.WK) / T;
+    if (c > cta_steps) cta_steps = c;
+  }
+  const size_t tbl_bytes = static_cast<size_t>(P::TABLE_BYTES_PER_WARP) * pl.WR * pl.WK;
+  const size_t x_bytes = static_cast<size_t>(cta_steps) * P::STEP_COLS * 2 * batch;
+  const size_t red_bytes = T > 1 ? static_cast<size_t>(T) * pl.WR * 16 * 8 * NB * sizeof(float) : 0;
+  if (x_bytes > kXBudget + 4096) return VQ_ERR_UNSUPPORTED;
   a.x_offset = static_cast<int>(tbl_bytes);
   a.red_offset = static_cast<int>(tbl_bytes + (x_bytes + 15) / 16 * 16);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(pl.S, (g.N + 16 * pl.WR - 1) / (16 * pl.WR), 1);
   cfg.blockDim = dim3(32 * pl.WR * pl.WK, 1, 1);
-  cfg.dynamicSmemBytes = a.red_offset + red_bytes + 4096;
+  cfg.dynamicSmemBytes = a.red_offset + red_bytes + 4096;   // + room to align the tables
   cfg.stream = s;
   cudaLaunchAttribute attr[2];
   int na = 0;
@@ -538,16 +523,11 @@ vq_status launch_gemm_rowcb(const Geometry& g, const LayerPtrs& p, const __half*
                             cudaStream_t s) {
   if (g.Br != 1 || g.b != 4) return VQ_ERR_UNSUPPORTED;
   const bool nb1 = batch <= 8;
-  if (g.cb_int8) {
-    const int use_lds = env_int("VQ_I8_LDS", 0);
-    if (g.d == 1) return nb1 ? launch<PrmtI8<1>, 1>(g, p, X, Y, batch, s) : launch<PrmtI8<1>, 2>(g, p, X, Y, batch, s);
-    if (g.d == 2) {
-      if (use_lds) return nb1 ? launch<LdsTbl<true>, 1>(g, p, X, Y, batch, s) : launch<LdsTbl<true>, 2>(g, p, X, Y, batch, s);
-      return nb1 ? launch<PrmtI8<2>, 1>(g, p, X, Y, batch, s) : launch<PrmtI8<2>, 2>(g, p, X, Y, batch, s);
-    }
-    return VQ_ERR_UNSUPPORTED;
-  }
-  if (g.d == 2) return nb1 ? launch<LdsTbl<false>, 1>(g, p, X, Y, batch, s) : launch<LdsTbl<false>, 2>(g, p, X, Y, batch, s);
+  if (g.cb_int8 && g.d == 1) return nb1 ? launch<PrmtI8, 1>(g, p, X, Y, batch, s) : launch<PrmtI8, 2>(g, p, X, Y, batch, s);
+  if (g.cb_int8 && g.d == 2)
+    return nb1 ? launch<LdsTbl<true>, 1>(g, p, X, Y, batch, s) : launch<LdsTbl<true>, 2>(g, p, X, Y, batch, s);
+  if (!g.cb_int8 && g.d == 2)
+    return nb1 ? launch<LdsTbl<false>, 1>(g, p, X, Y, batch, s) : launch<LdsTbl<false>, 2>(g, p, X, Y, batch, s);
   return VQ_ERR_UNSUPPORTED;
 }
 
