@@ -20,6 +20,7 @@
 // int8 codebooks: the block scale multiplies the block's fp32 partial sum (Sec. 3.1 scale factor).
 // Partial sums of the K parts (warps of the CTA, CTAs of a thread block cluster) meet in the
 // shared memory of cluster rank 0 and are added in a fixed order.
+#include <cstdio>
 #include <cstdlib>
 
 #include "vq_common.cuh"
@@ -414,9 +415,10 @@ int env_int(const char* name, int dflt) {
 // Choose the CTA shape (WR row tiles x WK column parts, at most 8 warps) and the cluster size S.
 // Model: an SM works through ceil(CTAs / SMs) CTAs; a warp costs its steps plus a fixed overhead
 // (prologue, table set-up, reduction; more with a cluster) plus its share of staging the CTA's
-// activations; the SM runs at full rate from about 24 resident warps on.  x_budget: bytes of
-// shared memory the activations of one CTA may take.
-Plan make_plan(int N, int n_steps, int step_cols, int batch, int sms, size_t x_budget) {
+// activations; the SM runs at full rate from about 24 resident warps on.  Shapes whose tables,
+// activations and reduction buffer exceed smem_budget bytes of shared memory are left out;
+// {0,0,0} if none fits.
+Plan make_plan(int N, int n_steps, int step_cols, int batch, int sms, int tbl_per_warp, int nb, size_t smem_budget) {
   const int row_tiles = (N + 15) / 16;
   Plan best = {0, 0, 0};
   double best_cost = -1.0;
@@ -426,10 +428,12 @@ Plan make_plan(int N, int n_steps, int step_cols, int batch, int sms, size_t x_b
         const int T = S * WK;
         if (T > n_steps || (T > 1 && 2 * T > n_steps)) continue;   // at least two steps per warp
         const double cta_steps = static_cast<double>(n_steps) / S;
-        if ((cta_steps + 1.0) * step_cols * 2.0 * batch > static_cast<double>(x_budget)) continue;
+        const int W = WR * WK;
+        const double smem_need = (cta_steps + 1.0) * step_cols * 2.0 * batch + static_cast<double>(tbl_per_warp) * W +
+                                 (T > 1 ? T * WR * 16.0 * 8.0 * nb * 4.0 : 0.0) + 4096.0 + 16.0;
+        if (smem_need > static_cast<double>(smem_budget)) continue;
         const long long ctas = static_cast<long long>((row_tiles + WR - 1) / WR) * S;
         const double per_sm = static_cast<double>((ctas + sms - 1) / sms);
-        const int W = WR * WK;
         const double steps = static_cast<double>(n_steps) / T;
         const double ovh = (S > 1 ? 4.0 : (WK > 1 ? 2.5 : 2.0)) + 0.25 * cta_steps * batch / W;
         double resident = per_sm * W;
@@ -474,8 +478,8 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
   a.n_steps = g.K / P::STEP_COLS;
   a.steps_per_block = g.Bc / P::STEP_COLS;
   a.blocks_per_row = g.blocks_per_row;
-  constexpr size_t kXBudget = 128 * 1024;
-  const Plan pl = make_plan(g.N, a.n_steps, P::STEP_COLS, batch, sms_of[dev], kXBudget);
+  constexpr size_t kSmemBudget = 200 * 1024;
+  const Plan pl = make_plan(g.N, a.n_steps, P::STEP_COLS, batch, sms_of[dev], P::TABLE_BYTES_PER_WARP, NB, kSmemBudget);
   const int T = pl.S * pl.WK;
   if (pl.WR < 1 || pl.WK < 1 || pl.WR * pl.WK > 8 || pl.S < 1 || pl.S > 8 || T > a.n_steps) return VQ_ERR_UNSUPPORTED;
   a.WR = pl.WR;
@@ -488,7 +492,7 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
   const size_t tbl_bytes = static_cast<size_t>(P::TABLE_BYTES_PER_WARP) * pl.WR * pl.WK;
   const size_t x_bytes = static_cast<size_t>(cta_steps) * P::STEP_COLS * 2 * batch;
   const size_t red_bytes = T > 1 ? static_cast<size_t>(T) * pl.WR * 16 * 8 * NB * sizeof(float) : 0;
-  if (x_bytes > kXBudget + 4096) return VQ_ERR_UNSUPPORTED;
+  if (tbl_bytes + x_bytes + 16 + red_bytes + 4096 > 208 * 1024) return VQ_ERR_UNSUPPORTED;
   a.x_offset = static_cast<int>(tbl_bytes);
   a.red_offset = static_cast<int>(tbl_bytes + (x_bytes + 15) / 16 * 16);
   cudaLaunchConfig_t cfg = {};
@@ -512,6 +516,17 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
   }
   cfg.attrs = attr;
   cfg.numAttrs = na;
+#ifdef VQ_TUNING
+  {
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, a);
+    if (e != cudaSuccess) {
+      fprintf(stderr, "rowcb launch failed: %s (grid %d,%d block %d smem %zu S %d WR %d WK %d)\n", cudaGetErrorString(e),
+              cfg.gridDim.x, cfg.gridDim.y, cfg.blockDim.x, cfg.dynamicSmemBytes, pl.S, pl.WR, pl.WK);
+      return VQ_ERR_CUDA;
+    }
+    return check_launch();
+  }
+#endif
   if (cudaLaunchKernelEx(&cfg, kern, a) != cudaSuccess) return VQ_ERR_CUDA;
   return check_launch();
 }
