@@ -147,6 +147,32 @@ vq_status vq_gemm_small_batch_host(const vq_format* fmt, const void* d_idx, cons
                                    void* d_ws, size_t ws_bytes, void* stream);
 size_t vq_workspace_bytes_host(const vq_format* fmt, int batch);
 
+/* The same computation as vq_gemm_small_batch_host for callers that cannot allocate device memory
+ * at all: code that runs where cudaMalloc is forbidden or unavailable - inside a region whose
+ * memory is owned and budgeted by another allocator (an inference server's arena, a real-time
+ * loop that may not block on the driver's allocator), or a plug-in that is handed device
+ * pointers to the weights but no allocator.  (The paper has no counterpart: this is a packaging
+ * variant of the entry point above, not a step of the method.)
+ * Instead of a caller-provided workspace, the device copies of X and Y live in a fixed array of
+ * vq_static_scratch_bytes() = 2 MiB that is part of the library image; every GPU that loads the
+ * library holds it until the process exits.  The call performs no cudaMalloc / cudaFree and calls
+ * no allocating routine.
+ *   Limit: round256(2*batch*K) + round256(2*batch*N) must not exceed vq_static_scratch_bytes();
+ *   larger problems return VQ_ERR_WORKSPACE and launch nothing.
+ *   The first call on each device looks the array's device address up (cudaGetSymbolAddress, with
+ *   that device current); make that first call outside any stream capture.
+ *   All calls on a device share the one array, which keeps the previous call's contents; nothing
+ *   in it has to be cleared between calls (X is overwritten by the copy in, Y by the kernel).
+ *   Two calls that may overlap on the GPU (different streams, no ordering between them) race on
+ *   it: order them on one stream or with events.
+ *   As with vq_gemm_small_batch_host the three steps are enqueued on `stream` and the call
+ *   returns without synchronising; synchronise before reading h_Y.
+ * Errors: NULL, FORMAT, SHAPE, ALIGN, BATCH, WORKSPACE (problem larger than the scratch), CUDA. */
+vq_status vq_gemm_small_batch_host_static(const vq_format* fmt, const void* d_idx, const void* d_cb,
+                                          const void* d_scale, const void* h_X, void* h_Y, int batch,
+                                          void* stream);
+size_t vq_static_scratch_bytes(void);
+
 /* Uniform INT4 group-128 reference GEMV used as the bandwidth yard-stick beside the VQ
  * kernels (paper Sec. 2.1 symmetric uniform quantiser x ~ s*x_int; Sec. 5 "INT4 g128", 4.125 bpv).
  *   d_q     : device, N rows of K/2 bytes; column k of row n is nibble (k mod 2) of byte k/2

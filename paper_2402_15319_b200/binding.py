@@ -75,6 +75,8 @@ _SIGNATURES = {
     "vq_gemm_small_batch": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
     "vq_gemm_small_batch_impl": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_int]),
     "vq_gemm_small_batch_host": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
+    "vq_gemm_small_batch_host_static": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p]),
+    "vq_static_scratch_bytes": (ctypes.c_size_t, []),
     "vq_int4g128_gemm_small_batch": (ctypes.c_int, [ctypes.c_int32, ctypes.c_int32] + [ctypes.c_void_p] * 4 + [ctypes.c_int, ctypes.c_void_p]),
     "vq_status_string": (ctypes.c_char_p, [ctypes.c_int]),
 }
@@ -173,6 +175,21 @@ def vq_gemm_small_batch_host(fmt: VQFormat, d_idx, d_cb, d_scale, h_X, h_Y, batc
                                            _ptr(h_Y), int(batch), _ptr(d_ws),
                                            d_ws.numel() * d_ws.element_size(), _stream(stream)),
            "vq_gemm_small_batch_host")
+
+
+def vq_gemm_small_batch_host_static(fmt: VQFormat, d_idx, d_cb, d_scale, h_X, h_Y, batch: int, stream=None) -> None:
+    """Host-buffer skinny GEMM that allocates nothing: the device copies of X and Y live in a
+    fixed 2 MiB array inside the library (vq_static_scratch_bytes()).  For callers that may not
+    call cudaMalloc.  Calls on one device share that array: keep them ordered on the GPU.
+    Synchronise before reading h_Y."""
+    c = fmt.c()
+    _check(load().vq_gemm_small_batch_host_static(ctypes.byref(c), _ptr(d_idx), _ptr(d_cb), _ptr(d_scale),
+                                                  _ptr(h_X), _ptr(h_Y), int(batch), _stream(stream)),
+           "vq_gemm_small_batch_host_static")
+
+
+def vq_static_scratch_bytes() -> int:
+    return load().vq_static_scratch_bytes()
 
 
 def vq_int4g128_gemm_small_batch(n_rows: int, k_cols: int, d_q, d_scale, d_X, d_Y, batch: int, stream=None) -> None:
