@@ -184,6 +184,13 @@ vq_status vq_int4g128_gemm_small_batch(int32_t n_rows, int32_t k_cols, const voi
                                        const void* d_scale, const void* d_X, void* d_Y,
                                        int batch, void* stream);
 
+/* Diagnostics.  The tuned kernels wait for their asynchronous copies (Sec. 3.2 index stream) with a
+ * bounded number of polls; a wait that runs out increments a per-device counter and the kernel
+ * carries on (its output is then wrong, but the device stays usable).  This call copies the
+ * counter of the current device to *h_count; it synchronises the device.  0 in a healthy run.
+ * Errors: NULL, CUDA. */
+vq_status vq_device_wait_failures(int* h_count);
+
 /* Human-readable name of a status code; never NULL. */
 const char* vq_status_string(vq_status s);
 

@@ -78,6 +78,7 @@ _SIGNATURES = {
     "vq_gemm_small_batch_host_static": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p]),
     "vq_static_scratch_bytes": (ctypes.c_size_t, []),
     "vq_int4g128_gemm_small_batch": (ctypes.c_int, [ctypes.c_int32, ctypes.c_int32] + [ctypes.c_void_p] * 4 + [ctypes.c_int, ctypes.c_void_p]),
+    "vq_device_wait_failures": (ctypes.c_int, [ctypes.c_void_p]),
     "vq_status_string": (ctypes.c_char_p, [ctypes.c_int]),
 }
 
@@ -190,6 +191,13 @@ def vq_gemm_small_batch_host_static(fmt: VQFormat, d_idx, d_cb, d_scale, h_X, h_
 
 def vq_static_scratch_bytes() -> int:
     return load().vq_static_scratch_bytes()
+
+
+def vq_device_wait_failures() -> int:
+    """Bounded in-kernel waits that ran out on the current device (0 in a healthy run); synchronises."""
+    out = ctypes.c_int(-1)
+    _check(load().vq_device_wait_failures(ctypes.byref(out)), "vq_device_wait_failures")
+    return out.value
 
 
 def vq_int4g128_gemm_small_batch(n_rows: int, k_cols: int, d_q, d_scale, d_X, d_Y, batch: int, stream=None) -> None:

@@ -1,106 +1,69 @@
 // Tuned skinny-GEMM kernels for formats whose codebook is shared by a tall block of rows
 // (block_rows a multiple of the CTA's rows): the 2-D 6-bit and 4-D 8-bit fp16-codebook families.
 //
-// Per CTA: a tile of CTA_ROWS x CTA_COLS weights.  Each warp owns 32 rows x 256 columns:
-// lane (g = lane/4, t = lane%4) streams its own 64 columns of rows g, g+8, g+16, g+24 straight
-// from the packed index stream into registers, looks every index up in a lane-private copy of
-// its block's codebook in shared memory (bank = lane, so the gather is conflict-free for any
-// index pattern) and feeds the fp16 pairs, untouched, into mma.sync m16n8k16 as the A fragment.
-// The activations of the lane's 64 columns sit in registers as the B fragment (batch row = g),
-// accumulation is fp32 in the tensor core.  The K dimension is split over the CTAs of a thread
-// block cluster; their partial sums are combined in a fixed order through distributed shared
-// memory, rounded once to fp16 and stored.  Paper: Sec. 3.2 (packed indices -> LUT -> mat-vec),
-// App. A (Q is a look-up of C); the tiling, the replication and the reduction are this library's.
-#include <cooperative_groups.h>
+// A CTA owns one block-row slab (128 or 256 rows: every warp 32 of them) and a range of 256-column
+// chunks; a thread block cluster of S CTAs splits K.  Per chunk and warp the packed indices of 32
+// rows arrive as ONE tiled TMA box (32 rows x 96 or 64 bytes) in a warp-private ring of shared
+// memory, a few chunks ahead, completion counted on an mbarrier; lane (g = lane/4, t = lane%4)
+// reads its own 64 columns of rows g, g+8, g+16, g+24 from the box (conflict-free), looks every
+// index up in a lane-private copy of the chunk's codebook ([entry][lane] words: bank = lane, so
+// the gather is conflict-free for any index pattern; index bits and lane bits of the address are
+// merged by one logic operation) and feeds the fp16 pairs, untouched, into mma.sync m16n8k16 as
+// the A fragment.  The activations of the CTA's column range are staged once in shared memory in
+// the order the lanes consume them (B fragment, batch row = g); accumulation is fp32.  Codebook
+// tables are double buffered: the next one is replicated while the current chunk is computed, its
+// entries fetched from global memory two tables ahead.  Partial sums of the K parts travel through
+// distributed shared memory to the cluster rank that owns the rows, are added in rank order,
+// rounded once to fp16 and stored.
+// Paper: Sec. 3.2 (packed indices -> LUT -> mat-vec), App. A (Q is a look-up of C); the tiling,
+// the replication and the reduction are this library's.
+#include <cuda.h>
 
+#include <cstdio>
 #include <cstdlib>
-#include <type_traits>
 #include <utility>
 
 #include "vq_common.cuh"
-
-namespace cg = cooperative_groups;
-
-#ifdef VQ_TUNING
-__device__ unsigned long long* g_vq_trace = nullptr;
-extern "C" void vq_debug_set_trace(unsigned long long* p) { cudaMemcpyToSymbol(g_vq_trace, &p, sizeof(p)); }
-#define VQ_TRACE(slot)                                                                            \
-  do {                                                                                            \
-    if (g_vq_trace && threadIdx.x == 0) {                                                         \
-      unsigned long long t_;                                                                      \
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                      \
-      g_vq_trace[(static_cast<size_t>(blockIdx.y) * gridDim.x + blockIdx.x) * 8 + (slot)] = t_;   \
-    }                                                                                             \
-  } while (0)
-#else
-#define VQ_TRACE(slot) do {} while (0)
-#endif
+#include "vq_device.cuh"
 
 namespace vq {
 namespace {
 
-__device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                         uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
+using namespace dev;
 
-__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
-  uint32_t v;
-  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr));
-  return v;
-}
+#ifndef VQ_BLOCK_STAGES
+#define VQ_BLOCK_STAGES 3   // chunks of the index stream a warp keeps in flight
+#endif
+constexpr int kStages = VQ_BLOCK_STAGES;
+constexpr int kWaitTries = 1 << 18;   // mbarrier polls before a warp gives up and flags an error
 
-__device__ __forceinline__ uint2 lds64(uint32_t addr) {
-  uint2 v;
-  asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
-  return v;
-}
-
-// 24-byte pieces: the three 8-byte loads of a lane share sectors, so let L1 keep the line.
-__device__ __forceinline__ uint2 ldg64_stream(const void* p) {
-  uint2 v;
-  asm volatile("ld.global.nc.v2.b32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
-  return v;
-}
-
-// Cluster barrier split into arrive / wait so that independent work overlaps the wait.
-__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
-__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
-__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
-
-// fp32 store into the shared memory of CTA `rank` of this cluster (same offset as `local_addr`).
-__device__ __forceinline__ void st_cluster_f32(uint32_t local_addr, int rank, float v) {
-  uint32_t remote;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
-}
-
-__device__ __forceinline__ uint4 ldg128_stream(const void* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.b32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
-}
+struct BlockArgs {
+  const void* cb;
+  const __half* X;
+  __half* Y;
+  int* error_flag;       // device counter of waits that ran out
+  int N, K, batch;
+  int n_chunks;          // K / 256
+  int blocks_per_row;    // K / block_cols
+  int Br, Bc;
+  // byte offsets from the aligned start of dynamic shared memory
+  int compact_off, ring_off, bar_off, x_off, recv_off;
+};
 
 // ---- format policies -----------------------------------------------------------------------
-// LANE_WORDS : 32-bit words of index stream a lane owns per row (64 columns)
-// ENTRY_BYTES: bytes of one codebook entry; TABLE_BYTES: one lane-private table set
 template <int D, int B>
 struct Policy;
 
-// 2-D, 6-bit indices: 64 columns = 32 indices = 24 bytes per lane and row
+// 2-D, 6-bit indices: 256 columns = 128 indices = 96 bytes per row; a lane owns 24 of them
 template <>
 struct Policy<2, 6> {
-  static constexpr int LANE_WORDS = 6, ENTRY_BYTES = 4, ENTRIES = 64;
-  static constexpr int WARPS = 4, TASKS = 1, SLICES = 1;     // CTA = 128 rows x 256 cols
+  static constexpr int LANE_WORDS = 6, ENTRIES = 64, SEG = 96;
+  static constexpr int WARPS = 4;                           // CTA = 128 rows
   static constexpr int TABLE_BYTES = ENTRIES * 128;          // [entry][lane] words
-  static constexpr uint32_t MASK = 0x1F80u;                  // 6 index bits at byte offset * 128
+  static constexpr int COMPACT_BYTES = ENTRIES * 8;          // [entry][half] words
+  static constexpr uint32_t MASK = 0x1F80u;                  // 6 index bits at address bits 7..12
 
-  // byte offset (entry * 128) of index I (0..31) of a lane's 6 words
-  template <int I>
+  template <int I>   // (index I of the lane's 32) * 128
   static __device__ __forceinline__ uint32_t entry_off(const uint32_t (&w)[LANE_WORDS]) {
     constexpr int p = 6 * I;
     if constexpr (p < 7) {
@@ -114,12 +77,13 @@ struct Policy<2, 6> {
   }
 };
 
-// 4-D, 8-bit indices: 64 columns = 16 indices = 16 bytes per lane and row
+// 4-D, 8-bit indices: 256 columns = 64 indices = 64 bytes per row; a lane owns 16 of them
 template <>
 struct Policy<4, 8> {
-  static constexpr int LANE_WORDS = 4, ENTRY_BYTES = 8, ENTRIES = 256;
-  static constexpr int WARPS = 8, TASKS = 2, SLICES = 2;     // CTA = 256 rows x 512 cols
+  static constexpr int LANE_WORDS = 4, ENTRIES = 256, SEG = 64;
+  static constexpr int WARPS = 8;                           // CTA = 256 rows
   static constexpr int TABLE_BYTES = ENTRIES * 128;          // [entry][lane%16] 8-byte entries
+  static constexpr int COMPACT_BYTES = ENTRIES * 8;
   static constexpr uint32_t MASK = 0x7F80u;
 
   template <int I>
@@ -130,50 +94,54 @@ struct Policy<4, 8> {
   }
 };
 
-// bytes of the compact codebook staging area behind the replicated tables
-template <int D, int B>
-constexpr int kCompactBytes = Policy<D, B>::ENTRIES * 8;
-
 template <int D, int B>
 struct Tile {
   using P = Policy<D, B>;
-  static constexpr int ROWS_PER_TASK = 32;
-  static constexpr int CTA_ROWS = ROWS_PER_TASK * P::WARPS * P::TASKS / P::SLICES;
-  static constexpr int CTA_COLS = 256 * P::SLICES;
+  static constexpr int CTA_ROWS = 32 * P::WARPS;
   static constexpr int THREADS = 32 * P::WARPS;
-  // resident CTAs per SM the register budget is tuned for (NB = 1 / NB = 2)
-  static constexpr int min_ctas(int nb) { return D == 2 ? (nb == 1 ? 6 : 4) : (nb == 1 ? 2 : 1); }
+  static constexpr int STAGE_BYTES = 32 * P::SEG;            // one TMA box
 };
 
-// Gather the A fragments of NSTEPS mma steps (each step = 4 columns per lane) of one 16-row tile:
-// wa / wb are the lane's index words of rows g and g+8.
+__device__ __forceinline__ void tma_box_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ uint2 lds64_ordered(uint32_t addr) {   // ring reads: stay behind the barrier wait
+  uint2 v;
+  asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr) : "memory");
+  return v;
+}
+
+// A fragments of NSTEPS mma steps (each step = 4 columns per lane) of one 16-row tile; wa / wb are
+// the lane's index words of rows g and g+8 of the tile, tbl the lane's table address.
 template <int D, int B, int STEP0, int NSTEPS>
 __device__ __forceinline__ void gather_steps(uint32_t (&a)[NSTEPS][4], const uint32_t (&wa)[Policy<D, B>::LANE_WORDS],
                                              const uint32_t (&wb)[Policy<D, B>::LANE_WORDS], uint32_t tbl) {
   using P = Policy<D, B>;
   if constexpr (D == 2) {
     [&]<int... S>(std::integer_sequence<int, S...>) {
-      ((a[S][0] = lds32(tbl + P::template entry_off<2 * (STEP0 + S)>(wa)),
-        a[S][1] = lds32(tbl + P::template entry_off<2 * (STEP0 + S)>(wb)),
-        a[S][2] = lds32(tbl + P::template entry_off<2 * (STEP0 + S) + 1>(wa)),
-        a[S][3] = lds32(tbl + P::template entry_off<2 * (STEP0 + S) + 1>(wb))), ...);
+      ((a[S][0] = lds32(P::template entry_off<2 * (STEP0 + S)>(wa) | tbl),
+        a[S][1] = lds32(P::template entry_off<2 * (STEP0 + S)>(wb) | tbl),
+        a[S][2] = lds32(P::template entry_off<2 * (STEP0 + S) + 1>(wa) | tbl),
+        a[S][3] = lds32(P::template entry_off<2 * (STEP0 + S) + 1>(wb) | tbl)), ...);
     }(std::make_integer_sequence<int, NSTEPS>{});
   } else {
     [&]<int... S>(std::integer_sequence<int, S...>) {
       (([&] {
-         const uint2 u = lds64(tbl + P::template entry_off<STEP0 + S>(wa));
-         const uint2 v = lds64(tbl + P::template entry_off<STEP0 + S>(wb));
+         const uint2 u = lds64(P::template entry_off<STEP0 + S>(wa) | tbl);
+         const uint2 v = lds64(P::template entry_off<STEP0 + S>(wb) | tbl);
          a[S][0] = u.x; a[S][2] = u.y; a[S][1] = v.x; a[S][3] = v.y;
        }()), ...);
     }(std::make_integer_sequence<int, NSTEPS>{});
   }
 }
 
-// One task = two 16-row tiles x 64 columns per lane.  The tiles' accumulator chains are
-// independent, so their look-ups are issued together and their mmas alternate.
+// Both 16-row tiles of a warp for NSTEPS steps: their accumulator chains are independent, so the
+// look-ups are issued together and the mmas alternate.
 template <int D, int B, int NB, int STEP0, int NSTEPS>
-__device__ __forceinline__ void task_steps(float (&acc)[2][NB][4], const uint32_t (&w)[4][Policy<D, B>::LANE_WORDS],
-                                           const uint32_t (&xr)[NB][32], uint32_t tbl) {
+__device__ __forceinline__ void chunk_steps(float (&acc)[2][NB][4], const uint32_t (&w)[4][Policy<D, B>::LANE_WORDS],
+                                            const uint32_t (&xr)[NB][32], uint32_t tbl) {
   uint32_t a0[NSTEPS][4], a1[NSTEPS][4];
   gather_steps<D, B, STEP0, NSTEPS>(a0, w[0], w[1], tbl);
   gather_steps<D, B, STEP0, NSTEPS>(a1, w[2], w[3], tbl);
@@ -186,286 +154,387 @@ __device__ __forceinline__ void task_steps(float (&acc)[2][NB][4], const uint32_
     }
 }
 
-template <int D, int B, int NB>
-__device__ __forceinline__ void task_all(float (&acc)[2][NB][4], const uint32_t (&w)[4][Policy<D, B>::LANE_WORDS],
-                                         const uint32_t (&xr)[NB][32], uint32_t tbl) {
-  task_steps<D, B, NB, 0, 4>(acc, w, xr, tbl);
-  task_steps<D, B, NB, 4, 4>(acc, w, xr, tbl);
-  task_steps<D, B, NB, 8, 4>(acc, w, xr, tbl);
-  task_steps<D, B, NB, 12, 4>(acc, w, xr, tbl);
+// Fetch this thread's share of the codebook entries of table k (global memory -> register).
+// 2-D: thread (e = tid%64, h = tid/64) takes entry e of the block under columns h*128.. of the
+// chunk; 4-D: thread tid takes entry tid of the block the table's chunks lie in.
+template <int D, int B>
+__device__ __forceinline__ uint2 fetch_entry(const BlockArgs& a, long long blk_row, int chunk, int tid) {
+  using P = Policy<D, B>;
+  uint2 v = make_uint2(0u, 0u);
+  if constexpr (D == 2) {
+    const int e = tid & 63, h = tid >> 6;
+    const int col = chunk * 256 + h * 128;
+    v.x = __ldg(static_cast<const uint32_t*>(a.cb) + (blk_row + col / a.Bc) * P::ENTRIES + e);
+  } else {
+    v = __ldg(static_cast<const uint2*>(a.cb) + (blk_row + (chunk * 256) / a.Bc) * P::ENTRIES + tid);
+  }
+  return v;
 }
 
+template <int D, int B>
+__device__ __forceinline__ void store_compact(unsigned char* compact, uint2 v, int tid) {
+  if constexpr (D == 2) reinterpret_cast<uint32_t*>(compact)[2 * (tid & 63) + (tid >> 6)] = v.x;   // [entry][half]
+  else reinterpret_cast<uint2*>(compact)[tid] = v;
+}
+
+// Replicate a compact codebook into the lane-private layout with 128-bit stores (the 8 lanes of a
+// quarter warp write 8 different 16-byte bank groups).
+template <int D, int B>
+__device__ __forceinline__ void replicate(uint32_t table, const unsigned char* compact, int tid) {
+  using P = Policy<D, B>;
+  constexpr int THREADS = Tile<D, B>::THREADS;
+#pragma unroll
+  for (int j = 0; j < P::ENTRIES * 8 / THREADS; ++j) {
+    const int item = tid + j * THREADS;   // (entry, 16-byte group)
+    const int e = item >> 3, u = item & 7;
+    const uint2 c = reinterpret_cast<const uint2*>(compact)[e];
+    // 2-D: lanes 4u..4u+3 = columns 0-127 (two lanes, half 0) and 128-255 (half 1) of the chunk
+    const uint4 v = D == 2 ? make_uint4(c.x, c.x, c.y, c.y) : make_uint4(c.x, c.y, c.x, c.y);
+    sts128(table + e * 128 + u * 16, v);
+  }
+}
+
+// Grid (S, N / CTA_ROWS), cluster (S, 1, 1).  Dynamic shared memory from its first TABLE_BYTES
+// boundary: two tables, two compact codebooks, the warps' index rings, their barriers, the
+// activations, the receive buffer of the reduction.
 template <int D, int B, int NB>
-__global__ void __launch_bounds__(Tile<D, B>::THREADS, Tile<D, B>::min_ctas(NB))
-blockcb_kernel(Geometry g, LayerPtrs p, const __half* __restrict__ X, __half* __restrict__ Y, int batch, int n_chunks) {
+__global__ void __launch_bounds__(Tile<D, B>::THREADS)
+blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
   using P = Policy<D, B>;
   using T = Tile<D, B>;
   constexpr int LW = P::LANE_WORDS;
   constexpr int NBT = 8 * NB;
-  extern __shared__ __align__(16) unsigned char smem[];
-  // smem: [0, TABLE_BYTES) lane-private tables; afterwards reused for the partial sums
-  const uint32_t smem_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
-
-  cg::cluster_group cluster = cg::this_cluster();
-  const int n_split = static_cast<int>(cluster.num_blocks());
-  const int rank = static_cast<int>(cluster.block_rank());
-  cluster_arrive_relaxed();  // waited on just before the first remote store
-  // Programmatic dependent launch: the next kernel in the stream may start its own weight
-  // streaming now; this kernel waits for its predecessor only where it first touches X.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  bool dep_waited = false;
-  VQ_TRACE(0);
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const uint32_t raw_u32 = smem_u32(smem_raw);
+  const uint32_t base = (raw_u32 + P::TABLE_BYTES - 1) & ~static_cast<uint32_t>(P::TABLE_BYTES - 1);
+  unsigned char* smem = smem_raw + (base - raw_u32);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int gq = lane >> 2, t = lane & 3;
+  const int g = lane >> 2, t = lane & 3;
+  const int S = gridDim.x, rank = blockIdx.x;
+  if (S > 1) cluster_arrive_relaxed();   // matched by the wait in front of the first remote store
+  pdl_launch_dependents();
+
+  const int c0 = a.n_chunks * rank / S, c1 = a.n_chunks * (rank + 1) / S, n = c1 - c0;
   const int row0 = blockIdx.y * T::CTA_ROWS;
-  const int slice = warp % P::SLICES;
-  const int rgroup0 = warp / P::SLICES;                          // first row group of this warp
-  constexpr int RGROUP_STEP = P::WARPS / P::SLICES;             // next task's row group
-  const long long blk_row = static_cast<long long>(row0 / g.Br) * g.blocks_per_row;
+  const long long blk_row = static_cast<long long>(row0 / a.Br) * a.blocks_per_row;
+  const int cpt = D == 2 ? 1 : a.Bc / 256;   // chunks that share one table
+  const int t0 = c0 / cpt, nt = n > 0 ? (c1 - 1) / cpt - t0 + 1 : 0;
 
-  const uint32_t tbl = smem_u32 + (D == 2 ? lane * 4 : (lane & 15) * 8);
+  // ---- index ring: warp-private stages, one TMA box each ----
+  const uint32_t bars = base + a.bar_off + warp * kStages * 8;
+  const uint32_t ring = base + a.ring_off + warp * kStages * T::STAGE_BYTES;
+  if (lane == 0) {
+    for (int s = 0; s < kStages; ++s) mbar_init(bars + 8 * s, 1);
+    mbar_init_fence();
+  }
+  __syncwarp();
+  auto issue = [&](int i) {   // lane 0 only
+    const int st = i % kStages;
+    mbar_arrive_expect_tx(bars + 8 * st, T::STAGE_BYTES);
+    tma_box_2d(ring + st * T::STAGE_BYTES, &tm, (c0 + i) * P::SEG, row0 + 32 * warp, bars + 8 * st);
+  };
+  if (lane == 0)
+    for (int i = 0; i < kStages && i < n; ++i) issue(i);
 
-  float acc[P::TASKS][2][NB][4];
-#pragma unroll
-  for (int a = 0; a < P::TASKS; ++a)
-#pragma unroll
-    for (int b = 0; b < 2; ++b)
-#pragma unroll
-      for (int c = 0; c < NB; ++c)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) acc[a][b][c][e] = 0.f;
+  // ---- first two codebook tables ----
+  unsigned char* compact = smem + a.compact_off;
+  if (nt > 0) store_compact<D, B>(compact, fetch_entry<D, B>(a, blk_row, t0 * cpt, tid), tid);
+  if (nt > 1) store_compact<D, B>(compact + P::COMPACT_BYTES, fetch_entry<D, B>(a, blk_row, (t0 + 1) * cpt, tid), tid);
 
-  for (int chunk = rank; chunk < n_chunks; chunk += n_split) {
-    const int col_cta = chunk * T::CTA_COLS;
-    const int col_lane = col_cta + slice * 256 + t * 64;
-    const bool lane_on = col_lane < g.K;
-
-    // ---- 0. this thread's share of the chunk's codebooks (the whole CTA waits on these) ----
-    typename std::conditional<D == 2, uint32_t, uint2>::type cbv;
-    if constexpr (D == 2) {
-      const int e = tid & 63, h = tid >> 6;
-      const int col = col_cta + h * 128;
-      cbv = 0u;
-      if (col < g.K) cbv = __ldg(static_cast<const uint32_t*>(p.cb) + (blk_row + col / g.Bc) * P::ENTRIES + e);
-    } else {
-      cbv = __ldg(static_cast<const uint2*>(p.cb) + (blk_row + col_cta / g.Bc) * P::ENTRIES + tid);
-    }
-
-    // ---- 1. index stream -> registers (everything this warp will need for the chunk) ----
-    uint32_t w[P::TASKS][4][LW];
-#pragma unroll
-    for (int task = 0; task < P::TASKS; ++task) {
-      const int r = row0 + (rgroup0 + task * RGROUP_STEP) * 32 + gq;
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const uint8_t* src = p.idx + static_cast<long long>(r + 8 * q) * g.stride + (static_cast<long long>(col_lane) / D) * B / 8;
-        if (lane_on) {
-          if constexpr (LW == 6) {
-#pragma unroll
-            for (int i = 0; i < 3; ++i) {
-              const uint2 v = ldg64_stream(src + 8 * i);
-              w[task][q][2 * i] = v.x;
-              w[task][q][2 * i + 1] = v.y;
-            }
-          } else {
-            const uint4 v = ldg128_stream(src);
-            w[task][q][0] = v.x; w[task][q][1] = v.y; w[task][q][2] = v.z; w[task][q][3] = v.w;
-          }
-        } else {
-#pragma unroll
-          for (int i = 0; i < LW; ++i) w[task][q][i] = 0u;
-        }
+  // ---- activations of the CTA's column range: chunk i, 16-byte piece j of a lane's 64 columns,
+  // batch row m, lane quarter tt at ((i*8 + j)*batch + m)*4 + tt ----
+  pdl_wait();   // the activations (and Y) belong to the previous kernel until here
+  {
+    uint4* xs = reinterpret_cast<uint4*>(smem + a.x_off);
+    const int n16 = n * 32;   // 16-byte pieces per batch row
+    for (int m = 0; m < a.batch; ++m) {
+      const uint4* src = reinterpret_cast<const uint4*>(a.X + static_cast<long long>(m) * a.K + c0 * 256);
+      for (int q = tid; q < n16; q += T::THREADS) {
+        const int i = q >> 5, tt = (q >> 3) & 3, j = q & 7;
+        xs[((i * 8 + j) * a.batch + m) * 4 + tt] = __ldg(src + q);
       }
     }
+  }
+  __syncthreads();
+  if (nt > 0) replicate<D, B>(base, compact, tid);
+  __syncthreads();
 
-    // ---- 2. activations of the lane's 64 columns -> B fragments ----
-    if (!dep_waited) {
-      asm volatile("griddepcontrol.wait;" ::: "memory");  // X (and Y) belong to the predecessor until here
-      dep_waited = true;
-    }
-    uint32_t xr[NB][32];
+  float acc[2][NB][4];
 #pragma unroll
-    for (int nb = 0; nb < NB; ++nb) {
-      const int n = nb * 8 + gq;
-      if (lane_on && n < batch) {
-        const uint4* xs = reinterpret_cast<const uint4*>(X + static_cast<long long>(n) * g.K + col_lane);
+  for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const uint4 v = __ldg(xs + i);
-          xr[nb][4 * i] = v.x; xr[nb][4 * i + 1] = v.y; xr[nb][4 * i + 2] = v.z; xr[nb][4 * i + 3] = v.w;
+    for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[mt][nb][e] = 0.f;
+  uint32_t xr[NB][32];
+  bool on[NB];
+  uint32_t xaddr[NB];
+#pragma unroll
+  for (int nb = 0; nb < NB; ++nb) {
+    on[nb] = nb * 8 + g < a.batch;
+    xaddr[nb] = base + a.x_off + ((nb * 8 + g) * 4 + t) * 16;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) xr[nb][i] = 0u;
+  }
+  const uint32_t xstride = a.batch * 64;
+  const uint32_t lane_off = D == 2 ? lane * 4 : (lane & 15) * 8;
+  const uint32_t row_off = (D == 2 ? t * 24 : t * 16) + g * P::SEG;
+
+  for (int i = 0; i < n; ++i) {
+    const int c = c0 + i;
+    const int k = c / cpt - t0;
+    const bool first_of_table = i == 0 || (c - 1) / cpt - t0 != k;
+    const bool last_of_table = i == n - 1 || (c + 1) / cpt - t0 != k;
+    // codebook two tables ahead: request now, park in shared memory after the chunk's math
+    const bool fetch2 = first_of_table && k + 2 < nt;
+    uint2 vnext = make_uint2(0u, 0u);
+    if (fetch2) vnext = fetch_entry<D, B>(a, blk_row, (t0 + k + 2) * cpt, tid);
+    if (first_of_table && k + 1 < nt)
+      replicate<D, B>(base + ((k + 1) & 1) * P::TABLE_BYTES, compact + ((k + 1) & 1) * P::COMPACT_BYTES, tid);
+
+    // ---- this warp's indices of the chunk ----
+    const int st = i % kStages;
+    if (!mbar_wait(bars + 8 * st, (i / kStages) & 1, kWaitTries) && lane == 0) atomicAdd(a.error_flag, 1);
+    uint32_t w[4][LW];
+    const uint32_t src = ring + st * T::STAGE_BYTES + row_off;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if constexpr (LW == 6) {
+#pragma unroll
+        for (int h = 0; h < 3; ++h) {
+          const uint2 v = lds64_ordered(src + q * 8 * P::SEG + 8 * h);
+          w[q][2 * h] = v.x;
+          w[q][2 * h + 1] = v.y;
         }
       } else {
-#pragma unroll
-        for (int i = 0; i < 32; ++i) xr[nb][i] = 0u;
+        const uint4 v = lds128(src + q * 8 * P::SEG);
+        w[q][0] = v.x; w[q][1] = v.y; w[q][2] = v.z; w[q][3] = v.w;
       }
+    }
+    __syncwarp();   // every lane has read the stage: refill it
+    if (lane == 0 && i + kStages < n) {
+      fence_proxy_async();
+      issue(i + kStages);
     }
 
-    // ---- 3. stage the lane-private codebook copies ----
-    // One global load per thread fetches the chunk's codebooks into a compact staging area; after
-    // a barrier every thread replicates them into the [entry][lane] layout with 128-bit stores.
-    if constexpr (D == 2) {
-      // compact[e][h] = entry e of the chunk's block h (two 128-column blocks when Bc = 128)
-      uint32_t* compact = reinterpret_cast<uint32_t*>(smem + P::TABLE_BYTES);
-      {
-        const int e = tid & 63, h = tid >> 6;             // 128 threads = 64 entries x 2 halves
-        const int col = col_cta + h * 128;
-        uint32_t v = 0u;
-        if (col < g.K) v = cbv;
-        compact[2 * e + h] = v;
-      }
-      VQ_TRACE(1);
-      __syncthreads();
-      // lanes 4u..4u+3 of entry e own columns 0-63, 64-127 (half 0) and 128-191, 192-255 (half 1)
+    // ---- activations of the lane's 64 columns -> B fragments ----
 #pragma unroll
-      for (int j = 0; j < P::ENTRIES * 8 / T::THREADS; ++j) {
-        const int item = tid + j * T::THREADS;            // (entry, 4-lane group)
-        const int e = item >> 3, u = item & 7;
-        const uint2 c = *reinterpret_cast<const uint2*>(compact + 2 * e);
-        uint4 v;
-        v.x = c.x; v.y = c.x; v.z = c.y; v.w = c.y;
-        *reinterpret_cast<uint4*>(smem + e * 128 + u * 16) = v;
-      }
-    } else {
-      // 8-byte word (e, c) <- entry e of the chunk's single codebook, 16 copies
-      uint2* compact = reinterpret_cast<uint2*>(smem + P::TABLE_BYTES);
-      compact[tid] = cbv;                                 // 256 threads = 256 entries
-      __syncthreads();
+    for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-      for (int j = 0; j < P::ENTRIES * 8 / T::THREADS; ++j) {
-        const int item = tid + j * T::THREADS;            // (entry, pair of copies)
-        const int e = item >> 3, u = item & 7;
-        const uint2 c = compact[e];
-        *reinterpret_cast<uint4*>(smem + e * 128 + u * 16) = make_uint4(c.x, c.y, c.x, c.y);
+      for (int j = 0; j < 8; ++j) {
+        uint4 v = make_uint4(xr[nb][4 * j], xr[nb][4 * j + 1], xr[nb][4 * j + 2], xr[nb][4 * j + 3]);
+        lds128_if(v, xaddr[nb] + (i * 8 + j) * xstride, on[nb]);
+        xr[nb][4 * j] = v.x; xr[nb][4 * j + 1] = v.y; xr[nb][4 * j + 2] = v.z; xr[nb][4 * j + 3] = v.w;
       }
-    }
-    __syncthreads();
 
-    VQ_TRACE(2);
-    // ---- 4. look up + multiply-accumulate ----
-#pragma unroll
-    for (int task = 0; task < P::TASKS; ++task) {
-      task_all<D, B, NB>(acc[task], w[task], xr, tbl);
-    }
-    if (chunk + n_split < n_chunks) __syncthreads();  // the next chunk rewrites the tables
+    // ---- look up + multiply-accumulate ----
+    const uint32_t tbl = (base + (k & 1) * P::TABLE_BYTES) | lane_off;
+    chunk_steps<D, B, NB, 0, 4>(acc, w, xr, tbl);
+    chunk_steps<D, B, NB, 4, 4>(acc, w, xr, tbl);
+    chunk_steps<D, B, NB, 8, 4>(acc, w, xr, tbl);
+    chunk_steps<D, B, NB, 12, 4>(acc, w, xr, tbl);
+
+    if (fetch2) store_compact<D, B>(compact + (k & 1) * P::COMPACT_BYTES, vnext, tid);
+    if (last_of_table && i != n - 1) __syncthreads();   // table k is done with, table k+1 complete
   }
 
-  // ---- 5. push the partial sums to the cluster rank that owns each row ----
-  // Row r of the tile is owned by rank r % n_split; the owner receives, from every (rank, slice),
-  // one value per (row slot, batch row): recv[src][slot][n], src = rank * SLICES + slice.
-  const int slots = (T::CTA_ROWS + n_split - 1) / n_split;
-  const uint32_t recv_u32 = smem_u32 + P::TABLE_BYTES + kCompactBytes<D, B>;
-  float* recv = reinterpret_cast<float*>(smem + P::TABLE_BYTES + kCompactBytes<D, B>);
-  const int src = rank * P::SLICES + slice;
-  VQ_TRACE(3);
-  cluster_wait_acquire();  // matches the arrive at kernel entry: every CTA of the cluster is running
+  // ---- combine the K parts ----
+  // acc[mt][nb][e]: row 32*warp + 16*mt + g + 8*(e/2) of the slab, batch row nb*8 + 2t + (e&1)
+  if (S == 1) {
 #pragma unroll
-  for (int task = 0; task < P::TASKS; ++task)
-#pragma unroll
-    for (int half = 0; half < 2; ++half)
+    for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
       for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const int r = (rgroup0 + task * RGROUP_STEP) * 32 + half * 16 + gq + (e >> 1) * 8;
-          const int n = nb * 8 + 2 * t + (e & 1);
-          if (n < batch) {
-            const int owner = r % n_split, slot = r / n_split;
-            st_cluster_f32(recv_u32 + ((src * slots + slot) * batch + n) * 4, owner, acc[task][half][nb][e]);
-          }
+          const int r = row0 + 32 * warp + 16 * mt + g + 8 * (e >> 1), nn = nb * 8 + 2 * t + (e & 1);
+          if (nn < a.batch) a.Y[static_cast<long long>(nn) * a.N + r] = __float2half_rn(acc[mt][nb][e]);
         }
-  VQ_TRACE(4);
+    return;
+  }
+  // Rows [q*rpo, (q+1)*rpo) of the slab are summed by cluster rank q, which receives one value per
+  // (source rank, row, batch row): recv[src][row % rpo][n].  rpo is a multiple of 16.
+  const int rpo = T::CTA_ROWS / S;
+  const uint32_t recv_u32 = base + a.recv_off;
+  cluster_wait_acquire();   // every CTA of the cluster has started: its shared memory exists
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt) {
+    const int r16 = 32 * warp + 16 * mt;             // first row of the 16-row tile
+    const int owner = r16 / rpo, slot = r16 % rpo + g;
+    const uint32_t dst = map_to_rank(recv_u32 + ((rank * rpo + slot) * NBT + 2 * t) * 4, owner);
+#pragma unroll
+    for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) st_cluster_f32(dst + ((e >> 1) * 8 * NBT + nb * 8 + (e & 1)) * 4, acc[mt][nb][e]);
+  }
   cluster_arrive_release();
   cluster_wait_acquire();
-  VQ_TRACE(5);
-
-  // ---- 6. fixed-order sum over (rank, slice), one rounding, store ----
-  const int n_src = n_split * P::SLICES;
-  for (int o = tid; o < slots * batch; o += T::THREADS) {
-    const int slot = o / batch, n = o % batch;
-    const int r = slot * n_split + rank;
-    if (r < T::CTA_ROWS) {
-      float sum = 0.f;
-      for (int q = 0; q < n_src; ++q) sum += recv[(q * slots + slot) * batch + n];
-      Y[static_cast<long long>(n) * g.N + row0 + r] = __float2half_rn(sum);
-    }
+  const float* recv = reinterpret_cast<const float*>(smem + a.recv_off);
+  for (int o = tid; o < rpo * a.batch; o += T::THREADS) {
+    const int nn = o / rpo, slot = o % rpo;
+    float sum = 0.f;
+    for (int q = 0; q < S; ++q) sum += recv[(q * rpo + slot) * NBT + nn];
+    a.Y[static_cast<long long>(nn) * a.N + row0 + rank * rpo + slot] = __float2half_rn(sum);
   }
-  VQ_TRACE(6);
 }
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+int env_int(const char* name, int dflt) {
+#ifdef VQ_TUNING
+  if (const char* e = getenv(name)) return atoi(e);
+#else
+  (void)name;
+#endif
+  return dflt;
+}
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up once through the runtime (no link against libcuda).
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 template <int D, int B, int NB>
 vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch, cudaStream_t s) {
   using P = Policy<D, B>;
   using T = Tile<D, B>;
-  const int n_chunks = (g.K + T::CTA_COLS - 1) / T::CTA_COLS;
-  const int row_blocks = g.N / T::CTA_ROWS;
-  // tables + compact staging + receive buffer for the cluster reduction (worst case over splits)
-  const size_t recv_bytes = static_cast<size_t>(P::SLICES) * (T::CTA_ROWS + 16) * 8 * NB * sizeof(float);
-  const size_t smem_bytes = static_cast<size_t>(P::TABLE_BYTES) + kCompactBytes<D, B> + recv_bytes;
   auto kern = blockcb_kernel<D, B, NB>;
-  // one-time, per-kernel attributes and occupancy (immutable properties of the device + kernel)
-  static int slots = 0;
-  if (slots == 0) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes)) != cudaSuccess ||
-        cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
-      return VQ_ERR_CUDA;
-    int per_sm = 0, dev = 0, sms = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, T::THREADS, smem_bytes) != cudaSuccess ||
-        cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || per_sm < 1)
-      return VQ_ERR_CUDA;
-    slots = per_sm * sms;
+  static int sms_of[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VQ_ERR_CUDA;
+  if (sms_of[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return VQ_ERR_CUDA;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess) return VQ_ERR_CUDA;
+    sms_of[dev] = n;
   }
-  // K is split over the CTAs of a cluster (<= 16).  Model: time ~ waves * chunks per CTA; ties go
-  // to the larger split (more, shorter CTAs balance the tail better).
-  int best = 1;
-  long long best_cost = -1;
-  for (int sp = 1; sp <= 16 && sp <= n_chunks; ++sp) {
-    const long long per = (n_chunks + sp - 1) / sp;
-    const long long waves = (static_cast<long long>(row_blocks) * sp + slots - 1) / slots;
-    const long long cost = per * waves;
-    if (best_cost < 0 || cost <= best_cost) {
+  const int sms = sms_of[dev];
+  EncodeTiledFn encode = encode_tiled_fn();
+  int* error_flag = nullptr;
+  if (!encode || device_error_counter(&error_flag) != VQ_OK) return VQ_ERR_CUDA;
+
+  BlockArgs a;
+  a.cb = p.cb;
+  a.X = X;
+  a.Y = Y;
+  a.error_flag = error_flag;
+  a.N = g.N;
+  a.K = g.K;
+  a.batch = batch;
+  a.n_chunks = g.K / 256;
+  a.blocks_per_row = g.blocks_per_row;
+  a.Br = g.Br;
+  a.Bc = g.Bc;
+  const int row_blocks = g.N / T::CTA_ROWS;
+
+  // Shared memory of a CTA whose column range is `chunks` long.
+  auto smem_for = [&](int chunks, BlockArgs* out) {
+    size_t off = 2 * P::TABLE_BYTES;
+    const size_t compact_off = off; off += 2 * P::COMPACT_BYTES;
+    const size_t ring_off = round_up(off, 128); off = ring_off + static_cast<size_t>(P::WARPS) * kStages * T::STAGE_BYTES;
+    const size_t bar_off = off; off += static_cast<size_t>(P::WARPS) * kStages * 8;
+    const size_t x_off = round_up(off, 16); off = x_off + static_cast<size_t>(chunks) * 512 * batch;
+    const size_t recv_off = round_up(off, 16); off = recv_off + static_cast<size_t>(T::CTA_ROWS) * 8 * NB * sizeof(float);
+    if (out) {
+      out->compact_off = static_cast<int>(compact_off); out->ring_off = static_cast<int>(ring_off);
+      out->bar_off = static_cast<int>(bar_off); out->x_off = static_cast<int>(x_off); out->recv_off = static_cast<int>(recv_off);
+    }
+    return off + P::TABLE_BYTES;   // + room to align the tables
+  };
+  // K split: waves of co-resident CTAs times (chunks per CTA + fixed overhead); ties to the larger split.
+  int best = 0;
+  double best_cost = -1.0;
+  for (int S = 1; S <= 8; S *= 2) {
+    if (S > a.n_chunks) break;
+    const int chunks = (a.n_chunks + S - 1) / S;
+    const size_t smem = smem_for(chunks, nullptr);
+    if (smem > 220 * 1024) continue;
+    const int per_sm = static_cast<int>((227 * 1024) / (smem + 1024));
+    const long long ctas = static_cast<long long>(row_blocks) * S;
+    const long long slots = static_cast<long long>(per_sm < 1 ? 1 : per_sm) * sms;
+    const double waves = static_cast<double>((ctas + slots - 1) / slots);
+    const double busy = ctas >= sms ? 1.0 : static_cast<double>(sms) / ctas;   // idle SMs
+    const double cost = waves * (chunks + (S > 1 ? 2.0 : 1.5)) * busy;
+    if (best_cost < 0.0 || cost <= best_cost) {
       best_cost = cost;
-      best = sp;
+      best = S;
     }
   }
-#ifdef VQ_TUNING
-  if (const char* e = getenv("VQ_SPLIT")) { const int v = atoi(e); if (v >= 1 && v <= 16 && v <= n_chunks) best = v; }
-#endif
+  best = env_int("VQ_SPLIT", best);
+  if (best < 1 || best > 8 || (best & (best - 1)) || best > a.n_chunks) return VQ_ERR_UNSUPPORTED;
+  const size_t smem_bytes = smem_for((a.n_chunks + best - 1) / best, &a);
+  if (smem_bytes > 220 * 1024) return VQ_ERR_UNSUPPORTED;
+
+  // index stream as a 2-D byte tensor: rows of `stride` bytes; one box = 32 rows x SEG bytes
+  CUtensorMap tm;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(g.stride), static_cast<cuuint64_t>(g.N)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(g.stride)};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(P::SEG), 32u};
+  const cuuint32_t elem_strides[2] = {1u, 1u};
+  if (encode(&tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(p.idx), dims, strides, box, elem_strides,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return VQ_ERR_CUDA;
+
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(best, row_blocks, 1);
   cfg.blockDim = dim3(T::THREADS, 1, 1);
   cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = s;
   cudaLaunchAttribute attr[2];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = best;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  int na = 0;
+  if (best > 1) {
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = best;
+    attr[na].val.clusterDim.y = 1;
+    attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  if (env_int("VQ_PDL", 1)) {
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
   cfg.attrs = attr;
-  cfg.numAttrs = 1;  // programmatic dependent launch measured slower here; attribute left off
+  cfg.numAttrs = na;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tm, a);
+  if (e != cudaSuccess) {
 #ifdef VQ_TUNING
-  if (getenv("VQ_PDL")) cfg.numAttrs = 2;
+    fprintf(stderr, "blockcb launch failed: %s (S %d smem %zu)\n", cudaGetErrorString(e), best, smem_bytes);
 #endif
-  if (cudaLaunchKernelEx(&cfg, kern, g, p, X, Y, batch, n_chunks) != cudaSuccess) return VQ_ERR_CUDA;
+    return VQ_ERR_CUDA;
+  }
   return check_launch();
 }
 
 }  // namespace
 
-// Shared-codebook families: fp16 codebooks, block rows a multiple of the CTA tile height,
-// block columns a multiple of what one lane (64) / one CTA chunk covers.
+// Shared-codebook families: fp16 codebooks, block rows a multiple of the CTA's rows, block columns
+// a multiple of 128 (2-D) / 256 (4-D), K a multiple of the 256-column chunk.
 vq_status launch_gemm_blockcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
                               cudaStream_t s) {
-  if (g.cb_int8) return VQ_ERR_UNSUPPORTED;
-  if (g.K % 64) return VQ_ERR_UNSUPPORTED;
+  if (g.cb_int8 || g.K % 256) return VQ_ERR_UNSUPPORTED;
   if (g.d == 2 && g.b == 6) {
     if (g.Br % Tile<2, 6>::CTA_ROWS || g.Bc % 128) return VQ_ERR_UNSUPPORTED;
     return batch <= 8 ? launch<2, 6, 1>(g, p, X, Y, batch, s) : launch<2, 6, 2>(g, p, X, Y, batch, s);
   }
   if (g.d == 4 && g.b == 8) {
-    if (g.Br % Tile<4, 8>::CTA_ROWS || g.Bc % Tile<4, 8>::CTA_COLS) return VQ_ERR_UNSUPPORTED;
+    if (g.Br % Tile<4, 8>::CTA_ROWS || g.Bc % 256) return VQ_ERR_UNSUPPORTED;
     return batch <= 8 ? launch<4, 8, 1>(g, p, X, Y, batch, s) : launch<4, 8, 2>(g, p, X, Y, batch, s);
   }
   return VQ_ERR_UNSUPPORTED;

@@ -45,6 +45,10 @@ vq_status launch_gemm_rowcb(const Geometry& g, const LayerPtrs& p, const __half*
                             cudaStream_t s);
 vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s);
 
+// Device address of this device's counter of bounded waits that ran out inside a kernel (a copy
+// that never completed); looked up once per device.
+vq_status device_error_counter(int** d_counter);
+
 inline vq_status check_launch() {
   return cudaGetLastError() == cudaSuccess ? VQ_OK : VQ_ERR_CUDA;
 }
