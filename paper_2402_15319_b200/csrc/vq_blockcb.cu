@@ -456,7 +456,8 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
     }
     return off + P::TABLE_BYTES;   // + room to align the tables
   };
-  // K split: waves of co-resident CTAs times (chunks per CTA + fixed overhead); ties to the larger split.
+  // K split: waves of co-resident CTAs times (chunks per CTA + fixed overhead, in chunk times); ties
+  // go to the larger split.
   int best = 0;
   double best_cost = -1.0;
   for (int S = 1; S <= 8; S *= 2) {
@@ -468,8 +469,7 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
     const long long ctas = static_cast<long long>(row_blocks) * S;
     const long long slots = static_cast<long long>(per_sm < 1 ? 1 : per_sm) * sms;
     const double waves = static_cast<double>((ctas + slots - 1) / slots);
-    const double busy = ctas >= sms ? 1.0 : static_cast<double>(sms) / ctas;   // idle SMs
-    const double cost = waves * (chunks + (S > 1 ? 2.0 : 1.5)) * busy;
+    const double cost = waves * (chunks + (S > 1 ? 2.0 : 1.5));
     if (best_cost < 0.0 || cost <= best_cost) {
       best_cost = cost;
       best = S;
