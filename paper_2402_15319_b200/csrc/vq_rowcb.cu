@@ -413,33 +413,39 @@ int env_int(const char* name, int dflt) {
 }
 
 // Choose the CTA shape (WR row tiles x WK column parts, at most 8 warps) and the cluster size S.
-// Model: an SM works through ceil(CTAs / SMs) CTAs; a warp costs its steps plus a fixed overhead
-// (prologue, table set-up, reduction; more with a cluster) plus its share of staging the CTA's
-// activations; the SM runs at full rate from about 24 resident warps on.  Shapes whose tables,
-// activations and reduction buffer exceed smem_budget bytes of shared memory are left out;
-// {0,0,0} if none fits.
+// Model fitted to sweeps on B200: time ~ waves x (steps per warp + a fixed per-CTA overhead of
+// about 3 steps, 4 with a cluster), where a wave is as many CTAs as are co-resident (registers
+// allow about 16 warps per SM, 8 for the two-tile batch variant).  One wave of 8-warp CTAs with
+// as many column parts per CTA as possible wins; ties go to more column parts, then fewer CTAs
+// per cluster.  Shapes whose tables, activations and reduction buffer exceed smem_budget bytes of
+// shared memory are left out; {0,0,0} if none fits.
 Plan make_plan(int N, int n_steps, int step_cols, int batch, int sms, int tbl_per_warp, int nb, size_t smem_budget) {
   const int row_tiles = (N + 15) / 16;
+  const int warps_per_sm = nb == 1 ? 16 : 8;
   Plan best = {0, 0, 0};
   double best_cost = -1.0;
   for (int S = 1; S <= 8; S *= 2)
-    for (int WK = 1; WK <= 8; WK *= 2)
+    for (int WK = 8; WK >= 1; WK /= 2)
       for (int WR = 1; WR * WK <= 8; WR *= 2) {
         const int T = S * WK;
         if (T > n_steps || (T > 1 && 2 * T > n_steps)) continue;   // at least two steps per warp
-        const double cta_steps = static_cast<double>(n_steps) / S;
         const int W = WR * WK;
+        const double cta_steps = static_cast<double>(n_steps) / S;
         const double smem_need = (cta_steps + 1.0) * step_cols * 2.0 * batch + static_cast<double>(tbl_per_warp) * W +
                                  (T > 1 ? T * WR * 16.0 * 8.0 * nb * 4.0 : 0.0) + 4096.0 + 16.0;
         if (smem_need > static_cast<double>(smem_budget)) continue;
+        int per_sm = warps_per_sm / W;
+        const int by_smem = static_cast<int>(227.0 * 1024.0 / (smem_need + 1024.0));
+        if (per_sm > by_smem) per_sm = by_smem;
+        if (per_sm < 1) per_sm = 1;
         const long long ctas = static_cast<long long>((row_tiles + WR - 1) / WR) * S;
-        const double per_sm = static_cast<double>((ctas + sms - 1) / sms);
+        const long long slots = static_cast<long long>(per_sm) * sms;
+        const double waves = static_cast<double>((ctas + slots - 1) / slots);
         const double steps = static_cast<double>(n_steps) / T;
-        const double ovh = (S > 1 ? 4.0 : (WK > 1 ? 2.5 : 2.0)) + 0.25 * cta_steps * batch / W;
-        double resident = per_sm * W;
-        if (resident > 32.0) resident = 32.0;
-        const double rate = resident >= 24.0 ? 1.0 : resident / 24.0;
-        const double cost = per_sm * W * (steps + ovh) / rate;
+        // few resident warps hide latency badly
+        const double resident = static_cast<double>(ctas < slots ? ctas : slots) * W / sms;
+        const double slow = resident >= 8.0 ? 1.0 : 8.0 / (resident < 1.0 ? 1.0 : resident);
+        const double cost = waves * (steps * slow + (S > 1 ? 4.0 : 3.0));
         if (best_cost < 0.0 || cost < best_cost) {
           best_cost = cost;
           best = {WR, WK, S};
