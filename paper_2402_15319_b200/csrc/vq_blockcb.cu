@@ -102,11 +102,6 @@ struct Tile {
   static constexpr int STAGE_BYTES = 32 * P::SEG;            // one TMA box
 };
 
-__device__ __forceinline__ void tma_box_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-               ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-
 __device__ __forceinline__ uint2 lds64_ordered(uint32_t addr) {   // ring reads: stay behind the barrier wait
   uint2 v;
   asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr) : "memory");
@@ -390,23 +385,6 @@ int env_int(const char* name, int dflt) {
   return dflt;
 }
 
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// The driver's tensor-map encoder, looked up once through the runtime (no link against libcuda).
-EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
 size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 template <int D, int B, int NB>
@@ -424,9 +402,8 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
     sms_of[dev] = n;
   }
   const int sms = sms_of[dev];
-  EncodeTiledFn encode = encode_tiled_fn();
   int* error_flag = nullptr;
-  if (!encode || device_error_counter(&error_flag) != VQ_OK) return VQ_ERR_CUDA;
+  if (device_error_counter(&error_flag) != VQ_OK) return VQ_ERR_CUDA;
 
   BlockArgs a;
   a.cb = p.cb;
@@ -482,14 +459,7 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
 
   // index stream as a 2-D byte tensor: rows of `stride` bytes; one box = 32 rows x SEG bytes
   CUtensorMap tm;
-  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(g.stride), static_cast<cuuint64_t>(g.N)};
-  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(g.stride)};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(P::SEG), 32u};
-  const cuuint32_t elem_strides[2] = {1u, 1u};
-  if (encode(&tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(p.idx), dims, strides, box, elem_strides,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return VQ_ERR_CUDA;
+  if (encode_index_map(&tm, p.idx, g.stride, g.N, P::SEG, 32) != VQ_OK) return VQ_ERR_CUDA;
 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(best, row_blocks, 1);

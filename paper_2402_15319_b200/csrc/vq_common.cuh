@@ -1,6 +1,7 @@
 // Shared declarations of the CUDA side of the VQ-decode library (sm_100a).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -48,6 +49,10 @@ vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, 
 // Device address of this device's counter of bounded waits that ran out inside a kernel (a copy
 // that never completed); looked up once per device.
 vq_status device_error_counter(int** d_counter);
+
+// Tensor map of the packed index stream seen as a 2-D byte tensor (N rows of `stride` bytes) with
+// boxes of box_rows rows x box_bytes bytes, for tiled TMA loads without swizzle or multicast.
+vq_status encode_index_map(CUtensorMap* tm, const uint8_t* idx, long long stride, int N, int box_bytes, int box_rows);
 
 inline vq_status check_launch() {
   return cudaGetLastError() == cudaSuccess ? VQ_OK : VQ_ERR_CUDA;

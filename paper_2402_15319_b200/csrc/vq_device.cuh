@@ -2,6 +2,7 @@
 // loads, cluster barriers / distributed shared memory, programmatic dependent launch.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_fp16.h>
 #include <stdint.h>
 
@@ -129,6 +130,12 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// Tiled TMA load of one box of a 2-D tensor map (x = innermost coordinate in elements, a multiple
+// of 16 bytes; y = row) into this CTA's shared memory; completion is counted on `bar`.
+__device__ __forceinline__ void tma_box_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 // Wait for phase `parity` of the barrier, at most `max_tries` attempts (each attempt itself blocks
 // for a hardware-defined short time).  Returns false if the phase did not complete: the caller
