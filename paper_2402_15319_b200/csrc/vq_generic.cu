@@ -59,6 +59,52 @@ __global__ void decode_generic_kernel(Geometry g, LayerPtrs p, __half* __restric
   }
 }
 
+// Vectorised decode for formats whose rows hold a whole number of 8-index groups (K/d % 8 == 0):
+// one thread expands one group (b bytes of indices) into 8*D weights and writes them with D
+// 128-bit stores; a warp writes 512*D contiguous bytes of one row.  The kernel is bound by the
+// fp16 output it has to write (2 B per weight); the codebook look-ups go through L1.
+template <int D>
+__global__ void __launch_bounds__(256) decode_vec_kernel(Geometry g, LayerPtrs p, __half* __restrict__ W) {
+  const int groups = g.J / 8;
+  const long long total = static_cast<long long>(g.N) * groups;
+  const bool block_per_group = g.Bc % (8 * D) == 0;   // a group never straddles two codebook blocks
+  for (long long it = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; it < total;
+       it += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const int n = static_cast<int>(it / groups);
+    const int grp = static_cast<int>(it - static_cast<long long>(n) * groups);
+    const uint8_t* src = p.idx + n * g.stride + static_cast<long long>(grp) * g.b;
+    unsigned long long bits = 0;
+    for (int i = 0; i < g.b; ++i) bits |= static_cast<unsigned long long>(__ldg(src + i)) << (8 * i);
+    const long long blk_row = static_cast<long long>(n / g.Br) * g.blocks_per_row;
+    const int k0 = grp * 8 * D;
+    long long blk = blk_row + k0 / g.Bc;
+    float sc = g.cb_int8 ? __half2float(__ldg(p.scale + blk)) : 0.f;
+    __align__(16) __half out[8 * D];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int e = static_cast<int>((bits >> (i * g.b)) & (g.entries - 1));
+      if (!block_per_group) {
+        blk = blk_row + (k0 + i * D) / g.Bc;
+        if (g.cb_int8) sc = __half2float(__ldg(p.scale + blk));
+      }
+      const long long at = (blk * g.entries + e) * D;
+      if (g.cb_int8) {
+        const int8_t* c = static_cast<const int8_t*>(p.cb) + at;
+#pragma unroll
+        for (int t = 0; t < D; ++t) out[i * D + t] = __float2half_rn(sc * static_cast<float>(__ldg(c + t)));   // exact product, one rounding
+      } else {
+        const __half* c = static_cast<const __half*>(p.cb) + at;   // bit copies
+        if constexpr (D == 1) out[i] = __ldg(c);
+        else if constexpr (D == 2) *reinterpret_cast<uint32_t*>(&out[2 * i]) = __ldg(reinterpret_cast<const uint32_t*>(c));
+        else *reinterpret_cast<uint2*>(&out[4 * i]) = __ldg(reinterpret_cast<const uint2*>(c));
+      }
+    }
+    uint4* dst = reinterpret_cast<uint4*>(W + static_cast<long long>(n) * g.K + k0);
+#pragma unroll
+    for (int q = 0; q < D; ++q) dst[q] = reinterpret_cast<const uint4*>(out)[q];
+  }
+}
+
 template <int MB>
 __global__ void __launch_bounds__(256) gemm_generic_kernel(Geometry g, LayerPtrs p, const __half* __restrict__ X,
                                                            __half* __restrict__ Y, int batch) {
@@ -101,6 +147,16 @@ __global__ void __launch_bounds__(256) gemm_generic_kernel(Geometry g, LayerPtrs
 }  // namespace
 
 vq_status launch_decode_generic(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s) {
+  if (g.J % 8 == 0) {   // K % 8 == 0 follows: every 128-bit store is aligned
+    const long long total = static_cast<long long>(g.N) * (g.J / 8);
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148LL * 32) blocks = 148LL * 32;
+    const unsigned nb = static_cast<unsigned>(blocks);
+    if (g.d == 1) decode_vec_kernel<1><<<nb, 256, 0, s>>>(g, p, W);
+    else if (g.d == 2) decode_vec_kernel<2><<<nb, 256, 0, s>>>(g, p, W);
+    else decode_vec_kernel<4><<<nb, 256, 0, s>>>(g, p, W);
+    return check_launch();
+  }
   const long long total = static_cast<long long>(g.N) * ((g.J + 7) / 8);
   long long blocks = (total + 255) / 256;
   if (blocks > 148LL * 64) blocks = 148LL * 64;
