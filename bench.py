@@ -285,12 +285,56 @@ def run_reference(args):
 
 
 def dram_traffic_note(cfg_name: str):
-    """Per-launch DRAM traffic of the dominant kernel from the committed ncu summary, if any."""
+    """Average DRAM bytes (read + write) per launch of the dominant kernel, from the committed ncu
+    summary (profiles/dram_traffic.json); None when no capture of the current kernel exists."""
     try:
         with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
-            return json.load(f).get(cfg_name)
+            entry = json.load(f).get(cfg_name)
+        return None if not entry or not entry.get("current", False) else float(entry["avg_bytes_per_launch"])
     except Exception:
         return None
+
+
+KERNEL_OF = {"cfg1": "rowcb_kernel<LdsTbl<false>,1>", "cfg2": "rowcb_kernel<PrmtI8,1>", "cfg3": "blockcb_kernel<2,6,1>",
+             "cfg4": "blockcb_kernel<4,8,NB>", "cfg5": "rowcb_kernel<LdsTbl<true>,NB>"}
+
+
+def max_over_ranks(value: float, dist=None, device=None) -> float:
+    """Slowest rank's time: the whole job is done when the last replica is."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(step_bytes_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Replicas only: every rank moves step_bytes_per_rank per step; value = all ranks' bytes / slowest time."""
+    return world * step_bytes_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
+def time_decode(ds, reps: int = 3):
+    """vq_decode_weights on the largest layer of the set: (us, GB/s over indices + codebooks + fp16 output)."""
+    torch, vq = ds.torch, ds.vq
+    i = max(range(len(ds.specs)), key=lambda j: ds.specs[j].n_weights)
+    spec, fmt = ds.specs[i], ds.fmts[i]
+    outs = [torch.empty((spec.N, spec.K), dtype=torch.float16, device=ds.device) for _ in range(max(2, min(6, (2 * L2_BYTES) // (2 * spec.n_weights) + 1)))]
+    idx, cb, sc = ds.dev[0][i]
+    for w in outs:
+        vq.vq_decode_weights(fmt, idx, cb, sc, w)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        for c, w in enumerate(outs):
+            lay = ds.dev[c % ds.copies][i]
+            vq.vq_decode_weights(fmt, lay[0], lay[1], lay[2], w)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / (reps * len(outs))
+    nbytes = ds.bytes_per_layer[i] - 2 * ds.batch * (spec.K + spec.N) + 2 * spec.n_weights
+    return {"layer": spec.name, "us": us, "GBps": nbytes / us / 1e3, "bytes": nbytes}
 
 
 def run_ours(args):
@@ -329,20 +373,14 @@ def run_ours(args):
             time_steps(ds, args.steps, 0)
         sampler.stop()
         clock_src = "timed region too short to poll; polled during immediate repeats of the same loop"
-    if dist:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, dist, dev)
     ms_per_step = ms / args.steps
-    value = world * ds.step_bytes / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_gbs(ds.step_bytes, world, ms_per_step)
 
     e2e_steps = max(5, min(args.steps, 200))
     ms_e2e = time_e2e(ds, e2e_steps, args.warmup) if not args.no_e2e else float("nan")
-    if dist:
-        t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    e2e_val = world * ds.step_bytes / (ms_e2e / e2e_steps * 1e-3) / 1e9
+    ms_e2e = max_over_ranks(ms_e2e, dist, dev)
+    e2e_val = whole_job_gbs(ds.step_bytes, world, ms_e2e / e2e_steps)
 
     launches = len(ds.fmts) * args.steps
     per_launch_gbs = ds.step_bytes / (ms_per_step * 1e-3) / 1e9  # one GPU's kernels
@@ -369,7 +407,7 @@ def run_ours(args):
                 "what": "vq_gemm_small_batch_host per layer: pinned-host activations copied in, kernel, outputs copied back, stream synchronised every step; compressed weights resident in HBM"},
         "gpu_launches": launches,
         "roofline": {
-            "bound": "hbm", "kernel": "vq gemm kernel (one launch per layer)", "achieved": per_launch_gbs, "peak": peak,
+            "bound": "hbm", "kernel": KERNEL_OF.get(args.config, "vq gemm kernel") + " (one launch per layer)", "achieved": per_launch_gbs, "peak": peak,
             "unit": "GB/s", "frac": per_launch_gbs / peak, "peak_source": peak_src,
             "algorithmic_bytes_per_launch": ds.step_bytes / len(ds.fmts),
             "avg_launch_us": ms_per_step * 1e3 / len(ds.fmts), "traffic": traffic,
@@ -394,6 +432,10 @@ def run_ours(args):
                 g = d2.step_bytes / (m * 1e-3) / 1e9
                 per[f"{cfg}.b{b}"] = {"us_per_step": m * 1e3, "GBps": g, "frac_of_measured": g / peak,
                                       "pct_of_nominal_8TBps": 100 * g / NOMINAL_HBM_GBS, "bytes": d2.step_bytes}
+                if b == vq_synth.CONFIGS[cfg]["batches"][0]:
+                    dec = time_decode(d2)
+                    dec["frac_of_measured"] = dec["GBps"] / peak
+                    per[f"{cfg}.decode_weights"] = dec
                 del d2
                 torch.cuda.empty_cache()
         line["per_config"] = per

@@ -79,6 +79,28 @@ def test_benchmark_families_medium(spec):
     _check_layer(spec, seed=77, batches=(1, 2, 4, 8, 16))
 
 
+@pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+def test_tuned_kernels_cover_every_benchmark_format(cfg):
+    """VQ_IMPL_TUNED never falls back: it must run (not VQ_ERR_UNSUPPORTED) on every layer shape of
+    the five configurations, at every batch of the configuration (row count cut to two tiles)."""
+    conf = vq_synth.CONFIGS[cfg]
+    seen = set()
+    for spec in conf["layers"]:
+        if spec.K in seen:
+            continue
+        seen.add(spec.K)
+        small = vq_synth.LayerSpec(spec.name + ".cut", N=2 * max(spec.Br, 128), K=spec.K, d=spec.d, b=spec.b, Br=spec.Br,
+                                   Bc=spec.Bc, int8=spec.int8, cb_sigma=spec.cb_sigma)
+        _check_layer(small, seed=conf["seed"], batches=conf["batches"], impls=[vq.VQ_IMPL_TUNED], decode=False)
+
+
+def test_no_wait_ran_out_inside_a_kernel():
+    # bounded waits on asynchronous copies never expired in anything this process has run so far
+    import torch
+    torch.cuda.synchronize()
+    assert vq.vq_device_wait_failures() == 0
+
+
 # ---- properties that hold at any size ---------------------------------------------------------
 def test_unit_vectors_return_decoded_columns():
     spec = vq_synth.LayerSpec("unit", N=256, K=256, d=2, b=6, Br=128, Bc=128, int8=False)
