@@ -314,6 +314,45 @@ def whole_job_gbs(step_bytes_per_rank: int, world: int, ms_per_step: float) -> f
     return world * step_bytes_per_rank / (ms_per_step * 1e-3) / 1e9
 
 
+def time_int4g128(cfg_name: str, batch: int, device, torch, vq):
+    """The uniform INT4 group-128 yard-stick on the shapes of a configuration: us per layer set and
+    GB/s over its own bytes (nibbles + fp16 scale per 128 columns + x + y), cold cache."""
+    conf = vq_synth.CONFIGS[cfg_name]
+    layers, set_bytes = [], 0
+    for lid, spec in enumerate(conf["layers"]):
+        if spec.K % 128:
+            return None
+        q, sc = vq_synth.make_int4g128(spec.N, spec.K, conf["seed"], lid)
+        X = vq_synth.make_x(spec, conf["seed"], batch, lid)
+        nbytes = q.size + sc.size * 2 + 2 * batch * (spec.N + spec.K)
+        set_bytes += nbytes
+        layers.append((spec, torch.from_numpy(q).to(device), torch.from_numpy(sc).to(device), torch.from_numpy(X).to(device),
+                       torch.empty((batch, spec.N), dtype=torch.float16, device=device)))
+    copies = max(2, -(-2 * L2_BYTES // set_bytes))
+    dev = [layers] + [[(sp, q.clone(), sc.clone(), X, Y) for (sp, q, sc, X, Y) in layers] for _ in range(copies - 1)]
+
+    def step(c):
+        for sp, q, sc, X, Y in dev[c]:
+            vq.vq_int4g128_gemm_small_batch(sp.N, sp.K, q, sc, X, Y, batch)
+    step(0)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for c in range(copies):
+            step(c)
+    for _ in range(2):
+        g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(10):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / (10 * copies)
+    return {"us_per_step": us, "GBps": set_bytes / us / 1e3, "bytes": set_bytes}
+
+
 def time_decode(ds, reps: int = 3):
     """vq_decode_weights on the largest layer of the set: (us, GB/s over indices + codebooks + fp16 output)."""
     torch, vq = ds.torch, ds.vq
@@ -437,6 +476,12 @@ def run_ours(args):
                     dec["frac_of_measured"] = dec["GBps"] / peak
                     per[f"{cfg}.decode_weights"] = dec
                 del d2
+                torch.cuda.empty_cache()
+            for b in vq_synth.CONFIGS[cfg]["batches"][:1]:
+                r = time_int4g128(cfg, b, dev, torch, vq)
+                if r:
+                    r["frac_of_measured"] = r["GBps"] / peak
+                    per[f"{cfg}.int4g128_yardstick.b{b}"] = r
                 torch.cuda.empty_cache()
         line["per_config"] = per
     if rank == 0:

@@ -44,6 +44,8 @@ vq_status launch_gemm_blockcb(const Geometry& g, const LayerPtrs& p, const __hal
                               cudaStream_t s);
 vq_status launch_gemm_rowcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
                             cudaStream_t s);
+vq_status launch_int4g128_rowcb(int N, int K, const uint8_t* q, const __half* scale, const __half* X, __half* Y, int batch,
+                                cudaStream_t s);
 vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s);
 
 // Device address of this device's counter of bounded waits that ran out inside a kernel (a copy

@@ -55,6 +55,12 @@ extern "C" vq_status vq_int4g128_gemm_small_batch(int32_t N, int32_t K, const vo
                            reinterpret_cast<uintptr_t>(d_X) | reinterpret_cast<uintptr_t>(d_Y);
   if (bitsor & 15u) return VQ_ERR_ALIGN;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  {
+    // tensor-core path shared with the per-row VQ kernels; the plain kernel below covers the rest
+    const vq_status st = launch_int4g128_rowcb(N, K, static_cast<const uint8_t*>(d_q), static_cast<const __half*>(d_scale),
+                                               static_cast<const __half*>(d_X), static_cast<__half*>(d_Y), batch, s);
+    if (st != VQ_ERR_UNSUPPORTED) return st;
+  }
   long long blocks = (N + 7) / 8;
   if (blocks > 148LL * 8) blocks = 148LL * 8;
   const unsigned nb = static_cast<unsigned>(blocks);

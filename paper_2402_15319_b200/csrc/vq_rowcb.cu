@@ -76,6 +76,7 @@ struct PrmtI8 {
   static constexpr bool SCALED = true;
   static constexpr int TABLE_BYTES_PER_WARP = 0;
   static constexpr int CB_ROW_BYTES = 16;
+  static __device__ __forceinline__ uint4 permute_x(uint4 in) { return in; }   // natural column order
 
   struct State {
     uint32_t T[2][4];   // [row g / g+8][entries 4q..4q+3], biased by +128
@@ -134,6 +135,7 @@ struct LdsTbl {
   static constexpr bool SCALED = INT8;
   static constexpr int TABLE_BYTES_PER_WARP = 4096;
   static constexpr int CB_ROW_BYTES = INT8 ? 32 : 64;
+  static __device__ __forceinline__ uint4 permute_x(uint4 in) { return in; }   // natural column order
 
   struct State {
     const uint8_t* cb_row[2];
@@ -203,6 +205,67 @@ struct LdsTbl {
 };
 
 // ---------------------------------------------------------------------------------------------
+// Int4G128: the uniform INT4 group-128 yard-stick run through the same skeleton (paper Sec. 2.1
+// symmetric uniform quantiser x ~ s*x_int; Sec. 5 "INT4 g128").  No table: a nibble q becomes the
+// fp16 value q - 8 by the exponent trick, (1024 + q) - 1032; a "block" is one 128-column group whose
+// fp16 scale multiplies the group's fp32 partial sum.  The two nibbles that share a mask
+// (columns c and c+4 of an 8-column word) land in one fp16 pair, so the activations are staged in
+// the matching order.
+// ---------------------------------------------------------------------------------------------
+struct Int4G128 {
+  static constexpr int D = 1;
+  static constexpr int STEP_COLS = 128;
+  static constexpr int WORD_CHUNKS = 1;
+  static constexpr bool SCALED = true;
+  static constexpr int TABLE_BYTES_PER_WARP = 0;
+  // (x0x1, x2x3, x4x5, x6x7) -> (x0x4, x1x5, x2x6, x3x7)
+  static __device__ __forceinline__ uint4 permute_x(uint4 in) {
+    return make_uint4(prmt(in.x, in.z, 0x5410), prmt(in.x, in.z, 0x7632), prmt(in.y, in.w, 0x5410), prmt(in.y, in.w, 0x7632));
+  }
+
+  struct State {
+    const __half* sc_row[2];
+    float sc[2], sc_next[2];
+    int n_blocks;
+
+    __device__ __forceinline__ void init(const RowArgs& a, int, int rl, int rh, int, uint32_t) {
+      sc_row[0] = a.scale + static_cast<long long>(rl) * a.blocks_per_row;
+      sc_row[1] = a.scale + static_cast<long long>(rh) * a.blocks_per_row;
+      n_blocks = a.blocks_per_row;
+      sc_next[0] = sc_next[1] = __int_as_float(0x7fc00000);   // "not loaded"
+    }
+
+    // scale of group blk; the next group's scale is requested one step ahead
+    __device__ __forceinline__ void load_block(int blk) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const float cur = sc_next[h];
+        sc[h] = cur == cur ? cur : __half2float(__ldg(sc_row[h] + blk));
+        sc_next[h] = blk + 1 < n_blocks ? __half2float(__ldg(sc_row[h] + blk + 1)) : 0.f;
+      }
+    }
+
+    __device__ __forceinline__ void decode(uint32_t wl, uint32_t wh, uint32_t (&a)[1][2][4]) const {
+      constexpr uint32_t kBias1032 = 0x64086408u;   // fp16 pair (1032, 1032) = 1024 + 8
+      const uint32_t w[2] = {wl, wh};
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        uint32_t p[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t m = ((w[h] >> (4 * i)) & 0x000F000Fu) | 0x64006400u;   // nibbles i and i+4
+          asm("sub.f16x2 %0, %1, %2;" : "=r"(p[i]) : "r"(m), "r"(kBias1032));
+        }
+        a[0][0][h] = p[0];       // columns 0,4
+        a[0][0][h + 2] = p[1];   // columns 1,5
+        a[0][1][h] = p[2];       // columns 2,6
+        a[0][1][h + 2] = p[3];   // columns 3,7
+      }
+    }
+  };
+};
+
+// ---------------------------------------------------------------------------------------------
 // The kernel.  Grid (S, ceil(N / (16*WR))), cluster (S, 1, 1); CTA = WR*WK warps.
 // Activations in shared memory: 16-byte chunk (step, chunk c of the lane's columns, batch row m,
 // lane quarter t) at index ((step*CHUNKS + c)*batch + m)*4 + t, so that the lanes of a warp that
@@ -265,7 +328,7 @@ __global__ void __launch_bounds__(256, VQ_ROW_MIN_CTAS) rowcb_kernel(const RowAr
         const int col = c8 * 8;
         const int step = col / P::STEP_COLS, within = col % P::STEP_COLS;
         const int tt = within / LANE_COLS, chunk = (within % LANE_COLS) / 8;
-        xs[((step * CHUNKS + chunk) * a.batch + m) * 4 + tt] = __ldg(src + c8);
+        xs[((step * CHUNKS + chunk) * a.batch + m) * 4 + tt] = P::permute_x(__ldg(src + c8));
       }
     }
   }
@@ -550,6 +613,21 @@ vq_status launch_gemm_rowcb(const Geometry& g, const LayerPtrs& p, const __half*
   if (!g.cb_int8 && g.d == 2)
     return nb1 ? launch<LdsTbl<false>, 1>(g, p, X, Y, batch, s) : launch<LdsTbl<false>, 2>(g, p, X, Y, batch, s);
   return VQ_ERR_UNSUPPORTED;
+}
+
+// Uniform INT4 group-128 yard-stick through the row-kernel skeleton; UNSUPPORTED if K is not a
+// multiple of 128.
+vq_status launch_int4g128_rowcb(int N, int K, const uint8_t* q, const __half* scale, const __half* X, __half* Y, int batch,
+                                cudaStream_t s) {
+  if (K % 128) return VQ_ERR_UNSUPPORTED;
+  Geometry g = {};
+  g.N = N; g.K = K; g.d = 1; g.b = 4; g.Br = 1; g.Bc = 128;
+  g.cb_int8 = 1; g.entries = 16; g.J = K; g.blocks_per_row = K / 128; g.stride = K / 2;
+  LayerPtrs p;
+  p.idx = q;
+  p.cb = nullptr;
+  p.scale = scale;
+  return batch <= 8 ? launch<Int4G128, 1>(g, p, X, Y, batch, s) : launch<Int4G128, 2>(g, p, X, Y, batch, s);
 }
 
 }  // namespace vq
