@@ -231,27 +231,53 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
   if (lane == 0)
     for (int i = 0; i < kStages && i < n; ++i) issue(i);
 
-  // ---- first two codebook tables ----
+  // ---- first two codebook tables and the activations: all global loads are requested before any
+  // of them is waited for ----
   unsigned char* compact = smem + a.compact_off;
-  if (nt > 0) store_compact<D, B>(compact, fetch_entry<D, B>(a, blk_row, t0 * cpt, tid), tid);
-  if (nt > 1) store_compact<D, B>(compact + P::COMPACT_BYTES, fetch_entry<D, B>(a, blk_row, (t0 + 1) * cpt, tid), tid);
+  uint2 cb0 = make_uint2(0u, 0u), cb1 = cb0;
+  if (nt > 0) cb0 = fetch_entry<D, B>(a, blk_row, t0 * cpt, tid);
+  if (nt > 1) cb1 = fetch_entry<D, B>(a, blk_row, (t0 + 1) * cpt, tid);
 
-  // ---- activations of the CTA's column range: chunk i, 16-byte piece j of a lane's 64 columns,
-  // batch row m, lane quarter tt at ((i*8 + j)*batch + m)*4 + tt ----
+  // Activations of the CTA's column range: chunk i, 16-byte piece j of a lane's 64 columns, batch
+  // row m, lane quarter tt at ((i*8 + j)*batch + m)*4 + tt.
   pdl_wait();   // the activations (and Y) belong to the previous kernel until here
   {
     uint4* xs = reinterpret_cast<uint4*>(smem + a.x_off);
     const int n16 = n * 32;   // 16-byte pieces per batch row
-    for (int m = 0; m < a.batch; ++m) {
-      const uint4* src = reinterpret_cast<const uint4*>(a.X + static_cast<long long>(m) * a.K + c0 * 256);
-      for (int q = tid; q < n16; q += T::THREADS) {
-        const int i = q >> 5, tt = (q >> 3) & 3, j = q & 7;
-        xs[((i * 8 + j) * a.batch + m) * 4 + tt] = __ldg(src + q);
+    const int total = n16 * a.batch;
+    constexpr int kInReg = 4;   // pieces a thread keeps in registers: enough for the usual ranges
+    uint4 xv[kInReg];
+#pragma unroll
+    for (int u = 0; u < kInReg; ++u) {
+      const int item = tid + u * T::THREADS;
+      xv[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (item < total) {
+        const int m = item / n16, q = item - m * n16;
+        xv[u] = __ldg(reinterpret_cast<const uint4*>(a.X + static_cast<long long>(m) * a.K + c0 * 256) + q);
       }
+    }
+    if (nt > 0) store_compact<D, B>(compact, cb0, tid);
+    if (nt > 1) store_compact<D, B>(compact + P::COMPACT_BYTES, cb1, tid);
+    auto put = [&](int item, uint4 v) {
+      const int m = item / n16, q = item - m * n16;
+      const int i = q >> 5, tt = (q >> 3) & 3, j = q & 7;
+      xs[((i * 8 + j) * a.batch + m) * 4 + tt] = v;
+    };
+#pragma unroll
+    for (int u = 0; u < kInReg; ++u) {
+      const int item = tid + u * T::THREADS;
+      if (item < total) put(item, xv[u]);
+    }
+    for (int item = tid + kInReg * T::THREADS; item < total; item += T::THREADS) {
+      const int m = item / n16, q = item - m * n16;
+      put(item, __ldg(reinterpret_cast<const uint4*>(a.X + static_cast<long long>(m) * a.K + c0 * 256) + q));
     }
   }
   __syncthreads();
   if (nt > 0) replicate<D, B>(base, compact, tid);
+  // every CTA of the cluster has started long ago; the wait that proves it (needed before the first
+  // remote store) costs a few hundred ns and hides here behind the first index box
+  if (S > 1) cluster_wait_acquire();
   __syncthreads();
 
   float acc[2][NB][4];
@@ -351,7 +377,6 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
   // (source rank, row, batch row): recv[src][row % rpo][n].  rpo is a multiple of 16.
   const int rpo = T::CTA_ROWS / S;
   const uint32_t recv_u32 = base + a.recv_off;
-  cluster_wait_acquire();   // every CTA of the cluster has started: its shared memory exists
 #pragma unroll
   for (int mt = 0; mt < 2; ++mt) {
     const int r16 = 32 * warp + 16 * mt;             // first row of the 16-row tile
@@ -360,7 +385,9 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
 #pragma unroll
     for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) st_cluster_f32(dst + ((e >> 1) * 8 * NBT + nb * 8 + (e & 1)) * 4, acc[mt][nb][e]);
+      for (int e = 0; e < 4; ++e)
+        if (nb * 8 + 2 * t + (e & 1) < a.batch)
+          st_cluster_f32(dst + ((e >> 1) * 8 * NBT + nb * 8 + (e & 1)) * 4, acc[mt][nb][e]);
   }
   cluster_arrive_release();
   cluster_wait_acquire();
