@@ -91,13 +91,24 @@ struct PrmtI8 {
       sc_row[1] = a.scale + static_cast<long long>(rh) * a.blocks_per_row;
     }
 
-    __device__ __forceinline__ void load_block(int blk) {
+    uint4 raw[2];     // requested entries of the next block
+    float sc_raw[2];
+
+    // Request the entries and the scale of block blk (global loads, not waited for here) ...
+    __device__ __forceinline__ void fetch(int blk) {
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
-        const uint4 v = ldg128_nc(cb_row[h] + static_cast<long long>(blk) * CB_ROW_BYTES);
-        T[h][0] = v.x ^ 0x80808080u; T[h][1] = v.y ^ 0x80808080u;
-        T[h][2] = v.z ^ 0x80808080u; T[h][3] = v.w ^ 0x80808080u;
-        sc[h] = __half2float(__ldg(sc_row[h] + blk));
+        raw[h] = ldg128_nc(cb_row[h] + static_cast<long long>(blk) * CB_ROW_BYTES);
+        sc_raw[h] = __half2float(__ldg(sc_row[h] + blk));
+      }
+    }
+    // ... and make them the current look-up table.
+    __device__ __forceinline__ void install() {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        T[h][0] = raw[h].x ^ 0x80808080u; T[h][1] = raw[h].y ^ 0x80808080u;
+        T[h][2] = raw[h].z ^ 0x80808080u; T[h][3] = raw[h].w ^ 0x80808080u;
+        sc[h] = sc_raw[h];
       }
     }
 
@@ -160,22 +171,40 @@ struct LdsTbl {
       fill = warp_tbl + (4 * tb) * 128 + gb * 16;   // entries 4tb..4tb+3, the 4 copies of row gb
     }
 
-    // Each fetched entry is written 4 times (one copy per lane of the row's quad).
-    __device__ __forceinline__ void load_block(int blk) {
-      uint32_t e[2][4];
+    uint32_t raw[2][4];   // requested entries of the next block (int8: still packed)
+    float sc_raw[2];
+
+    // Request this lane's share of the entries (and the scales) of block blk; not waited for here.
+    __device__ __forceinline__ void fetch(int blk) {
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         const uint8_t* p = cb_row[h] + static_cast<long long>(blk) * CB_ROW_BYTES;
         if constexpr (INT8) {
           const uint2 v = ldg64_nc(p);   // 4 entries x (c0, c1)
-          e[h][0] = sub_bias(prmt(v.x ^ 0x80808080u, kMagic, 0x4140));
-          e[h][1] = sub_bias(prmt(v.x ^ 0x80808080u, kMagic, 0x4342));
-          e[h][2] = sub_bias(prmt(v.y ^ 0x80808080u, kMagic, 0x4140));
-          e[h][3] = sub_bias(prmt(v.y ^ 0x80808080u, kMagic, 0x4342));
-          sc[h] = __half2float(__ldg(sc_row[h] + blk));
+          raw[h][0] = v.x; raw[h][1] = v.y; raw[h][2] = raw[h][3] = 0u;
+          sc_raw[h] = __half2float(__ldg(sc_row[h] + blk));
         } else {
           const uint4 v = ldg128_nc(p);
-          e[h][0] = v.x; e[h][1] = v.y; e[h][2] = v.z; e[h][3] = v.w;
+          raw[h][0] = v.x; raw[h][1] = v.y; raw[h][2] = v.z; raw[h][3] = v.w;
+        }
+      }
+    }
+
+    // Build the table from the requested entries: each is written 4 times (one copy per lane of the
+    // row's quad).
+    __device__ __forceinline__ void install() {
+      uint32_t e[2][4];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if constexpr (INT8) {
+          e[h][0] = sub_bias(prmt(raw[h][0] ^ 0x80808080u, kMagic, 0x4140));
+          e[h][1] = sub_bias(prmt(raw[h][0] ^ 0x80808080u, kMagic, 0x4342));
+          e[h][2] = sub_bias(prmt(raw[h][1] ^ 0x80808080u, kMagic, 0x4140));
+          e[h][3] = sub_bias(prmt(raw[h][1] ^ 0x80808080u, kMagic, 0x4342));
+          sc[h] = sc_raw[h];
+        } else {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) e[h][i] = raw[h][i];
         }
       }
       __syncwarp();   // every lane is done with the previous block's table
@@ -232,17 +261,15 @@ struct Int4G128 {
       sc_row[0] = a.scale + static_cast<long long>(rl) * a.blocks_per_row;
       sc_row[1] = a.scale + static_cast<long long>(rh) * a.blocks_per_row;
       n_blocks = a.blocks_per_row;
-      sc_next[0] = sc_next[1] = __int_as_float(0x7fc00000);   // "not loaded"
     }
 
-    // scale of group blk; the next group's scale is requested one step ahead
-    __device__ __forceinline__ void load_block(int blk) {
+    __device__ __forceinline__ void fetch(int blk) {
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const float cur = sc_next[h];
-        sc[h] = cur == cur ? cur : __half2float(__ldg(sc_row[h] + blk));
-        sc_next[h] = blk + 1 < n_blocks ? __half2float(__ldg(sc_row[h] + blk + 1)) : 0.f;
-      }
+      for (int h = 0; h < 2; ++h) sc_next[h] = __half2float(__ldg(sc_row[h] + blk));
+    }
+    __device__ __forceinline__ void install() {
+      sc[0] = sc_next[0];
+      sc[1] = sc_next[1];
     }
 
     __device__ __forceinline__ void decode(uint32_t wl, uint32_t wh, uint32_t (&a)[1][2][4]) const {
@@ -314,7 +341,7 @@ __global__ void __launch_bounds__(256, VQ_ROW_MIN_CTAS) rowcb_kernel(const RowAr
       qh[u] = ldg128_stream(ph + u * 64);
     }
   }
-  if (s0 < s1) st.load_block(s0 / a.steps_per_block);
+  if (s0 < s1) st.fetch(s0 / a.steps_per_block);
 
   // ---- activations of the CTA's column range ----
   pdl_wait();   // the activations (and Y) belong to the previous kernel until here
@@ -332,7 +359,11 @@ __global__ void __launch_bounds__(256, VQ_ROW_MIN_CTAS) rowcb_kernel(const RowAr
       }
     }
   }
+  if (s0 < s1) st.install();   // the first block's entries were requested ahead of the activations
   __syncthreads();
+  // every CTA of the cluster started long ago; the wait that proves it (needed before the first
+  // remote store) hides here behind the first index loads
+  if (S > 1) cluster_wait_acquire();
 
   float acc[NB][4], total[NB][4];
 #pragma unroll
@@ -366,6 +397,8 @@ __global__ void __launch_bounds__(256, VQ_ROW_MIN_CTAS) rowcb_kernel(const RowAr
       }
       pl += 64;
       ph += 64;
+      // last step of a codebook block: request the next block's entries one step ahead
+      if (in_blk + 1 == a.steps_per_block && s + 1 < s1) st.fetch(blk + 1);
       const uint32_t wl[4] = {cl.x, cl.y, cl.z, cl.w}, wh[4] = {ch.x, ch.y, ch.z, ch.w};
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -402,7 +435,7 @@ __global__ void __launch_bounds__(256, VQ_ROW_MIN_CTAS) rowcb_kernel(const RowAr
         }
         in_blk = 0;
         ++blk;
-        if (s + 1 < s1) st.load_block(blk);
+        if (s + 1 < s1) st.install();
       }
     }
   }
@@ -430,19 +463,21 @@ __global__ void __launch_bounds__(256, VQ_ROW_MIN_CTAS) rowcb_kernel(const RowAr
   const uint32_t red_local = smem_base + a.red_offset;
   const uint32_t mine = red_local + (((part * a.WR + wr) * 16 + g) * NBT + 2 * t) * 4;
   if (S > 1) {
-    cluster_wait_acquire();   // every CTA of the cluster has started: rank 0's shared memory exists
     const uint32_t dst = map_to_rank(mine, 0);
 #pragma unroll
     for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) st_cluster_f32(dst + ((e >> 1) * 8 * NBT + nb * 8 + (e & 1)) * 4, total[nb][e]);
+      for (int e = 0; e < 4; ++e)
+        if (nb * 8 + 2 * t + (e & 1) < a.batch)   // only existing batch rows travel
+          st_cluster_f32(dst + ((e >> 1) * 8 * NBT + nb * 8 + (e & 1)) * 4, total[nb][e]);
     cluster_arrive_release();
     cluster_wait_acquire();
   } else {
 #pragma unroll
     for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) sts32f(mine + ((e >> 1) * 8 * NBT + nb * 8 + (e & 1)) * 4, total[nb][e]);
+      for (int e = 0; e < 4; ++e)
+        if (nb * 8 + 2 * t + (e & 1) < a.batch) sts32f(mine + ((e >> 1) * 8 * NBT + nb * 8 + (e & 1)) * 4, total[nb][e]);
     __syncthreads();
   }
   if (rank != 0) return;
