@@ -206,7 +206,19 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int S = gridDim.x, rank = blockIdx.x;
-  if (S > 1) cluster_arrive_relaxed();   // matched by the wait in front of the first remote store
+  // Receive barrier of the K-part reduction: S * rpo * batch values of 4 bytes arrive through
+  // asynchronous remote stores.  Initialised before the start-up arrive so that every CTA of the
+  // cluster sees it once its start-up wait (in front of the first remote store) returns.
+  const uint32_t recv_bar = base + a.bar_off + P::WARPS * kStages * 8;
+  if (S > 1) {
+    if (tid == 0) {
+      mbar_init(recv_bar, 1);
+      mbar_init_fence();
+      mbar_arrive_expect_tx(recv_bar, static_cast<uint32_t>(T::CTA_ROWS * a.batch * 4));
+    }
+    __syncwarp();
+    cluster_arrive_release();
+  }
   pdl_launch_dependents();
 
   const int c0 = a.n_chunks * rank / S, c1 = a.n_chunks * (rank + 1) / S, n = c1 - c0;
@@ -382,15 +394,17 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
     const int r16 = 32 * warp + 16 * mt;             // first row of the 16-row tile
     const int owner = r16 / rpo, slot = r16 % rpo + g;
     const uint32_t dst = map_to_rank(recv_u32 + ((rank * rpo + slot) * NBT + 2 * t) * 4, owner);
+    const uint32_t dst_bar = map_to_rank(recv_bar, owner);
 #pragma unroll
     for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
       for (int e = 0; e < 4; ++e)
         if (nb * 8 + 2 * t + (e & 1) < a.batch)
-          st_cluster_f32(dst + ((e >> 1) * 8 * NBT + nb * 8 + (e & 1)) * 4, acc[mt][nb][e]);
+          st_async_f32(dst + ((e >> 1) * 8 * NBT + nb * 8 + (e & 1)) * 4, acc[mt][nb][e], dst_bar);
   }
-  cluster_arrive_release();
-  cluster_wait_acquire();
+  // every value this CTA sums has been counted on its barrier; nobody writes here afterwards, so the
+  // CTA may leave without a cluster barrier
+  if (!mbar_wait(recv_bar, 0, kWaitTries) && tid == 0) atomicAdd(a.error_flag, 1);
   const float* recv = reinterpret_cast<const float*>(smem + a.recv_off);
   for (int o = tid; o < rpo * a.batch; o += T::THREADS) {
     const int nn = o / rpo, slot = o % rpo;
@@ -451,7 +465,7 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
     size_t off = 2 * P::TABLE_BYTES;
     const size_t compact_off = off; off += 2 * P::COMPACT_BYTES;
     const size_t ring_off = round_up(off, 128); off = ring_off + static_cast<size_t>(P::WARPS) * kStages * T::STAGE_BYTES;
-    const size_t bar_off = off; off += static_cast<size_t>(P::WARPS) * kStages * 8;
+    const size_t bar_off = off; off += static_cast<size_t>(P::WARPS) * kStages * 8 + 8;   // rings + receive barrier
     const size_t x_off = round_up(off, 16); off = x_off + static_cast<size_t>(chunks) * 512 * batch;
     const size_t recv_off = round_up(off, 16); off = recv_off + static_cast<size_t>(T::CTA_ROWS) * 8 * NB * sizeof(float);
     if (out) {

@@ -110,6 +110,14 @@ __device__ __forceinline__ void st_cluster_f32(uint32_t cluster_addr, float v) {
   asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
 }
 
+// Asynchronous remote store: writes `v` into the shared memory of another CTA of the cluster and
+// counts 4 bytes on that CTA's mbarrier (both addresses from map_to_rank with the same rank), so
+// the receiver learns of the data by waiting on its own barrier: no cluster-wide barrier needed.
+__device__ __forceinline__ void st_async_f32(uint32_t cluster_addr, float v, uint32_t cluster_bar) {
+  asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];"
+               ::"r"(cluster_addr), "f"(v), "r"(cluster_bar) : "memory");
+}
+
 // ---- bulk asynchronous copies (TMA, untiled, no multicast) tracked by an mbarrier ----------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t arrivals) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(arrivals) : "memory");

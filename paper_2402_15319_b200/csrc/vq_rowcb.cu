@@ -44,6 +44,7 @@ struct RowArgs {
   const __half* scale;
   const __half* X;
   __half* Y;
+  int* error_flag;      // device counter of waits that ran out
   long long stride;     // bytes between index rows
   int N, K, batch;
   int n_steps;          // K / STEP_COLS
@@ -54,8 +55,10 @@ struct RowArgs {
   // activations (x_offset), then the reduction buffer (red_offset)
   int x_offset;
   int red_offset;
+  int bar_offset;   // receive barrier of the reduction (8 bytes), behind the reduction buffer
 };
 
+constexpr int kWaitTries = 1 << 18;            // mbarrier polls before rank 0 gives up and flags an error
 constexpr uint32_t kMagic = 0x64646464u;      // high byte of fp16 1024.0
 constexpr uint32_t kBias2 = 0x64806480u;      // fp16 pair (1152, 1152) = 1024 + 128
 
@@ -311,7 +314,20 @@ __global__ void __launch_bounds__(256, VQ_ROW_MIN_CTAS) rowcb_kernel(const RowAr
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int S = gridDim.x, rank = blockIdx.x;
-  if (S > 1) cluster_arrive_relaxed();   // matched by the wait in front of the first remote store
+  // Receive barrier of the K-part reduction in cluster rank 0: every warp of the cluster sends its
+  // 16 rows x batch partial sums there by asynchronous remote stores that count on this barrier.
+  // Initialised before the start-up arrive, so that it is visible to every CTA whose start-up wait
+  // (in front of the first remote store) has returned.
+  const uint32_t red_bar = smem_base + a.bar_offset;
+  if (S > 1) {
+    if (tid == 0) {
+      mbar_init(red_bar, 1);
+      mbar_init_fence();
+      mbar_arrive_expect_tx(red_bar, static_cast<uint32_t>(S * (blockDim.x / 32) * 16 * a.batch * 4));
+    }
+    __syncwarp();
+    cluster_arrive_release();
+  }
   pdl_launch_dependents();
 
   const int wr = warp % a.WR, wk = warp / a.WR;
@@ -463,15 +479,16 @@ __global__ void __launch_bounds__(256, VQ_ROW_MIN_CTAS) rowcb_kernel(const RowAr
   const uint32_t red_local = smem_base + a.red_offset;
   const uint32_t mine = red_local + (((part * a.WR + wr) * 16 + g) * NBT + 2 * t) * 4;
   if (S > 1) {
-    const uint32_t dst = map_to_rank(mine, 0);
+    const uint32_t dst = map_to_rank(mine, 0), dst_bar = map_to_rank(red_bar, 0);
 #pragma unroll
     for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
       for (int e = 0; e < 4; ++e)
         if (nb * 8 + 2 * t + (e & 1) < a.batch)   // only existing batch rows travel
-          st_cluster_f32(dst + ((e >> 1) * 8 * NBT + nb * 8 + (e & 1)) * 4, total[nb][e]);
-    cluster_arrive_release();
-    cluster_wait_acquire();
+          st_async_f32(dst + ((e >> 1) * 8 * NBT + nb * 8 + (e & 1)) * 4, total[nb][e], dst_bar);
+    // nobody writes into the other ranks' shared memory: they are done; rank 0 waits for the values
+    if (rank != 0) return;
+    if (!mbar_wait(red_bar, 0, kWaitTries) && tid == 0) atomicAdd(a.error_flag, 1);
   } else {
 #pragma unroll
     for (int nb = 0; nb < NB; ++nb)
@@ -575,6 +592,7 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
   a.scale = p.scale;
   a.X = X;
   a.Y = Y;
+  if (device_error_counter(&a.error_flag) != VQ_OK) return VQ_ERR_CUDA;
   a.stride = g.stride;
   a.N = g.N;
   a.K = g.K;
@@ -596,13 +614,14 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
   const size_t tbl_bytes = static_cast<size_t>(P::TABLE_BYTES_PER_WARP) * pl.WR * pl.WK;
   const size_t x_bytes = static_cast<size_t>(cta_steps) * P::STEP_COLS * 2 * batch;
   const size_t red_bytes = T > 1 ? static_cast<size_t>(T) * pl.WR * 16 * 8 * NB * sizeof(float) : 0;
-  if (tbl_bytes + x_bytes + 16 + red_bytes + 4096 > 208 * 1024) return VQ_ERR_UNSUPPORTED;
+  if (tbl_bytes + x_bytes + 16 + red_bytes + 16 + 4096 > 208 * 1024) return VQ_ERR_UNSUPPORTED;
   a.x_offset = static_cast<int>(tbl_bytes);
   a.red_offset = static_cast<int>(tbl_bytes + (x_bytes + 15) / 16 * 16);
+  a.bar_offset = a.red_offset + static_cast<int>(red_bytes);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(pl.S, (g.N + 16 * pl.WR - 1) / (16 * pl.WR), 1);
   cfg.blockDim = dim3(32 * pl.WR * pl.WK, 1, 1);
-  cfg.dynamicSmemBytes = a.red_offset + red_bytes + 4096;   // + room to align the tables
+  cfg.dynamicSmemBytes = a.red_offset + red_bytes + 16 + 4096;   // + barrier, + room to align the tables
   cfg.stream = s;
   cudaLaunchAttribute attr[2];
   int na = 0;
