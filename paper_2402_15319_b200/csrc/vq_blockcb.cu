@@ -1,5 +1,6 @@
 // Tuned skinny-GEMM kernels for formats whose codebook is shared by a tall block of rows
-// (block_rows a multiple of the CTA's rows): the 2-D 6-bit and 4-D 8-bit fp16-codebook families.
+// (block_rows a multiple of the CTA's rows): the 2-D 5- and 6-bit and the 4-D 8-bit families, with
+// fp16 codebooks or int8 codebooks (whose entries enter the tables as fp16(scale * c)).
 //
 // A CTA owns one block-row slab (128 or 256 rows: every warp 32 of them) and a range of 256-column
 // chunks; a thread block cluster of S CTAs splits K.  Per chunk and warp the packed indices of 32
@@ -39,6 +40,7 @@ constexpr int kWaitTries = 1 << 18;   // mbarrier polls before a warp gives up a
 
 struct BlockArgs {
   const void* cb;
+  const __half* scale;   // one per block for int8 codebooks, else null
   const __half* X;
   __half* Y;
   int* error_flag;       // device counter of waits that ran out
@@ -54,28 +56,33 @@ struct BlockArgs {
 template <int D, int B>
 struct Policy;
 
-// 2-D, 6-bit indices: 256 columns = 128 indices = 96 bytes per row; a lane owns 24 of them
-template <>
-struct Policy<2, 6> {
-  static constexpr int LANE_WORDS = 6, ENTRIES = 64, SEG = 96;
+// 2-D, B-bit indices (B = 5, 6): 256 columns = 128 indices = 16*B bytes per row; a lane owns 32
+// indices = B words of them
+template <int B>
+struct PolicyD2 {
+  static constexpr int LANE_WORDS = B, ENTRIES = 1 << B, SEG = 16 * B;
   static constexpr int WARPS = 4;                           // CTA = 128 rows
   static constexpr int TABLE_BYTES = ENTRIES * 128;          // [entry][lane] words
   static constexpr int COMPACT_BYTES = ENTRIES * 8;          // [entry][half] words
-  static constexpr uint32_t MASK = 0x1F80u;                  // 6 index bits at address bits 7..12
+  static constexpr uint32_t MASK = static_cast<uint32_t>(ENTRIES - 1) << 7;   // index bits at address bits 7..
 
   template <int I>   // (index I of the lane's 32) * 128
   static __device__ __forceinline__ uint32_t entry_off(const uint32_t (&w)[LANE_WORDS]) {
-    constexpr int p = 6 * I;
+    constexpr int p = B * I;
     if constexpr (p < 7) {
       return (w[0] << (7 - p)) & MASK;
     } else {
       constexpr int q = p - 7, wi = q >> 5, s = q & 31;
       if constexpr (s == 0) return w[wi] & MASK;
-      else if constexpr (s + 13 > 32) return __funnelshift_r(w[wi], w[wi + 1], s) & MASK;
+      else if constexpr (s + 7 + B > 32) return __funnelshift_r(w[wi], w[wi + 1], s) & MASK;
       else return (w[wi] >> s) & MASK;
     }
   }
 };
+template <>
+struct Policy<2, 6> : PolicyD2<6> {};
+template <>
+struct Policy<2, 5> : PolicyD2<5> {};
 
 // 4-D, 8-bit indices: 256 columns = 64 indices = 64 bytes per row; a lane owns 16 of them
 template <>
@@ -102,6 +109,11 @@ struct Tile {
   static constexpr int STAGE_BYTES = 32 * P::SEG;            // one TMA box
 };
 
+__device__ __forceinline__ uint32_t lds32_ordered(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+  return v;
+}
 __device__ __forceinline__ uint2 lds64_ordered(uint32_t addr) {   // ring reads: stay behind the barrier wait
   uint2 v;
   asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr) : "memory");
@@ -156,19 +168,41 @@ template <int D, int B>
 __device__ __forceinline__ uint2 fetch_entry(const BlockArgs& a, long long blk_row, int chunk, int tid) {
   using P = Policy<D, B>;
   uint2 v = make_uint2(0u, 0u);
+  // int8 codebooks: the table holds fp16(scale * c), the value vq_decode_weights writes for the weight
+  auto pair = [](float s, int lo, int hi) {
+    const __half2 hv = __halves2half2(__float2half_rn(s * static_cast<float>(lo)), __float2half_rn(s * static_cast<float>(hi)));
+    return *reinterpret_cast<const uint32_t*>(&hv);
+  };
   if constexpr (D == 2) {
-    const int e = tid & 63, h = tid >> 6;
-    const int col = chunk * 256 + h * 128;
-    v.x = __ldg(static_cast<const uint32_t*>(a.cb) + (blk_row + col / a.Bc) * P::ENTRIES + e);
+    const int e = tid % P::ENTRIES, h = tid / P::ENTRIES;
+    if (h >= 2) return v;
+    const long long blk = blk_row + (chunk * 256 + h * 128) / a.Bc;
+    if (a.scale == nullptr) {
+      v.x = __ldg(static_cast<const uint32_t*>(a.cb) + blk * P::ENTRIES + e);
+    } else {
+      const uint16_t raw = __ldg(static_cast<const uint16_t*>(a.cb) + blk * P::ENTRIES + e);
+      v.x = pair(__half2float(__ldg(a.scale + blk)), static_cast<int8_t>(raw & 0xff), static_cast<int8_t>(raw >> 8));
+    }
   } else {
-    v = __ldg(static_cast<const uint2*>(a.cb) + (blk_row + (chunk * 256) / a.Bc) * P::ENTRIES + tid);
+    const long long blk = blk_row + (chunk * 256) / a.Bc;
+    if (a.scale == nullptr) {
+      v = __ldg(static_cast<const uint2*>(a.cb) + blk * P::ENTRIES + tid);
+    } else {
+      const uint32_t raw = __ldg(static_cast<const uint32_t*>(a.cb) + blk * P::ENTRIES + tid);
+      const float s = __half2float(__ldg(a.scale + blk));
+      v.x = pair(s, static_cast<int8_t>(raw & 0xff), static_cast<int8_t>((raw >> 8) & 0xff));
+      v.y = pair(s, static_cast<int8_t>((raw >> 16) & 0xff), static_cast<int8_t>(raw >> 24));
+    }
   }
   return v;
 }
 
 template <int D, int B>
 __device__ __forceinline__ void store_compact(unsigned char* compact, uint2 v, int tid) {
-  if constexpr (D == 2) reinterpret_cast<uint32_t*>(compact)[2 * (tid & 63) + (tid >> 6)] = v.x;   // [entry][half]
+  if constexpr (D == 2) {
+    constexpr int E = Policy<D, B>::ENTRIES;
+    if (tid / E < 2) reinterpret_cast<uint32_t*>(compact)[2 * (tid % E) + tid / E] = v.x;   // [entry][half]
+  }
   else reinterpret_cast<uint2*>(compact)[tid] = v;
 }
 
@@ -311,7 +345,7 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
   }
   const uint32_t xstride = a.batch * 64;
   const uint32_t lane_off = D == 2 ? lane * 4 : (lane & 15) * 8;
-  const uint32_t row_off = (D == 2 ? t * 24 : t * 16) + g * P::SEG;
+  const uint32_t row_off = t * (LW * 4) + g * P::SEG;
 
   for (int i = 0; i < n; ++i) {
     const int c = c0 + i;
@@ -332,13 +366,16 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
     const uint32_t src = ring + st * T::STAGE_BYTES + row_off;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      if constexpr (LW == 6) {
+      if constexpr (D == 2 && LW == 6) {
 #pragma unroll
         for (int h = 0; h < 3; ++h) {
           const uint2 v = lds64_ordered(src + q * 8 * P::SEG + 8 * h);
           w[q][2 * h] = v.x;
           w[q][2 * h + 1] = v.y;
         }
+      } else if constexpr (D == 2) {   // odd word counts: 32-bit reads, conflict-free for odd B
+#pragma unroll
+        for (int h = 0; h < LW; ++h) w[q][h] = lds32_ordered(src + q * 8 * P::SEG + 4 * h);
       } else {
         const uint4 v = lds128(src + q * 8 * P::SEG);
         w[q][0] = v.x; w[q][1] = v.y; w[q][2] = v.z; w[q][3] = v.w;
@@ -448,6 +485,7 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
 
   BlockArgs a;
   a.cb = p.cb;
+  a.scale = g.cb_int8 ? p.scale : nullptr;
   a.X = X;
   a.Y = Y;
   a.error_flag = error_flag;
@@ -535,14 +573,18 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
 
 }  // namespace
 
-// Shared-codebook families: fp16 codebooks, block rows a multiple of the CTA's rows, block columns
+// Shared-codebook families: fp16 or int8 codebooks, block rows a multiple of the CTA's rows, block columns
 // a multiple of 128 (2-D) / 256 (4-D), K a multiple of the 256-column chunk.
 vq_status launch_gemm_blockcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
                               cudaStream_t s) {
-  if (g.cb_int8 || g.K % 256) return VQ_ERR_UNSUPPORTED;
+  if (g.K % 256) return VQ_ERR_UNSUPPORTED;
   if (g.d == 2 && g.b == 6) {
     if (g.Br % Tile<2, 6>::CTA_ROWS || g.Bc % 128) return VQ_ERR_UNSUPPORTED;
     return batch <= 8 ? launch<2, 6, 1>(g, p, X, Y, batch, s) : launch<2, 6, 2>(g, p, X, Y, batch, s);
+  }
+  if (g.d == 2 && g.b == 5) {
+    if (g.Br % Tile<2, 5>::CTA_ROWS || g.Bc % 128) return VQ_ERR_UNSUPPORTED;
+    return batch <= 8 ? launch<2, 5, 1>(g, p, X, Y, batch, s) : launch<2, 5, 2>(g, p, X, Y, batch, s);
   }
   if (g.d == 4 && g.b == 8) {
     if (g.Br % Tile<4, 8>::CTA_ROWS || g.Bc % 256) return VQ_ERR_UNSUPPORTED;

@@ -73,10 +73,26 @@ FAMILY = [
     vq_synth.LayerSpec("fam5", N=208, K=4096, d=2, b=4, Br=1, Bc=2048, int8=True),
 ]
 
+# further format points of the paper served by the tall-block kernel: int8 codebooks (Sec. 3.2:
+# 8-bit codebook entries with a scale per group), 5-bit indices (2.5 bits per dimension), 256-column groups
+TALL_BLOCK_EXTRA = [
+    vq_synth.LayerSpec("tb_d2b6_i8", N=384, K=1024, d=2, b=6, Br=128, Bc=128, int8=True),
+    vq_synth.LayerSpec("tb_d2b6_i8_256", N=256, K=2816, d=2, b=6, Br=256, Bc=256, int8=True),
+    vq_synth.LayerSpec("tb_d2b5", N=256, K=1280, d=2, b=5, Br=128, Bc=256, int8=False),
+    vq_synth.LayerSpec("tb_d2b5_i8", N=128, K=5632, d=2, b=5, Br=128, Bc=128, int8=True),
+    vq_synth.LayerSpec("tb_d4b8_i8", N=512, K=1536, d=4, b=8, Br=256, Bc=512, int8=True),
+]
+
 
 @pytest.mark.parametrize("spec", FAMILY, ids=lambda s: s.name)
 def test_benchmark_families_medium(spec):
     _check_layer(spec, seed=77, batches=(1, 2, 4, 8, 16))
+
+
+@pytest.mark.parametrize("spec", TALL_BLOCK_EXTRA, ids=lambda s: s.name)
+def test_tall_block_kernel_extra_formats(spec):
+    # tuned kernel only (no fallback), every batch size class, against the oracle
+    _check_layer(spec, seed=91, batches=(1, 3, 8, 16), impls=[vq.VQ_IMPL_TUNED, vq.VQ_IMPL_GENERIC], decode=True)
 
 
 @pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
