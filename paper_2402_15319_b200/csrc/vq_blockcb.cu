@@ -161,6 +161,18 @@ __device__ __forceinline__ void chunk_steps(float (&acc)[2][NB][4], const uint32
     }
 }
 
+// Compiler-level ordering point: everything that produced the accumulators (the mmas, hence the
+// gathers that feed them) is emitted before whatever follows.
+template <int NB>
+__device__ __forceinline__ void fence_acc(float (&acc)[2][NB][4]) {
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+    for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) asm volatile("" : "+f"(acc[mt][nb][e])::"memory");
+}
+
 // Fetch this thread's share of the codebook entries of table k (global memory -> register).
 // 2-D: thread (e = tid%64, h = tid/64) takes entry e of the block under columns h*128.. of the
 // chunk; 4-D: thread tid takes entry tid of the block the table's chunks lie in.
@@ -223,12 +235,72 @@ __device__ __forceinline__ void replicate(uint32_t table, const unsigned char* c
   }
 }
 
+// ---- warp-private tables (2-D formats whose block is 32 or 64 rows tall: every warp's 32 rows have
+// their own codebooks).  Lane l takes entries l*EPL .. +EPL-1 (EPL = ENTRIES / 32) of the two blocks
+// under the chunk's column halves: requested by load_private(), converted and written by
+// write_private() with the same rotation of the 16-byte groups as replicate().
+template <int B>
+struct PrivateRegs {
+  static constexpr int EPL = (1 << B) / 32;
+  uint32_t raw[2][EPL];   // fp16 codebooks: the entries; int8: EPL entries of 2 bytes in raw[h][0]
+  float scale[2];
+};
+template <int B>
+__device__ __forceinline__ void load_private(PrivateRegs<B>& r, const BlockArgs& a, long long blk_row, int chunk, int lane) {
+  constexpr int E = 1 << B, EPL = PrivateRegs<B>::EPL;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const long long blk = blk_row + (chunk * 256 + h * 128) / a.Bc;
+    if (a.scale == nullptr) {
+      const uint32_t* src = static_cast<const uint32_t*>(a.cb) + blk * E + lane * EPL;
+      if constexpr (EPL == 2) {
+        const uint2 q = ldg64_nc(src);
+        r.raw[h][0] = q.x;
+        r.raw[h][1] = q.y;
+      } else {
+        r.raw[h][0] = __ldg(src);
+      }
+      r.scale[h] = 1.f;
+    } else {
+      const uint16_t* src = static_cast<const uint16_t*>(a.cb) + blk * E + lane * EPL;
+      if constexpr (EPL == 2) r.raw[h][0] = __ldg(reinterpret_cast<const uint32_t*>(src));
+      else r.raw[h][0] = __ldg(src);
+      r.scale[h] = __half2float(__ldg(a.scale + blk));
+    }
+  }
+}
+template <int B>
+__device__ __forceinline__ void write_private(uint32_t table, const PrivateRegs<B>& r, bool int8, int lane) {
+  constexpr int EPL = PrivateRegs<B>::EPL;
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) {
+    uint32_t e[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      if (!int8) {
+        e[h] = r.raw[h][i];
+      } else {
+        const uint32_t two = r.raw[h][0] >> (16 * i);
+        const __half2 hv = __halves2half2(__float2half_rn(r.scale[h] * static_cast<float>(static_cast<int8_t>(two & 0xff))),
+                                          __float2half_rn(r.scale[h] * static_cast<float>(static_cast<int8_t>((two >> 8) & 0xff))));
+        e[h] = *reinterpret_cast<const uint32_t*>(&hv);
+      }
+    }
+    const uint4 v = make_uint4(e[0], e[0], e[1], e[1]);
+    const uint32_t row = table + (lane * EPL + i) * 128;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sts128(row + ((j + lane) & 7) * 16, v);
+  }
+}
+
 // Grid (S, N / CTA_ROWS), cluster (S, 1, 1).  Dynamic shared memory from its first TABLE_BYTES
 // boundary: two tables, two compact codebooks, the warps' index rings, their barriers, the
 // activations, the receive buffer of the reduction.
-template <int D, int B, int NB>
+// PRIV: every warp keeps its own pair of tables (block rows a multiple of 32, 2-D only).
+template <int D, int B, int NB, bool PRIV>
 __global__ void __launch_bounds__(Tile<D, B>::THREADS)
 blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
+  static_assert(!PRIV || D == 2, "warp-private tables exist for 2-D codebooks only");
   using P = Policy<D, B>;
   using T = Tile<D, B>;
   constexpr int LW = P::LANE_WORDS;
@@ -257,7 +329,8 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
 
   const int c0 = a.n_chunks * rank / S, c1 = a.n_chunks * (rank + 1) / S, n = c1 - c0;
   const int row0 = blockIdx.y * T::CTA_ROWS;
-  const long long blk_row = static_cast<long long>(row0 / a.Br) * a.blocks_per_row;
+  // first block of the block row the CTA's (PRIV: the warp's) rows lie in
+  const long long blk_row = static_cast<long long>((row0 + (PRIV ? 32 * warp : 0)) / a.Br) * a.blocks_per_row;
   const int cpt = D == 2 ? 1 : a.Bc / 256;   // chunks that share one table
   const int t0 = c0 / cpt, nt = n > 0 ? (c1 - 1) / cpt - t0 + 1 : 0;
 
@@ -281,8 +354,14 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
   // of them is waited for ----
   unsigned char* compact = smem + a.compact_off;
   uint2 cb0 = make_uint2(0u, 0u), cb1 = cb0;
-  if (nt > 0) cb0 = fetch_entry<D, B>(a, blk_row, t0 * cpt, tid);
-  if (nt > 1) cb1 = fetch_entry<D, B>(a, blk_row, (t0 + 1) * cpt, tid);
+  PrivateRegs<PRIV ? B : 5> mine;   // PRIV: this warp's entries of the table that is written next
+  const uint32_t my_tables = base + (PRIV ? warp * 2 * P::TABLE_BYTES : 0);
+  if constexpr (PRIV) {
+    if (n > 0) load_private<B>(mine, a, blk_row, c0, lane);
+  } else {
+    if (nt > 0) cb0 = fetch_entry<D, B>(a, blk_row, t0 * cpt, tid);
+    if (nt > 1) cb1 = fetch_entry<D, B>(a, blk_row, (t0 + 1) * cpt, tid);
+  }
 
   // Activations of the CTA's column range: chunk i, 16-byte piece j of a lane's 64 columns, batch
   // row m, lane quarter tt at ((i*8 + j)*batch + m)*4 + tt.
@@ -302,8 +381,13 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
         xv[u] = __ldg(reinterpret_cast<const uint4*>(a.X + static_cast<long long>(m) * a.K + c0 * 256) + q);
       }
     }
-    if (nt > 0) store_compact<D, B>(compact, cb0, tid);
-    if (nt > 1) store_compact<D, B>(compact + P::COMPACT_BYTES, cb1, tid);
+    if constexpr (PRIV) {
+      if (n > 0) write_private<B>(my_tables, mine, a.scale != nullptr, lane);
+      if (n > 1) load_private<B>(mine, a, blk_row, c0 + 1, lane);
+    } else {
+      if (nt > 0) store_compact<D, B>(compact, cb0, tid);
+      if (nt > 1) store_compact<D, B>(compact + P::COMPACT_BYTES, cb1, tid);
+    }
     auto put = [&](int item, uint4 v) {
       const int m = item / n16, q = item - m * n16;
       const int i = q >> 5, tt = (q >> 3) & 3, j = q & 7;
@@ -320,7 +404,8 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
     }
   }
   __syncthreads();
-  if (nt > 0) replicate<D, B>(base, compact, tid);
+  if constexpr (!PRIV)
+    if (nt > 0) replicate<D, B>(base, compact, tid);
   // every CTA of the cluster has started long ago; the wait that proves it (needed before the first
   // remote store) costs a few hundred ns and hides here behind the first index box
   if (S > 1) cluster_wait_acquire();
@@ -353,11 +438,13 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
     const bool first_of_table = i == 0 || (c - 1) / cpt - t0 != k;
     const bool last_of_table = i == n - 1 || (c + 1) / cpt - t0 != k;
     // codebook two tables ahead: request now, park in shared memory after the chunk's math
-    const bool fetch2 = first_of_table && k + 2 < nt;
+    const bool fetch2 = !PRIV && first_of_table && k + 2 < nt;
     uint2 vnext = make_uint2(0u, 0u);
-    if (fetch2) vnext = fetch_entry<D, B>(a, blk_row, (t0 + k + 2) * cpt, tid);
-    if (first_of_table && k + 1 < nt)
-      replicate<D, B>(base + ((k + 1) & 1) * P::TABLE_BYTES, compact + ((k + 1) & 1) * P::COMPACT_BYTES, tid);
+    if constexpr (!PRIV) {
+      if (fetch2) vnext = fetch_entry<D, B>(a, blk_row, (t0 + k + 2) * cpt, tid);
+      if (first_of_table && k + 1 < nt)
+        replicate<D, B>(base + ((k + 1) & 1) * P::TABLE_BYTES, compact + ((k + 1) & 1) * P::COMPACT_BYTES, tid);
+    }
 
     // ---- this warp's indices of the chunk ----
     const int st = i % kStages;
@@ -398,14 +485,26 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
       }
 
     // ---- look up + multiply-accumulate ----
-    const uint32_t tbl = (base + (k & 1) * P::TABLE_BYTES) | lane_off;
+    uint32_t tbl = (my_tables + (k & 1) * P::TABLE_BYTES) | lane_off;
+    if constexpr (PRIV) fence_value(tbl);   // the gathers stay behind the warp's own table writes
     chunk_steps<D, B, NB, 0, 4>(acc, w, xr, tbl);
     chunk_steps<D, B, NB, 4, 4>(acc, w, xr, tbl);
     chunk_steps<D, B, NB, 8, 4>(acc, w, xr, tbl);
     chunk_steps<D, B, NB, 12, 4>(acc, w, xr, tbl);
 
-    if (fetch2) store_compact<D, B>(compact + (k & 1) * P::COMPACT_BYTES, vnext, tid);
-    if (last_of_table && i != n - 1) __syncthreads();   // table k is done with, table k+1 complete
+    if constexpr (PRIV) {
+      // the warp's table for the next chunk goes into its other buffer (the previous chunk's, which
+      // only this warp read); the entries of the chunk after it are requested at once
+      if (i + 1 < n) {
+        fence_acc(acc);   // this chunk's and the previous chunk's gathers are emitted before the writes
+        write_private<B>(my_tables + ((k + 1) & 1) * P::TABLE_BYTES, mine, a.scale != nullptr, lane);
+        if (i + 2 < n) load_private<B>(mine, a, blk_row, c + 2, lane);
+        __syncwarp();
+      }
+    } else {
+      if (fetch2) store_compact<D, B>(compact + (k & 1) * P::COMPACT_BYTES, vnext, tid);
+      if (last_of_table && i != n - 1) __syncthreads();   // table k is done with, table k+1 complete
+    }
   }
 
   // ---- combine the K parts ----
@@ -465,11 +564,11 @@ int env_int(const char* name, int dflt) {
 
 size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-template <int D, int B, int NB>
+template <int D, int B, int NB, bool PRIV = false>
 vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch, cudaStream_t s) {
   using P = Policy<D, B>;
   using T = Tile<D, B>;
-  auto kern = blockcb_kernel<D, B, NB>;
+  auto kern = blockcb_kernel<D, B, NB, PRIV>;
   static int sms_of[kMaxDevices] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VQ_ERR_CUDA;
@@ -500,7 +599,7 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
 
   // Shared memory of a CTA whose column range is `chunks` long.
   auto smem_for = [&](int chunks, BlockArgs* out) {
-    size_t off = 2 * P::TABLE_BYTES;
+    size_t off = (PRIV ? 2 * P::WARPS : 2) * static_cast<size_t>(P::TABLE_BYTES);
     const size_t compact_off = off; off += 2 * P::COMPACT_BYTES;
     const size_t ring_off = round_up(off, 128); off = ring_off + static_cast<size_t>(P::WARPS) * kStages * T::STAGE_BYTES;
     const size_t bar_off = off; off += static_cast<size_t>(P::WARPS) * kStages * 8 + 8;   // rings + receive barrier
@@ -578,13 +677,18 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
 vq_status launch_gemm_blockcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
                               cudaStream_t s) {
   if (g.K % 256) return VQ_ERR_UNSUPPORTED;
-  if (g.d == 2 && g.b == 6) {
-    if (g.Br % Tile<2, 6>::CTA_ROWS || g.Bc % 128) return VQ_ERR_UNSUPPORTED;
-    return batch <= 8 ? launch<2, 6, 1>(g, p, X, Y, batch, s) : launch<2, 6, 2>(g, p, X, Y, batch, s);
-  }
-  if (g.d == 2 && g.b == 5) {
-    if (g.Br % Tile<2, 5>::CTA_ROWS || g.Bc % 128) return VQ_ERR_UNSUPPORTED;
-    return batch <= 8 ? launch<2, 5, 1>(g, p, X, Y, batch, s) : launch<2, 5, 2>(g, p, X, Y, batch, s);
+  if (g.d == 2 && (g.b == 6 || g.b == 5)) {
+    if (g.Bc % 128) return VQ_ERR_UNSUPPORTED;
+    // blocks of 128 rows or more: one pair of tables per CTA; 32 or 64 rows (the CTA's 128 rows must
+    // consist of whole blocks): a pair per warp
+    const bool shared_tables = g.Br % 128 == 0;
+    if (!shared_tables && (g.Br % 32 || 128 % g.Br || g.N % 128)) return VQ_ERR_UNSUPPORTED;
+    if (g.b == 6) {
+      if (shared_tables) return batch <= 8 ? launch<2, 6, 1>(g, p, X, Y, batch, s) : launch<2, 6, 2>(g, p, X, Y, batch, s);
+      return batch <= 8 ? launch<2, 6, 1, true>(g, p, X, Y, batch, s) : launch<2, 6, 2, true>(g, p, X, Y, batch, s);
+    }
+    if (shared_tables) return batch <= 8 ? launch<2, 5, 1>(g, p, X, Y, batch, s) : launch<2, 5, 2>(g, p, X, Y, batch, s);
+    return batch <= 8 ? launch<2, 5, 1, true>(g, p, X, Y, batch, s) : launch<2, 5, 2, true>(g, p, X, Y, batch, s);
   }
   if (g.d == 4 && g.b == 8) {
     if (g.Br % Tile<4, 8>::CTA_ROWS || g.Bc % 256) return VQ_ERR_UNSUPPORTED;

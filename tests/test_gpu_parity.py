@@ -81,6 +81,11 @@ TALL_BLOCK_EXTRA = [
     vq_synth.LayerSpec("tb_d2b5", N=256, K=1280, d=2, b=5, Br=128, Bc=256, int8=False),
     vq_synth.LayerSpec("tb_d2b5_i8", N=128, K=5632, d=2, b=5, Br=128, Bc=128, int8=True),
     vq_synth.LayerSpec("tb_d4b8_i8", N=512, K=1536, d=4, b=8, Br=256, Bc=512, int8=True),
+    # groups of 8192 weights with at most 256 columns (Sec. 4.1): 32 x 256 blocks, one pair of tables per warp
+    vq_synth.LayerSpec("wb_d2b6_i8_32x256", N=256, K=2304, d=2, b=6, Br=32, Bc=256, int8=True),
+    vq_synth.LayerSpec("wb_d2b6_64x128", N=384, K=1024, d=2, b=6, Br=64, Bc=128, int8=False),
+    vq_synth.LayerSpec("wb_d2b5_i8_32x256", N=128, K=4352, d=2, b=5, Br=32, Bc=256, int8=True),
+    vq_synth.LayerSpec("wb_d2b5_32x128", N=256, K=768, d=2, b=5, Br=32, Bc=128, int8=False),
 ]
 
 
