@@ -296,7 +296,8 @@ def dram_traffic_note(cfg_name: str):
 
 
 KERNEL_OF = {"cfg1": "rowcb_kernel<LdsTbl<false>,1>", "cfg2": "rowcb_kernel<PrmtI8,1>", "cfg3": "blockcb_kernel<2,6,1>",
-             "cfg4": "blockcb_kernel<4,8,NB>", "cfg5": "rowcb_kernel<LdsTbl<true>,NB>"}
+             "cfg4": "blockcb_kernel<4,8,NB>", "cfg5": "rowcb_kernel<LdsTbl<true>,NB>",
+             "llama3_8b": "blockcb_kernel<2,6,NB,warp-private tables>"}
 
 
 def max_over_ranks(value: float, dist=None, device=None) -> float:

@@ -100,7 +100,7 @@ def test_tall_block_kernel_extra_formats(spec):
     _check_layer(spec, seed=91, batches=(1, 3, 8, 16), impls=[vq.VQ_IMPL_TUNED, vq.VQ_IMPL_GENERIC], decode=True)
 
 
-@pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+@pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "llama3_8b"])
 def test_tuned_kernels_cover_every_benchmark_format(cfg):
     """VQ_IMPL_TUNED never falls back: it must run (not VQ_ERR_UNSUPPORTED) on every layer shape of
     the five configurations, at every batch of the configuration (row count cut to two tiles)."""
@@ -178,7 +178,7 @@ def _decode_slab_check(spec, L, dev_W, block_row):
     assert np.array_equal(dev_W[r0:r0 + spec.Br].view(np.uint16), W16), f"{spec.name}: decode rows {r0}.."
 
 
-@pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+@pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "llama3_8b"])
 def test_benchmark_configs_full_size(cfg):
     conf = vq_synth.CONFIGS[cfg]
     seen = set()

@@ -118,7 +118,8 @@ def _set(prefix, shapes, **fmt):
     return [LayerSpec(name=f"{prefix}.{nm}", N=n, K=k, **fmt) for nm, n, k in shapes]
 
 
-# The five benchmark configurations (seeded synthetic layers with LLM projection shapes).
+# The five benchmark configurations (seeded synthetic layers with LLM projection shapes) and, last,
+# the paper's deployed format on the shapes of the model it was deployed for.
 CONFIGS = {
     # single 4096x4096 layer, 2-D VQ, 4-bit indices, 16-entry fp16 codebook per 1x1024 block
     "cfg1": dict(seed=0, batches=(1,), layers=_set("l4096", [("w", 4096, 4096)],
@@ -141,6 +142,12 @@ CONFIGS = {
                  ("q", 8192, 8192), ("k", 1024, 8192), ("v", 1024, 8192), ("o", 8192, 8192),
                  ("gate", 28672, 8192), ("up", 28672, 8192), ("down", 8192, 28672)],
                  d=2, b=4, Br=1, Bc=2048, int8=True)),
+    # Llama-3-8B-shaped (GQA) layer set in the format the paper deploys (Sec. 4.1, Table 1, App. B):
+    # 2-D, 6-bit indices, int8 codebook + scale per group of 8192 weights of at most 256 columns
+    "llama3_8b": dict(seed=5, batches=(1, 8), layers=_set("llama3_8b", [
+                 ("q", 4096, 4096), ("k", 1024, 4096), ("v", 1024, 4096), ("o", 4096, 4096),
+                 ("gate", 14336, 4096), ("up", 14336, 4096), ("down", 4096, 14336)],
+                 d=2, b=6, Br=32, Bc=256, int8=True)),
 }
 
 
