@@ -364,12 +364,17 @@ def time_decode(ds, reps: int = 3):
     for w in outs:
         vq.vq_decode_weights(fmt, idx, cb, sc, w)
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(reps):
+    graph = torch.cuda.CUDAGraph()   # replayed, so that small layers are not timed at the host's launch rate
+    with torch.cuda.graph(graph):
         for c, w in enumerate(outs):
             lay = ds.dev[c % ds.copies][i]
             vq.vq_decode_weights(fmt, lay[0], lay[1], lay[2], w)
+    graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        graph.replay()
     e1.record()
     torch.cuda.synchronize()
     us = e0.elapsed_time(e1) * 1e3 / (reps * len(outs))

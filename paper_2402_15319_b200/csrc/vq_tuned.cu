@@ -54,9 +54,6 @@ vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half*
   return launch_gemm_rowcb(g, p, X, Y, batch, s);
 }
 
-vq_status launch_decode_tuned(const Geometry&, const LayerPtrs&, __half*, cudaStream_t) {
-  return VQ_ERR_UNSUPPORTED;
-}
 
 }  // namespace vq
 
