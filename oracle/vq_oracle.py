@@ -198,5 +198,31 @@ def int4g128_gemm(q: np.ndarray, scale, X, threads: int = 1):
     return Y, A
 
 
+def unpack_uniform(kind: str, src: np.ndarray, scale=None) -> np.ndarray:
+    """Uniformly quantized weights expanded to binary16, the yard-sticks of the transfer + decode
+    experiment (App. B; Sec. 2.1 symmetric uniform quantizer w = s * q):
+      "fp16":     the weights themselves, copied;
+      "int8row":  signed 8-bit q [N][K], one binary16 scale per row;
+      "int4g128": unsigned nibbles [N][K/2] (low nibble = lower column) meaning q - 8, one binary16
+                  scale per row and group of 128 columns.
+    The product s * q is exact in float64 (11-bit by 8-bit significands); it is rounded once to
+    binary16 (round to nearest even), as decode() does for int8 codebooks."""
+    if kind == "fp16":
+        return np.array(src, dtype=np.float16, copy=True)
+    if kind == "int8row":
+        q = np.asarray(src, dtype=np.int8).astype(np.float64)
+        s = np.asarray(scale, dtype=np.float16).astype(np.float64).reshape(-1, 1)
+        return (q * s).astype(np.float16)
+    if kind == "int4g128":
+        b = np.asarray(src, dtype=np.uint8)
+        N, K = b.shape[0], b.shape[1] * 2
+        q = np.empty((N, K), np.float64)
+        q[:, 0::2] = (b & 15).astype(np.float64) - 8.0
+        q[:, 1::2] = (b >> 4).astype(np.float64) - 8.0
+        s = np.asarray(scale, dtype=np.float16).astype(np.float64).reshape(N, K // 128)
+        return (q * np.repeat(s, 128, axis=1)).astype(np.float16)
+    raise ValueError(kind)
+
+
 def hardware_threads() -> int:
     return _load().ref_hardware_threads()

@@ -412,3 +412,31 @@ def test_synth_is_deterministic_and_distributed():
     assert L.cb.min() >= -127 and L.cb.max() <= 127
     assert 0.0005 <= float(L.scale.min()) and float(L.scale.max()) <= 0.002
     assert spec.N == 4096 and spec.K == 4096
+
+
+def test_unpack_uniform_hand_values():
+    """Yard-stick unpackers against values worked out by hand (Sec. 2.1: w = s * q)."""
+    # int4 g128: nibble 0 -> -8, nibble 15 -> +7; low nibble is the lower column; scale per 128 columns
+    b = np.zeros((1, 128), np.uint8)        # K = 256: two groups
+    b[0, 0] = 0xF0                          # columns 0, 1 = nibbles 0, 15
+    b[0, 64] = 0x9A                         # columns 128, 129 = nibbles 10, 9
+    s = np.array([[0.5, 2.0]], np.float16)
+    W = orc.unpack_uniform("int4g128", b, s)
+    assert W.dtype == np.float16 and W.shape == (1, 256)
+    assert W[0, 0] == -4.0 and W[0, 1] == 3.5 and W[0, 2] == -4.0
+    assert W[0, 128] == 4.0 and W[0, 129] == 2.0 and W[0, 130] == -16.0
+    # int8 with a row scale; 0.1 is not a binary16 value: s = 0.0999755859375, s * 127 rounds once
+    q = np.array([[-128, 127, 0, 3]], np.int8)
+    W8 = orc.unpack_uniform("int8row", q, np.array([0.1], np.float16))
+    s16 = float(np.float16(0.1))
+    assert s16 == 0.0999755859375
+    assert W8[0, 0] == np.float16(-128 * s16) and W8[0, 1] == np.float16(127 * s16) and W8[0, 2] == 0 and W8[0, 3] == np.float16(3 * s16)
+    assert float(W8[0, 0]) == -12.796875      # -128 * s is a power-of-two multiple: exact
+    # the rounding is one rounding of the exact product, not of a float32-rounded scale times q twice
+    exact = 127 * s16
+    lo, hi = np.float16(12.6953125), np.float16(12.703125)   # neighbours around 12.696899...
+    assert float(lo) < exact < float(hi) and W8[0, 1] == lo
+    # fp16 is a copy
+    w = np.array([[1.5, -0.0, 65504.0]], np.float16)
+    assert np.array_equal(orc.unpack_uniform("fp16", w).view(np.uint16), w.view(np.uint16))
+
