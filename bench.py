@@ -354,6 +354,61 @@ def time_int4g128(cfg_name: str, batch: int, device, torch, vq):
     return {"us_per_step": us, "GBps": set_bytes / us / 1e3, "bytes": set_bytes}
 
 
+def time_transfer_decode(device, torch, vq, N: int = 11008, K: int = 4096, reps: int = 5):
+    """The transfer + decode experiment of App. B on a gate_proj-shaped layer: time to read one stored
+    layer and write it out as fp16, for FP16 / INT8 / INT4-g128 storage and for three VQ formats
+    (the format points of cfg3, cfg5 and cfg4).  Latencies relative to INT4, as the paper's table."""
+    n_out = max(2, min(6, (2 * L2_BYTES) // (2 * N * K) + 1))
+    outs = [torch.empty((N, K), dtype=torch.float16, device=device) for _ in range(n_out)]
+
+    def timed(call):
+        for w in outs:
+            call(w)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for w in outs:
+                call(w)
+        g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (reps * n_out)
+
+    rows = {}
+    w16 = torch.from_numpy(vq_synth.normal(21, 1, N * K).astype(np.float16).reshape(N, K)).to(device)
+    rows["fp16"] = {"bits_per_weight": 16.0, "us": timed(lambda w: vq.vq_unpack_uniform(vq.VQ_UNPACK_FP16, N, K, w16, None, w))}
+    del w16
+    q8 = torch.from_numpy(vq_synth.random_bytes(21, 2, N * K).reshape(N, K).view(np.int8)).to(device)
+    s8 = torch.from_numpy((0.001 + 0.003 * vq_synth.uniform01(21, 3, N)).astype(np.float16)).to(device)
+    rows["int8_row"] = {"bits_per_weight": 8.0 + 16.0 / K, "us": timed(lambda w: vq.vq_unpack_uniform(vq.VQ_UNPACK_INT8_ROW, N, K, q8, s8, w))}
+    del q8
+    q4, s4 = vq_synth.make_int4g128(N, K, 21)
+    q4, s4 = torch.from_numpy(q4).to(device), torch.from_numpy(s4).to(device)
+    rows["int4_g128"] = {"bits_per_weight": 4.125, "us": timed(lambda w: vq.vq_unpack_uniform(vq.VQ_UNPACK_INT4_G128, N, K, q4, s4, w))}
+    del q4
+    for name, src in (("vq_2d_3.125", "cfg3"), ("vq_2d_2.125", "cfg5"), ("vq_4d_2.125", "cfg4")):
+        t = vq_synth.CONFIGS[src]["layers"][0]
+        spec = vq_synth.LayerSpec(name, N, K, t.d, t.b, t.Br, t.Bc, t.int8, cb_sigma=t.cb_sigma)
+        fmt = vq.VQFormat(N, K, spec.d, spec.b, spec.Br, spec.Bc, vq.VQ_CB_INT8_SCALED if spec.int8 else vq.VQ_CB_FP16)
+        info = vq.vq_pack_info(fmt)
+        L = vq_synth.make_layer(spec, info.row_stride_bytes, 21, 4)
+        idx, cb = torch.from_numpy(L.idx).to(device), torch.from_numpy(L.cb).to(device)
+        sc = None if L.scale is None else torch.from_numpy(L.scale).to(device)
+        rows[name] = {"bits_per_weight": 8.0 * info.total_bytes / (N * K),
+                      "us": timed(lambda w: vq.vq_decode_weights(fmt, idx, cb, sc, w))}
+    base = rows["int4_g128"]
+    for r in rows.values():
+        r["rel_footprint"] = r["bits_per_weight"] / base["bits_per_weight"]
+        r["rel_latency"] = r["us"] / base["us"]
+        r["GBps"] = (r["bits_per_weight"] / 8.0 + 2.0) * N * K / r["us"] / 1e3
+    return {"layer": f"{N}x{K}", "output": "fp16 [N][K]", "rows": rows}
+
+
 def time_decode(ds, reps: int = 3):
     """vq_decode_weights on the largest layer of the set: (us, GB/s over indices + codebooks + fp16 output)."""
     torch, vq = ds.torch, ds.vq
@@ -490,6 +545,7 @@ def run_ours(args):
                     per[f"{cfg}.int4g128_yardstick.b{b}"] = r
                 torch.cuda.empty_cache()
         line["per_config"] = per
+        line["transfer_decode"] = time_transfer_decode(dev, torch, vq)
     if rank == 0:
         print(json.dumps(line))
     if dist:

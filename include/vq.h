@@ -184,6 +184,18 @@ vq_status vq_int4g128_gemm_small_batch(int32_t n_rows, int32_t k_cols, const voi
                                        const void* d_scale, const void* d_X, void* d_Y,
                                        int batch, void* stream);
 
+/* Uniformly quantized weights expanded to binary16: the yard-sticks of the transfer + decode
+ * experiment (paper App. B: time to move and unpack a layer stored as FP16, INT8, INT4 or VQ),
+ * timed beside vq_decode_weights.  w = s * q (Sec. 2.1), exact product rounded once to binary16.
+ *   kind VQ_UNPACK_FP16     : d_src binary16 [N][K], d_scale NULL; a copy.
+ *   kind VQ_UNPACK_INT8_ROW : d_src signed 8-bit q [N][K]; d_scale binary16 [N], one per row.
+ *   kind VQ_UNPACK_INT4_G128: d_src and d_scale as for vq_int4g128_gemm_small_batch (q-8).
+ *   d_W : device binary16 [N][K], written completely.  K % 128 == 0; pointers 16-byte aligned.
+ * Errors: NULL, FORMAT (unknown kind), SHAPE, ALIGN, CUDA. */
+typedef enum { VQ_UNPACK_FP16 = 0, VQ_UNPACK_INT8_ROW = 1, VQ_UNPACK_INT4_G128 = 2 } vq_unpack_kind;
+vq_status vq_unpack_uniform(int kind, int32_t n_rows, int32_t k_cols, const void* d_src,
+                            const void* d_scale, void* d_W, void* stream);
+
 /* Diagnostics.  The tuned kernels wait for their asynchronous copies (Sec. 3.2 index stream) with a
  * bounded number of polls; a wait that runs out increments a per-device counter and the kernel
  * carries on (its output is then wrong, but the device stays usable).  This call copies the

@@ -41,6 +41,44 @@ __global__ void __launch_bounds__(256) int4g128_kernel(int N, int K, const uint3
   }
 }
 
+// Uniform yard-stick unpackers (App. B transfer + decode experiment): one thread writes 8 adjacent
+// weights with one 128-bit store; a warp reads 512 / 256 / 128 contiguous bytes and writes 512.
+template <int KIND>
+__global__ void __launch_bounds__(256) unpack_uniform_kernel(long long groups8, int k8, const void* __restrict__ src,
+                                                             const __half* __restrict__ scale, uint4* __restrict__ W) {
+  for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < groups8;
+       i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    uint4 out;
+    if constexpr (KIND == VQ_UNPACK_FP16) {
+      out = __ldg(static_cast<const uint4*>(src) + i);
+    } else {
+      int q[8];
+      float s;
+      if constexpr (KIND == VQ_UNPACK_INT8_ROW) {
+        const uint2 raw = __ldg(static_cast<const uint2*>(src) + i);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          q[j] = static_cast<int8_t>((raw.x >> (8 * j)) & 0xff);
+          q[4 + j] = static_cast<int8_t>((raw.y >> (8 * j)) & 0xff);
+        }
+        s = __half2float(__ldg(scale + i / k8));   // one scale per row of k8 groups
+      } else {
+        const uint32_t raw = __ldg(static_cast<const uint32_t*>(src) + i);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) q[j] = static_cast<int>((raw >> (4 * j)) & 15u) - 8;
+        s = __half2float(__ldg(scale + i / 16));   // 16 groups of 8 columns share a scale
+      }
+      __half2 h[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j)   // exact fp32 products, one rounding each
+        h[j] = __halves2half2(__float2half_rn(s * static_cast<float>(q[2 * j])), __float2half_rn(s * static_cast<float>(q[2 * j + 1])));
+      out = make_uint4(*reinterpret_cast<uint32_t*>(&h[0]), *reinterpret_cast<uint32_t*>(&h[1]),
+                       *reinterpret_cast<uint32_t*>(&h[2]), *reinterpret_cast<uint32_t*>(&h[3]));
+    }
+    W[i] = out;
+  }
+}
+
 }  // namespace
 }  // namespace vq
 
@@ -73,5 +111,26 @@ extern "C" vq_status vq_int4g128_gemm_small_batch(int32_t N, int32_t K, const vo
   else if (batch <= 4) int4g128_kernel<4><<<nb, 256, 0, s>>>(N, K, q, sc, X, Y, batch);
   else if (batch <= 8) int4g128_kernel<8><<<nb, 256, 0, s>>>(N, K, q, sc, X, Y, batch);
   else int4g128_kernel<16><<<nb, 256, 0, s>>>(N, K, q, sc, X, Y, batch);
+  return check_launch();
+}
+
+extern "C" vq_status vq_unpack_uniform(int kind, int32_t N, int32_t K, const void* d_src, const void* d_scale,
+                                       void* d_W, void* stream) {
+  if (kind != VQ_UNPACK_FP16 && kind != VQ_UNPACK_INT8_ROW && kind != VQ_UNPACK_INT4_G128) return VQ_ERR_FORMAT;
+  if (!d_src || !d_W || (kind != VQ_UNPACK_FP16 && !d_scale)) return VQ_ERR_NULL;
+  if (N <= 0 || K <= 0 || K % 128) return VQ_ERR_SHAPE;
+  uintptr_t bitsor = reinterpret_cast<uintptr_t>(d_src) | reinterpret_cast<uintptr_t>(d_W);
+  if (kind != VQ_UNPACK_FP16) bitsor |= reinterpret_cast<uintptr_t>(d_scale);
+  if (bitsor & 15u) return VQ_ERR_ALIGN;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const long long groups8 = static_cast<long long>(N) * (K / 8);
+  long long blocks = (groups8 + 255) / 256;
+  if (blocks > 148LL * 64) blocks = 148LL * 64;
+  const unsigned nb = static_cast<unsigned>(blocks);
+  const __half* sc = static_cast<const __half*>(d_scale);
+  uint4* W = static_cast<uint4*>(d_W);
+  if (kind == VQ_UNPACK_FP16) unpack_uniform_kernel<VQ_UNPACK_FP16><<<nb, 256, 0, s>>>(groups8, K / 8, d_src, sc, W);
+  else if (kind == VQ_UNPACK_INT8_ROW) unpack_uniform_kernel<VQ_UNPACK_INT8_ROW><<<nb, 256, 0, s>>>(groups8, K / 8, d_src, sc, W);
+  else unpack_uniform_kernel<VQ_UNPACK_INT4_G128><<<nb, 256, 0, s>>>(groups8, K / 8, d_src, sc, W);
   return check_launch();
 }

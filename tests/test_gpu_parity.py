@@ -223,6 +223,31 @@ def test_int4g128(N, K):
         assert_outputs_close(dY.cpu().numpy(), Y, A, f"int4 {N}x{K} b{batch}")
 
 
+@pytest.mark.parametrize("N,K", [(37, 256), (300, 1408)])
+def test_unpack_uniform_bit_exact(N, K):
+    """App. B yard-sticks: fp16 copy, int8 with a row scale, int4 g128; every output bit against the oracle."""
+    import torch
+    q4, s4 = vq_synth.make_int4g128(N, K, seed=11)
+    rng_bytes = vq_synth.random_bytes(12, 1, N * K).reshape(N, K)
+    q8 = rng_bytes.view(np.int8)
+    s8 = (0.001 + 0.003 * vq_synth.uniform01(12, 2, N)).astype(np.float16)
+    w16 = vq_synth.normal(12, 3, N * K).astype(np.float16).reshape(N, K)
+    cases = [(vq.VQ_UNPACK_FP16, "fp16", w16, None), (vq.VQ_UNPACK_INT8_ROW, "int8row", q8, s8),
+             (vq.VQ_UNPACK_INT4_G128, "int4g128", q4, s4)]
+    for kind, name, src, scale in cases:
+        want = orc.unpack_uniform(name, src, scale)
+        d_src = torch.from_numpy(np.ascontiguousarray(src)).cuda()
+        d_scale = None if scale is None else torch.from_numpy(np.ascontiguousarray(scale)).cuda()
+        d_W = torch.full((N, K), float("nan"), dtype=torch.float16, device="cuda")
+        vq.vq_unpack_uniform(kind, N, K, d_src, d_scale, d_W)
+        torch.cuda.synchronize()
+        assert np.array_equal(d_W.cpu().numpy().view(np.uint16), want.view(np.uint16)), name
+    with pytest.raises(vq.VQError):
+        vq.vq_unpack_uniform(7, N, K, d_src, d_scale, d_W)           # unknown kind
+    with pytest.raises(vq.VQError):
+        vq.vq_unpack_uniform(vq.VQ_UNPACK_INT4_G128, N, K + 64, d_src, d_scale, d_W)   # K % 128
+
+
 def test_host_buffer_entry_point():
     import torch
     spec = vq_synth.LayerSpec("host", N=256, K=1024, d=2, b=6, Br=128, Bc=128, int8=False)
