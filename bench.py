@@ -461,6 +461,12 @@ def run_ours(args):
 
     peak, peak_src = measured_peaks()
     ds = DeviceSet(args.config, args.batch, dev)
+    if args.decode_only:   # vq_decode_weights alone on the configuration's largest layer (profiling runs)
+        dec = time_decode(ds)
+        dec["frac_of_measured"] = dec["GBps"] / peak
+        if rank == 0:
+            print(json.dumps({"metric": "vq_decode_weights_bandwidth", "unit": "GB/s", "value": dec["GBps"], "config": args.config, **dec}))
+        return
     sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
     sampler.start()
     ms = time_steps(ds, args.steps, args.warmup, barrier)
@@ -563,6 +569,7 @@ def main():
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--all-configs", action="store_true", help="also time every configuration and batch (adds per_config)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--decode-only", action="store_true", help="time vq_decode_weights on the configuration's largest layer and exit")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end loop (profiling runs)")
     args = ap.parse_args()
     if args.warmup < 3:

@@ -40,7 +40,7 @@ struct DecodeArgs {
   int N, K, b, Br, Bc, entries, blocks_per_row;
   int m;              // index bits per lane and segment = 8 b / d
   int tile_cols;      // columns of a tile, a multiple of 256; the last tile of a row may be shorter
-  int bc_shift;       // log2(Bc) when Bc is a power of two, else -1
+  int bc_shift;       // log2(Bc): block columns are a power of two
   int br_per_tile;    // codebook block rows a tile touches
   int bc_per_tile;    // codebook block columns a tile touches
   int rows_per_br;    // tile rows that share a block row = min(Br, kTileRows)
@@ -117,29 +117,32 @@ __global__ void __launch_bounds__(32 * kWarps) decode_tile_kernel(const DecodeAr
     const uint32_t* row32 = reinterpret_cast<const uint32_t*>(a.idx + n * a.stride) + static_cast<long long>(col0 / 256) * m;
     const __half* row_tabs = tables + (r / a.rows_per_br) * a.bc_per_tile * table_halves;
     uint4* dst = reinterpret_cast<uint4*>(a.W + static_cast<long long>(n) * a.K + col0) + lane;
-    for (int s0 = 0; s0 < segs; s0 += kUnroll) {
+    // block-column table of the lane's 8 columns: constant per segment group for wide blocks,
+    // per-lane offset for blocks narrower than a segment
+    const int lane_cols = lane * 8;
+    auto emit = [&](int seg, uint32_t word_u) {
+      const uint32_t w0 = __shfl_sync(0xffffffffu, word_u, src_lane);
+      const uint32_t w1 = __shfl_sync(0xffffffffu, word_u, src_lane2);
+      const uint32_t v = __funnelshift_r(w0, w1, sh) & vmask;
+      const __half* tab = row_tabs + ((seg * 256 + lane_cols) >> a.bc_shift) * table_halves;
+      dst[seg * 32] = lookup8<D>(tab, v, a.b, emask);
+    };
+    int s0 = 0;
+    for (; s0 + kUnroll <= segs; s0 += kUnroll) {   // full groups: no per-segment predicates
       uint32_t word[kUnroll];
 #pragma unroll
-      for (int u = 0; u < kUnroll; ++u)
-        word[u] = (s0 + u < segs && lane < m) ? __ldg(row32 + (s0 + u) * m + lane) : 0u;
+      for (int u = 0; u < kUnroll; ++u) word[u] = lane < m ? __ldg(row32 + (s0 + u) * m + lane) : 0u;
 #pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        if (s0 + u >= segs) break;
-        const uint32_t w0 = __shfl_sync(0xffffffffu, word[u], src_lane);
-        const uint32_t w1 = __shfl_sync(0xffffffffu, word[u], src_lane2);
-        const uint32_t v = __funnelshift_r(w0, w1, sh) & vmask;
-        const int col = (s0 + u) * 256 + lane * 8;   // within the tile
-        const __half* tab = row_tabs + (a.bc_shift >= 0 ? col >> a.bc_shift : col / a.Bc) * table_halves;
-        dst[(s0 + u) * 32] = lookup8<D>(tab, v, a.b, emask);
-      }
+      for (int u = 0; u < kUnroll; ++u) emit(s0 + u, word[u]);
     }
+    for (; s0 < segs; ++s0) emit(s0, lane < m ? __ldg(row32 + s0 * m + lane) : 0u);
   }
 }
 
 }  // namespace
 
 // Formats the tile kernel covers: K a multiple of 256, at most 32 index bits per lane and segment
-// (8 b / d <= 32), block columns a multiple of 8 that divide or are divided by the tile's columns,
+// (8 b / d <= 32), block columns a power of two >= 8 that divide or are divided by the tile's columns,
 // block rows that divide or are divided by 32, tables of the tile within 96 KB of shared memory.
 vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s) {
   if (g.K % 256 || (8 * g.b) % g.d || 8 * g.b / g.d > 32 || g.Bc % 8) return VQ_ERR_UNSUPPORTED;
@@ -148,6 +151,7 @@ vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, 
   a.bc_shift = -1;
   for (int sft = 3; sft < 31; ++sft)
     if ((1 << sft) == g.Bc) a.bc_shift = sft;
+  if (a.bc_shift < 0) return VQ_ERR_UNSUPPORTED;
   if (a.tile_cols % g.Bc && g.Bc % a.tile_cols) return VQ_ERR_UNSUPPORTED;
   if (kTileRows % g.Br && g.Br % kTileRows) return VQ_ERR_UNSUPPORTED;
   a.idx = p.idx;
