@@ -50,6 +50,7 @@ struct RowArgs {
   int n_steps;          // K / STEP_COLS
   int steps_per_block;  // block_cols / STEP_COLS
   int blocks_per_row;   // K / block_cols
+  int Br;               // rows that share a codebook block (1 for per-row codebooks)
   int WR, WK;           // warps of a CTA: row tiles x K parts
   // dynamic shared memory, from its first 4096-byte boundary: warp-private tables, then the
   // activations (x_offset), then the reduction buffer (red_offset)
@@ -88,10 +89,10 @@ struct PrmtI8 {
     float sc[2];
 
     __device__ __forceinline__ void init(const RowArgs& a, int, int rl, int rh, int, uint32_t) {
-      cb_row[0] = a.cb + static_cast<long long>(rl) * a.blocks_per_row * CB_ROW_BYTES;
-      cb_row[1] = a.cb + static_cast<long long>(rh) * a.blocks_per_row * CB_ROW_BYTES;
-      sc_row[0] = a.scale + static_cast<long long>(rl) * a.blocks_per_row;
-      sc_row[1] = a.scale + static_cast<long long>(rh) * a.blocks_per_row;
+      cb_row[0] = a.cb + static_cast<long long>(rl / a.Br) * a.blocks_per_row * CB_ROW_BYTES;
+      cb_row[1] = a.cb + static_cast<long long>(rh / a.Br) * a.blocks_per_row * CB_ROW_BYTES;
+      sc_row[0] = a.scale + static_cast<long long>(rl / a.Br) * a.blocks_per_row;
+      sc_row[1] = a.scale + static_cast<long long>(rh / a.Br) * a.blocks_per_row;
     }
 
     uint4 raw[2];     // requested entries of the next block
@@ -164,11 +165,11 @@ struct LdsTbl {
     __device__ __forceinline__ void init(const RowArgs& a, int row0, int rl, int rh, int lane, uint32_t warp_tbl) {
       const int gb = lane & 7, tb = lane >> 3;
       const int b_lo = min(row0 + gb, a.N - 1), b_hi = min(row0 + gb + 8, a.N - 1);
-      cb_row[0] = a.cb + static_cast<long long>(b_lo) * a.blocks_per_row * CB_ROW_BYTES + tb * (CB_ROW_BYTES / 4);
-      cb_row[1] = a.cb + static_cast<long long>(b_hi) * a.blocks_per_row * CB_ROW_BYTES + tb * (CB_ROW_BYTES / 4);
+      cb_row[0] = a.cb + static_cast<long long>(b_lo / a.Br) * a.blocks_per_row * CB_ROW_BYTES + tb * (CB_ROW_BYTES / 4);
+      cb_row[1] = a.cb + static_cast<long long>(b_hi / a.Br) * a.blocks_per_row * CB_ROW_BYTES + tb * (CB_ROW_BYTES / 4);
       if constexpr (INT8) {
-        sc_row[0] = a.scale + static_cast<long long>(rl) * a.blocks_per_row;
-        sc_row[1] = a.scale + static_cast<long long>(rh) * a.blocks_per_row;
+        sc_row[0] = a.scale + static_cast<long long>(rl / a.Br) * a.blocks_per_row;
+        sc_row[1] = a.scale + static_cast<long long>(rh / a.Br) * a.blocks_per_row;
       }
       tbl = warp_tbl + lane * 4;
       fill = warp_tbl + (4 * tb) * 128 + gb * 16;   // entries 4tb..4tb+3, the 4 copies of row gb
@@ -600,6 +601,7 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
   a.n_steps = g.K / P::STEP_COLS;
   a.steps_per_block = g.Bc / P::STEP_COLS;
   a.blocks_per_row = g.blocks_per_row;
+  a.Br = g.Br;
   constexpr size_t kSmemBudget = 200 * 1024;
   const Plan pl = make_plan(g.N, a.n_steps, P::STEP_COLS, batch, sms_of[dev], P::TABLE_BYTES_PER_WARP, NB, kSmemBudget);
   const int T = pl.S * pl.WK;
@@ -656,10 +658,11 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
 
 }  // namespace
 
-// Per-row codebook families (block_rows == 1, 4-bit indices).
+// 4-bit families whose codebooks are looked up per row: block_rows == 1, or a few rows that share
+// a block (every lane then simply takes the entries of its own rows' block).
 vq_status launch_gemm_rowcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
                             cudaStream_t s) {
-  if (g.Br != 1 || g.b != 4) return VQ_ERR_UNSUPPORTED;
+  if (g.b != 4) return VQ_ERR_UNSUPPORTED;
   const bool nb1 = batch <= 8;
   if (g.cb_int8 && g.d == 1) return nb1 ? launch<PrmtI8, 1>(g, p, X, Y, batch, s) : launch<PrmtI8, 2>(g, p, X, Y, batch, s);
   if (g.cb_int8 && g.d == 2)

@@ -86,6 +86,12 @@ TALL_BLOCK_EXTRA = [
     vq_synth.LayerSpec("wb_d2b6_64x128", N=384, K=1024, d=2, b=6, Br=64, Bc=128, int8=False),
     vq_synth.LayerSpec("wb_d2b5_i8_32x256", N=128, K=4352, d=2, b=5, Br=32, Bc=256, int8=True),
     vq_synth.LayerSpec("wb_d2b5_32x128", N=256, K=768, d=2, b=5, Br=32, Bc=128, int8=False),
+    # 4-bit indices with a few rows per block (4 x 256 groups, Sec. 4.1): the row kernel, every lane
+    # taking its own rows' block
+    vq_synth.LayerSpec("rb_d2b4_4x256_i8", N=212, K=2048, d=2, b=4, Br=4, Bc=256, int8=True),
+    vq_synth.LayerSpec("rb_d2b4_4x256", N=64, K=4096, d=2, b=4, Br=4, Bc=256, int8=False),
+    vq_synth.LayerSpec("rb_d1b4_4x256_i8", N=132, K=1024, d=1, b=4, Br=4, Bc=256, int8=True),
+    vq_synth.LayerSpec("rb_d2b4_128x512", N=256, K=1024, d=2, b=4, Br=128, Bc=512, int8=False),
 ]
 
 
