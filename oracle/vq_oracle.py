@@ -224,5 +224,50 @@ def unpack_uniform(kind: str, src: np.ndarray, scale=None) -> np.ndarray:
     raise ValueError(kind)
 
 
+def assign(f: Fmt, W: np.ndarray, cb, scale=None, hdiag=None) -> np.ndarray:
+    """E-step / VQ_quant (Sec. 3, Eq. 5): for every d-vector x of W (d adjacent columns of one row)
+    the index m of the centroid of its block that minimises (x - c_m)^T D (x - c_m), D = the diagonal
+    weights of the vector's columns (hdiag[k] = 1 / [H^-1]_kk; None = identity, plain K-means).
+    Returns I[N][K/d] uint8.
+
+    The decision is taken in binary32, the arithmetic of the CUDA kernel, so that both sides break
+    near-ties alike: per coordinate t  diff = x_t - c_t,  sq = diff * diff,  term = D_t * sq, every
+    operation rounded to binary32, the terms added left to right; the lowest index wins among equal
+    distances.  int8 centroids are c = scale * c_int (exact in binary32)."""
+    W = np.ascontiguousarray(W, dtype=np.float16)
+    assert W.shape == (f.N, f.K)
+    e, d = f.entries, f.d
+    if f.int8:
+        C = np.asarray(cb, dtype=np.int8).reshape(f.n_blocks, e, d).astype(np.float32)
+        C = C * np.asarray(scale, dtype=np.float16).astype(np.float32).reshape(f.n_blocks, 1, 1)
+    else:
+        C = np.asarray(cb, dtype=np.float16).reshape(f.n_blocks, e, d).astype(np.float32)
+    D = np.ones(f.K, np.float32) if hdiag is None else np.ascontiguousarray(hdiag, dtype=np.float32)
+    assert D.shape == (f.K,)
+    I = np.empty((f.N, f.K // d), np.uint8)
+    bpr = f.K // f.Bc
+    for br in range(f.N // f.Br):
+        for bc in range(bpr):
+            r0, k0 = br * f.Br, bc * f.Bc
+            X = W[r0:r0 + f.Br, k0:k0 + f.Bc].astype(np.float32).reshape(f.Br, f.Bc // d, d)
+            Dv = D[k0:k0 + f.Bc].reshape(f.Bc // d, d)
+            Cb = C[br * bpr + bc]                                   # [e][d]
+            acc = None
+            for t in range(d):
+                diff = X[:, :, t, None] - Cb[None, None, :, t]       # binary32 throughout
+                term = Dv[None, :, t, None] * (diff * diff)
+                acc = term if acc is None else acc + term
+            assert acc.dtype == np.float32
+            I[r0:r0 + f.Br, k0 // d:(k0 + f.Bc) // d] = np.argmin(acc, axis=2)   # first minimum = lowest index
+    return I
+
+
+def sqnr_db(W: np.ndarray, Q: np.ndarray) -> float:
+    """Signal-to-quantization-noise ratio in dB (Sec. 2.2): 10 log10( E[W^2] / E[(W - Q)^2] )."""
+    W = np.asarray(W, dtype=np.float64)
+    Q = np.asarray(Q, dtype=np.float64)
+    return float(10.0 * np.log10(np.mean(W * W) / np.mean((W - Q) ** 2)))
+
+
 def hardware_threads() -> int:
     return _load().ref_hardware_threads()

@@ -440,3 +440,95 @@ def test_unpack_uniform_hand_values():
     w = np.array([[1.5, -0.0, 65504.0]], np.float16)
     assert np.array_equal(orc.unpack_uniform("fp16", w).view(np.uint16), w.view(np.uint16))
 
+
+# ---- E-step (Eq. 5) and SQNR (Sec. 2.2) ------------------------------------------------------------
+def _exact_assign(x, C, D):
+    """Brute force in exact rational arithmetic: all minimisers of sum_t D_t (x_t - c_mt)^2."""
+    from fractions import Fraction as Fr
+    dist = [sum(Fr(float(D[t])) * (Fr(float(x[t])) - Fr(float(c[t]))) ** 2 for t in range(len(x))) for c in C]
+    best = min(dist)
+    return [m for m, v in enumerate(dist) if v == best], dist
+
+
+@pytest.mark.parametrize("d,b,int8", [(1, 3, False), (2, 4, True), (2, 6, False), (4, 5, True)])
+def test_assign_is_an_exact_minimiser_or_a_rounding_tie(d, b, int8):
+    """Every index the oracle picks minimises the weighted distance exactly, or is within binary32
+    rounding (2^-20 relative) of the exact minimum; plain brute force with Fractions."""
+    spec = vq_synth.LayerSpec("e", N=8, K=16 * d, d=d, b=b, Br=4, Bc=8 * d, int8=int8)
+    f = orc.Fmt(spec.N, spec.K, d, b, spec.Br, spec.Bc, int8)
+    L = vq_synth.make_layer(spec, f.stride, 5)
+    W = (0.03 * vq_synth.normal(5, 40, spec.N * spec.K)).astype(np.float16).reshape(spec.N, spec.K)
+    h = (0.5 + vq_synth.uniform01(5, 41, spec.K)).astype(np.float32)
+    I = orc.assign(f, W, L.cb, L.scale, h)
+    assert I.shape == (spec.N, spec.K // d) and I.max() < (1 << b)
+    bpr = spec.K // spec.Bc
+    exact_hits = 0
+    for n in range(spec.N):
+        for j in range(spec.K // d):
+            blk = (n // spec.Br) * bpr + (j * d) // spec.Bc
+            C = L.cb[blk].astype(np.float64) * (float(L.scale[blk]) if int8 else 1.0)
+            mins, dist = _exact_assign(W[n, j * d:(j + 1) * d], C, h[j * d:(j + 1) * d])
+            if I[n, j] in mins:
+                exact_hits += 1
+            else:
+                assert float(dist[I[n, j]] - dist[mins[0]]) <= 2.0 ** -20 * float(dist[mins[0]])
+    assert exact_hits >= 0.99 * spec.N * (spec.K // d)
+
+
+def test_assign_identity_weights_is_nearest_centroid():
+    """D = I: the E-step is K-means' assignment (Sec. 3); scipy's vector quantiser is the library routine."""
+    from scipy.cluster.vq import vq as scipy_vq
+    spec = vq_synth.LayerSpec("km", N=16, K=64, d=2, b=4, Br=16, Bc=64, int8=False)
+    f = orc.Fmt(16, 64, 2, 4, 16, 64, False)
+    L = vq_synth.make_layer(spec, f.stride, 6)
+    W = (0.02 * vq_synth.normal(6, 40, 16 * 64)).astype(np.float16).reshape(16, 64)
+    I = orc.assign(f, W, L.cb, None, None)
+    code, _ = scipy_vq(W.astype(np.float64).reshape(-1, 2), L.cb[0].astype(np.float64))
+    # scipy decides in binary64: allow only disagreements that are binary32-level ties
+    diff = np.flatnonzero(code != I.reshape(-1))
+    X = W.astype(np.float64).reshape(-1, 2)
+    C = L.cb[0].astype(np.float64)
+    for i in diff:
+        da = ((X[i] - C[code[i]]) ** 2).sum()
+        db = ((X[i] - C[I.reshape(-1)[i]]) ** 2).sum()
+        assert abs(da - db) <= 2.0 ** -20 * da
+    assert diff.size <= 2
+
+
+def test_assign_special_cases():
+    # 1-D, centroids on a uniform grid: the E-step is round-to-nearest of x / step (Sec. 2.1 uniform quantizer)
+    f = orc.Fmt(2, 32, 1, 3, 1, 32, False)
+    grid = (np.arange(8) - 4) * 0.25
+    cb = np.tile(grid.astype(np.float16), (2, 1)).reshape(2, 8, 1)
+    W = np.linspace(-1.2, 0.9, 64).astype(np.float16).reshape(2, 32)
+    I = orc.assign(f, W, cb)
+    want = np.clip(np.floor(W.astype(np.float64) / 0.25 + 0.5), -4, 3) + 4     # half-way cases go up = lower |distance| tie -> check separately
+    ties = np.isclose((W.astype(np.float64) / 0.25) % 1.0, 0.5)
+    assert np.array_equal(I[~ties], want[~ties].astype(np.uint8))
+    # exact ties go to the lower index
+    assert orc.assign(orc.Fmt(1, 1, 1, 1, 1, 1, False), np.array([[0.5]], np.float16), np.array([[[0.0], [1.0]]], np.float16))[0, 0] == 0
+    # the weights matter: x = (1, 0) between c0 = (0, 0) and c1 = (1, 1); D = (1, 9) -> c0, D = (9, 1) -> c1
+    f2 = orc.Fmt(1, 2, 2, 1, 1, 2, False)
+    cb2 = np.array([[[0.0, 0.0], [1.0, 1.0]]], np.float16)
+    x = np.array([[1.0, 0.0]], np.float16)
+    assert orc.assign(f2, x, cb2, None, np.array([1.0, 9.0], np.float32))[0, 0] == 0
+    assert orc.assign(f2, x, cb2, None, np.array([9.0, 1.0], np.float32))[0, 0] == 1
+    # a weight that is itself a centroid maps to it; decode(pack(assign)) then returns the weight
+    f3 = orc.Fmt(4, 8, 2, 3, 2, 4, True)
+    spec3 = vq_synth.LayerSpec("rt", 4, 8, 2, 3, 2, 4, True)
+    L3 = vq_synth.make_layer(spec3, f3.stride, 8)
+    _, W16 = orc.decode(f3, L3.idx, L3.cb, L3.scale, exact=False)
+    Wq = W16.view(np.float16)
+    I3 = orc.assign(f3, Wq, L3.cb, L3.scale)
+    _, W16b = orc.decode(f3, orc.pack(f3, I3), L3.cb, L3.scale, exact=False)
+    assert np.array_equal(W16b, W16)          # idempotent: quantising a quantised matrix changes nothing
+
+
+def test_sqnr_closed_forms():
+    assert abs(orc.sqnr_db(np.array([1.0, -1.0]), np.array([0.5, -0.5])) - 10 * np.log10(4.0)) < 1e-12
+    # uniform quantizer with step q on a signal uniform in [-A, A]: noise power q^2/12, signal A^2/3
+    A, q = 1.0, 2.0 / 256
+    w = (np.arange(1 << 16) + 0.5) / (1 << 16) * 2 * A - A
+    qw = (np.floor(w / q) + 0.5) * q
+    assert abs(orc.sqnr_db(w, qw) - 10 * np.log10((A * A / 3) / (q * q / 12))) < 1e-3
+
