@@ -184,6 +184,23 @@ vq_status vq_int4g128_gemm_small_batch(int32_t n_rows, int32_t k_cols, const voi
                                        const void* d_scale, const void* d_X, void* d_Y,
                                        int batch, void* stream);
 
+/* E-step / VQ_quant of the quantizer (paper Sec. 3, Eq. 5; Algorithm 2's quantization step): for
+ * every d-vector x of the dense matrix W (d adjacent columns of one row) the index m of the centroid
+ * of its block that minimises (x - c_m)^T D (x - c_m), written in the packed index format above so
+ * that vq_decode_weights / vq_gemm_small_batch read the result directly.
+ *   d_W     : device binary16 [N][K].
+ *   d_cb, d_scale : the codebooks to assign to, layouts above.
+ *   d_hdiag : device binary32 [K], the diagonal of D (1 / [H^-1]_kk per column), or NULL for the
+ *             identity (plain nearest centroid).  16-byte aligned.
+ *   d_idx   : device, OUTPUT, N rows of row_stride_bytes; padding bytes are written as zero.
+ * The decision is taken in binary32, each operation rounded separately, terms added in column
+ * order; among equal distances the lowest index wins.
+ * Covered: formats with a whole number of 8-index groups per row (K / d % 8 == 0), block_cols a
+ * power of two >= 8 d, block_rows dividing or divided by 32; others return VQ_ERR_UNSUPPORTED.
+ * Errors: NULL, FORMAT, SHAPE, ALIGN, UNSUPPORTED, CUDA. */
+vq_status vq_assign_indices(const vq_format* fmt, const void* d_W, const void* d_cb,
+                            const void* d_scale, const void* d_hdiag, void* d_idx, void* stream);
+
 /* Uniformly quantized weights expanded to binary16: the yard-sticks of the transfer + decode
  * experiment (paper App. B: time to move and unpack a layer stored as FP16, INT8, INT4 or VQ),
  * timed beside vq_decode_weights.  w = s * q (Sec. 2.1), exact product rounded once to binary16.

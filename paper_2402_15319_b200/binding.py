@@ -78,6 +78,7 @@ _SIGNATURES = {
     "vq_gemm_small_batch_host_static": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p]),
     "vq_static_scratch_bytes": (ctypes.c_size_t, []),
     "vq_int4g128_gemm_small_batch": (ctypes.c_int, [ctypes.c_int32, ctypes.c_int32] + [ctypes.c_void_p] * 4 + [ctypes.c_int, ctypes.c_void_p]),
+    "vq_assign_indices": (ctypes.c_int, [ctypes.c_void_p] * 7),
     "vq_unpack_uniform": (ctypes.c_int, [ctypes.c_int, ctypes.c_int32, ctypes.c_int32] + [ctypes.c_void_p] * 4),
     "vq_device_wait_failures": (ctypes.c_int, [ctypes.c_void_p]),
     "vq_status_string": (ctypes.c_char_p, [ctypes.c_int]),
@@ -213,4 +214,11 @@ VQ_UNPACK_FP16, VQ_UNPACK_INT8_ROW, VQ_UNPACK_INT4_G128 = 0, 1, 2
 def vq_unpack_uniform(kind: int, n_rows: int, k_cols: int, d_src, d_scale, d_W, stream=None) -> None:
     _check(load().vq_unpack_uniform(int(kind), int(n_rows), int(k_cols), _ptr(d_src), _ptr(d_scale), _ptr(d_W),
                                     _stream(stream)), "vq_unpack_uniform")
+
+
+def vq_assign_indices(fmt: "VQFormat", d_W, d_cb, d_scale, d_hdiag, d_idx, stream=None) -> None:
+    """E-step (Eq. 5): nearest centroid under diagonal weights; writes the packed index stream d_idx."""
+    c = fmt.c()
+    _check(load().vq_assign_indices(ctypes.byref(c), _ptr(d_W), _ptr(d_cb), _ptr(d_scale), _ptr(d_hdiag), _ptr(d_idx),
+                                    _stream(stream)), "vq_assign_indices")
 

@@ -109,6 +109,18 @@ vq_status vq_decode_weights(const vq_format* fmt, const void* d_idx, const void*
   return st;
 }
 
+vq_status vq_assign_indices(const vq_format* fmt, const void* d_W, const void* d_cb, const void* d_scale,
+                            const void* d_hdiag, void* d_idx, void* stream) {
+  Geometry g;
+  LayerPtrs p;
+  vq_status st = check_layer(fmt, d_idx, d_cb, d_scale, &g, &p);   // d_idx: checked like an input, written here
+  if (st != VQ_OK) return st;
+  if (!d_W) return VQ_ERR_NULL;
+  if (!aligned16(d_W) || (d_hdiag && !aligned16(d_hdiag))) return VQ_ERR_ALIGN;
+  return launch_assign(g, p, static_cast<const __half*>(d_W), static_cast<const float*>(d_hdiag),
+                       static_cast<uint8_t*>(d_idx), static_cast<cudaStream_t>(stream));
+}
+
 vq_status vq_gemm_small_batch_impl(const vq_format* fmt, const void* d_idx, const void* d_cb,
                                    const void* d_scale, const void* d_X, void* d_Y, int batch,
                                    void* d_ws, size_t ws_bytes, void* stream, int impl) {

@@ -47,6 +47,9 @@ vq_status launch_gemm_rowcb(const Geometry& g, const LayerPtrs& p, const __half*
 vq_status launch_int4g128_rowcb(int N, int K, const uint8_t* q, const __half* scale, const __half* X, __half* Y, int batch,
                                 cudaStream_t s);
 vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s);
+// E-step: nearest centroid under diagonal weights, packed into the index stream `idx` (output).
+vq_status launch_assign(const Geometry& g, const LayerPtrs& p, const __half* W, const float* hdiag, uint8_t* idx,
+                        cudaStream_t s);
 
 // Device address of this device's counter of bounded waits that ran out inside a kernel (a copy
 // that never completed); looked up once per device.

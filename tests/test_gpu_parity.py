@@ -254,6 +254,55 @@ def test_unpack_uniform_bit_exact(N, K):
         vq.vq_unpack_uniform(vq.VQ_UNPACK_INT4_G128, N, K + 64, d_src, d_scale, d_W)   # K % 128
 
 
+ASSIGN_CASES = [
+    vq_synth.LayerSpec("as_d2b6", N=200, K=1024, d=2, b=6, Br=8, Bc=128, int8=False),
+    vq_synth.LayerSpec("as_d2b6_i8_32x256", N=96, K=2304, d=2, b=6, Br=32, Bc=256, int8=True),
+    vq_synth.LayerSpec("as_d1b3_1x256", N=37, K=768, d=1, b=3, Br=1, Bc=256, int8=False),
+    vq_synth.LayerSpec("as_d4b8", N=256, K=1024, d=4, b=8, Br=256, Bc=512, int8=False, cb_sigma=0.015),
+    vq_synth.LayerSpec("as_d2b4_i8_rows", N=130, K=4096, d=2, b=4, Br=1, Bc=2048, int8=True),
+    vq_synth.LayerSpec("as_d2b5", N=64, K=1280, d=2, b=5, Br=64, Bc=256, int8=False),
+]
+
+
+@pytest.mark.parametrize("weighted", [False, True])
+@pytest.mark.parametrize("spec", ASSIGN_CASES, ids=lambda s: s.name)
+def test_assign_indices_bit_exact(spec, weighted):
+    """E-step (Eq. 5): the packed index stream the library writes equals pack(assign) of the oracle,
+    byte for byte (padding included), and re-decoding it gives the oracle's quantized matrix."""
+    import torch
+    f = oracle_fmt(spec)
+    L = draw(spec, 31)
+    sigma = 0.02 if not spec.int8 else 0.1
+    W = (sigma * vq_synth.normal(31, 40, spec.N * spec.K)).astype(np.float16).reshape(spec.N, spec.K)
+    h = (0.25 + 2.0 * vq_synth.uniform01(31, 41, spec.K)).astype(np.float32) if weighted else None
+    want = orc.pack(f, orc.assign(f, W, L.cb, L.scale, h))
+    dev = DeviceLayer(spec, L)
+    d_W = torch.from_numpy(W).cuda()
+    d_h = None if h is None else torch.from_numpy(h).cuda()
+    d_idx = torch.full((spec.N, f.stride), 0xA5, dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        vq.vq_assign_indices(dev.fmt, d_W, dev.cb, dev.scale, d_h, d_idx)
+    torch.cuda.synchronize()
+    got = d_idx.cpu().numpy()
+    assert np.array_equal(got, want), f"{spec.name}: {np.count_nonzero(got != want)} bytes differ"
+    # the stream feeds the decode path: quantize -> decode is the oracle's Q(W); SQNR is finite and positive
+    dev.idx = d_idx
+    Q = dev.decode()
+    _, Q16 = orc.decode(f, want, L.cb, L.scale, exact=False)
+    assert np.array_equal(Q.view(np.uint16), Q16)
+    assert orc.sqnr_db(W, Q) > 0.0
+
+
+def test_assign_indices_rejects_what_it_does_not_cover():
+    import torch
+    spec = vq_synth.LayerSpec("as_bad", N=8, K=24, d=2, b=3, Br=1, Bc=12, int8=False)   # 12 indices per row
+    L = draw(spec, 1)
+    dev = DeviceLayer(spec, L)
+    d_W = torch.zeros((8, 24), dtype=torch.float16, device="cuda")
+    with pytest.raises(vq.VQError):
+        vq.vq_assign_indices(dev.fmt, d_W, dev.cb, dev.scale, None, dev.idx)
+
+
 def test_host_buffer_entry_point():
     import torch
     spec = vq_synth.LayerSpec("host", N=256, K=1024, d=2, b=6, Br=128, Bc=128, int8=False)
