@@ -409,6 +409,44 @@ def time_transfer_decode(device, torch, vq, N: int = 11008, K: int = 4096, reps:
     return {"layer": f"{N}x{K}", "output": "fp16 [N][K]", "rows": rows}
 
 
+def time_assign(device, torch, vq, cfg_name: str = "cfg3", N: int = 11008, K: int = 4096, reps: int = 5):
+    """E-step (Eq. 5) on a gate_proj-shaped dense matrix against the codebooks of a configuration's
+    format: us per call, vectors per second, and the arithmetic rate against the fp32 lanes of the
+    GPU (148 SMs x 128 lanes x SM clock, one operation per lane and clock)."""
+    t = vq_synth.CONFIGS[cfg_name]["layers"][0]
+    spec = vq_synth.LayerSpec("assign", N, K, t.d, t.b, t.Br, t.Bc, t.int8, cb_sigma=t.cb_sigma)
+    fmt = vq.VQFormat(N, K, spec.d, spec.b, spec.Br, spec.Bc, vq.VQ_CB_INT8_SCALED if spec.int8 else vq.VQ_CB_FP16)
+    info = vq.vq_pack_info(fmt)
+    L = vq_synth.make_layer(spec, info.row_stride_bytes, 22, 0)
+    W = (spec.cb_sigma * vq_synth.normal(22, 40, N * K)).astype(np.float16).reshape(N, K)
+    h = (0.25 + 2.0 * vq_synth.uniform01(22, 41, K)).astype(np.float32)
+    d_W, d_h = torch.from_numpy(W).to(device), torch.from_numpy(h).to(device)
+    cb = torch.from_numpy(L.cb).to(device)
+    sc = None if L.scale is None else torch.from_numpy(L.scale).to(device)
+    d_idx = torch.empty((N, info.row_stride_bytes), dtype=torch.uint8, device=device)
+    vq.vq_assign_indices(fmt, d_W, cb, sc, d_h, d_idx)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        vq.vq_assign_indices(fmt, d_W, cb, sc, d_h, d_idx)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / reps
+    Q = torch.empty((N, K), dtype=torch.float16, device=device)
+    vq.vq_decode_weights(fmt, d_idx, cb, sc, Q)
+    torch.cuda.synchronize()
+    err = (d_W.double() - Q.double()).pow(2).mean().item()
+    sqnr = 10.0 * np.log10(d_W.double().pow(2).mean().item() / err)
+    vectors = N * K // spec.d
+    ops = vectors * (1 << spec.b) * (4 * spec.d + 2)   # per (vector, centroid): d sub, 2d mul, d-1 add, compare, 2 selects
+    sm_mhz = torch.cuda.get_device_properties(device).clock_rate / 1e3 if hasattr(torch.cuda.get_device_properties(device), "clock_rate") else 1965.0
+    peak = 148 * 128 * sm_mhz * 1e6
+    return {"layer": f"{N}x{K}", "format": f"d={spec.d} b={spec.b} {spec.Br}x{spec.Bc}", "us": us,
+            "Gvectors_per_s": vectors / us / 1e3, "alu_ops_per_s": ops / us * 1e6, "alu_peak_ops_per_s": peak,
+            "alu_frac": ops / us * 1e6 / peak, "sqnr_db_random_codebook": sqnr}
+
+
 def time_decode(ds, reps: int = 3):
     """vq_decode_weights on the largest layer of the set: (us, GB/s over indices + codebooks + fp16 output)."""
     torch, vq = ds.torch, ds.vq
@@ -552,6 +590,7 @@ def run_ours(args):
                 torch.cuda.empty_cache()
         line["per_config"] = per
         line["transfer_decode"] = time_transfer_decode(dev, torch, vq)
+        line["assign"] = time_assign(dev, torch, vq)
     if rank == 0:
         print(json.dumps(line))
     if dist:
