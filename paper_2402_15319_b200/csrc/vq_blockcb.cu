@@ -36,6 +36,9 @@ using namespace dev;
 #define VQ_BLOCK_STAGES 3   // chunks of the index stream a warp keeps in flight
 #endif
 constexpr int kStages = VQ_BLOCK_STAGES;
+// Warp-private tables take 32 KB of a CTA's shared memory: two ring stages keep three CTAs on an SM.
+template <bool PRIV>
+constexpr int kStagesOf = PRIV ? 2 : kStages;
 constexpr int kWaitTries = 1 << 18;   // mbarrier polls before a warp gives up and flags an error
 
 struct BlockArgs {
@@ -301,6 +304,7 @@ template <int D, int B, int NB, bool PRIV>
 __global__ void __launch_bounds__(Tile<D, B>::THREADS)
 blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
   static_assert(!PRIV || D == 2, "warp-private tables exist for 2-D codebooks only");
+  constexpr int ST = kStagesOf<PRIV>;   // ring stages per warp
   using P = Policy<D, B>;
   using T = Tile<D, B>;
   constexpr int LW = P::LANE_WORDS;
@@ -315,7 +319,7 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
   // Receive barrier of the K-part reduction: S * rpo * batch values of 4 bytes arrive through
   // asynchronous remote stores.  Initialised before the start-up arrive so that every CTA of the
   // cluster sees it once its start-up wait (in front of the first remote store) returns.
-  const uint32_t recv_bar = base + a.bar_off + P::WARPS * kStages * 8;
+  const uint32_t recv_bar = base + a.bar_off + P::WARPS * ST * 8;
   if (S > 1) {
     if (tid == 0) {
       mbar_init(recv_bar, 1);
@@ -335,27 +339,27 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
   const int t0 = c0 / cpt, nt = n > 0 ? (c1 - 1) / cpt - t0 + 1 : 0;
 
   // ---- index ring: warp-private stages, one TMA box each ----
-  const uint32_t bars = base + a.bar_off + warp * kStages * 8;
-  const uint32_t ring = base + a.ring_off + warp * kStages * T::STAGE_BYTES;
+  const uint32_t bars = base + a.bar_off + warp * ST * 8;
+  const uint32_t ring = base + a.ring_off + warp * ST * T::STAGE_BYTES;
   if (lane == 0) {
-    for (int s = 0; s < kStages; ++s) mbar_init(bars + 8 * s, 1);
+    for (int s = 0; s < ST; ++s) mbar_init(bars + 8 * s, 1);
     mbar_init_fence();
   }
   __syncwarp();
   auto issue = [&](int i) {   // lane 0 only
-    const int st = i % kStages;
+    const int st = i % ST;
     mbar_arrive_expect_tx(bars + 8 * st, T::STAGE_BYTES);
     tma_box_2d(ring + st * T::STAGE_BYTES, &tm, (c0 + i) * P::SEG, row0 + 32 * warp, bars + 8 * st);
   };
   if (lane == 0)
-    for (int i = 0; i < kStages && i < n; ++i) issue(i);
+    for (int i = 0; i < ST && i < n; ++i) issue(i);
 
   // ---- first two codebook tables and the activations: all global loads are requested before any
   // of them is waited for ----
   unsigned char* compact = smem + a.compact_off;
   uint2 cb0 = make_uint2(0u, 0u), cb1 = cb0;
   PrivateRegs<PRIV ? B : 5> mine;   // PRIV: this warp's entries of the table that is written next
-  const uint32_t my_tables = base + (PRIV ? warp * 2 * P::TABLE_BYTES : 0);
+  const uint32_t my_tables = base + (PRIV ? warp * P::TABLE_BYTES : 0);   // PRIV: one table per warp
   if constexpr (PRIV) {
     if (n > 0) load_private<B>(mine, a, blk_row, c0, lane);
   } else {
@@ -447,8 +451,8 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
     }
 
     // ---- this warp's indices of the chunk ----
-    const int st = i % kStages;
-    if (!mbar_wait(bars + 8 * st, (i / kStages) & 1, kWaitTries) && lane == 0) atomicAdd(a.error_flag, 1);
+    const int st = i % ST;
+    if (!mbar_wait(bars + 8 * st, (i / ST) & 1, kWaitTries) && lane == 0) atomicAdd(a.error_flag, 1);
     uint32_t w[4][LW];
     const uint32_t src = ring + st * T::STAGE_BYTES + row_off;
 #pragma unroll
@@ -469,9 +473,9 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
       }
     }
     __syncwarp();   // every lane has read the stage: refill it
-    if (lane == 0 && i + kStages < n) {
+    if (lane == 0 && i + ST < n) {
       fence_proxy_async();
-      issue(i + kStages);
+      issue(i + ST);
     }
 
     // ---- activations of the lane's 64 columns -> B fragments ----
@@ -485,7 +489,7 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
       }
 
     // ---- look up + multiply-accumulate ----
-    uint32_t tbl = (my_tables + (k & 1) * P::TABLE_BYTES) | lane_off;
+    uint32_t tbl = (my_tables + (PRIV ? 0 : (k & 1) * P::TABLE_BYTES)) | lane_off;
     if constexpr (PRIV) fence_value(tbl);   // the gathers stay behind the warp's own table writes
     chunk_steps<D, B, NB, 0, 4>(acc, w, xr, tbl);
     chunk_steps<D, B, NB, 4, 4>(acc, w, xr, tbl);
@@ -493,11 +497,12 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
     chunk_steps<D, B, NB, 12, 4>(acc, w, xr, tbl);
 
     if constexpr (PRIV) {
-      // the warp's table for the next chunk goes into its other buffer (the previous chunk's, which
-      // only this warp read); the entries of the chunk after it are requested at once
+      // the warp's table for the next chunk replaces the one it has just finished with (only this
+      // warp reads it); the entries of the chunk after it are requested at once
       if (i + 1 < n) {
-        fence_acc(acc);   // this chunk's and the previous chunk's gathers are emitted before the writes
-        write_private<B>(my_tables + ((k + 1) & 1) * P::TABLE_BYTES, mine, a.scale != nullptr, lane);
+        fence_acc(acc);   // this chunk's gathers are emitted before the writes
+        __syncwarp();     // ... by every lane of the warp
+        write_private<B>(my_tables, mine, a.scale != nullptr, lane);
         if (i + 2 < n) load_private<B>(mine, a, blk_row, c + 2, lane);
         __syncwarp();
       }
@@ -599,10 +604,11 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
 
   // Shared memory of a CTA whose column range is `chunks` long.
   auto smem_for = [&](int chunks, BlockArgs* out) {
-    size_t off = (PRIV ? 2 * P::WARPS : 2) * static_cast<size_t>(P::TABLE_BYTES);
+    constexpr int ST = kStagesOf<PRIV>;
+    size_t off = (PRIV ? P::WARPS : 2) * static_cast<size_t>(P::TABLE_BYTES);
     const size_t compact_off = off; off += 2 * P::COMPACT_BYTES;
-    const size_t ring_off = round_up(off, 128); off = ring_off + static_cast<size_t>(P::WARPS) * kStages * T::STAGE_BYTES;
-    const size_t bar_off = off; off += static_cast<size_t>(P::WARPS) * kStages * 8 + 8;   // rings + receive barrier
+    const size_t ring_off = round_up(off, 128); off = ring_off + static_cast<size_t>(P::WARPS) * ST * T::STAGE_BYTES;
+    const size_t bar_off = off; off += static_cast<size_t>(P::WARPS) * ST * 8 + 8;   // rings + receive barrier
     const size_t x_off = round_up(off, 16); off = x_off + static_cast<size_t>(chunks) * 512 * batch;
     const size_t recv_off = round_up(off, 16); off = recv_off + static_cast<size_t>(T::CTA_ROWS) * 8 * NB * sizeof(float);
     if (out) {
