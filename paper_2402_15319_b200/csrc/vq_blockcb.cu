@@ -37,8 +37,18 @@ using namespace dev;
 #endif
 constexpr int kStages = VQ_BLOCK_STAGES;
 // Warp-private tables take 32 KB of a CTA's shared memory: two ring stages keep three CTAs on an SM.
-template <bool PRIV>
-constexpr int kStagesOf = PRIV ? 2 : kStages;
+#ifndef VQ_BLOCK_STAGES_D4
+#define VQ_BLOCK_STAGES_D4 2
+#endif
+#ifndef VQ_BLOCK_TB_D4
+#define VQ_BLOCK_TB_D4 1
+#endif
+template <int D, bool PRIV>
+constexpr int kStagesOf = PRIV ? 2 : (D == 4 ? VQ_BLOCK_STAGES_D4 : kStages);
+// Table buffers of the shared-table mode: 2 = the next table is replicated during the current one's
+// math; 1 = it replaces the current one between two block-wide barriers (saves TABLE_BYTES).
+template <int D>
+constexpr int kTableBuffers = D == 4 ? VQ_BLOCK_TB_D4 : 2;
 constexpr int kWaitTries = 1 << 18;   // mbarrier polls before a warp gives up and flags an error
 
 struct BlockArgs {
@@ -304,7 +314,7 @@ template <int D, int B, int NB, bool PRIV>
 __global__ void __launch_bounds__(Tile<D, B>::THREADS)
 blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
   static_assert(!PRIV || D == 2, "warp-private tables exist for 2-D codebooks only");
-  constexpr int ST = kStagesOf<PRIV>;   // ring stages per warp
+  constexpr int ST = kStagesOf<D, PRIV>;   // ring stages per warp
   using P = Policy<D, B>;
   using T = Tile<D, B>;
   constexpr int LW = P::LANE_WORDS;
@@ -446,7 +456,7 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
     uint2 vnext = make_uint2(0u, 0u);
     if constexpr (!PRIV) {
       if (fetch2) vnext = fetch_entry<D, B>(a, blk_row, (t0 + k + 2) * cpt, tid);
-      if (first_of_table && k + 1 < nt)
+      if (kTableBuffers<D> == 2 && first_of_table && k + 1 < nt)
         replicate<D, B>(base + ((k + 1) & 1) * P::TABLE_BYTES, compact + ((k + 1) & 1) * P::COMPACT_BYTES, tid);
     }
 
@@ -489,7 +499,8 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
       }
 
     // ---- look up + multiply-accumulate ----
-    uint32_t tbl = (my_tables + (PRIV ? 0 : (k & 1) * P::TABLE_BYTES)) | lane_off;
+    uint32_t tbl = (my_tables + (PRIV || kTableBuffers<D> == 1 ? 0 : (k & 1) * P::TABLE_BYTES)) | lane_off;
+    if constexpr (!PRIV && kTableBuffers<D> == 1) fence_value(tbl);
     if constexpr (PRIV) fence_value(tbl);   // the gathers stay behind the warp's own table writes
     chunk_steps<D, B, NB, 0, 4>(acc, w, xr, tbl);
     chunk_steps<D, B, NB, 4, 4>(acc, w, xr, tbl);
@@ -508,7 +519,14 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
       }
     } else {
       if (fetch2) store_compact<D, B>(compact + (k & 1) * P::COMPACT_BYTES, vnext, tid);
-      if (last_of_table && i != n - 1) __syncthreads();   // table k is done with, table k+1 complete
+      if (last_of_table && i != n - 1) {
+        if constexpr (kTableBuffers<D> == 1) {
+          fence_acc(acc);
+          __syncthreads();   // every warp has left table k
+          replicate<D, B>(base, compact + ((k + 1) & 1) * P::COMPACT_BYTES, tid);
+        }
+        __syncthreads();   // table k is done with, table k+1 complete
+      }
     }
   }
 
@@ -604,8 +622,8 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
 
   // Shared memory of a CTA whose column range is `chunks` long.
   auto smem_for = [&](int chunks, BlockArgs* out) {
-    constexpr int ST = kStagesOf<PRIV>;
-    size_t off = (PRIV ? P::WARPS : 2) * static_cast<size_t>(P::TABLE_BYTES);
+    constexpr int ST = kStagesOf<D, PRIV>;
+    size_t off = (PRIV ? P::WARPS : kTableBuffers<D>) * static_cast<size_t>(P::TABLE_BYTES);
     const size_t compact_off = off; off += 2 * P::COMPACT_BYTES;
     const size_t ring_off = round_up(off, 128); off = ring_off + static_cast<size_t>(P::WARPS) * ST * T::STAGE_BYTES;
     const size_t bar_off = off; off += static_cast<size_t>(P::WARPS) * ST * 8 + 8;   // rings + receive barrier
