@@ -121,6 +121,54 @@ def test_tuned_kernels_cover_every_benchmark_format(cfg):
         _check_layer(small, seed=conf["seed"], batches=conf["batches"], impls=[vq.VQ_IMPL_TUNED], decode=False)
 
 
+def _sweep_specs():
+    """Seeded draw of valid formats inside and around what the tuned kernels cover: block shapes,
+    index widths, codebook types, row counts with tails, column counts with short last chunks."""
+    rng = np.random.default_rng(20240229)
+    specs = []
+    for i in range(28):
+        fam = i % 4
+        if fam == 0:      # tall blocks, 2-D, 5/6 bits (shared or warp-private tables)
+            Br = int(rng.choice([32, 64, 128, 256])); Bc = int(rng.choice([128, 256, 512]))
+            N = Br * int(rng.integers(1, 4)) if Br >= 128 else 128 * int(rng.integers(1, 3))
+            K = Bc * int(rng.integers(1, 12)); K += (-K) % 256
+            K = K if K % Bc == 0 else Bc * (K // Bc + 1)
+            specs.append(vq_synth.LayerSpec(f"sw{i}", N, K, 2, int(rng.choice([5, 6])), Br, Bc, bool(rng.integers(2))))
+        elif fam == 1:    # 4-D 8-bit, 256-row blocks
+            Bc = int(rng.choice([256, 512, 1024]))
+            specs.append(vq_synth.LayerSpec(f"sw{i}", 256 * int(rng.integers(1, 3)), Bc * int(rng.integers(1, 7)), 4, 8, 256, Bc,
+                                            bool(rng.integers(2)), cb_sigma=0.015))
+        elif fam == 2:    # 4-bit, few rows per block (row kernel)
+            d = int(rng.choice([1, 2])); Br = int(rng.choice([1, 2, 4, 8])); Bc = int(rng.choice([256, 512, 1024, 2048]))
+            int8 = True if d == 1 else bool(rng.integers(2))
+            specs.append(vq_synth.LayerSpec(f"sw{i}", Br * int(rng.integers(3, 60)), Bc * int(rng.integers(1, 5)), d, 4, Br, Bc, int8))
+        else:             # anything valid: generic kernels (and the tuned decode / E-step where they apply)
+            d = int(rng.choice([1, 2, 4])); b = int(rng.integers(1, 9)); Br = int(rng.choice([1, 3, 16, 32]))
+            Bc = d * 8 * int(rng.choice([1, 4, 16, 32]))
+            specs.append(vq_synth.LayerSpec(f"sw{i}", Br * int(rng.integers(1, 9)), Bc * int(rng.integers(1, 6)), d, b, Br, Bc,
+                                            bool(rng.integers(2))))
+    return specs
+
+
+@pytest.mark.parametrize("spec", _sweep_specs(), ids=lambda s: f"{s.name}_{s.N}x{s.K}_d{s.d}b{s.b}_{s.Br}x{s.Bc}_{'i8' if s.int8 else 'f16'}")
+def test_randomized_format_sweep(spec):
+    batch = 1 + (spec.N + spec.K) % 16
+    _check_layer(spec, seed=spec.N + spec.K, batches=(1, batch))
+    # E-step on the same format where the kernel covers it: byte-exact stream
+    import torch
+    f = oracle_fmt(spec)
+    tables = (32 // spec.Br if spec.Br < 32 else 1) * max(1, 256 * spec.d // spec.Bc) * (1 << spec.b) * spec.d * 4   # bytes per tile
+    if ((spec.K // spec.d) % 8 == 0 and spec.Bc % (8 * spec.d) == 0 and (spec.Bc & (spec.Bc - 1)) == 0
+            and (32 % spec.Br == 0 or spec.Br % 32 == 0) and tables <= 96 * 1024):
+        L = draw(spec, spec.N + spec.K)
+        W = (0.05 * vq_synth.normal(spec.N, 40, spec.N * spec.K)).astype(np.float16).reshape(spec.N, spec.K)
+        dev = DeviceLayer(spec, L)
+        d_idx = torch.zeros((spec.N, f.stride), dtype=torch.uint8, device="cuda")
+        vq.vq_assign_indices(dev.fmt, torch.from_numpy(W).cuda(), dev.cb, dev.scale, None, d_idx)
+        torch.cuda.synchronize()
+        assert np.array_equal(d_idx.cpu().numpy(), orc.pack(f, orc.assign(f, W, L.cb, L.scale)))
+
+
 def test_no_wait_ran_out_inside_a_kernel():
     # bounded waits on asynchronous copies never expired in anything this process has run so far
     import torch
