@@ -530,7 +530,7 @@ int env_int(const char* name, int dflt) {
 
 // Choose the CTA shape (WR row tiles x WK column parts, at most 8 warps) and the cluster size S.
 // Model fitted to sweeps on B200: time ~ waves x (steps per warp + a fixed per-CTA overhead of
-// about 3 steps, 4 with a cluster), where a wave is as many CTAs as are co-resident (registers
+// about 3 steps, 4 with a cluster, + the CTA's activation staging), where a wave is as many CTAs as are co-resident (registers
 // allow about 16 warps per SM, 8 for the two-tile batch variant).  One wave of 8-warp CTAs with
 // as many column parts per CTA as possible wins; ties go to more column parts, then fewer CTAs
 // per cluster.  Shapes whose tables, activations and reduction buffer exceed smem_budget bytes of
@@ -556,12 +556,19 @@ Plan make_plan(int N, int n_steps, int step_cols, int batch, int sms, int tbl_pe
         if (per_sm < 1) per_sm = 1;
         const long long ctas = static_cast<long long>((row_tiles + WR - 1) / WR) * S;
         const long long slots = static_cast<long long>(per_sm) * sms;
-        const double waves = static_cast<double>((ctas + slots - 1) / slots);
+        // more CTAs than fit at once: between the work-conserving ratio and whole waves
+        const double ratio = static_cast<double>(ctas) / static_cast<double>(slots);
+        const double whole = static_cast<double>((ctas + slots - 1) / slots);
+        // (measured at batch 1 and 2; with more batch rows the staging of a late CTA is not hidden)
+        const double waves = batch <= 2 ? 0.5 * (ratio < 1.0 ? 2.0 : ratio + whole) : whole;
         const double steps = static_cast<double>(n_steps) / T;
+        // every CTA stages the activations of its whole column range: about a tenth of a step of
+        // work per staged step, shared by its warps
+        const double stage = batch <= 2 ? 0.1 * cta_steps / W : 0.0;
         // few resident warps hide latency badly
         const double resident = static_cast<double>(ctas < slots ? ctas : slots) * W / sms;
         const double slow = resident >= 8.0 ? 1.0 : 8.0 / (resident < 1.0 ? 1.0 : resident);
-        const double cost = waves * (steps * slow + (S > 1 ? 4.0 : 3.0));
+        const double cost = waves * (steps * slow + (S > 1 ? 4.0 : 3.0) + stage);
         if (best_cost < 0.0 || cost < best_cost) {
           best_cost = cost;
           best = {WR, WK, S};
