@@ -548,7 +548,7 @@ def run_ours(args):
         "clocks": sampler.summary(clock_src),
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": ds.h2d, "d2h_bytes_per_step": ds.d2h,
                 "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps,
-                "what": "vq_gemm_small_batch_host per layer: pinned-host activations copied in, kernel, outputs copied back, stream synchronised every step; compressed weights resident in HBM"},
+                "what": "vq_gemm_small_batch_host per layer: activations read from pinned host memory, kernel, outputs written back to pinned host memory, stream synchronised every step; compressed weights resident in HBM"},
         "gpu_launches": launches,
         "roofline": {
             "bound": "hbm", "kernel": KERNEL_OF.get(args.config, "vq gemm kernel") + " (one launch per layer)", "achieved": per_launch_gbs, "peak": peak,

@@ -137,7 +137,10 @@ vq_status vq_gemm_small_batch_impl(const vq_format* fmt, const void* d_idx, cons
  * device, runs vq_gemm_small_batch, copies Y back into h_Y (binary16 [batch][N]); all three
  * steps are enqueued on `stream` and the call returns without synchronising, so the caller
  * must synchronise the stream before reading h_Y.  Pinned host memory keeps the copies
- * asynchronous.  The compressed weights stay resident on the device (paper Sec. 1: every
+ * asynchronous; when both buffers are pinned (page-locked and mapped, as cudaHostAlloc and
+ * cudaHostRegister make them) and 16-byte aligned, a small kernel fetches X and the mat-vec
+ * kernel stores Y directly into h_Y instead of the two copies (same results, no hand-over to
+ * the copy engines).  The compressed weights stay resident on the device (paper Sec. 1: every
  * weight is read once per generated token; only activations cross the host boundary).
  *   d_ws must hold vq_workspace_bytes(fmt, batch) + 2*batch*(K+N) bytes rounded up to 256:
  *   use vq_workspace_bytes_host(fmt, batch).

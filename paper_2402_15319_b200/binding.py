@@ -4,6 +4,7 @@ streams are torch's); there is no CPU fallback — a missing library is an error
 from __future__ import annotations
 
 import ctypes
+import functools
 import os
 from dataclasses import dataclass
 
@@ -46,8 +47,13 @@ class VQFormat:
     cb_type: int
 
     def c(self) -> _CFormat:
-        return _CFormat(self.n_rows, self.k_cols, self.vq_dim, self.index_bits, self.block_rows,
-                        self.block_cols, self.cb_type)
+        return _c_format(self)
+
+
+@functools.lru_cache(maxsize=4096)
+def _c_format(f: "VQFormat") -> _CFormat:
+    # one struct per distinct format, reused by every call (the library only reads it)
+    return _CFormat(f.n_rows, f.k_cols, f.vq_dim, f.index_bits, f.block_rows, f.block_cols, f.cb_type)
 
 
 @dataclass(frozen=True)
@@ -117,14 +123,14 @@ def _check(code: int, where: str):
 
 
 def _ptr(t):
-    return None if t is None else ctypes.c_void_p(t.data_ptr())
+    return None if t is None else t.data_ptr()
 
 
 def _stream(stream):
     if stream is None:
         import torch
         stream = torch.cuda.current_stream()
-    return ctypes.c_void_p(stream.cuda_stream)
+    return stream.cuda_stream
 
 
 def vq_pack_info(fmt: VQFormat) -> PackInfo:

@@ -56,6 +56,22 @@ static vq_status check_layer(const vq_format* fmt, const void* d_idx, const void
 
 }  // namespace vq
 
+namespace {
+// Device-side address of a pinned (page-locked, mapped) host allocation, or null for any other memory.
+const void* mapped_device_pointer(const void* h) {
+  cudaPointerAttributes at;
+  if (cudaPointerGetAttributes(&at, h) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return nullptr;
+  }
+  return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+}
+// X from mapped host memory into device memory: 16-byte pieces, grid-stride.
+__global__ void __launch_bounds__(256) fetch_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int n16) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += gridDim.x * blockDim.x) dst[i] = src[i];
+}
+}  // namespace
+
 using namespace vq;
 
 extern "C" {
@@ -174,6 +190,24 @@ vq_status vq_gemm_small_batch_host(const vq_format* fmt, const void* d_idx, cons
   void* d_X = ws + base;
   void* d_Y = ws + base + round256(x_bytes);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // Pinned host buffers are mapped into the device's address space: one small kernel fetches X and
+  // the mat-vec kernel stores Y straight into host memory, so the step stays on the compute engine
+  // (two copy-engine hand-overs cost more than the kernel they surround).  Anything else (pageable
+  // memory, unaligned Y) takes the two asynchronous copies below.
+  {
+    const void* dx = mapped_device_pointer(h_X);
+    void* dy = const_cast<void*>(mapped_device_pointer(h_Y));
+    if (dx && dy && aligned16(dx) && aligned16(dy)) {
+      const int n16 = static_cast<int>(x_bytes / 16);
+      if (x_bytes % 16 == 0) {   // whole 16-byte pieces only
+        int blocks = (n16 + 255) / 256;
+        if (blocks > 8) blocks = 8;
+        fetch_kernel<<<blocks, 256, 0, s>>>(static_cast<const uint4*>(dx), static_cast<uint4*>(d_X), n16);
+        if (check_launch() != VQ_OK) return VQ_ERR_CUDA;
+        return vq_gemm_small_batch(fmt, d_idx, d_cb, d_scale, d_X, dy, batch, d_ws, base, stream);
+      }
+    }
+  }
   if (cudaMemcpyAsync(d_X, h_X, x_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return VQ_ERR_CUDA;
   st = vq_gemm_small_batch(fmt, d_idx, d_cb, d_scale, d_X, d_Y, batch, d_ws, base, stream);
   if (st != VQ_OK) return st;
