@@ -12,10 +12,12 @@
 // merged by one logic operation) and feeds the fp16 pairs, untouched, into mma.sync m16n8k16 as
 // the A fragment.  The activations of the CTA's column range are staged once in shared memory in
 // the order the lanes consume them (B fragment, batch row = g); accumulation is fp32.  Codebook
-// tables are double buffered: the next one is replicated while the current chunk is computed, its
-// entries fetched from global memory two tables ahead.  Partial sums of the K parts travel through
-// distributed shared memory to the cluster rank that owns the rows, are added in rank order,
-// rounded once to fp16 and stored.
+// tables are double buffered for 2-D formats (the next one is replicated while the current chunk
+// is computed, its entries fetched from global memory two tables ahead); the 32 KB tables of the
+// 4-D format use one buffer rewritten between two block-wide barriers, and blocks of 32 or 64 rows
+// one table per warp.  Partial sums of the K parts travel as asynchronous remote stores, counted
+// on an mbarrier, to the cluster rank that owns the rows, are added in rank order, rounded once to
+// fp16 and stored.
 // Paper: Sec. 3.2 (packed indices -> LUT -> mat-vec), App. A (Q is a look-up of C); the tiling,
 // the replication and the reduction are this library's.
 #include <cuda.h>
