@@ -100,7 +100,9 @@ struct Layer {
 };
 
 // Exact value of weight (n, k): Sec. 3.1 tuple + App. A look-up.  For int8 codebooks the
-// value is scale * c (Sec. 2.1 symmetric quantiser x ~ s * x_int), exact in fp64.
+// value is scale * c (Sec. 2.1 symmetric quantiser x ~ s * x_int), exact in fp64.  cb_int8: 0 = fp16
+// entries, 1 = int8 entries with one scale per block, 2 = int4 entries with one scale per row and
+// group of 128 columns.
 inline double weight_exact(const Layer& L, int n, int k) {
   const uint8_t* row = L.idx + static_cast<long long>(n) * L.stride;
   const int e = read_index(row, k / L.d, L.b);
@@ -108,9 +110,18 @@ inline double weight_exact(const Layer& L, int n, int k) {
   const long long blk = static_cast<long long>(n / L.Br) * blocks_per_row + (k / L.Bc);
   const long long entries = 1LL << L.b;
   const long long at = (blk * entries + e) * L.d + (k % L.d);
-  if (L.cb_int8) {
+  if (L.cb_int8 == 1) {
     const int8_t c = static_cast<const int8_t*>(L.cb)[at];
     return half_bits_to_double(L.scale[blk]) * static_cast<double>(c);
+  }
+  if (L.cb_int8 == 2) {
+    // INT4 codebook with "codebook quantization groups" of 128 values (Sec. 4.2, INT4 codebooks): the
+    // entry is a signed 4-bit integer (two nibbles per byte, low nibble first), the weight is that
+    // integer times the scale of its row's group of 128 columns
+    const uint8_t byte = static_cast<const uint8_t*>(L.cb)[at / 2];
+    const int nib = (at % 2) ? (byte >> 4) : (byte & 15);
+    const int c = nib >= 8 ? nib - 16 : nib;
+    return half_bits_to_double(L.scale[static_cast<long long>(n) * (L.K / 128) + k / 128]) * static_cast<double>(c);
   }
   return half_bits_to_double(static_cast<const uint16_t*>(L.cb)[at]);
 }

@@ -73,7 +73,7 @@ class Fmt:
     b: int
     Br: int
     Bc: int
-    int8: bool
+    int8: bool   # False: fp16 codebook; True: int8 codebook + scale per block; 2: int4 codebook + scale per row and 128 columns
 
     @property
     def entries(self) -> int:
@@ -138,6 +138,12 @@ def unpack(f: Fmt, idx: np.ndarray) -> np.ndarray:
 def _check_layer(f: Fmt, idx, cb, scale):
     idx = np.ascontiguousarray(idx, dtype=np.uint8)
     assert idx.size == f.N * f.stride
+    if int(f.int8) == 2:      # int4 codebook, scales per (row, 128-column group)
+        cb = np.ascontiguousarray(cb, dtype=np.uint8)
+        scale = _u16(scale)
+        assert f.K % 128 == 0 and scale.size == f.N * (f.K // 128)
+        assert cb.size == f.n_blocks * f.entries * f.d // 2
+        return idx, cb, scale
     if f.int8:
         cb = np.ascontiguousarray(cb, dtype=np.int8)
         scale = _u16(scale)
@@ -236,6 +242,7 @@ def assign(f: Fmt, W: np.ndarray, cb, scale=None, hdiag=None) -> np.ndarray:
     distances.  int8 centroids are c = scale * c_int (exact in binary32)."""
     W = np.ascontiguousarray(W, dtype=np.float16)
     assert W.shape == (f.N, f.K)
+    assert int(f.int8) != 2, "the E-step is defined here for fp16 and int8 codebooks"
     e, d = f.entries, f.d
     if f.int8:
         C = np.asarray(cb, dtype=np.int8).reshape(f.n_blocks, e, d).astype(np.float32)

@@ -532,3 +532,26 @@ def test_sqnr_closed_forms():
     qw = (np.floor(w / q) + 0.5) * q
     assert abs(orc.sqnr_db(w, qw) - 10 * np.log10((A * A / 3) / (q * q / 12))) < 1e-3
 
+
+def test_int4_codebook_with_group_scales_hand_values():
+    """INT4 codebooks decoded with a scale per row and group of 128 columns (Sec. 4.2): values by hand."""
+    f = orc.Fmt(2, 256, 2, 2, 2, 256, 2)            # one block, 4 entries of 2 nibbles, two groups per row
+    cb = np.array([[0x10, 0xF7, 0x8F, 0x23]], np.uint8)   # entries: (0,1) (7,-1) (-1,-8) (3,2)
+    I = np.zeros((2, 128), np.uint8)
+    I[0, 0], I[0, 1], I[0, 64], I[1, 127] = 1, 2, 3, 2
+    idx = orc.pack(f, I)
+    scale = np.array([[0.5, 2.0], [0.25, 3.0]], np.float16)
+    W, W16 = orc.decode(f, idx, cb, scale)
+    assert W[0, 0] == 3.5 and W[0, 1] == -0.5           # entry 1 = (7,-1), group 0 of row 0: x0.5
+    assert W[0, 2] == -0.5 and W[0, 3] == -4.0          # entry 2 = (-1,-8)
+    assert W[0, 4] == 0.0 and W[0, 5] == 0.5            # entry 0 = (0,1)
+    assert W[0, 128] == 6.0 and W[0, 129] == 4.0        # entry 3 = (3,2), group 1 of row 0: x2
+    assert W[1, 254] == -3.0 and W[1, 255] == -24.0     # row 1, group 1: x3
+    assert np.array_equal(W16.view(np.float16).astype(np.float64), W)   # all exactly representable here
+    # bits per value: 2/2 index + 4*2*4/512 codebook = 1.0625 (Sec. 4 formula, b_c = 4)
+    assert abs(orc.bpv(4, 2, 4, 512) - 1.0625) < 1e-12
+    # mat-vec = dense product on the decoded matrix
+    x = vq_synth.normal(3, 1, 256).astype(np.float16)
+    Y, A = orc.gemm(f, idx, cb, scale, x)
+    assert np.allclose(Y[0], W @ x.astype(np.float64), rtol=1e-14, atol=0)
+
