@@ -23,6 +23,7 @@
  *   codebook: cb[blk][entry][t], t < d; blk = (n / block_rows)*(K / block_cols) + (k / block_cols).
  *             VQ_CB_FP16: IEEE binary16.  VQ_CB_INT8_SCALED: signed 8-bit.
  *   scale   : VQ_CB_INT8_SCALED only: one binary16 per block, w = scale * int8.
+ *             (VQ_CB_INT4_G128: 4-bit entries and a scale per row and 128 columns, described at vq_cb_type.)
  *   x / X   : activations, binary16, X[batch][K] row-major.
  *   y / Y   : outputs, binary16, Y[batch][N] row-major; accumulated in fp32, rounded once.
  *
@@ -56,7 +57,17 @@ typedef enum {
   VQ_ERR_CUDA = 8         /* a CUDA runtime call or the launch itself reported an error                 */
 } vq_status;
 
-typedef enum { VQ_CB_FP16 = 0, VQ_CB_INT8_SCALED = 1 } vq_cb_type;
+/* VQ_CB_INT4_G128 (paper Sec. 4.2, "INT4 codebooks" with codebook quantization groups of 128 values):
+ *   d_cb    : per block 2^index_bits * vq_dim signed 4-bit integers (-8..7), two per byte, value
+ *             v = entry * vq_dim + t in nibble v mod 2 (low nibble first) of byte v / 2;
+ *   d_scale : binary16 [N][K/128]; w[n][k] = scale[n][k/128] * c.  K % 128 == 0.
+ * Served by the format-generic kernels (decode and skinny GEMM); the tuned kernels and
+ * vq_assign_indices do not take it. */
+typedef enum {
+  VQ_CB_FP16 = 0,         /* binary16 entries                                                        */
+  VQ_CB_INT8_SCALED = 1,  /* signed 8-bit entries, one binary16 scale per block                       */
+  VQ_CB_INT4_G128 = 2     /* signed 4-bit entries, one binary16 scale per row and group of 128 columns */
+} vq_cb_type;
 
 /* Kernel selection for the *_impl entry points.  VQ_IMPL_AUTO is what the plain entry points use. */
 typedef enum {

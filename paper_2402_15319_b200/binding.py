@@ -8,7 +8,7 @@ import functools
 import os
 from dataclasses import dataclass
 
-VQ_CB_FP16, VQ_CB_INT8_SCALED = 0, 1
+VQ_CB_FP16, VQ_CB_INT8_SCALED, VQ_CB_INT4_G128 = 0, 1, 2
 VQ_IMPL_AUTO, VQ_IMPL_GENERIC, VQ_IMPL_TUNED = 0, 1, 2
 
 _PKG = os.path.dirname(os.path.abspath(__file__))

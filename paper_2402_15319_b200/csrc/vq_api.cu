@@ -11,9 +11,10 @@ static vq_status check_format(const vq_format* f) {
   if (!f) return VQ_ERR_NULL;
   if (!(f->vq_dim == 1 || f->vq_dim == 2 || f->vq_dim == 4)) return VQ_ERR_FORMAT;
   if (f->index_bits < 1 || f->index_bits > 8) return VQ_ERR_FORMAT;
-  if (!(f->cb_type == VQ_CB_FP16 || f->cb_type == VQ_CB_INT8_SCALED)) return VQ_ERR_FORMAT;
+  if (!(f->cb_type == VQ_CB_FP16 || f->cb_type == VQ_CB_INT8_SCALED || f->cb_type == VQ_CB_INT4_G128)) return VQ_ERR_FORMAT;
   if (f->n_rows <= 0 || f->k_cols <= 0 || f->block_rows <= 0 || f->block_cols <= 0) return VQ_ERR_SHAPE;
   if (f->n_rows % f->block_rows || f->k_cols % f->block_cols || f->block_cols % f->vq_dim) return VQ_ERR_SHAPE;
+  if (f->cb_type == VQ_CB_INT4_G128 && f->k_cols % 128) return VQ_ERR_SHAPE;
   return VQ_OK;
 }
 
@@ -32,6 +33,7 @@ vq_status make_geometry(const vq_format* f, Geometry* g) {
   g->Br = f->block_rows;
   g->Bc = f->block_cols;
   g->cb_int8 = f->cb_type == VQ_CB_INT8_SCALED;
+  g->cb_int4 = f->cb_type == VQ_CB_INT4_G128;
   g->entries = 1 << f->index_bits;
   g->J = f->k_cols / f->vq_dim;
   g->blocks_per_row = f->k_cols / f->block_cols;
@@ -46,7 +48,7 @@ static vq_status check_layer(const vq_format* fmt, const void* d_idx, const void
   vq_status st = make_geometry(fmt, g);
   if (st != VQ_OK) return st;
   if (!d_idx || !d_cb) return VQ_ERR_NULL;
-  if (g->cb_int8 ? d_scale == nullptr : d_scale != nullptr) return VQ_ERR_NULL;
+  if ((g->cb_int8 || g->cb_int4) ? d_scale == nullptr : d_scale != nullptr) return VQ_ERR_NULL;
   if (!aligned16(d_idx) || !aligned16(d_cb) || !aligned16(d_scale)) return VQ_ERR_ALIGN;
   p->idx = static_cast<const uint8_t*>(d_idx);
   p->cb = d_cb;
@@ -82,7 +84,7 @@ vq_status vq_pack_info(const vq_format* fmt, vq_pack_info_t* out) {
   if (st != VQ_OK) return st;
   const long long N = fmt->n_rows, K = fmt->k_cols, d = fmt->vq_dim;
   const long long k = 1LL << fmt->index_bits;
-  const int b_c = fmt->cb_type == VQ_CB_INT8_SCALED ? 8 : 16;
+  const int b_c = fmt->cb_type == VQ_CB_INT8_SCALED ? 8 : fmt->cb_type == VQ_CB_INT4_G128 ? 4 : 16;
   const long long l = static_cast<long long>(fmt->block_rows) * fmt->block_cols;
   out->entries = static_cast<int32_t>(k);
   out->codebook_bits = b_c;
@@ -92,7 +94,7 @@ vq_status vq_pack_info(const vq_format* fmt, vq_pack_info_t* out) {
   out->n_blocks = (N / fmt->block_rows) * (K / fmt->block_cols);
   out->codebook_bytes_per_block = k * d * b_c / 8;
   out->codebook_bytes = out->n_blocks * out->codebook_bytes_per_block;
-  out->scale_bytes = fmt->cb_type == VQ_CB_INT8_SCALED ? 2 * out->n_blocks : 0;
+  out->scale_bytes = fmt->cb_type == VQ_CB_INT8_SCALED ? 2 * out->n_blocks : fmt->cb_type == VQ_CB_INT4_G128 ? 2 * N * (K / 128) : 0;
   out->total_bytes = out->index_bytes + out->codebook_bytes + out->scale_bytes;
   out->bpv_paper = static_cast<double>(fmt->index_bits) / d + static_cast<double>(k * d * b_c) / static_cast<double>(l);
   out->bpv_stored = 8.0 * static_cast<double>(out->total_bytes) / static_cast<double>(N * K);

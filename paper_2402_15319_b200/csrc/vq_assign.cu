@@ -131,7 +131,7 @@ __global__ void __launch_bounds__(32 * kWarps) assign_kernel(const AssignArgs a)
 vq_status launch_assign(const Geometry& g, const LayerPtrs& p, const __half* W, const float* hdiag, uint8_t* idx,
                         cudaStream_t s) {
   const int seg_cols = 256 * g.d;
-  if (g.J % 8 || g.Bc % (8 * g.d)) return VQ_ERR_UNSUPPORTED;
+  if (g.cb_int4 || g.J % 8 || g.Bc % (8 * g.d)) return VQ_ERR_UNSUPPORTED;
   int bc_shift = -1;
   for (int sft = 3; sft < 31; ++sft)
     if ((1 << sft) == g.Bc) bc_shift = sft;

@@ -14,6 +14,7 @@ namespace vq {
 struct Geometry {
   int N, K, d, b, Br, Bc;
   int cb_int8;            // 0: fp16 codebook, 1: int8 codebook + fp16 block scale
+  int cb_int4;            // 1: int4 codebook + fp16 scale per row and group of 128 columns (cb_int8 is 0 then)
   int entries;            // 2^b
   int J;                  // indices per row = K/d
   int blocks_per_row;     // K/Bc

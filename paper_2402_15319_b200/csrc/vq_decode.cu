@@ -145,7 +145,7 @@ __global__ void __launch_bounds__(32 * kWarps) decode_tile_kernel(const DecodeAr
 // (8 b / d <= 32), block columns a power of two >= 8 that divide or are divided by the tile's columns,
 // block rows that divide or are divided by 32, tables of the tile within 96 KB of shared memory.
 vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s) {
-  if (g.K % 256 || (8 * g.b) % g.d || 8 * g.b / g.d > 32 || g.Bc % 8) return VQ_ERR_UNSUPPORTED;
+  if (g.cb_int4 || g.K % 256 || (8 * g.b) % g.d || 8 * g.b / g.d > 32 || g.Bc % 8) return VQ_ERR_UNSUPPORTED;
   DecodeArgs a;
   a.tile_cols = g.K < kTileCols ? g.K : kTileCols;
   a.bc_shift = -1;

@@ -21,8 +21,14 @@ __device__ __forceinline__ unsigned long long load_group_bits(const uint8_t* row
 
 // One codebook value as fp32; for int8 codebooks scale*c, exact in fp32 (App. A look-up,
 // Sec. 3.1 scale factor).
-__device__ __forceinline__ float lut_value(const Geometry& g, const LayerPtrs& p, long long blk, int e, int t) {
+// int4 codebooks: scale of row n's group of 128 columns times the signed nibble, exact in fp32.
+__device__ __forceinline__ float lut_value(const Geometry& g, const LayerPtrs& p, long long blk, int e, int t, int n, int k) {
   const long long at = (blk * g.entries + e) * g.d + t;
+  if (g.cb_int4) {
+    const uint8_t byte = static_cast<const uint8_t*>(p.cb)[at >> 1];
+    const int nib = (at & 1) ? (byte >> 4) : (byte & 15);
+    return __half2float(p.scale[static_cast<long long>(n) * (g.K / 128) + k / 128]) * static_cast<float>(nib >= 8 ? nib - 16 : nib);
+  }
   if (g.cb_int8) {
     const float c = static_cast<float>(static_cast<const int8_t*>(p.cb)[at]);
     return __half2float(p.scale[blk]) * c;
@@ -48,8 +54,8 @@ __global__ void decode_generic_kernel(Geometry g, LayerPtrs p, __half* __restric
       const long long blk = blk_row + k0 / g.Bc;
       for (int t = 0; t < g.d; ++t) {
         __half h;
-        if (g.cb_int8) {
-          h = __float2half_rn(lut_value(g, p, blk, e, t));
+        if (g.cb_int8 || g.cb_int4) {
+          h = __float2half_rn(lut_value(g, p, blk, e, t, n, k0 + t));
         } else {
           h = static_cast<const __half*>(p.cb)[(blk * g.entries + e) * g.d + t];  // bit copy
         }
@@ -127,7 +133,7 @@ __global__ void __launch_bounds__(256) gemm_generic_kernel(Geometry g, LayerPtrs
         const int k0 = j * g.d;
         const long long blk = blk_row + k0 / g.Bc;
         for (int t = 0; t < g.d; ++t) {
-          const float w = lut_value(g, p, blk, e, t);
+          const float w = lut_value(g, p, blk, e, t, n, k0 + t);
 #pragma unroll
           for (int m = 0; m < MB; ++m)
             if (m < batch) acc[m] = fmaf(w, __half2float(__ldg(X + static_cast<long long>(m) * g.K + k0 + t)), acc[m]);
@@ -147,7 +153,7 @@ __global__ void __launch_bounds__(256) gemm_generic_kernel(Geometry g, LayerPtrs
 }  // namespace
 
 vq_status launch_decode_generic(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s) {
-  if (g.J % 8 == 0) {   // K % 8 == 0 follows: every 128-bit store is aligned
+  if (g.J % 8 == 0 && !g.cb_int4) {   // K % 8 == 0 follows: every 128-bit store is aligned
     const long long total = static_cast<long long>(g.N) * (g.J / 8);
     long long blocks = (total + 255) / 256;
     if (blocks > 148LL * 32) blocks = 148LL * 32;

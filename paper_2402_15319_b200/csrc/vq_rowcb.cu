@@ -746,7 +746,7 @@ vq_status launch_int4g128_rowcb(int N, int K, const uint8_t* q, const __half* sc
   if (K % 128) return VQ_ERR_UNSUPPORTED;
   Geometry g = {};
   g.N = N; g.K = K; g.d = 1; g.b = 4; g.Br = 1; g.Bc = 128;
-  g.cb_int8 = 1; g.entries = 16; g.J = K; g.blocks_per_row = K / 128; g.stride = K / 2;
+  g.cb_int8 = 1; g.cb_int4 = 0; g.entries = 16; g.J = K; g.blocks_per_row = K / 128; g.stride = K / 2;
   LayerPtrs p;
   p.idx = q;
   p.cb = nullptr;

@@ -42,7 +42,7 @@ extern "C" vq_status vq_gemm_small_batch_host_static(const vq_format* fmt, const
   vq_status st = make_geometry(fmt, &g);
   if (st != VQ_OK) return st;
   if (!d_idx || !d_cb || !h_X || !h_Y) return VQ_ERR_NULL;
-  if (g.cb_int8 ? d_scale == nullptr : d_scale != nullptr) return VQ_ERR_NULL;
+  if ((g.cb_int8 || g.cb_int4) ? d_scale == nullptr : d_scale != nullptr) return VQ_ERR_NULL;
   if ((reinterpret_cast<uintptr_t>(d_idx) | reinterpret_cast<uintptr_t>(d_cb) | reinterpret_cast<uintptr_t>(d_scale)) & 15u)
     return VQ_ERR_ALIGN;
   if (batch < 1 || batch > 16) return VQ_ERR_BATCH;

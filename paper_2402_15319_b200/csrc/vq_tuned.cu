@@ -49,6 +49,7 @@ vq_status device_error_counter(int** d_counter) {
 vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch, float* ws,
                             cudaStream_t s) {
   (void)ws;
+  if (g.cb_int4) return VQ_ERR_UNSUPPORTED;   // int4 codebooks: format-generic kernels only
   vq_status st = launch_gemm_blockcb(g, p, X, Y, batch, s);
   if (st != VQ_ERR_UNSUPPORTED) return st;
   return launch_gemm_rowcb(g, p, X, Y, batch, s);

@@ -16,7 +16,7 @@ def oracle_fmt(spec: vq_synth.LayerSpec) -> orc.Fmt:
 def lib_fmt(spec: vq_synth.LayerSpec):
     import paper_2402_15319_b200 as vq
     return vq.VQFormat(spec.N, spec.K, spec.d, spec.b, spec.Br, spec.Bc,
-                       vq.VQ_CB_INT8_SCALED if spec.int8 else vq.VQ_CB_FP16)
+                       vq.VQ_CB_INT4_G128 if int(spec.int8) == 2 else vq.VQ_CB_INT8_SCALED if spec.int8 else vq.VQ_CB_FP16)
 
 
 def draw(spec: vq_synth.LayerSpec, seed: int, layer_id: int = 0) -> vq_synth.Layer:

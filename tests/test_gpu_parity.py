@@ -351,6 +351,27 @@ def test_assign_indices_rejects_what_it_does_not_cover():
         vq.vq_assign_indices(dev.fmt, d_W, dev.cb, dev.scale, None, dev.idx)
 
 
+INT4_CODEBOOK_CASES = [
+    vq_synth.LayerSpec("i4cb_d2b3", N=64, K=1024, d=2, b=3, Br=32, Bc=256, int8=2),
+    vq_synth.LayerSpec("i4cb_d2b6", N=37, K=256, d=2, b=6, Br=37, Bc=128, int8=2),
+    vq_synth.LayerSpec("i4cb_d1b4", N=20, K=384, d=1, b=4, Br=4, Bc=96, int8=2),
+    vq_synth.LayerSpec("i4cb_d4b8", N=16, K=1280, d=4, b=8, Br=16, Bc=640, int8=2),
+]
+
+
+@pytest.mark.parametrize("spec", INT4_CODEBOOK_CASES, ids=lambda s: s.name)
+def test_int4_codebooks_with_group_scales(spec):
+    """INT4 codebooks decoded with a scale per row and group of 128 columns (Sec. 4.2): bit-exact
+    decode, mat-vec within the tolerance, through the format-generic kernels (the only ones that take
+    this codebook type: VQ_IMPL_TUNED must refuse it)."""
+    _check_layer(spec, seed=55, batches=(1, 5, 16), impls=[vq.VQ_IMPL_GENERIC, vq.VQ_IMPL_AUTO])
+    L = draw(spec, 55)
+    dev = DeviceLayer(spec, L)
+    with pytest.raises(vq.VQError) as err:
+        dev.gemm(vq_synth.make_x(spec, 1, 1), vq.VQ_IMPL_TUNED)
+    assert err.value.code == 7
+
+
 def test_host_buffer_entry_point():
     import torch
     spec = vq_synth.LayerSpec("host", N=256, K=1024, d=2, b=6, Br=128, Bc=128, int8=False)

@@ -84,7 +84,7 @@ def _replace(fmt, **kw):
 
 @pytest.mark.parametrize("kw,code", [
     (dict(vq_dim=3), 2), (dict(vq_dim=0), 2), (dict(index_bits=0), 2), (dict(index_bits=9), 2),
-    (dict(cb_type=2), 2), (dict(n_rows=0), 3), (dict(k_cols=-4), 3), (dict(block_rows=3), 3),
+    (dict(cb_type=3), 2), (dict(cb_type=-1), 2), (dict(n_rows=0), 3), (dict(k_cols=-4), 3), (dict(block_rows=3), 3),
     (dict(block_cols=5), 3), (dict(block_cols=0), 3), (dict(vq_dim=4, block_cols=2, k_cols=16), 3),
 ])
 def test_bad_formats_rejected(kw, code):
@@ -145,3 +145,19 @@ def test_missing_library_is_an_error(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "_LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError, match="missing"):
         binding.load()
+
+
+def test_pack_info_int4_codebook_with_group_scales():
+    """INT4 codebooks (Sec. 4.2): 4 bits per codebook value, one binary16 scale per row and 128 columns."""
+    f = vq.VQFormat(256, 1024, 2, 3, 32, 256, vq.VQ_CB_INT4_G128)
+    info = vq.vq_pack_info(f)
+    assert info.codebook_bits == 4 and info.entries == 8
+    assert info.codebook_bytes_per_block == 8 * 2 // 2
+    assert info.n_blocks == (256 // 32) * (1024 // 256)
+    assert info.scale_bytes == 2 * 256 * (1024 // 128)
+    assert info.total_bytes == info.index_bytes + info.codebook_bytes + info.scale_bytes
+    assert abs(info.bpv_paper - (3 / 2 + 8 * 2 * 4 / (32 * 256))) < 1e-12
+    with pytest.raises(vq.VQError) as e:          # K must hold whole groups of 128 columns
+        vq.vq_pack_info(vq.VQFormat(256, 1024 + 64, 2, 3, 32, 32, vq.VQ_CB_INT4_G128))
+    assert e.value.code == 3
+

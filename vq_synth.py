@@ -64,7 +64,7 @@ class LayerSpec:
     b: int          # index bits
     Br: int         # block rows
     Bc: int         # block cols
-    int8: bool      # int8 codebook with one fp16 scale per block, else fp16 codebook
+    int8: bool      # int8 codebook with one fp16 scale per block, else fp16 codebook; 2 = int4 codebook, scale per row and 128 columns
     cb_sigma: float = 0.02                 # fp16 codebook entries ~ N(0, sigma^2)
     scale_range: tuple = (0.0005, 0.002)   # int8: block scale ~ U(lo, hi)
 
@@ -97,7 +97,10 @@ def make_layer(spec: LayerSpec, stride: int, seed: int, layer_id: int = 0) -> La
     s0 = 16 * layer_id
     idx = random_bytes(seed, s0 + 1, spec.N * stride).reshape(spec.N, stride)
     n_cb = spec.n_blocks * spec.entries * spec.d
-    if spec.int8:
+    if int(spec.int8) == 2:   # int4 codebook (two nibbles per byte), scale per row and group of 128 columns
+        cb = random_bytes(seed, s0 + 2, n_cb // 2).reshape(spec.n_blocks, spec.entries * spec.d // 2)
+        scale = (0.001 + 0.003 * uniform01(seed, s0 + 3, spec.N * (spec.K // 128))).astype(np.float16).reshape(spec.N, spec.K // 128)
+    elif spec.int8:
         cb = (raw_u64(seed, s0 + 2, n_cb) % np.uint64(255)).astype(np.int64) - 127
         cb = cb.astype(np.int8).reshape(spec.n_blocks, spec.entries, spec.d)
         lo, hi = spec.scale_range
