@@ -61,8 +61,8 @@ typedef enum {
  *   d_cb    : per block 2^index_bits * vq_dim signed 4-bit integers (-8..7), two per byte, value
  *             v = entry * vq_dim + t in nibble v mod 2 (low nibble first) of byte v / 2;
  *   d_scale : binary16 [N][K/128]; w[n][k] = scale[n][k/128] * c.  K % 128 == 0.
- * Served by the format-generic kernels (decode and skinny GEMM); the tuned kernels and
- * vq_assign_indices do not take it. */
+ * vq_decode_weights decodes it with its tile kernel; the skinny GEMM runs in the format-generic
+ * kernel (VQ_IMPL_TUNED returns VQ_ERR_UNSUPPORTED); vq_assign_indices does not take it. */
 typedef enum {
   VQ_CB_FP16 = 0,         /* binary16 entries                                                        */
   VQ_CB_INT8_SCALED = 1,  /* signed 8-bit entries, one binary16 scale per block                       */

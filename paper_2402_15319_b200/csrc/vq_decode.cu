@@ -35,6 +35,7 @@ struct DecodeArgs {
   const uint8_t* idx;
   const void* cb;
   const __half* scale;
+  const __half* row_scale;   // int4 codebooks: [N][K/128] scales applied after the look-up, else null
   __half* W;
   long long stride;
   int N, K, b, Br, Bc, entries, blocks_per_row;
@@ -94,7 +95,12 @@ __global__ void __launch_bounds__(32 * kWarps) decode_tile_kernel(const DecodeAr
       if (bcol >= a.blocks_per_row) bcol = a.blocks_per_row - 1;   // short last tile: never looked up
       const long long blk = brow * a.blocks_per_row + bcol;
       __half v;
-      if (a.scale == nullptr) {
+      if (a.row_scale != nullptr) {   // signed nibble, kept unscaled (exact in fp16)
+        const long long at = blk * table_halves + within;
+        const uint8_t byte = __ldg(static_cast<const uint8_t*>(a.cb) + (at >> 1));
+        const int nib = (at & 1) ? (byte >> 4) : (byte & 15);
+        v = __int2half_rn(nib >= 8 ? nib - 16 : nib);
+      } else if (a.scale == nullptr) {
         v = __ldg(static_cast<const __half*>(a.cb) + blk * table_halves + within);
       } else {
         const float c = static_cast<float>(__ldg(static_cast<const int8_t*>(a.cb) + blk * table_halves + within));
@@ -125,7 +131,18 @@ __global__ void __launch_bounds__(32 * kWarps) decode_tile_kernel(const DecodeAr
       const uint32_t w1 = __shfl_sync(0xffffffffu, word_u, src_lane2);
       const uint32_t v = __funnelshift_r(w0, w1, sh) & vmask;
       const __half* tab = row_tabs + ((seg * 256 + lane_cols) >> a.bc_shift) * table_halves;
-      dst[seg * 32] = lookup8<D>(tab, v, a.b, emask);
+      uint4 out = lookup8<D>(tab, v, a.b, emask);
+      if (a.row_scale != nullptr) {   // the lane's 8 columns lie in one group of 128: exact fp32 product, one rounding
+        const float sc = __half2float(__ldg(a.row_scale + static_cast<long long>(n) * (a.K / 128) + (col0 + seg * 256 + lane_cols) / 128));
+        uint32_t* o32 = reinterpret_cast<uint32_t*>(&out);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const __half2 hv = *reinterpret_cast<const __half2*>(&o32[q]);
+          const __half2 r = __halves2half2(__float2half_rn(sc * __low2float(hv)), __float2half_rn(sc * __high2float(hv)));
+          o32[q] = *reinterpret_cast<const uint32_t*>(&r);
+        }
+      }
+      dst[seg * 32] = out;
     };
     int s0 = 0;
     for (; s0 + kUnroll <= segs; s0 += kUnroll) {   // full groups: no per-segment predicates
@@ -145,7 +162,7 @@ __global__ void __launch_bounds__(32 * kWarps) decode_tile_kernel(const DecodeAr
 // (8 b / d <= 32), block columns a power of two >= 8 that divide or are divided by the tile's columns,
 // block rows that divide or are divided by 32, tables of the tile within 96 KB of shared memory.
 vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s) {
-  if (g.cb_int4 || g.K % 256 || (8 * g.b) % g.d || 8 * g.b / g.d > 32 || g.Bc % 8) return VQ_ERR_UNSUPPORTED;
+  if (g.K % 256 || (8 * g.b) % g.d || 8 * g.b / g.d > 32 || g.Bc % 8) return VQ_ERR_UNSUPPORTED;
   DecodeArgs a;
   a.tile_cols = g.K < kTileCols ? g.K : kTileCols;
   a.bc_shift = -1;
@@ -157,6 +174,7 @@ vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, 
   a.idx = p.idx;
   a.cb = p.cb;
   a.scale = g.cb_int8 ? p.scale : nullptr;
+  a.row_scale = g.cb_int4 ? p.scale : nullptr;
   a.W = W;
   a.stride = g.stride;
   a.N = g.N;

@@ -356,6 +356,8 @@ INT4_CODEBOOK_CASES = [
     vq_synth.LayerSpec("i4cb_d2b6", N=37, K=256, d=2, b=6, Br=37, Bc=128, int8=2),
     vq_synth.LayerSpec("i4cb_d1b4", N=20, K=384, d=1, b=4, Br=4, Bc=96, int8=2),
     vq_synth.LayerSpec("i4cb_d4b8", N=16, K=1280, d=4, b=8, Br=16, Bc=640, int8=2),
+    vq_synth.LayerSpec("i4cb_d4b8_tile", N=96, K=2560, d=4, b=8, Br=32, Bc=512, int8=2),   # tile decode kernel
+    vq_synth.LayerSpec("i4cb_d1b4_tile", N=40, K=512, d=1, b=4, Br=8, Bc=128, int8=2),
 ]
 
 
