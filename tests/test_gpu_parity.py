@@ -169,6 +169,22 @@ def test_randomized_format_sweep(spec):
         assert np.array_equal(d_idx.cpu().numpy(), orc.pack(f, orc.assign(f, W, L.cb, L.scale)))
 
 
+@pytest.mark.parametrize("spec,batch", [
+    (vq_synth.LayerSpec("rep_tall", N=1024, K=4096, d=2, b=6, Br=128, Bc=128, int8=False), 3),
+    (vq_synth.LayerSpec("rep_row", N=2048, K=8192, d=2, b=4, Br=1, Bc=2048, int8=True), 16),
+    (vq_synth.LayerSpec("rep_d4", N=512, K=5120, d=4, b=8, Br=256, Bc=512, int8=False), 8),
+], ids=lambda v: v.name if hasattr(v, "name") else str(v))
+def test_repeated_calls_are_bitwise_identical(spec, batch):
+    """The K-part reduction adds in a fixed order whatever order the partial sums arrive in: sixty
+    launches on the same inputs give the same bits (cluster split, remote stores, streamed activations)."""
+    L = draw(spec, 7)
+    dev = DeviceLayer(spec, L)
+    X = vq_synth.make_x(spec, 8, batch)
+    first = dev.gemm(X, vq.VQ_IMPL_TUNED).view(np.uint16)
+    for _ in range(60):
+        assert np.array_equal(dev.gemm(X, vq.VQ_IMPL_TUNED).view(np.uint16), first)
+
+
 def test_no_wait_ran_out_inside_a_kernel():
     # bounded waits on asynchronous copies never expired in anything this process has run so far
     import torch
