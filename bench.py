@@ -143,11 +143,11 @@ class DeviceSet:
             self.dev.append([tuple(None if t is None else t.clone() for t in lay) for lay in base])
         self.X = [torch.from_numpy(X).to(device) for (_, X) in self.host]
         self.Y = [torch.empty((batch, s.N), dtype=torch.float16, device=device) for s in self.specs]
-        self.ws = [torch.empty(vq.vq_workspace_bytes(f, batch), dtype=torch.uint8, device=device) for f in self.fmts]
+        self.ws = [torch.zeros(vq.vq_workspace_bytes(f, batch), dtype=torch.uint8, device=device) for f in self.fmts]
         # host side of the end-to-end path
         self.hX = [torch.from_numpy(X).pin_memory() for (_, X) in self.host]
         self.hY = [torch.empty((batch, s.N), dtype=torch.float16).pin_memory() for s in self.specs]
-        self.ws_host = [torch.empty(vq.vq_workspace_bytes_host(f, batch), dtype=torch.uint8, device=device) for f in self.fmts]
+        self.ws_host = [torch.zeros(vq.vq_workspace_bytes_host(f, batch), dtype=torch.uint8, device=device) for f in self.fmts]
         self.h2d = sum(int(x.numel()) * 2 for x in self.hX)
         self.d2h = sum(int(y.numel()) * 2 for y in self.hY)
 
@@ -328,13 +328,14 @@ def time_int4g128(cfg_name: str, batch: int, device, torch, vq):
         nbytes = q.size + sc.size * 2 + 2 * batch * (spec.N + spec.K)
         set_bytes += nbytes
         layers.append((spec, torch.from_numpy(q).to(device), torch.from_numpy(sc).to(device), torch.from_numpy(X).to(device),
-                       torch.empty((batch, spec.N), dtype=torch.float16, device=device)))
+                       torch.empty((batch, spec.N), dtype=torch.float16, device=device),
+                       torch.zeros(vq.vq_int4g128_workspace_bytes(spec.N, batch), dtype=torch.uint8, device=device)))
     copies = max(2, -(-2 * L2_BYTES // set_bytes))
-    dev = [layers] + [[(sp, q.clone(), sc.clone(), X, Y) for (sp, q, sc, X, Y) in layers] for _ in range(copies - 1)]
+    dev = [layers] + [[(sp, q.clone(), sc.clone(), X, Y, ws) for (sp, q, sc, X, Y, ws) in layers] for _ in range(copies - 1)]
 
     def step(c):
-        for sp, q, sc, X, Y in dev[c]:
-            vq.vq_int4g128_gemm_small_batch(sp.N, sp.K, q, sc, X, Y, batch)
+        for sp, q, sc, X, Y, ws in dev[c]:
+            vq.vq_int4g128_gemm_small_batch(sp.N, sp.K, q, sc, X, Y, batch, ws)
     step(0)
     torch.cuda.synchronize()
     g = torch.cuda.CUDAGraph()

@@ -196,7 +196,8 @@ size_t vq_static_scratch_bytes(void);
  * Errors: NULL, SHAPE, ALIGN, BATCH, CUDA. */
 vq_status vq_int4g128_gemm_small_batch(int32_t n_rows, int32_t k_cols, const void* d_q,
                                        const void* d_scale, const void* d_X, void* d_Y,
-                                       int batch, void* stream);
+                                       int batch, void* d_ws, size_t ws_bytes, void* stream);
+size_t vq_int4g128_workspace_bytes(int32_t n_rows, int batch);
 
 /* E-step / VQ_quant of the quantizer (paper Sec. 3, Eq. 5; Algorithm 2's quantization step): for
  * every d-vector x of the dense matrix W (d adjacent columns of one row) the index m of the centroid

@@ -83,7 +83,8 @@ _SIGNATURES = {
     "vq_gemm_small_batch_host": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
     "vq_gemm_small_batch_host_static": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p]),
     "vq_static_scratch_bytes": (ctypes.c_size_t, []),
-    "vq_int4g128_gemm_small_batch": (ctypes.c_int, [ctypes.c_int32, ctypes.c_int32] + [ctypes.c_void_p] * 4 + [ctypes.c_int, ctypes.c_void_p]),
+    "vq_int4g128_gemm_small_batch": (ctypes.c_int, [ctypes.c_int32, ctypes.c_int32] + [ctypes.c_void_p] * 4 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
+    "vq_int4g128_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int32, ctypes.c_int]),
     "vq_assign_indices": (ctypes.c_int, [ctypes.c_void_p] * 7),
     "vq_unpack_uniform": (ctypes.c_int, [ctypes.c_int, ctypes.c_int32, ctypes.c_int32] + [ctypes.c_void_p] * 4),
     "vq_device_wait_failures": (ctypes.c_int, [ctypes.c_void_p]),
@@ -208,9 +209,14 @@ def vq_device_wait_failures() -> int:
     return out.value
 
 
-def vq_int4g128_gemm_small_batch(n_rows: int, k_cols: int, d_q, d_scale, d_X, d_Y, batch: int, stream=None) -> None:
+def vq_int4g128_workspace_bytes(n_rows: int, batch: int) -> int:
+    return load().vq_int4g128_workspace_bytes(int(n_rows), int(batch))
+
+
+def vq_int4g128_gemm_small_batch(n_rows: int, k_cols: int, d_q, d_scale, d_X, d_Y, batch: int, d_ws, stream=None) -> None:
     _check(load().vq_int4g128_gemm_small_batch(int(n_rows), int(k_cols), _ptr(d_q), _ptr(d_scale), _ptr(d_X),
-                                               _ptr(d_Y), int(batch), _stream(stream)),
+                                               _ptr(d_Y), int(batch), _ptr(d_ws), d_ws.numel() * d_ws.element_size(),
+                                               _stream(stream)),
            "vq_int4g128_gemm_small_batch")
 
 

@@ -103,8 +103,7 @@ vq_status vq_pack_info(const vq_format* fmt, vq_pack_info_t* out) {
 
 size_t vq_workspace_bytes(const vq_format* fmt, int batch) {
   if (check_format(fmt) != VQ_OK || batch < 1 || batch > 16) return 0;
-  // fp32 partial sums of every K-split: [kMaxSplits][batch][N]
-  return round256(static_cast<size_t>(kMaxSplits) * batch * fmt->n_rows * sizeof(float));
+  return stream_workspace_bytes(fmt->n_rows, batch);
 }
 
 size_t vq_workspace_bytes_host(const vq_format* fmt, int batch) {
@@ -156,7 +155,7 @@ vq_status vq_gemm_small_batch_impl(const vq_format* fmt, const void* d_idx, cons
   const __half* X = static_cast<const __half*>(d_X);
   __half* Y = static_cast<__half*>(d_Y);
   if (impl != VQ_IMPL_GENERIC) {
-    st = launch_gemm_tuned(g, p, X, Y, batch, static_cast<float*>(d_ws), s);
+    st = launch_gemm_tuned(g, p, X, Y, batch, d_ws, ws_bytes, s);
     if (st != VQ_ERR_UNSUPPORTED || impl == VQ_IMPL_TUNED) return st;
   }
   return launch_gemm_generic(g, p, X, Y, batch, s);

@@ -27,8 +27,12 @@ struct LayerPtrs {
   const __half* scale;
 };
 
-// Maximum number of K-splits any kernel uses; fixes the workspace size.
-constexpr int kMaxSplits = 8;
+// Workspace of the persistent kernel (vq_stream.cu): one ticket counter per 16 rows at most, and
+// two slabs (at most 256 rows each) of fp32 partial sums per persistent CTA.
+constexpr int kMaxStreamCtas = 320;
+constexpr int kMaxSlabRows = 256;
+// Layers of one grouped call (they share the activations).
+constexpr int kMaxSegments = 4;
 // Devices per process the launchers keep per-device set-up state for.
 constexpr int kMaxDevices = 64;
 
@@ -40,7 +44,26 @@ vq_status launch_decode_generic(const Geometry& g, const LayerPtrs& p, __half* W
 vq_status launch_gemm_generic(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y,
                               int batch, cudaStream_t s);
 vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y,
-                            int batch, float* ws, cudaStream_t s);
+                            int batch, void* ws, size_t ws_bytes, cudaStream_t s);
+
+// One call of the persistent kernel: n_seg layers of one format and one K that share X.
+struct StreamCall {
+  Geometry g;          // format and K; g.N is not used (rows per layer are in N[])
+  int n_seg;
+  const uint8_t* idx[kMaxSegments];
+  const void* cb[kMaxSegments];
+  const __half* scale[kMaxSegments];
+  __half* Y[kMaxSegments];
+  int N[kMaxSegments];
+  const __half* X;
+  int batch;
+  void* ws;            // ticket counters (zero on entry, zero on exit) + partial sums
+  size_t ws_bytes;
+};
+size_t stream_workspace_bytes(long long rows, int batch);
+vq_status launch_gemm_stream(const StreamCall& call, cudaStream_t s);
+vq_status launch_int4g128_stream(int N, int K, const uint8_t* q, const __half* scale, const __half* X, __half* Y, int batch,
+                                 void* ws, size_t ws_bytes, cudaStream_t s);
 vq_status launch_gemm_blockcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
                               cudaStream_t s);
 vq_status launch_gemm_rowcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
@@ -58,7 +81,14 @@ vq_status device_error_counter(int** d_counter);
 
 // Tensor map of the packed index stream seen as a 2-D byte tensor (N rows of `stride` bytes) with
 // boxes of box_rows rows x box_bytes bytes, for tiled TMA loads without swizzle or multicast.
-vq_status encode_index_map(CUtensorMap* tm, const uint8_t* idx, long long stride, int N, int box_bytes, int box_rows);
+// swizzle128: rows of the box (box_bytes == 128) land with the 128-byte swizzle pattern.
+vq_status encode_index_map(CUtensorMap* tm, const uint8_t* idx, long long stride, int N, int box_bytes, int box_rows,
+                           bool swizzle128 = false);
+
+// General tiled tensor map (no multicast is ever used with it): elements of 1 or 2 bytes, rank <= 5,
+// dims / box in elements, strides of dimensions 1.. in bytes; swizzle 0 none, 1 64-byte, 2 128-byte.
+vq_status encode_tensor_map(CUtensorMap* tm, const void* base, int elem_bytes, int rank, const uint64_t* dims,
+                            const uint64_t* strides, const uint32_t* box, int swizzle);
 
 inline vq_status check_launch() {
   return cudaGetLastError() == cudaSuccess ? VQ_OK : VQ_ERR_CUDA;

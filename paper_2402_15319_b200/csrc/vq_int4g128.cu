@@ -84,19 +84,29 @@ __global__ void __launch_bounds__(256) unpack_uniform_kernel(long long groups8, 
 
 using namespace vq;
 
+extern "C" size_t vq_int4g128_workspace_bytes(int32_t N, int batch) {
+  if (N <= 0 || batch < 1 || batch > 16) return 0;
+  return stream_workspace_bytes(N, batch);
+}
+
 extern "C" vq_status vq_int4g128_gemm_small_batch(int32_t N, int32_t K, const void* d_q, const void* d_scale,
-                                                  const void* d_X, void* d_Y, int batch, void* stream) {
+                                                  const void* d_X, void* d_Y, int batch, void* d_ws, size_t ws_bytes,
+                                                  void* stream) {
   if (!d_q || !d_scale || !d_X || !d_Y) return VQ_ERR_NULL;
   if (N <= 0 || K <= 0 || K % 128 || (K / 2) % 16) return VQ_ERR_SHAPE;
   if (batch < 1 || batch > 16) return VQ_ERR_BATCH;
   const uintptr_t bitsor = reinterpret_cast<uintptr_t>(d_q) | reinterpret_cast<uintptr_t>(d_scale) |
                            reinterpret_cast<uintptr_t>(d_X) | reinterpret_cast<uintptr_t>(d_Y);
   if (bitsor & 15u) return VQ_ERR_ALIGN;
+  if (!d_ws || ws_bytes < vq_int4g128_workspace_bytes(N, batch)) return VQ_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(d_ws) & 15u) return VQ_ERR_ALIGN;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   {
-    // tensor-core path shared with the per-row VQ kernels; the plain kernel below covers the rest
-    const vq_status st = launch_int4g128_rowcb(N, K, static_cast<const uint8_t*>(d_q), static_cast<const __half*>(d_scale),
-                                               static_cast<const __half*>(d_X), static_cast<__half*>(d_Y), batch, s);
+    // the persistent tensor-core kernel shared with the per-row VQ formats; the plain kernel below
+    // covers rows that are not whole 128-byte chunks
+    const vq_status st = launch_int4g128_stream(N, K, static_cast<const uint8_t*>(d_q), static_cast<const __half*>(d_scale),
+                                                static_cast<const __half*>(d_X), static_cast<__half*>(d_Y), batch, d_ws,
+                                                ws_bytes, s);
     if (st != VQ_ERR_UNSUPPORTED) return st;
   }
   long long blocks = (N + 7) / 8;

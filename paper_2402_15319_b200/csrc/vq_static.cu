@@ -60,7 +60,7 @@ extern "C" vq_status vq_gemm_small_batch_host_static(const vq_format* fmt, const
   p.idx = static_cast<const uint8_t*>(d_idx);
   p.cb = d_cb;
   p.scale = static_cast<const __half*>(d_scale);
-  st = launch_gemm_tuned(g, p, d_X, d_Y, batch, nullptr, s);
+  st = launch_gemm_tuned(g, p, d_X, d_Y, batch, nullptr, 0, s);
   if (st == VQ_ERR_UNSUPPORTED) st = launch_gemm_generic(g, p, d_X, d_Y, batch, s);
   if (st != VQ_OK) return st;
   if (cudaMemcpyAsync(h_Y, d_Y, y_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return VQ_ERR_CUDA;

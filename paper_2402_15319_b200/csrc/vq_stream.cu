@@ -1,0 +1,1099 @@
+// Persistent, warp-specialised skinny-GEMM kernel for the VQ-decode linear layer (paper Sec. 3.2:
+// packed indices -> look-up table -> mat-vec; App. A: the weight matrix is a look-up of the
+// codebook).  The tiling, the pipeline and the reduction are this library's.
+//
+// Work.  The rows of every layer of a call ("segment": layers that share the activations, e.g. the
+// q/k/v or gate/up projections) are cut into slabs of 16*WR rows, a row's index stream into chunks
+// of CHUNK_BYTES.  A slab takes S = chunks / WK pipeline stages; in stage s consumer warp (wr, wk)
+// multiplies its 16 rows by chunk wk*S + s.  Every persistent CTA (one per SM) first takes q =
+// slabs / P whole slabs; the stages of the slabs left over form one sequence that is cut into equal
+// contiguous pieces, one per CTA, so that every SM streams the same number of bytes whatever the
+// layer shape.
+//
+// Pipeline.  One elected producer thread walks the CTA's stages D deep ahead of the consumers with
+// two tiled TMA loads per stage, both counted on the stage's "full" mbarrier: a box {CHUNK_BYTES,
+// 16*WR rows, WK parts} of the index stream and a box of the activations of the same columns, laid
+// out [part][w][batch row][row bytes] so that the B fragments of mma.sync m16n8k16 (batch row =
+// lane / 4) are read without bank conflicts.  Consumers wait on "full", expand indices to fp16
+// weights (A fragments), run the tensor-core steps with fp32 accumulation, and release the stage
+// through its "empty" mbarrier.
+//
+// Reduction.  The partial sums of the WK column parts meet in shared memory and are added in part
+// order.  A slab whose stages all belong to one CTA is rounded to fp16 and stored.  A left-over
+// slab spans several CTAs: each writes its fp32 partial sums into the workspace; at the end of the
+// kernel it draws a ticket from the slab's counter, and the CTA that draws the last ticket adds
+// the partial sums in CTA order (fixed order: results do not depend on timing), stores the outputs
+// and resets the counter to 0.
+//
+// Every wait is bounded; a wait that runs out increments a device counter, and the warp stops
+// waiting for anything else but still takes part in every block-level barrier, so that the kernel
+// ends.
+#include <cstdio>
+#include <cstdlib>
+
+#include "vq_common.cuh"
+#include "vq_device.cuh"
+
+namespace vq {
+namespace {
+
+using namespace dev;
+
+constexpr int kWaitTries = 1 << 18;   // polls (with a sleep of 40-500 ns in between) before a wait gives up
+
+struct Segment {
+  const void* cb;
+  const __half* scale;
+  __half* Y;
+  int N;
+  int slab0;   // first slab of the segment in the call's slab sequence
+};
+
+struct StreamArgs {
+  Segment seg[kMaxSegments];
+  int n_seg;
+  float* ws_part;     // [CTA][2][16*WR * batch] partial sums
+  int* ws_ticket;     // [slab], zero between calls
+  int* error_flag;
+  int K, batch;
+  int S;                 // stages per slab
+  int WR, WK, D;
+  int q;                 // whole slabs per CTA
+  int tail_units;        // stages of the left-over slabs
+  int tail_ctas;         // CTAs that share them (each at least one stage)
+  int blocks_per_row;
+  int cpb_shift;         // row policies: log2 of the chunks that share one codebook block
+  int br_shift;          // log2 of the rows that share one codebook block
+  int sr_shift;          // log2 of the rows of a slab (16*WR)
+  // byte offsets from the 4096-byte aligned start of dynamic shared memory
+  int red_off, bar_off, stage_off;
+  int stage_bytes;       // a stage: WK index boxes, then WK activation boxes
+  int x_off;             // activations inside a stage
+  int idx_part_bytes, x_part_bytes;
+  uint32_t tx_bytes;     // bytes the two loads of a stage bring
+};
+
+struct Maps {
+  CUtensorMap idx[kMaxSegments];
+  CUtensorMap x;
+};
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Bounded wait for phase `parity` that sleeps `ns` nanoseconds between polls, so that a waiting warp
+// leaves the issue slots of its scheduler to the warps that compute.  Returns false if the phase
+// did not complete within the attempts.
+__device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity, int max_tries, unsigned ns) {
+  for (int i = 0; i < max_tries; ++i) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) return true;
+    __nanosleep(ns);
+  }
+  return false;
+}
+__device__ __forceinline__ void named_barrier(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ float ldcg_f32(const float* p) {
+  float v;
+  asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void tma_box_3d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+               ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_box_4d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+               ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* tm) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
+}
+template <int NB>
+__device__ __forceinline__ void fence_acc(float (&acc)[NB][4]) {
+#pragma unroll
+  for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) asm volatile("" : "+f"(acc[nb][e])::"memory");
+}
+
+constexpr uint32_t kMagic = 0x64646464u;      // high byte of fp16 1024.0
+constexpr uint32_t kBias2 = 0x64806480u;      // fp16 pair (1152, 1152) = 1024 + 128
+// (1024 + u) - 1152 = u - 128, exact in fp16
+__device__ __forceinline__ uint32_t sub_bias(uint32_t h) {
+  uint32_t r;
+  asm("sub.f16x2 %0, %1, %2;" : "=r"(r) : "r"(h), "r"(kBias2));
+  return r;
+}
+
+// The CTA's walk over its stages: first its piece of the left-over stages (so that the slabs shared
+// with other CTAs are summed while the whole slabs are still being computed), then its q whole slabs.
+struct Walk {
+  int n;           // stages of this CTA
+  int n_tail;      // of which in left-over slabs (they come first)
+  int t0, t1;      // its piece of the left-over sequence
+  int slab, s;     // current stage
+  int k;
+  int whole0;      // first whole slab of this CTA
+  int tail_slab0;  // first left-over slab of the call
+
+  __device__ __forceinline__ void init(const StreamArgs& a, int c, int P) {
+    t0 = t1 = 0;
+    if (c < a.tail_ctas) {
+      t0 = static_cast<int>(static_cast<long long>(a.tail_units) * c / a.tail_ctas);
+      t1 = static_cast<int>(static_cast<long long>(a.tail_units) * (c + 1) / a.tail_ctas);
+    }
+    n_tail = t1 - t0;
+    n = n_tail + a.q * a.S;
+    whole0 = c * a.q;
+    tail_slab0 = a.q * P;
+    k = 0;
+    if (n_tail > 0) {
+      slab = tail_slab0 + t0 / a.S;
+      s = t0 % a.S;
+    } else {
+      slab = whole0;
+      s = 0;
+    }
+  }
+  __device__ __forceinline__ void next(const StreamArgs& a) {
+    ++k;
+    if (k == n_tail) {
+      slab = whole0;
+      s = 0;
+    } else if (++s == a.S) {
+      s = 0;
+      ++slab;
+    }
+  }
+  // last stage of its slab that this CTA works on
+  __device__ __forceinline__ bool slab_end(const StreamArgs& a) const { return s == a.S - 1 || k == n_tail - 1; }
+  // does this CTA hold every stage of the current slab?
+  __device__ __forceinline__ bool complete(const StreamArgs& a) const {
+    if (k >= n_tail) return true;
+    const int first_u = (slab - tail_slab0) * a.S;
+    return first_u >= t0 && first_u + a.S <= t1;
+  }
+};
+
+// What a consumer warp knows about the stage it works on.
+struct Where {
+  int seg;       // segment of the slab
+  int row0;      // first of the warp's 16 rows inside the segment
+  int ch;        // chunk of the row
+  int key;       // identifies (slab, codebook block): equal keys share a table
+};
+
+// =============================================================================================
+// Row policies: codebooks that belong to one row (or a few rows), 4-bit indices.  Chunk = 128 bytes
+// of a row, boxes land with the 128-byte swizzle (16-byte piece p of box row r at p ^ (r & 7)), lane
+// (g, t) reads index word 4w + t of rows g and g+8 for w = 0..7: conflict-free 32-bit reads.
+// The activations of the 16*d columns that index word 4w + t covers are X_ROW_BYTES / 4 bytes at
+// t * X_ROW_BYTES / 4 of row (w, batch row) of the stage's activation box.
+// =============================================================================================
+
+// Index words of rows g and g+8: idx = address of the warp's box rows + g*128 + t*4.
+__device__ __forceinline__ void load_words(const unsigned char* idx, int ww, uint32_t sw, uint32_t& wl, uint32_t& wh) {
+  const unsigned char* p = idx + ((16u * ww) ^ sw);
+  wl = *reinterpret_cast<const uint32_t*>(p);
+  wh = *reinterpret_cast<const uint32_t*>(p + 1024);
+}
+
+// ---- 2-D codebooks of 16 entries (fp16, or int8 + block scale): lane-private fp16 tables in shared
+// memory, word (entry, row half, lane) at entry*256 + half*128 + lane*4 from a 4096-byte boundary:
+// the entry index sits in address bits 8..11 and merges with the lane's address by one logic op.
+template <bool INT8>
+struct RowD2B4 {
+  static constexpr int CHUNK_BYTES = 128, CHUNK_COLS = 512, X_ROW_BYTES = 128;
+  static constexpr bool X_SWIZZLE = true;
+  static constexpr int TILE_TABLE_BYTES = 4096;   // per 16-row tile
+  static constexpr int CB_ROW_BYTES = INT8 ? 32 : 64;
+  static constexpr int RAW = INT8 ? 2 : 4;
+
+  template <int NB, int R>
+  struct State {
+    float acc[R][NB][4];
+    float sc[R][2], sc_raw[R][2];
+    uint32_t raw[R][2][RAW];
+    uint32_t tbl, fill;
+    int cur_key, pend_key;
+
+    __device__ __forceinline__ void init(uint32_t warp_tbl, int lane) {
+      tbl = warp_tbl + lane * 4;
+      fill = warp_tbl + (4 * (lane >> 3)) * 256 + (lane & 7) * 16;   // entries 4tb..4tb+3, the quad of row gb
+      cur_key = pend_key = -1;
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        sc[r][0] = sc[r][1] = 1.f;
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) acc[r][nb][e] = 0.f;
+      }
+    }
+
+    // Request the entries (and scales) of the block of `w`; lane l takes entries 4*(l/8)..+3 of rows
+    // l%8 and l%8+8 of every tile (the mapping the table is WRITTEN with), the scales of its own rows.
+    __device__ __forceinline__ void fetch(const StreamArgs& a, const Where& w, int lane) {
+      const Segment& sg = a.seg[w.seg];
+      const int blk = w.ch >> a.cpb_shift;
+      const int gb = lane & 7, tb = lane >> 3, g = lane >> 2;
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int rb = min(w.row0 + 16 * r + gb + 8 * h, sg.N - 1);
+          const uint8_t* p = static_cast<const uint8_t*>(sg.cb) +
+                             (static_cast<long long>(rb >> a.br_shift) * a.blocks_per_row + blk) * CB_ROW_BYTES + tb * (CB_ROW_BYTES / 4);
+          if constexpr (INT8) {
+            const uint2 v = ldg64_nc(p);
+            raw[r][h][0] = v.x; raw[r][h][1] = v.y;
+            const int rr = min(w.row0 + 16 * r + g + 8 * h, sg.N - 1);
+            sc_raw[r][h] = __half2float(__ldg(sg.scale + static_cast<long long>(rr >> a.br_shift) * a.blocks_per_row + blk));
+          } else {
+            const uint4 v = ldg128_nc(p);
+            raw[r][h][0] = v.x; raw[r][h][1] = v.y; raw[r][h][2] = v.z; raw[r][h][3] = v.w;
+          }
+        }
+      pend_key = w.key;
+    }
+
+    __device__ __forceinline__ void install() {
+      __syncwarp();   // every lane is done with the previous tables
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          uint32_t e[4];
+          if constexpr (INT8) {
+            e[0] = sub_bias(prmt(raw[r][h][0] ^ 0x80808080u, kMagic, 0x4140));
+            e[1] = sub_bias(prmt(raw[r][h][0] ^ 0x80808080u, kMagic, 0x4342));
+            e[2] = sub_bias(prmt(raw[r][h][1] ^ 0x80808080u, kMagic, 0x4140));
+            e[3] = sub_bias(prmt(raw[r][h][1] ^ 0x80808080u, kMagic, 0x4342));
+            sc[r][h] = sc_raw[r][h];
+          } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) e[i] = raw[r][h][i];
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) sts128(fill + r * TILE_TABLE_BYTES + i * 256 + h * 128, make_uint4(e[i], e[i], e[i], e[i]));
+        }
+      __syncwarp();
+      fence_value(tbl);   // gathers of the new block stay behind the rewrite
+    }
+
+    // Close the current block: its scale multiplies its fp32 partial sums.
+    __device__ __forceinline__ void flush(float (&total)[R][NB][4]) {
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) {
+          total[r][nb][0] = fmaf(sc[r][0], acc[r][nb][0], total[r][nb][0]);
+          total[r][nb][1] = fmaf(sc[r][0], acc[r][nb][1], total[r][nb][1]);
+          total[r][nb][2] = fmaf(sc[r][1], acc[r][nb][2], total[r][nb][2]);
+          total[r][nb][3] = fmaf(sc[r][1], acc[r][nb][3], total[r][nb][3]);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) acc[r][nb][e] = 0.f;
+        }
+    }
+
+    __device__ __forceinline__ void prefetch(const StreamArgs& a, const Where& next, int lane) {
+      if (next.key != cur_key && next.key != pend_key) fetch(a, next, lane);
+    }
+
+    // Make the block of `w` the current one (its tables must be complete before the stage's look-ups).
+    __device__ __forceinline__ void begin(const StreamArgs& a, const Where& w, int lane, float (&total)[R][NB][4]) {
+      if (w.key != cur_key) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) fence_acc(acc[r]);
+        flush(total);
+        if (pend_key != w.key) fetch(a, w, lane);
+        install();
+        cur_key = w.key;
+      }
+    }
+
+    template <int I, int OFF>
+    __device__ __forceinline__ uint32_t gather(uint32_t w) const {
+      constexpr int p = 4 * I;
+      const uint32_t x = p < 8 ? w << (8 - p) : w >> (p - 8);
+      return lds32_off<OFF>((x & 0xF00u) | tbl);
+    }
+
+    template <int RR>
+    __device__ __forceinline__ void tile_step(const unsigned char* idx, int ww, uint32_t sw, const uint4 (&b)[NB][2]) {
+      uint32_t wl, wh;
+      load_words(idx + RR * 2048, ww, sw, wl, wh);
+      constexpr int T0 = RR * TILE_TABLE_BYTES, T1 = T0 + 128;
+      uint32_t af[4][4];
+      af[0][0] = gather<0, T0>(wl); af[0][1] = gather<0, T1>(wh); af[0][2] = gather<1, T0>(wl); af[0][3] = gather<1, T1>(wh);
+      af[1][0] = gather<2, T0>(wl); af[1][1] = gather<2, T1>(wh); af[1][2] = gather<3, T0>(wl); af[1][3] = gather<3, T1>(wh);
+      af[2][0] = gather<4, T0>(wl); af[2][1] = gather<4, T1>(wh); af[2][2] = gather<5, T0>(wl); af[2][3] = gather<5, T1>(wh);
+      af[3][0] = gather<6, T0>(wl); af[3][1] = gather<6, T1>(wh); af[3][2] = gather<7, T0>(wl); af[3][3] = gather<7, T1>(wh);
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb) {
+        mma16816(acc[RR][nb], af[0][0], af[0][1], af[0][2], af[0][3], b[nb][0].x, b[nb][0].y);
+        mma16816(acc[RR][nb], af[1][0], af[1][1], af[1][2], af[1][3], b[nb][0].z, b[nb][0].w);
+        mma16816(acc[RR][nb], af[2][0], af[2][1], af[2][2], af[2][3], b[nb][1].x, b[nb][1].y);
+        mma16816(acc[RR][nb], af[3][0], af[3][1], af[3][2], af[3][3], b[nb][1].z, b[nb][1].w);
+      }
+    }
+
+    // idx: the warp's box rows + g*128 + t*4 (tile r 2048 bytes further); xrow[nb]: row (w = 0, batch
+    // row) of the activation box, xstep = batch * 128 bytes to the next w.
+    __device__ __forceinline__ void compute(const unsigned char* idx, const unsigned char* const (&xrow)[NB], uint32_t xstep,
+                                            int lane, float (&)[R][NB][4]) {
+      const uint32_t sw = static_cast<uint32_t>(lane >> 2) << 4;
+      const uint32_t t32 = static_cast<uint32_t>(lane & 3) << 5;
+      uint4 b[NB][2];
+#pragma unroll
+      for (int ww = 0; ww < 8; ++ww) {
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) {
+          // 32 bytes at t*32 of the 128-byte row; the box is swizzled: piece p of row r at p ^ (r & 7)
+          const unsigned char* r = xrow[nb] + ww * xstep;
+          const uint32_t ph = (static_cast<uint32_t>(reinterpret_cast<uintptr_t>(r)) >> 3) & 0x70u;
+          b[nb][0] = *reinterpret_cast<const uint4*>(r + (t32 ^ ph));
+          b[nb][1] = *reinterpret_cast<const uint4*>(r + ((t32 + 16u) ^ ph));
+        }
+        tile_step<0>(idx, ww, sw, b);
+        if constexpr (R > 1) tile_step<1>(idx, ww, sw, b);
+        if constexpr (R > 2) tile_step<2>(idx, ww, sw, b);
+        if constexpr (R > 3) tile_step<3>(idx, ww, sw, b);
+      }
+    }
+  };
+};
+
+// ---- 1-D int8 codebooks of 16 entries + block scale: the row's entries live in 4 registers and
+// are looked up with byte permutes, the register-file analogue of the paper's LUT instruction
+// (Sec. 3.2: index -> 8-bit value); bytes become fp16 by the 0x6400 exponent trick, exactly.
+struct RowD1B4I8 {
+  static constexpr int CHUNK_BYTES = 128, CHUNK_COLS = 256, X_ROW_BYTES = 64;
+  static constexpr bool X_SWIZZLE = false;
+  static constexpr int TILE_TABLE_BYTES = 0;
+
+  template <int NB, int R>
+  struct State {
+    float acc[R][NB][4];
+    float sc[R][2], sc_raw[R][2];
+    uint32_t T[R][2][4];
+    uint4 raw[R][2];
+    int cur_key, pend_key;
+
+    __device__ __forceinline__ void init(uint32_t, int) {
+      cur_key = pend_key = -1;
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        sc[r][0] = sc[r][1] = 1.f;
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) acc[r][nb][e] = 0.f;
+      }
+    }
+    __device__ __forceinline__ void fetch(const StreamArgs& a, const Where& w, int lane) {
+      const Segment& sg = a.seg[w.seg];
+      const int blk = w.ch >> a.cpb_shift;
+      const int g = lane >> 2;
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int rr = min(w.row0 + 16 * r + g + 8 * h, sg.N - 1);
+          const long long b = static_cast<long long>(rr >> a.br_shift) * a.blocks_per_row + blk;
+          raw[r][h] = ldg128_nc(static_cast<const uint8_t*>(sg.cb) + b * 16);
+          sc_raw[r][h] = __half2float(__ldg(sg.scale + b));
+        }
+      pend_key = w.key;
+    }
+    __device__ __forceinline__ void install() {
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          T[r][h][0] = raw[r][h].x ^ 0x80808080u; T[r][h][1] = raw[r][h].y ^ 0x80808080u;
+          T[r][h][2] = raw[r][h].z ^ 0x80808080u; T[r][h][3] = raw[r][h].w ^ 0x80808080u;
+          sc[r][h] = sc_raw[r][h];
+        }
+    }
+    __device__ __forceinline__ void flush(float (&total)[R][NB][4]) {
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) {
+          total[r][nb][0] = fmaf(sc[r][0], acc[r][nb][0], total[r][nb][0]);
+          total[r][nb][1] = fmaf(sc[r][0], acc[r][nb][1], total[r][nb][1]);
+          total[r][nb][2] = fmaf(sc[r][1], acc[r][nb][2], total[r][nb][2]);
+          total[r][nb][3] = fmaf(sc[r][1], acc[r][nb][3], total[r][nb][3]);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) acc[r][nb][e] = 0.f;
+        }
+    }
+    __device__ __forceinline__ void prefetch(const StreamArgs& a, const Where& next, int lane) {
+      if (next.key != cur_key && next.key != pend_key) fetch(a, next, lane);
+    }
+    __device__ __forceinline__ void begin(const StreamArgs& a, const Where& w, int lane, float (&total)[R][NB][4]) {
+      if (w.key != cur_key) {
+        flush(total);
+        if (pend_key != w.key) fetch(a, w, lane);
+        install();
+        cur_key = w.key;
+      }
+    }
+    __device__ __forceinline__ void compute(const unsigned char* idx, const unsigned char* const (&xrow)[NB], uint32_t xstep,
+                                            int lane, float (&)[R][NB][4]) {
+      const uint32_t sw = static_cast<uint32_t>(lane >> 2) << 4;
+      const uint32_t t16 = static_cast<uint32_t>(lane & 3) << 4;
+      uint4 b[NB];
+#pragma unroll
+      for (int ww = 0; ww < 8; ++ww) {
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) b[nb] = *reinterpret_cast<const uint4*>(xrow[nb] + ww * xstep + t16);
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          uint32_t wd[2];
+          load_words(idx + r * 2048, ww, sw, wd[0], wd[1]);
+          uint32_t af[2][4];
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            // selector nibble = entry mod 8 (bit 3 would mean "replicate sign"), looked up in entries
+            // 0..7 and 8..15; a second permute picks per index by the index's bit 3
+            const uint32_t sel = wd[h] & 0x77777777u;
+            const uint32_t pick = ((wd[h] >> 1) & 0x44444444u) | 0x32103210u;
+            const uint32_t rL = prmt(prmt(T[r][h][0], T[r][h][1], sel), prmt(T[r][h][2], T[r][h][3], sel), pick);
+            const uint32_t rH = prmt(prmt(T[r][h][0], T[r][h][1], sel >> 16), prmt(T[r][h][2], T[r][h][3], sel >> 16), pick >> 16);
+            af[0][h] = sub_bias(prmt(rL, kMagic, 0x4140));       // columns 0,1
+            af[0][h + 2] = sub_bias(prmt(rL, kMagic, 0x4342));   // columns 2,3
+            af[1][h] = sub_bias(prmt(rH, kMagic, 0x4140));       // columns 4,5
+            af[1][h + 2] = sub_bias(prmt(rH, kMagic, 0x4342));   // columns 6,7
+          }
+#pragma unroll
+          for (int nb = 0; nb < NB; ++nb) {
+            mma16816(acc[r][nb], af[0][0], af[0][1], af[0][2], af[0][3], b[nb].x, b[nb].y);
+            mma16816(acc[r][nb], af[1][0], af[1][1], af[1][2], af[1][3], b[nb].z, b[nb].w);
+          }
+        }
+      }
+    }
+  };
+};
+
+// ---- uniform INT4 with an fp16 scale per 128 columns (paper Sec. 2.1 symmetric uniform quantiser;
+// Sec. 5 "INT4 g128"), the bandwidth yard-stick: no table.  Byte j of an index word holds columns
+// 2j (low nibble) and 2j+1 (high nibble): the byte is copied into both halves of a register, masked
+// to (q_lo, 16*q_hi) and merged with the fp16 exponent of 1024, giving the pair (1024 + q_lo,
+// 1024 + 16*q_hi); one fused multiply-add by (1, 1/16) and (-1032, -72) makes it (q_lo - 8, q_hi - 8),
+// exactly.
+struct RowInt4G128 {
+  static constexpr int CHUNK_BYTES = 128, CHUNK_COLS = 256, X_ROW_BYTES = 64;
+  static constexpr bool X_SWIZZLE = false;
+  static constexpr int TILE_TABLE_BYTES = 0;
+
+  template <int NB, int R>
+  struct State {
+    uint32_t sc_cur[R][2], sc_next[R][2];   // two fp16 scales (the chunk's two groups) per row
+    int cur_key, pend_key;
+
+    __device__ __forceinline__ void init(uint32_t, int) { cur_key = pend_key = -1; }
+    __device__ __forceinline__ void fetch(const StreamArgs& a, const Where& w, int lane) {
+      const Segment& sg = a.seg[w.seg];
+      const int g = lane >> 2;
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int rr = min(w.row0 + 16 * r + g + 8 * h, sg.N - 1);
+          sc_next[r][h] = __ldg(reinterpret_cast<const uint32_t*>(sg.scale + static_cast<long long>(rr) * (a.K / 128) + 2 * w.ch));
+        }
+      pend_key = w.key;
+    }
+    __device__ __forceinline__ void flush(float (&)[R][NB][4]) {}
+    __device__ __forceinline__ void prefetch(const StreamArgs& a, const Where& next, int lane) {
+      if (next.key != cur_key && next.key != pend_key) fetch(a, next, lane);
+    }
+    __device__ __forceinline__ void begin(const StreamArgs& a, const Where& w, int lane, float (&)[R][NB][4]) {
+      if (w.key != cur_key) {
+        if (pend_key != w.key) fetch(a, w, lane);
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          sc_cur[r][0] = sc_next[r][0];
+          sc_cur[r][1] = sc_next[r][1];
+        }
+        cur_key = w.key;
+      }
+    }
+    __device__ __forceinline__ void compute(const unsigned char* idx, const unsigned char* const (&xrow)[NB], uint32_t xstep,
+                                            int lane, float (&total)[R][NB][4]) {
+      constexpr uint32_t kMul = 0x2C003C00u;    // fp16 pair (1, 1/16)
+      constexpr uint32_t kAdd = 0xD480E408u;    // fp16 pair (-1032, -72)
+      const uint32_t sw = static_cast<uint32_t>(lane >> 2) << 4;
+      const uint32_t t16 = static_cast<uint32_t>(lane & 3) << 4;
+      uint4 b[NB];
+#pragma unroll
+      for (int grp = 0; grp < 2; ++grp) {
+        float acc[R][NB][4];
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+          for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[r][nb][e] = 0.f;
+#pragma unroll
+        for (int w4 = 0; w4 < 4; ++w4) {
+          const int ww = 4 * grp + w4;
+#pragma unroll
+          for (int nb = 0; nb < NB; ++nb) b[nb] = *reinterpret_cast<const uint4*>(xrow[nb] + ww * xstep + t16);
+#pragma unroll
+          for (int r = 0; r < R; ++r) {
+            uint32_t wd[2];
+            load_words(idx + r * 2048, ww, sw, wd[0], wd[1]);
+            uint32_t q[2][4];
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const uint32_t both = prmt(wd[h], 0u, 0x4040u + 0x0101u * i);      // byte i in bits 0..7 and 16..23
+                const uint32_t m = (both & 0x00F0000Fu) | 0x64006400u;             // (1024 + q_lo, 1024 + 16 q_hi)
+                asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(q[h][i]) : "r"(m), "r"(kMul), "r"(kAdd));
+              }
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb) {
+              mma16816(acc[r][nb], q[0][0], q[1][0], q[0][1], q[1][1], b[nb].x, b[nb].y);   // columns 0,1 | 2,3
+              mma16816(acc[r][nb], q[0][2], q[1][2], q[0][3], q[1][3], b[nb].z, b[nb].w);   // columns 4,5 | 6,7
+            }
+          }
+        }
+        // the group's scale multiplies its fp32 partial sums
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          const float s0 = __half2float(__ushort_as_half(static_cast<unsigned short>(grp ? sc_cur[r][0] >> 16 : sc_cur[r][0] & 0xffffu)));
+          const float s1 = __half2float(__ushort_as_half(static_cast<unsigned short>(grp ? sc_cur[r][1] >> 16 : sc_cur[r][1] & 0xffffu)));
+#pragma unroll
+          for (int nb = 0; nb < NB; ++nb) {
+            total[r][nb][0] = fmaf(s0, acc[r][nb][0], total[r][nb][0]);
+            total[r][nb][1] = fmaf(s0, acc[r][nb][1], total[r][nb][1]);
+            total[r][nb][2] = fmaf(s1, acc[r][nb][2], total[r][nb][2]);
+            total[r][nb][3] = fmaf(s1, acc[r][nb][3], total[r][nb][3]);
+          }
+        }
+      }
+    }
+  };
+};
+
+// =============================================================================================
+// The kernel.  Grid (P), block (W + 2) warps: warps 0..W-1 consume (warp = wk*WR + wr), warp W produces
+// (one thread), warp W+1 writes the results.  CW = the most consumer warps a launch may use (4: two
+// CTAs per SM, 8: one), which fixes the registers a thread may take.
+// =============================================================================================
+template <class P, int NB, int R, int CW>
+__global__ void __launch_bounds__((CW + 2) * 32, CW <= 4 ? 2 : 1)
+stream_kernel(const __grid_constant__ Maps maps, const StreamArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  const uint32_t sbase = (smem_u32(smem_raw) + 4095u) & ~4095u;
+  unsigned char* smem = smem_raw + (sbase - smem_u32(smem_raw));
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int W = a.WR * a.WK;
+  const int D = a.D;
+  // barriers: full[D], empty[D] (pipeline stages); out_full[2], out_empty[2] (results of a slab)
+  const uint32_t full0 = sbase + a.bar_off, empty0 = full0 + 8 * D;
+  const uint32_t out_full0 = empty0 + 8 * D, out_empty0 = out_full0 + 16;
+  constexpr int NBT = 8 * NB;
+  const int red_floats = W * R * 16 * NBT;   // one buffer of the slab's partial sums: [wk][16*R*WR rows][NBT]
+
+  if (tid == 0) {
+    for (int i = 0; i < D; ++i) {
+      mbar_init(full0 + 8 * i, 1);
+      mbar_init(empty0 + 8 * i, W);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(out_full0 + 8 * i, W);
+      mbar_init(out_empty0 + 8 * i, 1);
+    }
+    mbar_init_fence();
+  }
+  __syncthreads();
+  pdl_launch_dependents();
+
+  const int c = blockIdx.x, Pn = gridDim.x;
+  const int slab_rows = 16 * R * a.WR;
+  Walk wk_;
+  wk_.init(a, c, Pn);
+
+  auto segment_of = [&](int slab) {
+    int sgi = 0;
+#pragma unroll
+    for (int i = 1; i < kMaxSegments; ++i)
+      if (i < a.n_seg && slab >= a.seg[i].slab0) sgi = i;
+    return sgi;
+  };
+
+  // ------------------------------------------------------------------------------------------
+  // producer: one thread
+  // ------------------------------------------------------------------------------------------
+  if (warp == W) {
+    if (lane != 0) return;
+    prefetch_tensormap(&maps.x);
+    for (int i = 0; i < a.n_seg; ++i) prefetch_tensormap(&maps.idx[i]);
+    bool waited = false;
+    for (; wk_.k < wk_.n; wk_.next(a)) {
+      const int k = wk_.k, slot = k % D;
+      const uint32_t full = full0 + 8 * slot;
+      if (k >= D && !mbar_wait_idle(empty0 + 8 * slot, ((k / D) & 1) ^ 1, kWaitTries, 200)) {
+        atomicAdd(a.error_flag, 1);
+        break;
+      }
+      const int sg = segment_of(wk_.slab);
+      const int row0 = (wk_.slab - a.seg[sg].slab0) * slab_rows;
+      const uint32_t stage = sbase + a.stage_off + slot * a.stage_bytes;
+      mbar_arrive_expect_tx(full, a.tx_bytes);
+      // indices: {CHUNK_BYTES, slab rows, WK parts} at (byte s*CHUNK_BYTES of a part, row, part 0)
+      tma_box_3d(stage, &maps.idx[sg], wk_.s * P::CHUNK_BYTES, row0, 0, full);
+      if (!waited) {   // the activations belong to the previous kernel of the stream until here
+        pdl_wait();
+        waited = true;
+      }
+      // activations: {row bytes, batch, w = 0..7, WK parts} at (0, 0, box row s*8 of a part, part 0)
+      tma_box_4d(stage + a.x_off, &maps.x, 0, 0, wk_.s * 8, 0, full);
+    }
+    return;
+  }
+
+  // ------------------------------------------------------------------------------------------
+  // results: one warp takes the slabs' partial sums from the consumers, adds the WK column parts in
+  // part order and stores the outputs (or, for a slab shared with other CTAs, this CTA's share)
+  // ------------------------------------------------------------------------------------------
+  if (warp == W + 1) {
+    pdl_wait();   // outputs and workspace belong to earlier kernels of the stream until here
+    int ev = 0;                                   // slabs handed over so far
+    int n_partial = 0, partial_a = 0, partial_b = 0;
+    bool dead = false;
+    for (; wk_.k < wk_.n; wk_.next(a)) {
+      if (!wk_.slab_end(a)) continue;
+      const int buf = ev & 1;
+      if (!dead && !mbar_wait_idle(out_full0 + 8 * buf, (ev >> 1) & 1, kWaitTries, 500)) {
+        if (lane == 0) atomicAdd(a.error_flag, 1);
+        dead = true;
+      }
+      dead = __any_sync(0xffffffffu, dead);
+      const int slab = wk_.slab;
+      const bool complete = wk_.complete(a);
+      const Segment& sg = a.seg[segment_of(slab)];
+      const int srow0 = (slab - sg.slab0) * slab_rows;
+      const int n_out = slab_rows * a.batch;
+      const float* red = reinterpret_cast<const float*>(smem + a.red_off) + buf * red_floats;
+      // this CTA's share of a left-over slab goes to the workspace: slot 0 if the CTA's piece begins
+      // inside this slab, else slot 1
+      float* part = nullptr;
+      if (!complete) {
+        const int my_slot = (wk_.tail_slab0 + wk_.t0 / a.S == slab) ? 0 : 1;
+        part = a.ws_part + (static_cast<long long>(c) * 2 + my_slot) * n_out;
+        if (n_partial == 0) partial_a = slab;
+        else partial_b = slab;
+        ++n_partial;
+      }
+      if (!dead) {
+        for (int o = lane; o < n_out; o += 32) {
+          const int n = o >> a.sr_shift, rr = o & (slab_rows - 1);
+          float sum = 0.f;
+          for (int p = 0; p < a.WK; ++p) sum += red[(p * slab_rows + rr) * NBT + n];
+          if (complete) {
+            if (srow0 + rr < sg.N) sg.Y[static_cast<long long>(n) * sg.N + srow0 + rr] = __float2half_rn(sum);
+          } else {
+            part[o] = sum;
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(out_empty0 + 8 * buf);   // the buffer may be refilled
+      ++ev;
+
+      // ---- the CTA's piece of the left-over stages is done: tickets, and the sums of the slabs
+      // this CTA completes (the consumers are already at work on the whole slabs) ----
+      if (wk_.k == wk_.n_tail - 1 && n_partial > 0) {
+        if (n_partial > 2) n_partial = 2;   // (cannot happen: a piece is shorter than a slab)
+        const long long T = a.tail_units;
+        const int Pt = a.tail_ctas;
+        int last_mask = 0;
+        if (lane == 0) {
+          __threadfence();            // this warp's partial sums are visible to the GPU before a ticket is drawn
+          for (int i = 0; i < n_partial; ++i) {
+            const int ps = i == 0 ? partial_a : partial_b;
+            const int first_u = (ps - wk_.tail_slab0) * a.S, last_u = first_u + a.S - 1;
+            const int c_first = static_cast<int>((static_cast<long long>(first_u + 1) * Pt - 1) / T);
+            const int c_last = static_cast<int>((static_cast<long long>(last_u + 1) * Pt - 1) / T);
+            const int ticket = atomicAdd(a.ws_ticket + ps, 1);
+            if (ticket == c_last - c_first) {
+              a.ws_ticket[ps] = 0;   // nobody else touches the counter in this call
+              last_mask |= 1 << i;
+            }
+          }
+          if (last_mask) __threadfence();   // the other CTAs' partial sums are visible after the tickets
+        }
+        last_mask = __shfl_sync(0xffffffffu, last_mask, 0);
+        for (int i = 0; i < n_partial; ++i) {
+          if (!(last_mask >> i & 1)) continue;
+          const int ps = i == 0 ? partial_a : partial_b;
+          const Segment& sp = a.seg[segment_of(ps)];
+          const int prow0 = (ps - sp.slab0) * slab_rows;
+          const int first_u = (ps - wk_.tail_slab0) * a.S, last_u = first_u + a.S - 1;
+          const int c_first = static_cast<int>((static_cast<long long>(first_u + 1) * Pt - 1) / T);
+          const int c_last = static_cast<int>((static_cast<long long>(last_u + 1) * Pt - 1) / T);
+          for (int o = lane; o < n_out; o += 32) {
+            const int n = o >> a.sr_shift, rr = o & (slab_rows - 1);
+            float sum = 0.f;
+            for (int qc = c_first; qc <= c_last; ++qc) {
+              const int q_t0 = static_cast<int>(T * qc / Pt);
+              const int q_slot = (wk_.tail_slab0 + q_t0 / a.S == ps) ? 0 : 1;
+              sum += ldcg_f32(a.ws_part + (static_cast<long long>(qc) * 2 + q_slot) * n_out + o);
+            }
+            if (prow0 + rr < sp.N) sp.Y[static_cast<long long>(n) * sp.N + prow0 + rr] = __float2half_rn(sum);
+          }
+        }
+      }
+    }
+    return;
+  }
+  if (warp > W + 1) return;
+
+  // ------------------------------------------------------------------------------------------
+  // consumers
+  // ------------------------------------------------------------------------------------------
+  const int g = lane >> 2, t = lane & 3;
+  const int wr = warp % a.WR, wk = warp / a.WR;
+  bool dead = false;
+
+  typename P::template State<NB, R> st;
+  st.init(sbase + warp * (R * P::TILE_TABLE_BYTES), lane);
+  float total[R][NB][4];
+#pragma unroll
+  for (int r = 0; r < R; ++r)
+#pragma unroll
+    for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) total[r][nb][e] = 0.f;
+  // batch row of the lane's B fragments; lanes beyond the batch re-read the last row (their columns
+  // of the result are never stored)
+  int xm[NB];
+#pragma unroll
+  for (int nb = 0; nb < NB; ++nb) xm[nb] = min(nb * 8 + g, a.batch - 1);
+  const uint32_t xstep = a.batch * P::X_ROW_BYTES;
+
+  auto where = [&](int slab, int s) {
+    Where w;
+    w.seg = segment_of(slab);
+    w.row0 = (slab - a.seg[w.seg].slab0) * slab_rows + wr * (16 * R);
+    w.ch = wk * a.S + s;
+    w.key = slab * a.blocks_per_row + (w.ch >> a.cpb_shift);
+    return w;
+  };
+
+  int ev = 0;
+  Where cur = where(wk_.slab, wk_.s);
+  if (wk_.n > 0) st.prefetch(a, cur, lane);
+  for (; wk_.k < wk_.n;) {
+    const int k = wk_.k, slot = k % D;
+    const bool slab_end = wk_.slab_end(a);
+    st.begin(a, cur, lane, total);
+    wk_.next(a);
+    Where nxt = cur;
+    if (wk_.k < wk_.n) {   // the stage after this one: request its codebook if it is another block
+      nxt = where(wk_.slab, wk_.s);
+      st.prefetch(a, nxt, lane);
+    }
+    if (!dead && !mbar_wait_idle(full0 + 8 * slot, (k / D) & 1, kWaitTries, 40)) {
+      if (lane == 0) atomicAdd(a.error_flag, 1);
+      dead = true;
+    }
+    dead = __any_sync(0xffffffffu, dead);
+    if (!dead) {
+      const unsigned char* stage = smem + a.stage_off + slot * a.stage_bytes;
+      const unsigned char* idx = stage + wk * a.idx_part_bytes + (wr * (16 * R) + g) * P::CHUNK_BYTES + t * 4;
+      const unsigned char* xrow[NB];
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb) xrow[nb] = stage + a.x_off + wk * a.x_part_bytes + xm[nb] * P::X_ROW_BYTES;
+      st.compute(idx, xrow, xstep, lane, total);
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty0 + 8 * slot);
+
+    if (slab_end) {
+      // ---- hand the slab's partial sums to the results warp ----
+      st.flush(total);
+      const int buf = ev & 1;
+      if (ev >= 2 && !dead && !mbar_wait_idle(out_empty0 + 8 * buf, ((ev >> 1) & 1) ^ 1, kWaitTries, 100)) {
+        if (lane == 0) atomicAdd(a.error_flag, 1);
+        dead = true;
+      }
+      dead = __any_sync(0xffffffffu, dead);
+      // total[r][nb][e]: row 16r + g + 8*(e/2) of the warp's rows, batch row nb*8 + 2t + (e&1)
+      float* mine = reinterpret_cast<float*>(smem + a.red_off) + buf * red_floats + ((wk * a.WR + wr) * (16 * R) + g) * NBT + 2 * t;
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            mine[(r * 16 + (e >> 1) * 8) * NBT + nb * 8 + (e & 1)] = total[r][nb][e];
+            total[r][nb][e] = 0.f;
+          }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(out_full0 + 8 * buf);
+      ++ev;
+    }
+    cur = nxt;
+  }
+}
+
+// =============================================================================================
+// host side
+// =============================================================================================
+int env_int(const char* name, int dflt) {
+#ifdef VQ_TUNING
+  if (const char* e = getenv(name)) return atoi(e);
+#else
+  (void)name;
+#endif
+  return dflt;
+}
+
+size_t round_up(size_t v, size_t al) { return (v + al - 1) / al * al; }
+
+vq_status device_sms(int* out) {
+  static int sms_of[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VQ_ERR_CUDA;
+  int n = __atomic_load_n(&sms_of[dev], __ATOMIC_ACQUIRE);
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return VQ_ERR_CUDA;
+    __atomic_store_n(&sms_of[dev], n, __ATOMIC_RELEASE);
+  }
+  *out = n;
+  return VQ_OK;
+}
+
+constexpr size_t kSmemMax = 224 * 1024;
+
+template <class P, int NB, int R, int CW>
+vq_status launch(const StreamCall& call, int chunks_per_block, cudaStream_t s) {
+  auto kern = stream_kernel<P, NB, R, CW>;
+  static int attr_set[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VQ_ERR_CUDA;
+  if (!__atomic_load_n(&attr_set[dev], __ATOMIC_ACQUIRE)) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemMax)) != cudaSuccess)
+      return VQ_ERR_CUDA;
+    __atomic_store_n(&attr_set[dev], 1, __ATOMIC_RELEASE);
+  }
+  int sms = 0;
+  if (device_sms(&sms) != VQ_OK) return VQ_ERR_CUDA;
+
+  const Geometry& g = call.g;
+  const int batch = call.batch;
+  auto log2_exact = [](int v) {
+    int l = 0;
+    while ((1 << l) < v) ++l;
+    return (1 << l) == v ? l : -1;
+  };
+  StreamArgs a = {};
+  a.n_seg = call.n_seg;
+  a.K = g.K;
+  a.batch = batch;
+  a.blocks_per_row = g.blocks_per_row;
+  a.cpb_shift = log2_exact(chunks_per_block);
+  a.br_shift = log2_exact(g.Br);
+  if (a.cpb_shift < 0 || a.br_shift < 0) return VQ_ERR_UNSUPPORTED;
+  const int n_chunks = static_cast<int>(g.stride / P::CHUNK_BYTES);
+  if (device_error_counter(&a.error_flag) != VQ_OK) return VQ_ERR_CUDA;
+
+  // ---- CTA shape: W = WR row tiles x WK column parts (WK divides the chunks of a row); D stages ----
+  int W = CW;
+  int ctas_per_sm = env_int("VQ_CTAS", CW <= 4 ? 2 : 1);
+  int WK = n_chunks % 4 == 0 ? 4 : n_chunks % 2 == 0 ? 2 : 1;
+  WK = env_int("VQ_WK", WK);
+  if (WK < 1 || n_chunks % WK || W % WK) return VQ_ERR_UNSUPPORTED;
+  int WR = env_int("VQ_WR", W / WK);
+  if (WR < 1 || WR * WK > CW || log2_exact(WR) < 0 || 16 * R * WR > kMaxSlabRows) return VQ_ERR_UNSUPPORTED;
+  W = WR * WK;
+  a.sr_shift = 4 + log2_exact(WR * R);
+  a.WR = WR;
+  a.WK = WK;
+  a.S = n_chunks / WK;
+  const int slab_rows = 16 * R * WR;
+  int slabs = 0;
+  for (int i = 0; i < call.n_seg; ++i) {
+    a.seg[i].cb = call.cb[i];
+    a.seg[i].scale = call.scale[i];
+    a.seg[i].Y = call.Y[i];
+    a.seg[i].N = call.N[i];
+    a.seg[i].slab0 = slabs;
+    slabs += (call.N[i] + slab_rows - 1) / slab_rows;
+  }
+  if (static_cast<long long>(slabs) * a.S > 0x3fffffff || static_cast<long long>(slabs) * a.blocks_per_row > 0x3fffffff)
+    return VQ_ERR_UNSUPPORTED;
+
+  const size_t tbl_bytes = static_cast<size_t>(P::TILE_TABLE_BYTES) * R * W;
+  const size_t red_bytes = 2 * static_cast<size_t>(W) * R * 16 * 8 * NB * sizeof(float);   // two buffers
+  const size_t idx_part = static_cast<size_t>(slab_rows) * P::CHUNK_BYTES;       // multiple of 2048
+  const size_t x_part = static_cast<size_t>(8) * batch * P::X_ROW_BYTES;         // [w][batch][row bytes]
+  const size_t x_off = idx_part * WK;
+  const size_t stage_bytes = round_up(x_off + x_part * WK, 1024);
+  if (P::X_SWIZZLE && x_part % 1024) return VQ_ERR_UNSUPPORTED;
+  const size_t red_off = tbl_bytes;
+  const size_t bar_off = round_up(red_off + red_bytes, 16);
+  const size_t stage_off = round_up(bar_off + 16 * 16 + 32, 1024);
+  // shared memory of a CTA: the SM's 227 KB minus 1 KB per resident CTA, shared by the resident CTAs
+  size_t budget = (227 * 1024 - 1024 * ctas_per_sm) / ctas_per_sm;
+  if (budget > kSmemMax) budget = kSmemMax;
+  if (budget < stage_off + 4096 + 2 * stage_bytes) {   // does not fit twice: one CTA per SM
+    ctas_per_sm = 1;
+    budget = kSmemMax;
+  }
+  int D = static_cast<int>((budget - 4096 - stage_off) / stage_bytes);
+  if (D > 8) D = 8;
+  D = env_int("VQ_D", D);
+  if (D < 2 || D > 16) return VQ_ERR_UNSUPPORTED;
+  const size_t smem_bytes = stage_off + static_cast<size_t>(D) * stage_bytes + 4096;
+  if (smem_bytes > kSmemMax) return VQ_ERR_UNSUPPORTED;
+  a.D = D;
+  a.red_off = static_cast<int>(red_off);
+  a.bar_off = static_cast<int>(bar_off);
+  a.stage_off = static_cast<int>(stage_off);
+  a.stage_bytes = static_cast<int>(stage_bytes);
+  a.x_off = static_cast<int>(x_off);
+  a.idx_part_bytes = static_cast<int>(idx_part);
+  a.x_part_bytes = static_cast<int>(x_part);
+  a.tx_bytes = static_cast<uint32_t>((idx_part + x_part) * WK);
+
+  // ---- persistent CTAs: whole slabs first, the left-over stages shared evenly ----
+  int Pn = env_int("VQ_P", sms * ctas_per_sm);
+  if (Pn > kMaxStreamCtas) Pn = kMaxStreamCtas;
+  if (Pn < 1) return VQ_ERR_UNSUPPORTED;
+  a.q = slabs / Pn;
+  const int left = slabs - a.q * Pn;
+  const long long tail = static_cast<long long>(left) * a.S;
+  a.tail_units = static_cast<int>(tail);
+  a.tail_ctas = static_cast<int>(tail < Pn ? tail : Pn);
+  // left-over slabs are not split (a CTA takes a whole one) when that costs little balance
+  if (env_int("VQ_NOSPLIT", 0)) a.tail_ctas = left;
+  if (a.q == 0) Pn = a.tail_ctas;   // fewer stages than CTAs: the others would have nothing to do
+  if (Pn < 1) return VQ_ERR_UNSUPPORTED;
+  const size_t ticket_bytes = round_up(static_cast<size_t>(slabs) * sizeof(int), 256);
+  const size_t part_ws = static_cast<size_t>(Pn) * 2 * slab_rows * batch * sizeof(float);
+  if (!call.ws || call.ws_bytes < ticket_bytes + part_ws) return VQ_ERR_WORKSPACE;
+  a.ws_ticket = static_cast<int*>(call.ws);
+  a.ws_part = reinterpret_cast<float*>(static_cast<char*>(call.ws) + ticket_bytes);
+
+  // ---- tensor maps ----
+  Maps maps;
+  for (int i = 0; i < call.n_seg; ++i) {
+    // index stream: bytes of a part, rows, parts
+    const uint64_t dims[3] = {static_cast<uint64_t>(a.S) * P::CHUNK_BYTES, static_cast<uint64_t>(call.N[i]), static_cast<uint64_t>(WK)};
+    const uint64_t strides[2] = {static_cast<uint64_t>(g.stride), static_cast<uint64_t>(a.S) * P::CHUNK_BYTES};
+    const uint32_t box[3] = {P::CHUNK_BYTES, static_cast<uint32_t>(slab_rows), static_cast<uint32_t>(WK)};
+    if (encode_tensor_map(&maps.idx[i], call.idx[i], 1, 3, dims, strides, box, 2) != VQ_OK) return VQ_ERR_CUDA;
+  }
+  for (int i = call.n_seg; i < kMaxSegments; ++i) maps.idx[i] = maps.idx[0];
+  {
+    // activations: columns of a row of the box, batch rows, box rows of a part, parts
+    const uint32_t row_cols = P::X_ROW_BYTES / 2;
+    const uint64_t dims[4] = {row_cols, static_cast<uint64_t>(batch), static_cast<uint64_t>(a.S) * 8, static_cast<uint64_t>(WK)};
+    const uint64_t strides[3] = {static_cast<uint64_t>(g.K) * 2, P::X_ROW_BYTES, static_cast<uint64_t>(a.S) * 8 * P::X_ROW_BYTES};
+    const uint32_t box[4] = {row_cols, static_cast<uint32_t>(batch), 8u, static_cast<uint32_t>(WK)};
+    if (encode_tensor_map(&maps.x, call.X, 2, 4, dims, strides, box, P::X_SWIZZLE ? 2 : 0) != VQ_OK) return VQ_ERR_CUDA;
+  }
+
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(Pn, 1, 1);
+  cfg.blockDim = dim3((W + 2) * 32, 1, 1);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  int na = 0;
+  if (env_int("VQ_PDL", 1)) {
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = na;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, maps, a);
+  if (e != cudaSuccess) {
+#ifdef VQ_TUNING
+    fprintf(stderr, "stream launch failed: %s (P %d WR %d WK %d D %d smem %zu)\n", cudaGetErrorString(e), Pn, WR, WK, D, smem_bytes);
+#endif
+    return VQ_ERR_CUDA;
+  }
+  return check_launch();
+}
+
+// Row tiles per consumer warp: the activation fragments of a step are loaded once and used by every
+// tile, so more tiles per warp mean fewer shared-memory cycles per weight; small layers keep one
+// tile so that there are enough slabs for every SM.
+template <class P, int NB>
+vq_status launch_tiles(const StreamCall& call, int chunks_per_block, cudaStream_t s) {
+  long long rows = 0;
+  for (int i = 0; i < call.n_seg; ++i) rows += call.N[i];
+  int R = NB == 1 && rows >= 8192 ? 2 : 1;
+  R = env_int("VQ_R", R);
+  const int cw = env_int("VQ_W", 4);
+  if (cw == 8) {
+    if (NB == 1 && R == 2) return launch<P, NB, 2, 8>(call, chunks_per_block, s);
+    return launch<P, NB, 1, 8>(call, chunks_per_block, s);
+  }
+  if (NB == 1 && R == 2) return launch<P, NB, 2, 4>(call, chunks_per_block, s);
+  if (NB == 1 && R == 4) return launch<P, NB, 4, 4>(call, chunks_per_block, s);
+  return launch<P, NB, 1, 4>(call, chunks_per_block, s);
+}
+
+}  // namespace
+
+vq_status launch_gemm_stream(const StreamCall& call, cudaStream_t s) {
+  const Geometry& g = call.g;
+  if (call.n_seg < 1 || call.n_seg > kMaxSegments) return VQ_ERR_UNSUPPORTED;
+  if (g.cb_int4) return VQ_ERR_UNSUPPORTED;
+  const bool nb2 = call.batch > 8;
+  if (g.b == 4 && g.Br >= 1 && g.stride % 128 == 0 && g.stride * 8 == static_cast<long long>(g.J) * 4) {
+    if (g.d == 2) {
+      if (g.Bc % 512) return VQ_ERR_UNSUPPORTED;
+      const int cpb = g.Bc / 512;
+      if (g.cb_int8) return nb2 ? launch_tiles<RowD2B4<true>, 2>(call, cpb, s) : launch_tiles<RowD2B4<true>, 1>(call, cpb, s);
+      return nb2 ? launch_tiles<RowD2B4<false>, 2>(call, cpb, s) : launch_tiles<RowD2B4<false>, 1>(call, cpb, s);
+    }
+    if (g.d == 1 && g.cb_int8) {
+      if (g.Bc % 256) return VQ_ERR_UNSUPPORTED;
+      return nb2 ? launch_tiles<RowD1B4I8, 2>(call, g.Bc / 256, s) : launch_tiles<RowD1B4I8, 1>(call, g.Bc / 256, s);
+    }
+  }
+  return VQ_ERR_UNSUPPORTED;
+}
+
+// Uniform INT4 group-128 yard-stick through the same kernel; UNSUPPORTED if a row is not a whole
+// number of 128-byte chunks.
+vq_status launch_int4g128_stream(int N, int K, const uint8_t* q, const __half* scale, const __half* X, __half* Y, int batch,
+                                 void* ws, size_t ws_bytes, cudaStream_t s) {
+  if (K % 256) return VQ_ERR_UNSUPPORTED;
+  StreamCall call = {};
+  Geometry& g = call.g;
+  g.N = N; g.K = K; g.d = 1; g.b = 4; g.Br = 1; g.Bc = 128;
+  g.cb_int8 = 1; g.cb_int4 = 0; g.entries = 16; g.J = K; g.blocks_per_row = K / 256; g.stride = K / 2;
+  call.n_seg = 1;
+  call.idx[0] = q;
+  call.cb[0] = nullptr;
+  call.scale[0] = scale;
+  call.Y[0] = Y;
+  call.N[0] = N;
+  call.X = X;
+  call.batch = batch;
+  call.ws = ws;
+  call.ws_bytes = ws_bytes;
+  return batch > 8 ? launch_tiles<RowInt4G128, 2>(call, 1, s) : launch_tiles<RowInt4G128, 1>(call, 1, s);
+}
+
+}  // namespace vq

@@ -8,7 +8,8 @@ namespace {
 static __device__ int g_wait_failures;
 }  // namespace
 
-vq_status encode_index_map(CUtensorMap* tm, const uint8_t* idx, long long stride, int N, int box_bytes, int box_rows) {
+vq_status encode_index_map(CUtensorMap* tm, const uint8_t* idx, long long stride, int N, int box_bytes, int box_rows,
+                           bool swizzle128) {
   using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                      const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -27,7 +28,39 @@ vq_status encode_index_map(CUtensorMap* tm, const uint8_t* idx, long long stride
   const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_bytes), static_cast<cuuint32_t>(box_rows)};
   const cuuint32_t elem_strides[2] = {1u, 1u};
   if (encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(idx), dims, strides, box, elem_strides,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+             CU_TENSOR_MAP_L2_PROMOTION_NONE,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return VQ_ERR_CUDA;
+  return VQ_OK;
+}
+
+vq_status encode_tensor_map(CUtensorMap* tm, const void* base, int elem_bytes, int rank, const uint64_t* dims,
+                            const uint64_t* strides, const uint32_t* box, int swizzle) {
+  using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                     const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                     CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeTiledFn encode = nullptr;   // (a pointer-sized store; two first callers write the same value)
+  if (!encode) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess || !p)
+      return VQ_ERR_CUDA;
+    encode = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  if (rank < 1 || rank > 5 || (elem_bytes != 1 && elem_bytes != 2)) return VQ_ERR_CUDA;
+  cuuint64_t d[5], st[4];
+  cuuint32_t b[5], es[5];
+  for (int i = 0; i < rank; ++i) {
+    d[i] = dims[i];
+    b[i] = box[i];
+    es[i] = 1u;
+    if (i + 1 < rank) st[i] = strides[i];
+  }
+  const CUtensorMapSwizzle sw = swizzle == 2 ? CU_TENSOR_MAP_SWIZZLE_128B : swizzle == 1 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE;
+  if (encode(tm, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_UINT16, static_cast<cuuint32_t>(rank),
+             const_cast<void*>(base), d, st, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_NONE,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return VQ_ERR_CUDA;
   return VQ_OK;
@@ -46,11 +79,32 @@ vq_status device_error_counter(int** d_counter) {
   return VQ_OK;
 }
 
-vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch, float* ws,
-                            cudaStream_t s) {
-  (void)ws;
+size_t stream_workspace_bytes(long long rows, int batch) {
+  const size_t tickets = (static_cast<size_t>((rows + 15) / 16 + kMaxSegments) * sizeof(int) + 255) / 256 * 256;
+  return tickets + static_cast<size_t>(kMaxStreamCtas) * 2 * kMaxSlabRows * batch * sizeof(float);
+}
+
+vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch, void* ws,
+                            size_t ws_bytes, cudaStream_t s) {
   if (g.cb_int4) return VQ_ERR_UNSUPPORTED;   // int4 codebooks: format-generic kernels only
-  vq_status st = launch_gemm_blockcb(g, p, X, Y, batch, s);
+  vq_status st = VQ_ERR_UNSUPPORTED;
+  if (ws) {   // the persistent kernel needs the workspace; callers without one take the cluster kernels
+    StreamCall call = {};
+    call.g = g;
+    call.n_seg = 1;
+    call.idx[0] = p.idx;
+    call.cb[0] = p.cb;
+    call.scale[0] = p.scale;
+    call.Y[0] = Y;
+    call.N[0] = g.N;
+    call.X = X;
+    call.batch = batch;
+    call.ws = ws;
+    call.ws_bytes = ws_bytes;
+    st = launch_gemm_stream(call, s);
+    if (st != VQ_ERR_UNSUPPORTED) return st;
+  }
+  st = launch_gemm_blockcb(g, p, X, Y, batch, s);
   if (st != VQ_ERR_UNSUPPORTED) return st;
   return launch_gemm_rowcb(g, p, X, Y, batch, s);
 }

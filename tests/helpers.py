@@ -33,7 +33,8 @@ class DeviceLayer:
         self.idx = torch.from_numpy(layer.idx).to(device)
         self.cb = torch.from_numpy(layer.cb).to(device)
         self.scale = None if layer.scale is None else torch.from_numpy(layer.scale).to(device)
-        self.ws = torch.empty(vq.vq_workspace_bytes(self.fmt, max_batch), dtype=torch.uint8, device=device)
+        # ticket counters at the start of the workspace must be zero on first use (the kernels leave them zero)
+        self.ws = torch.zeros(vq.vq_workspace_bytes(self.fmt, max_batch), dtype=torch.uint8, device=device)
         self.device = device
 
     def gemm(self, X: np.ndarray, impl=None):

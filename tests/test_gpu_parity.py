@@ -288,7 +288,8 @@ def test_int4g128(N, K):
         Y, A = orc.int4g128_gemm(q, s, X, threads=4)
         dq, ds, dX = (torch.from_numpy(a).cuda() for a in (q, s, X))
         dY = torch.full((batch, N), float("nan"), dtype=torch.float16, device="cuda")
-        vq.vq_int4g128_gemm_small_batch(N, K, dq, ds, dX, dY, batch)
+        ws = torch.zeros(vq.vq_int4g128_workspace_bytes(N, batch), dtype=torch.uint8, device="cuda")
+        vq.vq_int4g128_gemm_small_batch(N, K, dq, ds, dX, dY, batch, ws)
         torch.cuda.synchronize()
         assert_outputs_close(dY.cpu().numpy(), Y, A, f"int4 {N}x{K} b{batch}")
 
@@ -399,7 +400,7 @@ def test_host_buffer_entry_point():
     X = vq_synth.make_x(spec, 2, batch)
     hX = torch.from_numpy(X).pin_memory()
     hY = torch.zeros((batch, spec.N), dtype=torch.float16).pin_memory()
-    ws = torch.empty(vq.vq_workspace_bytes_host(dev.fmt, batch), dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(vq.vq_workspace_bytes_host(dev.fmt, batch), dtype=torch.uint8, device="cuda")
     vq.vq_gemm_small_batch_host(dev.fmt, dev.idx, dev.cb, dev.scale, hX, hY, batch, ws)
     torch.cuda.synchronize()
     assert np.array_equal(hY.numpy().view(np.uint16), dev.gemm(X).view(np.uint16))

@@ -127,10 +127,13 @@ def test_argument_errors_before_any_launch():
     assert lib.vq_gemm_small_batch_host(ctypes.byref(c), FAKE, FAKE, None, None, FAKE, 1, FAKE, 1 << 30, None) == 1
     assert lib.vq_gemm_small_batch_host(ctypes.byref(c), FAKE, FAKE, None, FAKE, FAKE, 1, FAKE, 16, None) == 5
     # INT4 yard-stick
-    assert lib.vq_int4g128_gemm_small_batch(8, 100, FAKE, FAKE, FAKE, FAKE, 1, None) == 3
-    assert lib.vq_int4g128_gemm_small_batch(8, 256, None, FAKE, FAKE, FAKE, 1, None) == 1
-    assert lib.vq_int4g128_gemm_small_batch(8, 256, FAKE, FAKE, ODD, FAKE, 1, None) == 4
-    assert lib.vq_int4g128_gemm_small_batch(8, 256, FAKE, FAKE, FAKE, FAKE, 0, None) == 6
+    assert lib.vq_int4g128_gemm_small_batch(8, 100, FAKE, FAKE, FAKE, FAKE, 1, FAKE, 1 << 30, None) == 3
+    assert lib.vq_int4g128_gemm_small_batch(8, 256, None, FAKE, FAKE, FAKE, 1, FAKE, 1 << 30, None) == 1
+    assert lib.vq_int4g128_gemm_small_batch(8, 256, FAKE, FAKE, ODD, FAKE, 1, FAKE, 1 << 30, None) == 4
+    assert lib.vq_int4g128_gemm_small_batch(8, 256, FAKE, FAKE, FAKE, FAKE, 0, FAKE, 1 << 30, None) == 6
+    assert lib.vq_int4g128_gemm_small_batch(8, 256, FAKE, FAKE, FAKE, FAKE, 1, None, 1 << 30, None) == 5
+    assert lib.vq_int4g128_gemm_small_batch(8, 256, FAKE, FAKE, FAKE, FAKE, 1, FAKE, 16, None) == 5
+    assert vq.vq_int4g128_workspace_bytes(8, 1) > 0 and vq.vq_int4g128_workspace_bytes(8, 17) == 0
 
 
 def test_status_strings():

@@ -50,7 +50,7 @@ def test_static_scratch_variant_matches_workspace_variant_twice(spec):
         hX = torch.from_numpy(X).pin_memory()
         # existing entry point: caller-allocated workspace
         hY_ref = torch.zeros((batch, spec.N), dtype=torch.float16).pin_memory()
-        ws = torch.empty(vq.vq_workspace_bytes_host(dev.fmt, batch), dtype=torch.uint8, device="cuda")
+        ws = torch.zeros(vq.vq_workspace_bytes_host(dev.fmt, batch), dtype=torch.uint8, device="cuda")
         vq.vq_gemm_small_batch_host(dev.fmt, dev.idx, dev.cb, dev.scale, hX, hY_ref, batch, ws)
         torch.cuda.synchronize()
         # new entry point: no workspace argument at all
