@@ -39,6 +39,21 @@ namespace {
 
 using namespace dev;
 
+#ifndef VQ_UNROLL_D2
+#define VQ_UNROLL_D2 2   // index-word steps of the 2-D loop emitted back to back (the loop body must stay small: the
+#endif                  // kernel is sensitive to instruction-cache misses)
+#ifndef VQ_UNROLL_D1
+#define VQ_UNROLL_D1 4
+#endif
+// Index-word steps of the decode loops that are emitted back to back (8 = the whole chunk; measured
+// on B200: 1, 2, 4, 8 steps give 32.3 / 31.4 / 30.7 / 30.0 us on a 28672 x 8192 layer).
+#ifndef VQ_UNROLL_D2
+#define VQ_UNROLL_D2 8
+#endif
+#ifndef VQ_UNROLL_D1
+#define VQ_UNROLL_D1 8
+#endif
+constexpr int kUnrollD2 = VQ_UNROLL_D2, kUnrollD1 = VQ_UNROLL_D1;
 constexpr int kWaitTries = 1 << 18;   // polls (with a sleep of 40-500 ns in between) before a wait gives up
 
 struct Segment {
@@ -85,6 +100,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 // leaves the issue slots of its scheduler to the warps that compute.  Returns false if the phase
 // did not complete within the attempts.
 __device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity, int max_tries, unsigned ns) {
+#pragma unroll 1
   for (int i = 0; i < max_tries; ++i) {
     uint32_t done;
     asm volatile(
@@ -351,7 +367,7 @@ struct RowD2B4 {
       const uint32_t sw = static_cast<uint32_t>(lane >> 2) << 4;
       const uint32_t t32 = static_cast<uint32_t>(lane & 3) << 5;
       uint4 b[NB][2];
-#pragma unroll
+#pragma unroll kUnrollD2
       for (int ww = 0; ww < 8; ++ww) {
 #pragma unroll
         for (int nb = 0; nb < NB; ++nb) {
@@ -451,7 +467,7 @@ struct RowD1B4I8 {
       const uint32_t sw = static_cast<uint32_t>(lane >> 2) << 4;
       const uint32_t t16 = static_cast<uint32_t>(lane & 3) << 4;
       uint4 b[NB];
-#pragma unroll
+#pragma unroll kUnrollD1
       for (int ww = 0; ww < 8; ++ww) {
 #pragma unroll
         for (int nb = 0; nb < NB; ++nb) b[nb] = *reinterpret_cast<const uint4*>(xrow[nb] + ww * xstep + t16);
@@ -535,7 +551,7 @@ struct RowInt4G128 {
       const uint32_t sw = static_cast<uint32_t>(lane >> 2) << 4;
       const uint32_t t16 = static_cast<uint32_t>(lane & 3) << 4;
       uint4 b[NB];
-#pragma unroll
+#pragma unroll 1
       for (int grp = 0; grp < 2; ++grp) {
         float acc[R][NB][4];
 #pragma unroll
@@ -544,7 +560,7 @@ struct RowInt4G128 {
           for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc[r][nb][e] = 0.f;
-#pragma unroll
+#pragma unroll kUnrollD1
         for (int w4 = 0; w4 < 4; ++w4) {
           const int ww = 4 * grp + w4;
 #pragma unroll
@@ -795,23 +811,30 @@ stream_kernel(const __grid_constant__ Maps maps, const StreamArgs a) {
   };
 
   int ev = 0;
+  int slot = 0;             // k % D and the parity of k / D, kept incrementally
+  uint32_t phase = 0;
   Where cur = where(wk_.slab, wk_.s);
   if (wk_.n > 0) st.prefetch(a, cur, lane);
   for (; wk_.k < wk_.n;) {
-    const int k = wk_.k, slot = k % D;
     const bool slab_end = wk_.slab_end(a);
+    const int slab_before = wk_.slab;
     st.begin(a, cur, lane, total);
     wk_.next(a);
     Where nxt = cur;
     if (wk_.k < wk_.n) {   // the stage after this one: request its codebook if it is another block
-      nxt = where(wk_.slab, wk_.s);
+      if (wk_.slab == slab_before) {   // same slab: the next chunk of the same rows
+        nxt.ch = cur.ch + 1;
+        nxt.key = slab_before * a.blocks_per_row + (nxt.ch >> a.cpb_shift);
+      } else {
+        nxt = where(wk_.slab, wk_.s);
+      }
       st.prefetch(a, nxt, lane);
     }
-    if (!dead && !mbar_wait_idle(full0 + 8 * slot, (k / D) & 1, kWaitTries, 40)) {
+    if (!dead && !mbar_wait_idle(full0 + 8 * slot, phase, kWaitTries, 40)) {
       if (lane == 0) atomicAdd(a.error_flag, 1);
       dead = true;
     }
-    dead = __any_sync(0xffffffffu, dead);
+    dead = __any_sync(0xffffffffu, dead);   // (a vote outside the branch: the warp stays converged)
     if (!dead) {
       const unsigned char* stage = smem + a.stage_off + slot * a.stage_bytes;
       const unsigned char* idx = stage + wk * a.idx_part_bytes + (wr * (16 * R) + g) * P::CHUNK_BYTES + t * 4;
@@ -822,6 +845,10 @@ stream_kernel(const __grid_constant__ Maps maps, const StreamArgs a) {
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(empty0 + 8 * slot);
+    if (++slot == D) {
+      slot = 0;
+      phase ^= 1u;
+    }
 
     if (slab_end) {
       // ---- hand the slab's partial sums to the results warp ----
@@ -980,11 +1007,20 @@ vq_status launch(const StreamCall& call, int chunks_per_block, cudaStream_t s) {
   const long long tail = static_cast<long long>(left) * a.S;
   a.tail_units = static_cast<int>(tail);
   a.tail_ctas = static_cast<int>(tail < Pn ? tail : Pn);
-  // left-over slabs are not split (a CTA takes a whole one) when that costs little balance
-  if (env_int("VQ_NOSPLIT", 0)) a.tail_ctas = left;
+  // Left-over slabs are either cut into stages shared evenly by all CTAs (their partial sums then meet
+  // through the workspace, which costs about two stage times at the end of the kernel) or handed out
+  // whole, one per CTA, whichever ends earlier.
+  const double t_split = static_cast<double>(slabs) * a.S / Pn + 2.0;
+  const double t_whole = static_cast<double>(a.q + (left > 0 ? 1 : 0)) * a.S;
+  if (env_int("VQ_NOSPLIT", t_whole <= t_split ? 1 : 0)) a.tail_ctas = left;
   if (a.q == 0) Pn = a.tail_ctas;   // fewer stages than CTAs: the others would have nothing to do
   if (Pn < 1) return VQ_ERR_UNSUPPORTED;
-  const size_t ticket_bytes = round_up(static_cast<size_t>(slabs) * sizeof(int), 256);
+  // the counters take the same room whatever the slab height, so that the partial sums of one call
+  // never land where another call (other batch size, other tiling) keeps its counters
+  long long rows_total = 0;
+  for (int i = 0; i < call.n_seg; ++i) rows_total += call.N[i];
+  const size_t ticket_bytes = stream_ticket_bytes(rows_total);
+  if (static_cast<size_t>(slabs) * sizeof(int) > ticket_bytes) return VQ_ERR_UNSUPPORTED;
   const size_t part_ws = static_cast<size_t>(Pn) * 2 * slab_rows * batch * sizeof(float);
   if (!call.ws || call.ws_bytes < ticket_bytes + part_ws) return VQ_ERR_WORKSPACE;
   a.ws_ticket = static_cast<int*>(call.ws);

@@ -79,9 +79,12 @@ vq_status device_error_counter(int** d_counter) {
   return VQ_OK;
 }
 
+size_t stream_ticket_bytes(long long rows) {
+  return (static_cast<size_t>((rows + 15) / 16 + kMaxSegments) * sizeof(int) + 255) / 256 * 256;
+}
+
 size_t stream_workspace_bytes(long long rows, int batch) {
-  const size_t tickets = (static_cast<size_t>((rows + 15) / 16 + kMaxSegments) * sizeof(int) + 255) / 256 * 256;
-  return tickets + static_cast<size_t>(kMaxStreamCtas) * 2 * kMaxSlabRows * batch * sizeof(float);
+  return stream_ticket_bytes(rows) + static_cast<size_t>(kMaxStreamCtas) * 2 * kMaxSlabRows * batch * sizeof(float);
 }
 
 vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch, void* ws,
