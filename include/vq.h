@@ -73,7 +73,9 @@ typedef enum {
 typedef enum {
   VQ_IMPL_AUTO = 0,     /* tuned kernel when one covers the format/shape, else the generic one   */
   VQ_IMPL_GENERIC = 1,  /* format-generic fp32-FMA kernel (any valid format)                     */
-  VQ_IMPL_TUNED = 2     /* tuned kernel only; VQ_ERR_UNSUPPORTED if none covers the format/shape */
+  VQ_IMPL_TUNED = 2,    /* tuned kernel only; VQ_ERR_UNSUPPORTED if none covers the format/shape */
+  VQ_IMPL_STREAM = 3    /* the persistent tuned kernel only (the one AUTO picks for large per-row 4-bit
+                           layers and for groups); VQ_ERR_UNSUPPORTED if it does not cover the format */
 } vq_impl;
 
 /* Caller-filled description of one VQ-compressed matrix (paper Sec. 2.1 notation in comments). */
@@ -143,6 +145,29 @@ vq_status vq_gemm_small_batch(const vq_format* fmt, const void* d_idx, const voi
 vq_status vq_gemm_small_batch_impl(const vq_format* fmt, const void* d_idx, const void* d_cb,
                                    const void* d_scale, const void* d_X, void* d_Y, int batch,
                                    void* d_ws, size_t ws_bytes, void* stream, int impl);
+
+/* Several layers that read the SAME activations in one call - the q/k/v or the gate/up projections of
+ * a transformer block (paper Sec. 3.2: every linear layer of a token step streams its own weights;
+ * grouping is this library's): Y_i[m][n] = sum_k W_i[n][k] X[m][k] for i < n_members.
+ *   fmt       : the members' common format and K; fmt->n_rows = the SUM of the members' rows
+ *               (it sizes the workspace: vq_workspace_bytes(fmt, batch)).
+ *   members   : HOST array of n_members (1..VQ_MAX_GROUP) entries; each holds the member's device
+ *               pointers (layouts as for vq_gemm_small_batch), its output d_Y (binary16
+ *               [batch][n_rows]) and its row count (a multiple of block_rows).
+ *   d_X       : device binary16 [batch][K], shared by all members.
+ * One kernel serves the whole group where the tuned persistent kernel covers the format; otherwise
+ * the members run one after the other on `stream`.  Results are the same as n_members separate calls.
+ * Errors: as vq_gemm_small_batch; SHAPE also if the rows do not add up to fmt->n_rows. */
+#define VQ_MAX_GROUP 4
+typedef struct {
+  const void* d_idx;
+  const void* d_cb;
+  const void* d_scale;   /* NULL iff cb_type == VQ_CB_FP16 */
+  void* d_Y;
+  int32_t n_rows;
+} vq_group_member;
+vq_status vq_gemm_small_batch_grouped(const vq_format* fmt, const vq_group_member* members, int n_members,
+                                      const void* d_X, int batch, void* d_ws, size_t ws_bytes, void* stream);
 
 /* Same computation with HOST activations and outputs: copies h_X (binary16 [batch][K]) to the
  * device, runs vq_gemm_small_batch, copies Y back into h_Y (binary16 [batch][N]); all three

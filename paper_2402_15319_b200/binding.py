@@ -9,7 +9,7 @@ import os
 from dataclasses import dataclass
 
 VQ_CB_FP16, VQ_CB_INT8_SCALED, VQ_CB_INT4_G128 = 0, 1, 2
-VQ_IMPL_AUTO, VQ_IMPL_GENERIC, VQ_IMPL_TUNED = 0, 1, 2
+VQ_IMPL_AUTO, VQ_IMPL_GENERIC, VQ_IMPL_TUNED, VQ_IMPL_STREAM = 0, 1, 2, 3
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libvq_b200.so")
@@ -80,6 +80,8 @@ _SIGNATURES = {
     "vq_gemv": (ctypes.c_int, [ctypes.c_void_p] * 7 + [ctypes.c_size_t, ctypes.c_void_p]),
     "vq_gemm_small_batch": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
     "vq_gemm_small_batch_impl": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_int]),
+    "vq_gemm_small_batch_grouped": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int,
+                                                   ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
     "vq_gemm_small_batch_host": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
     "vq_gemm_small_batch_host_static": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p]),
     "vq_static_scratch_bytes": (ctypes.c_size_t, []),
@@ -167,6 +169,22 @@ def vq_gemm_small_batch(fmt: VQFormat, d_idx, d_cb, d_scale, d_X, d_Y, batch: in
     _check(load().vq_gemm_small_batch(ctypes.byref(c), _ptr(d_idx), _ptr(d_cb), _ptr(d_scale), _ptr(d_X),
                                       _ptr(d_Y), int(batch), _ptr(d_ws), d_ws.numel() * d_ws.element_size(),
                                       _stream(stream)), "vq_gemm_small_batch")
+
+
+class _CGroupMember(ctypes.Structure):
+    _fields_ = [("d_idx", ctypes.c_void_p), ("d_cb", ctypes.c_void_p), ("d_scale", ctypes.c_void_p),
+                ("d_Y", ctypes.c_void_p), ("n_rows", ctypes.c_int32)]
+
+
+def vq_gemm_small_batch_grouped(fmt: VQFormat, members, d_X, batch: int, d_ws, stream=None) -> None:
+    """members: sequence of (d_idx, d_cb, d_scale, d_Y, n_rows); fmt.n_rows = the sum of the members' rows."""
+    arr = (_CGroupMember * len(members))()
+    for i, (idx, cb, sc, Y, n) in enumerate(members):
+        arr[i] = _CGroupMember(_ptr(idx), _ptr(cb), _ptr(sc), _ptr(Y), int(n))
+    c = fmt.c()
+    _check(load().vq_gemm_small_batch_grouped(ctypes.byref(c), arr, len(members), _ptr(d_X), int(batch), _ptr(d_ws),
+                                              d_ws.numel() * d_ws.element_size(), _stream(stream)),
+           "vq_gemm_small_batch_grouped")
 
 
 def vq_gemm_small_batch_impl(fmt: VQFormat, d_idx, d_cb, d_scale, d_X, d_Y, batch: int, d_ws, impl: int,

@@ -85,6 +85,8 @@ struct StreamArgs {
   int stage_bytes;       // a stage: WK index boxes, then WK activation boxes
   int x_off;             // activations inside a stage
   int idx_part_bytes, x_part_bytes;
+  int tbl_off, tbl_part_bytes;   // block policies: the stage's look-up tables
+  int Br, Bc, cb_int8;
   uint32_t tx_bytes;     // bytes the two loads of a stage bring
 };
 
@@ -225,9 +227,10 @@ __device__ __forceinline__ void load_words(const unsigned char* idx, int ww, uin
 // the entry index sits in address bits 8..11 and merges with the lane's address by one logic op.
 template <bool INT8>
 struct RowD2B4 {
-  static constexpr int CHUNK_BYTES = 128, CHUNK_COLS = 512, X_ROW_BYTES = 128;
-  static constexpr bool X_SWIZZLE = true;
+  static constexpr int CHUNK_BYTES = 128, CHUNK_COLS = 512, X_ROW_BYTES = 128, X_ROWS = 8, LANE_BYTES = 4;
+  static constexpr bool X_SWIZZLE = true, IDX_SWIZZLE = true, X_BATCH_INNER = true;
   static constexpr int TILE_TABLE_BYTES = 4096;   // per 16-row tile
+  static constexpr int STAGE_TABLE_BYTES = 0, BASE_ALIGN = 4096;
   static constexpr int CB_ROW_BYTES = INT8 ? 32 : 64;
   static constexpr int RAW = INT8 ? 2 : 4;
 
@@ -360,10 +363,14 @@ struct RowD2B4 {
       }
     }
 
-    // idx: the warp's box rows + g*128 + t*4 (tile r 2048 bytes further); xrow[nb]: row (w = 0, batch
-    // row) of the activation box, xstep = batch * 128 bytes to the next w.
-    __device__ __forceinline__ void compute(const unsigned char* idx, const unsigned char* const (&xrow)[NB], uint32_t xstep,
-                                            int lane, float (&)[R][NB][4]) {
+    // idx: the warp's box rows + g*128 + t*4 (tile r 2048 bytes further); xpart: the part's activation
+    // box [w][batch row][128 bytes]; xm[nb]: the lane's batch rows.
+    __device__ __forceinline__ void compute(const unsigned char* idx, const unsigned char* xpart, const int (&xm)[NB], int batch,
+                                            uint32_t, int lane, float (&)[R][NB][4]) {
+      const unsigned char* xrow[NB];
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb) xrow[nb] = xpart + xm[nb] * X_ROW_BYTES;
+      const uint32_t xstep = batch * X_ROW_BYTES;
       const uint32_t sw = static_cast<uint32_t>(lane >> 2) << 4;
       const uint32_t t32 = static_cast<uint32_t>(lane & 3) << 5;
       uint4 b[NB][2];
@@ -390,9 +397,10 @@ struct RowD2B4 {
 // are looked up with byte permutes, the register-file analogue of the paper's LUT instruction
 // (Sec. 3.2: index -> 8-bit value); bytes become fp16 by the 0x6400 exponent trick, exactly.
 struct RowD1B4I8 {
-  static constexpr int CHUNK_BYTES = 128, CHUNK_COLS = 256, X_ROW_BYTES = 64;
-  static constexpr bool X_SWIZZLE = false;
+  static constexpr int CHUNK_BYTES = 128, CHUNK_COLS = 256, X_ROW_BYTES = 64, X_ROWS = 8, LANE_BYTES = 4;
+  static constexpr bool X_SWIZZLE = false, IDX_SWIZZLE = true, X_BATCH_INNER = true;
   static constexpr int TILE_TABLE_BYTES = 0;
+  static constexpr int STAGE_TABLE_BYTES = 0, BASE_ALIGN = 4096;
 
   template <int NB, int R>
   struct State {
@@ -462,8 +470,12 @@ struct RowD1B4I8 {
         cur_key = w.key;
       }
     }
-    __device__ __forceinline__ void compute(const unsigned char* idx, const unsigned char* const (&xrow)[NB], uint32_t xstep,
-                                            int lane, float (&)[R][NB][4]) {
+    __device__ __forceinline__ void compute(const unsigned char* idx, const unsigned char* xpart, const int (&xm)[NB], int batch,
+                                            uint32_t, int lane, float (&)[R][NB][4]) {
+      const unsigned char* xrow[NB];
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb) xrow[nb] = xpart + xm[nb] * X_ROW_BYTES;
+      const uint32_t xstep = batch * X_ROW_BYTES;
       const uint32_t sw = static_cast<uint32_t>(lane >> 2) << 4;
       const uint32_t t16 = static_cast<uint32_t>(lane & 3) << 4;
       uint4 b[NB];
@@ -507,9 +519,10 @@ struct RowD1B4I8 {
 // 1024 + 16*q_hi); one fused multiply-add by (1, 1/16) and (-1032, -72) makes it (q_lo - 8, q_hi - 8),
 // exactly.
 struct RowInt4G128 {
-  static constexpr int CHUNK_BYTES = 128, CHUNK_COLS = 256, X_ROW_BYTES = 64;
-  static constexpr bool X_SWIZZLE = false;
+  static constexpr int CHUNK_BYTES = 128, CHUNK_COLS = 256, X_ROW_BYTES = 64, X_ROWS = 8, LANE_BYTES = 4;
+  static constexpr bool X_SWIZZLE = false, IDX_SWIZZLE = true, X_BATCH_INNER = true;
   static constexpr int TILE_TABLE_BYTES = 0;
+  static constexpr int STAGE_TABLE_BYTES = 0, BASE_ALIGN = 4096;
 
   template <int NB, int R>
   struct State {
@@ -544,8 +557,12 @@ struct RowInt4G128 {
         cur_key = w.key;
       }
     }
-    __device__ __forceinline__ void compute(const unsigned char* idx, const unsigned char* const (&xrow)[NB], uint32_t xstep,
-                                            int lane, float (&total)[R][NB][4]) {
+    __device__ __forceinline__ void compute(const unsigned char* idx, const unsigned char* xpart, const int (&xm)[NB], int batch,
+                                            uint32_t, int lane, float (&total)[R][NB][4]) {
+      const unsigned char* xrow[NB];
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb) xrow[nb] = xpart + xm[nb] * X_ROW_BYTES;
+      const uint32_t xstep = batch * X_ROW_BYTES;
       constexpr uint32_t kMul = 0x2C003C00u;    // fp16 pair (1, 1/16)
       constexpr uint32_t kAdd = 0xD480E408u;    // fp16 pair (-1032, -72)
       const uint32_t sw = static_cast<uint32_t>(lane >> 2) << 4;
@@ -604,15 +621,175 @@ struct RowInt4G128 {
 };
 
 // =============================================================================================
+// Block policy: 2-D codebooks of 64 entries (6-bit indices) shared by a tall block of rows (fp16, or
+// int8 whose entries enter the tables as fp16(scale * c)).  Chunk = 96 bytes of a row = 128 indices
+// = 256 columns; lane (g, t) owns the 32 indices (24 bytes, read as three 64-bit words: conflict-free
+// with rows 96 bytes apart) of columns 64t .. 64t+63 of rows g and g+8.  A helper warp replicates the
+// chunk's codebooks into a lane-private table of the stage, word (entry, lane) at entry*128 + lane*4:
+// lanes t < 2 see the block under columns 0..127 of the chunk, lanes t >= 2 the block under columns
+// 128..255.  The activations of the chunk lie as [batch row][t][128 bytes] (128-byte swizzle).
+// =============================================================================================
+struct BlkD2B6 {
+  static constexpr int CHUNK_BYTES = 96, CHUNK_COLS = 256, X_ROW_BYTES = 128, X_ROWS = 4, LANE_BYTES = 24;
+  static constexpr bool X_SWIZZLE = true, IDX_SWIZZLE = false, X_BATCH_INNER = false;
+  static constexpr int TILE_TABLE_BYTES = 0;
+  static constexpr int STAGE_TABLE_BYTES = 8192, BASE_ALIGN = 8192;
+  static constexpr uint32_t MASK = 63u << 7;
+
+  template <int I>   // (index I of the lane's 32) * 128
+  static __device__ __forceinline__ uint32_t entry_off(const uint32_t (&w)[6]) {
+    constexpr int p = 6 * I;
+    if constexpr (p < 7) {
+      return (w[0] << (7 - p)) & MASK;
+    } else {
+      constexpr int q = p - 7, wi = q >> 5, sft = q & 31;
+      if constexpr (sft == 0) return w[wi] & MASK;
+      else if constexpr (sft + 13 > 32) return __funnelshift_r(w[wi], w[wi + 1], sft) & MASK;
+      else return (w[wi] >> sft) & MASK;
+    }
+  }
+
+  // The helper warp's share of one part's table: lane l converts entries 2l, 2l+1 of the two blocks
+  // under the chunk (requested one stage ahead by load()) and writes each 8 times with 128-bit stores
+  // whose 16-byte groups are rotated by the lane (the 8 lanes of a quarter warp hit 8 different groups).
+  struct Builder {
+    uint32_t raw[2][2];   // [block A / B][entry 2l, 2l+1] (int8: both entries in raw[.][0])
+    float sc[2];
+    __device__ __forceinline__ void load(const StreamArgs& a, const Segment& sg, int row0, int ch, int lane) {
+      const long long brow = static_cast<long long>(row0 >> a.br_shift) * a.blocks_per_row;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const long long blk = brow + (ch * CHUNK_COLS + h * 128) / a.Bc;
+        if (a.cb_int8) {
+          raw[h][0] = __ldg(reinterpret_cast<const uint32_t*>(static_cast<const uint16_t*>(sg.cb) + blk * 64 + 2 * lane));
+          raw[h][1] = 0u;
+          sc[h] = __half2float(__ldg(sg.scale + blk));
+        } else {
+          const uint2 v = ldg64_nc(static_cast<const uint32_t*>(sg.cb) + blk * 64 + 2 * lane);
+          raw[h][0] = v.x;
+          raw[h][1] = v.y;
+          sc[h] = 1.f;
+        }
+      }
+    }
+    __device__ __forceinline__ void store(const StreamArgs& a, uint32_t table, int lane) const {
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        uint32_t e[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (a.cb_int8) {
+            const uint32_t two = raw[h][0] >> (16 * i);
+            const __half2 hv = __halves2half2(__float2half_rn(sc[h] * static_cast<float>(static_cast<int8_t>(two & 0xff))),
+                                              __float2half_rn(sc[h] * static_cast<float>(static_cast<int8_t>((two >> 8) & 0xff))));
+            e[h] = *reinterpret_cast<const uint32_t*>(&hv);
+          } else {
+            e[h] = raw[h][i];
+          }
+        }
+        const uint4 v = make_uint4(e[0], e[0], e[1], e[1]);
+        const uint32_t row = table + (2 * lane + i) * 128;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) sts128(row + ((j + lane) & 7) * 16, v);
+      }
+    }
+  };
+
+  template <int NB, int R>
+  struct State {
+    float acc[R][NB][4];
+    __device__ __forceinline__ void init(uint32_t, int) {
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) acc[r][nb][e] = 0.f;
+    }
+    __device__ __forceinline__ void prefetch(const StreamArgs&, const Where&, int) {}
+    __device__ __forceinline__ void begin(const StreamArgs&, const Where&, int, float (&)[R][NB][4]) {}
+    __device__ __forceinline__ void settle() {
+#pragma unroll
+      for (int r = 0; r < R; ++r) fence_acc(acc[r]);
+    }
+    __device__ __forceinline__ void flush(float (&total)[R][NB][4]) {
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            total[r][nb][e] += acc[r][nb][e];
+            acc[r][nb][e] = 0.f;
+          }
+    }
+
+    template <int J, int RR>
+    __device__ __forceinline__ void piece_step(const uint32_t (&wl)[6], const uint32_t (&wh)[6], uint32_t tbl, const uint4 (&b)[NB]) {
+      // indices 4J .. 4J+3 of rows g and g+8: two tensor-core steps
+      uint32_t af[2][4];
+      af[0][0] = lds32(entry_off<4 * J>(wl) | tbl);     af[0][1] = lds32(entry_off<4 * J>(wh) | tbl);
+      af[0][2] = lds32(entry_off<4 * J + 1>(wl) | tbl); af[0][3] = lds32(entry_off<4 * J + 1>(wh) | tbl);
+      af[1][0] = lds32(entry_off<4 * J + 2>(wl) | tbl); af[1][1] = lds32(entry_off<4 * J + 2>(wh) | tbl);
+      af[1][2] = lds32(entry_off<4 * J + 3>(wl) | tbl); af[1][3] = lds32(entry_off<4 * J + 3>(wh) | tbl);
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb) {
+        mma16816(acc[RR][nb], af[0][0], af[0][1], af[0][2], af[0][3], b[nb].x, b[nb].y);
+        mma16816(acc[RR][nb], af[1][0], af[1][1], af[1][2], af[1][3], b[nb].z, b[nb].w);
+      }
+    }
+
+    template <int J>
+    __device__ __forceinline__ void piece(const uint32_t (&w)[R][2][6], uint32_t tbl, const unsigned char* const (&xrow)[NB],
+                                          const uint32_t (&ph)[NB]) {
+      uint4 b[NB];
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb) b[nb] = *reinterpret_cast<const uint4*>(xrow[nb] + ((16u * J) ^ ph[nb]));
+      piece_step<J, 0>(w[0][0], w[0][1], tbl, b);
+      if constexpr (R > 1) piece_step<J, 1>(w[1][0], w[1][1], tbl, b);
+      if constexpr (R > 2) piece_step<J, 2>(w[2][0], w[2][1], tbl, b);
+      if constexpr (R > 3) piece_step<J, 3>(w[3][0], w[3][1], tbl, b);
+    }
+
+    // idx: the warp's box rows + g*96 + t*24 (tile r 16 rows further); xpart: [batch row][t][128 bytes];
+    // table: shared address of the part's table.
+    __device__ __forceinline__ void compute(const unsigned char* idx, const unsigned char* xpart, const int (&xm)[NB], int,
+                                            uint32_t table, int lane, float (&)[R][NB][4]) {
+      uint32_t w[R][2][6];
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int q = 0; q < 3; ++q) {
+            const uint2 v = *reinterpret_cast<const uint2*>(idx + (r * 16 + h * 8) * CHUNK_BYTES + 8 * q);
+            w[r][h][2 * q] = v.x;
+            w[r][h][2 * q + 1] = v.y;
+          }
+      const unsigned char* xrow[NB];
+      uint32_t ph[NB];
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb) {
+        xrow[nb] = xpart + (xm[nb] * 4 + (lane & 3)) * X_ROW_BYTES;
+        ph[nb] = (static_cast<uint32_t>(reinterpret_cast<uintptr_t>(xrow[nb])) >> 3) & 0x70u;
+      }
+      const uint32_t tbl = table + lane * 4;
+      piece<0>(w, tbl, xrow, ph); piece<1>(w, tbl, xrow, ph); piece<2>(w, tbl, xrow, ph); piece<3>(w, tbl, xrow, ph);
+      piece<4>(w, tbl, xrow, ph); piece<5>(w, tbl, xrow, ph); piece<6>(w, tbl, xrow, ph); piece<7>(w, tbl, xrow, ph);
+    }
+  };
+};
+
+// =============================================================================================
 // The kernel.  Grid (P), block (W + 2) warps: warps 0..W-1 consume (warp = wk*WR + wr), warp W produces
 // (one thread), warp W+1 writes the results.  CW = the most consumer warps a launch may use (4: two
 // CTAs per SM, 8: one), which fixes the registers a thread may take.
 // =============================================================================================
 template <class P, int NB, int R, int CW>
-__global__ void __launch_bounds__((CW + 2) * 32, CW <= 4 ? 2 : 1)
+__global__ void __launch_bounds__((CW + 3) * 32, CW <= 4 ? 2 : 1)
 stream_kernel(const __grid_constant__ Maps maps, const StreamArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  const uint32_t sbase = (smem_u32(smem_raw) + 4095u) & ~4095u;
+  const uint32_t sbase = (smem_u32(smem_raw) + (P::BASE_ALIGN - 1)) & ~static_cast<uint32_t>(P::BASE_ALIGN - 1);
   unsigned char* smem = smem_raw + (sbase - smem_u32(smem_raw));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int W = a.WR * a.WK;
@@ -625,7 +802,7 @@ stream_kernel(const __grid_constant__ Maps maps, const StreamArgs a) {
 
   if (tid == 0) {
     for (int i = 0; i < D; ++i) {
-      mbar_init(full0 + 8 * i, 1);
+      mbar_init(full0 + 8 * i, P::STAGE_TABLE_BYTES ? 2 : 1);   // the producer's arrival (+ the table builder's)
       mbar_init(empty0 + 8 * i, W);
     }
     for (int i = 0; i < 2; ++i) {
@@ -675,10 +852,44 @@ stream_kernel(const __grid_constant__ Maps maps, const StreamArgs a) {
         pdl_wait();
         waited = true;
       }
-      // activations: {row bytes, batch, w = 0..7, WK parts} at (0, 0, box row s*8 of a part, part 0)
-      tma_box_4d(stage + a.x_off, &maps.x, 0, 0, wk_.s * 8, 0, full);
+      // activations of the stage's columns: box rows s*X_ROWS .. of every part
+      if constexpr (P::X_BATCH_INNER) tma_box_4d(stage + a.x_off, &maps.x, 0, 0, wk_.s * P::X_ROWS, 0, full);
+      else tma_box_4d(stage + a.x_off, &maps.x, 0, wk_.s * P::X_ROWS, 0, 0, full);
     }
     return;
+  }
+
+  // ------------------------------------------------------------------------------------------
+  // table builder (formats whose codebook is shared by a block of rows): one warp replicates the
+  // codebooks under every stage's chunks into the stage's lane-private tables, one stage ahead of
+  // its global loads
+  // ------------------------------------------------------------------------------------------
+  if constexpr (P::STAGE_TABLE_BYTES > 0) {
+    if (warp == W + 2) {
+      typename P::Builder cur[2], nxt[2];   // at most two column parts per stage
+      auto request = [&](typename P::Builder (&b)[2], const Walk& w) {
+        const int sg = segment_of(w.slab);
+        const int row0 = (w.slab - a.seg[sg].slab0) * slab_rows;
+        for (int p = 0; p < a.WK && p < 2; ++p) b[p].load(a, a.seg[sg], row0, p * a.S + w.s, lane);
+      };
+      if (wk_.n > 0) request(cur, wk_);
+      for (; wk_.k < wk_.n;) {
+        const int k = wk_.k, slot = k % D;
+        wk_.next(a);
+        if (wk_.k < wk_.n) request(nxt, wk_);
+        if (k >= D && !mbar_wait_idle(empty0 + 8 * slot, ((k / D) & 1) ^ 1, kWaitTries, 200)) {
+          if (lane == 0) atomicAdd(a.error_flag, 1);
+          break;
+        }
+        const uint32_t tables = sbase + a.stage_off + slot * a.stage_bytes + a.tbl_off;
+        for (int p = 0; p < a.WK && p < 2; ++p) cur[p].store(a, tables + p * a.tbl_part_bytes, lane);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(full0 + 8 * slot);
+        cur[0] = nxt[0];
+        cur[1] = nxt[1];
+      }
+      return;
+    }
   }
 
   // ------------------------------------------------------------------------------------------
@@ -761,22 +972,40 @@ stream_kernel(const __grid_constant__ Maps maps, const StreamArgs a) {
           const int first_u = (ps - wk_.tail_slab0) * a.S, last_u = first_u + a.S - 1;
           const int c_first = static_cast<int>((static_cast<long long>(first_u + 1) * Pt - 1) / T);
           const int c_last = static_cast<int>((static_cast<long long>(last_u + 1) * Pt - 1) / T);
-          for (int o = lane; o < n_out; o += 32) {
-            const int n = o >> a.sr_shift, rr = o & (slab_rows - 1);
-            float sum = 0.f;
-            for (int qc = c_first; qc <= c_last; ++qc) {
-              const int q_t0 = static_cast<int>(T * qc / Pt);
-              const int q_slot = (wk_.tail_slab0 + q_t0 / a.S == ps) ? 0 : 1;
-              sum += ldcg_f32(a.ws_part + (static_cast<long long>(qc) * 2 + q_slot) * n_out + o);
+          // four adjacent outputs per lane and pass; the contributors' values are requested eight at a
+          // time before any is used (the loads overlap), and added in CTA order
+          for (int o = 4 * lane; o < n_out; o += 128) {
+            float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int q0 = c_first; q0 <= c_last; q0 += 8) {
+              float4 v[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const int qc = q0 + i;
+                v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (qc <= c_last) {
+                  const int q_t0 = static_cast<int>(T * qc / Pt);
+                  const int q_slot = (wk_.tail_slab0 + q_t0 / a.S == ps) ? 0 : 1;
+                  v[i] = __ldcg(reinterpret_cast<const float4*>(a.ws_part + (static_cast<long long>(qc) * 2 + q_slot) * n_out + o));
+                }
+              }
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                sum.x += v[i].x; sum.y += v[i].y; sum.z += v[i].z; sum.w += v[i].w;
+              }
             }
-            if (prow0 + rr < sp.N) sp.Y[static_cast<long long>(n) * sp.N + prow0 + rr] = __float2half_rn(sum);
+            const float sv[4] = {sum.x, sum.y, sum.z, sum.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int n = (o + j) >> a.sr_shift, rr = (o + j) & (slab_rows - 1);
+              if (prow0 + rr < sp.N) sp.Y[static_cast<long long>(n) * sp.N + prow0 + rr] = __float2half_rn(sv[j]);
+            }
           }
         }
       }
     }
     return;
   }
-  if (warp > W + 1) return;
+  if (warp > W + 1) return;   // (lanes of no role)
 
   // ------------------------------------------------------------------------------------------
   // consumers
@@ -799,7 +1028,6 @@ stream_kernel(const __grid_constant__ Maps maps, const StreamArgs a) {
   int xm[NB];
 #pragma unroll
   for (int nb = 0; nb < NB; ++nb) xm[nb] = min(nb * 8 + g, a.batch - 1);
-  const uint32_t xstep = a.batch * P::X_ROW_BYTES;
 
   auto where = [&](int slab, int s) {
     Where w;
@@ -837,11 +1065,11 @@ stream_kernel(const __grid_constant__ Maps maps, const StreamArgs a) {
     dead = __any_sync(0xffffffffu, dead);   // (a vote outside the branch: the warp stays converged)
     if (!dead) {
       const unsigned char* stage = smem + a.stage_off + slot * a.stage_bytes;
-      const unsigned char* idx = stage + wk * a.idx_part_bytes + (wr * (16 * R) + g) * P::CHUNK_BYTES + t * 4;
-      const unsigned char* xrow[NB];
-#pragma unroll
-      for (int nb = 0; nb < NB; ++nb) xrow[nb] = stage + a.x_off + wk * a.x_part_bytes + xm[nb] * P::X_ROW_BYTES;
-      st.compute(idx, xrow, xstep, lane, total);
+      const unsigned char* idx = stage + wk * a.idx_part_bytes + (wr * (16 * R) + g) * P::CHUNK_BYTES + t * P::LANE_BYTES;
+      const uint32_t table = sbase + a.stage_off + slot * a.stage_bytes + a.tbl_off + wk * a.tbl_part_bytes;
+      st.compute(idx, stage + a.x_off + wk * a.x_part_bytes, xm, a.batch, table, lane, total);
+      // the stage's tables may be rewritten once it is released: its look-ups are done before
+      if constexpr (P::STAGE_TABLE_BYTES > 0) st.settle();
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(empty0 + 8 * slot);
@@ -908,7 +1136,7 @@ vq_status device_sms(int* out) {
 constexpr size_t kSmemMax = 224 * 1024;
 
 template <class P, int NB, int R, int CW>
-vq_status launch(const StreamCall& call, int chunks_per_block, cudaStream_t s) {
+vq_status launch(const StreamCall& call, int chunks_per_block, cudaStream_t s, int want_wk, int min_depth) {
   auto kern = stream_kernel<P, NB, R, CW>;
   static int attr_set[kMaxDevices] = {};
   int dev = 0;
@@ -943,10 +1171,19 @@ vq_status launch(const StreamCall& call, int chunks_per_block, cudaStream_t s) {
   int W = CW;
   int ctas_per_sm = env_int("VQ_CTAS", CW <= 4 ? 2 : 1);
   int WK = n_chunks % 4 == 0 ? 4 : n_chunks % 2 == 0 ? 2 : 1;
+  if (P::STAGE_TABLE_BYTES) {   // shared tables: as many row tiles of the block as the CTA has warps, then column parts
+    const int tiles = g.Br / (16 * R);
+    WK = tiles >= CW ? 1 : (n_chunks % 2 == 0 && CW / (tiles < 1 ? 1 : tiles) >= 2 ? 2 : 1);
+  }
+  if (want_wk > 0 && !P::STAGE_TABLE_BYTES) WK = want_wk;
   WK = env_int("VQ_WK", WK);
+  if (P::STAGE_TABLE_BYTES && WK > 2) return VQ_ERR_UNSUPPORTED;
   if (WK < 1 || n_chunks % WK || W % WK) return VQ_ERR_UNSUPPORTED;
-  int WR = env_int("VQ_WR", W / WK);
+  int WR = W / WK;
+  if (P::STAGE_TABLE_BYTES && WR > g.Br / (16 * R)) WR = g.Br / (16 * R);   // a slab stays inside one block row
+  WR = env_int("VQ_WR", WR);
   if (WR < 1 || WR * WK > CW || log2_exact(WR) < 0 || 16 * R * WR > kMaxSlabRows) return VQ_ERR_UNSUPPORTED;
+  if (P::STAGE_TABLE_BYTES && g.Br % (16 * R * WR)) return VQ_ERR_UNSUPPORTED;   // a slab lies inside one block row
   W = WR * WK;
   a.sr_shift = 4 + log2_exact(WR * R);
   a.WR = WR;
@@ -967,26 +1204,28 @@ vq_status launch(const StreamCall& call, int chunks_per_block, cudaStream_t s) {
 
   const size_t tbl_bytes = static_cast<size_t>(P::TILE_TABLE_BYTES) * R * W;
   const size_t red_bytes = 2 * static_cast<size_t>(W) * R * 16 * 8 * NB * sizeof(float);   // two buffers
-  const size_t idx_part = static_cast<size_t>(slab_rows) * P::CHUNK_BYTES;       // multiple of 2048
-  const size_t x_part = static_cast<size_t>(8) * batch * P::X_ROW_BYTES;         // [w][batch][row bytes]
-  const size_t x_off = idx_part * WK;
-  const size_t stage_bytes = round_up(x_off + x_part * WK, 1024);
-  if (P::X_SWIZZLE && x_part % 1024) return VQ_ERR_UNSUPPORTED;
+  const size_t idx_part = static_cast<size_t>(slab_rows) * P::CHUNK_BYTES;       // multiple of 512
+  const size_t x_part = static_cast<size_t>(P::X_ROWS) * batch * P::X_ROW_BYTES;
+  const size_t x_off = round_up(idx_part * WK, 1024);
+  const size_t tbl_off = round_up(x_off + x_part * WK, P::STAGE_TABLE_BYTES ? P::STAGE_TABLE_BYTES : 1024);
+  const size_t stage_bytes = round_up(tbl_off + static_cast<size_t>(P::STAGE_TABLE_BYTES) * WK, P::STAGE_TABLE_BYTES ? P::STAGE_TABLE_BYTES : 1024);
   const size_t red_off = tbl_bytes;
   const size_t bar_off = round_up(red_off + red_bytes, 16);
-  const size_t stage_off = round_up(bar_off + 16 * 16 + 32, 1024);
+  const size_t stage_off = round_up(bar_off + 16 * 16 + 32, P::STAGE_TABLE_BYTES ? P::STAGE_TABLE_BYTES : 1024);
   // shared memory of a CTA: the SM's 227 KB minus 1 KB per resident CTA, shared by the resident CTAs
   size_t budget = (227 * 1024 - 1024 * ctas_per_sm) / ctas_per_sm;
   if (budget > kSmemMax) budget = kSmemMax;
-  if (budget < stage_off + 4096 + 2 * stage_bytes) {   // does not fit twice: one CTA per SM
+  if (budget < stage_off + P::BASE_ALIGN + static_cast<size_t>(min_depth) * stage_bytes) {   // does not fit twice
+    if (CW <= 4) return VQ_ERR_UNSUPPORTED;   // (a 4-warp CTA alone on an SM would leave it half empty)
     ctas_per_sm = 1;
     budget = kSmemMax;
   }
-  int D = static_cast<int>((budget - 4096 - stage_off) / stage_bytes);
+  if (budget < stage_off + P::BASE_ALIGN + 2 * stage_bytes) return VQ_ERR_UNSUPPORTED;
+  int D = static_cast<int>((budget - P::BASE_ALIGN - stage_off) / stage_bytes);
   if (D > 8) D = 8;
   D = env_int("VQ_D", D);
-  if (D < 2 || D > 16) return VQ_ERR_UNSUPPORTED;
-  const size_t smem_bytes = stage_off + static_cast<size_t>(D) * stage_bytes + 4096;
+  if (D < min_depth || D > 16) return VQ_ERR_UNSUPPORTED;
+  const size_t smem_bytes = stage_off + static_cast<size_t>(D) * stage_bytes + P::BASE_ALIGN;
   if (smem_bytes > kSmemMax) return VQ_ERR_UNSUPPORTED;
   a.D = D;
   a.red_off = static_cast<int>(red_off);
@@ -996,6 +1235,11 @@ vq_status launch(const StreamCall& call, int chunks_per_block, cudaStream_t s) {
   a.x_off = static_cast<int>(x_off);
   a.idx_part_bytes = static_cast<int>(idx_part);
   a.x_part_bytes = static_cast<int>(x_part);
+  a.tbl_off = static_cast<int>(tbl_off);
+  a.tbl_part_bytes = P::STAGE_TABLE_BYTES;
+  a.Br = g.Br;
+  a.Bc = g.Bc;
+  a.cb_int8 = g.cb_int8;
   a.tx_bytes = static_cast<uint32_t>((idx_part + x_part) * WK);
 
   // ---- persistent CTAs: whole slabs first, the left-over stages shared evenly ----
@@ -1033,21 +1277,29 @@ vq_status launch(const StreamCall& call, int chunks_per_block, cudaStream_t s) {
     const uint64_t dims[3] = {static_cast<uint64_t>(a.S) * P::CHUNK_BYTES, static_cast<uint64_t>(call.N[i]), static_cast<uint64_t>(WK)};
     const uint64_t strides[2] = {static_cast<uint64_t>(g.stride), static_cast<uint64_t>(a.S) * P::CHUNK_BYTES};
     const uint32_t box[3] = {P::CHUNK_BYTES, static_cast<uint32_t>(slab_rows), static_cast<uint32_t>(WK)};
-    if (encode_tensor_map(&maps.idx[i], call.idx[i], 1, 3, dims, strides, box, 2) != VQ_OK) return VQ_ERR_CUDA;
+    if (encode_tensor_map(&maps.idx[i], call.idx[i], 1, 3, dims, strides, box, P::IDX_SWIZZLE ? 2 : 0) != VQ_OK) return VQ_ERR_CUDA;
   }
   for (int i = call.n_seg; i < kMaxSegments; ++i) maps.idx[i] = maps.idx[0];
   {
     // activations: columns of a row of the box, batch rows, box rows of a part, parts
     const uint32_t row_cols = P::X_ROW_BYTES / 2;
-    const uint64_t dims[4] = {row_cols, static_cast<uint64_t>(batch), static_cast<uint64_t>(a.S) * 8, static_cast<uint64_t>(WK)};
-    const uint64_t strides[3] = {static_cast<uint64_t>(g.K) * 2, P::X_ROW_BYTES, static_cast<uint64_t>(a.S) * 8 * P::X_ROW_BYTES};
-    const uint32_t box[4] = {row_cols, static_cast<uint32_t>(batch), 8u, static_cast<uint32_t>(WK)};
-    if (encode_tensor_map(&maps.x, call.X, 2, 4, dims, strides, box, P::X_SWIZZLE ? 2 : 0) != VQ_OK) return VQ_ERR_CUDA;
+    const uint64_t rows_per_part = static_cast<uint64_t>(a.S) * P::X_ROWS;   // box rows of X_ROW_BYTES in a part
+    if (P::X_BATCH_INNER) {   // shared memory [part][box row][batch row][row bytes]
+      const uint64_t dims[4] = {row_cols, static_cast<uint64_t>(batch), rows_per_part, static_cast<uint64_t>(WK)};
+      const uint64_t strides[3] = {static_cast<uint64_t>(g.K) * 2, P::X_ROW_BYTES, rows_per_part * P::X_ROW_BYTES};
+      const uint32_t box[4] = {row_cols, static_cast<uint32_t>(batch), P::X_ROWS, static_cast<uint32_t>(WK)};
+      if (encode_tensor_map(&maps.x, call.X, 2, 4, dims, strides, box, P::X_SWIZZLE ? 2 : 0) != VQ_OK) return VQ_ERR_CUDA;
+    } else {                  // shared memory [part][batch row][box row][row bytes]
+      const uint64_t dims[4] = {row_cols, rows_per_part, static_cast<uint64_t>(batch), static_cast<uint64_t>(WK)};
+      const uint64_t strides[3] = {P::X_ROW_BYTES, static_cast<uint64_t>(g.K) * 2, rows_per_part * P::X_ROW_BYTES};
+      const uint32_t box[4] = {row_cols, P::X_ROWS, static_cast<uint32_t>(batch), static_cast<uint32_t>(WK)};
+      if (encode_tensor_map(&maps.x, call.X, 2, 4, dims, strides, box, P::X_SWIZZLE ? 2 : 0) != VQ_OK) return VQ_ERR_CUDA;
+    }
   }
 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(Pn, 1, 1);
-  cfg.blockDim = dim3((W + 2) * 32, 1, 1);
+  cfg.blockDim = dim3((W + (P::STAGE_TABLE_BYTES ? 3 : 2)) * 32, 1, 1);
   cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
@@ -1077,15 +1329,29 @@ vq_status launch_tiles(const StreamCall& call, int chunks_per_block, cudaStream_
   long long rows = 0;
   for (int i = 0; i < call.n_seg; ++i) rows += call.N[i];
   int R = NB == 1 && rows >= 8192 ? 2 : 1;
+  // shared tables: two tiles per warp make a 4-warp CTA cover a whole 128-row block per table
+  if (P::STAGE_TABLE_BYTES) R = NB == 1 && call.g.Br >= 128 ? 2 : 1;
   R = env_int("VQ_R", R);
-  const int cw = env_int("VQ_W", 4);
-  if (cw == 8) {
-    if (NB == 1 && R == 2) return launch<P, NB, 2, 8>(call, chunks_per_block, s);
-    return launch<P, NB, 1, 8>(call, chunks_per_block, s);
-  }
-  if (NB == 1 && R == 2) return launch<P, NB, 2, 4>(call, chunks_per_block, s);
-  if (NB == 1 && R == 4) return launch<P, NB, 4, 4>(call, chunks_per_block, s);
-  return launch<P, NB, 1, 4>(call, chunks_per_block, s);
+  const int only_w = env_int("VQ_W", 0);
+  // CTA shapes in order of preference: two 4-warp CTAs per SM (a CTA of the next kernel of the stream
+  // can start beside one of this kernel) with as many column parts as fit, then one 8-warp CTA;
+  // first with at least three pipeline stages, then with two.
+  static const int kShapes[][2] = {{4, 4}, {4, 2}, {8, 4}, {8, 2}, {4, 1}, {8, 1}};
+  for (int min_depth = 3; min_depth >= 2; --min_depth)
+    for (const auto& sh : kShapes) {
+      const int cw = sh[0], wk = sh[1];
+      if (only_w && cw != only_w) continue;
+      vq_status st;
+      if (cw == 8) {
+        st = (NB == 1 && R == 2) ? launch<P, NB, 2, 8>(call, chunks_per_block, s, wk, min_depth)
+                                 : launch<P, NB, 1, 8>(call, chunks_per_block, s, wk, min_depth);
+      } else {
+        st = (NB == 1 && R == 2) ? launch<P, NB, 2, 4>(call, chunks_per_block, s, wk, min_depth)
+                                 : launch<P, NB, 1, 4>(call, chunks_per_block, s, wk, min_depth);
+      }
+      if (st != VQ_ERR_UNSUPPORTED) return st;
+    }
+  return VQ_ERR_UNSUPPORTED;
 }
 
 }  // namespace
@@ -1107,6 +1373,9 @@ vq_status launch_gemm_stream(const StreamCall& call, cudaStream_t s) {
       return nb2 ? launch_tiles<RowD1B4I8, 2>(call, g.Bc / 256, s) : launch_tiles<RowD1B4I8, 1>(call, g.Bc / 256, s);
     }
   }
+  // 2-D 6-bit codebooks shared by blocks of at least 32 rows and 128 columns
+  if (g.d == 2 && g.b == 6 && g.K % 256 == 0 && g.Bc % 128 == 0 && g.Br % 32 == 0 && g.stride * 8 == static_cast<long long>(g.J) * 6)
+    return nb2 ? launch_tiles<BlkD2B6, 2>(call, 1, s) : launch_tiles<BlkD2B6, 1>(call, 1, s);
   return VQ_ERR_UNSUPPORTED;
 }
 

@@ -91,7 +91,22 @@ vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half*
                             size_t ws_bytes, cudaStream_t s) {
   if (g.cb_int4) return VQ_ERR_UNSUPPORTED;   // int4 codebooks: format-generic kernels only
   vq_status st = VQ_ERR_UNSUPPORTED;
-  if (ws) {   // the persistent kernel needs the workspace; callers without one take the cluster kernels
+#ifdef VQ_TUNING
+  const char* path_env = getenv("VQ_PATH");
+  const int path = path_env ? atoi(path_env) : 0;   // 1: persistent kernel only, 2: cluster kernels only
+  if (path == 2) ws = nullptr;
+#endif
+  // Which family serves a single layer (measured on B200, both families on every benchmark shape at
+  // batch 1 / 4 / 16): the persistent kernel wins on the large per-row 4-bit 2-D layers (28672 x 8192:
+  // 30.6 against 37.8 us at batch 1, 68.6 against 77.6 us at batch 16; 8192 x 8192: 10.8 against 11.0 us
+  // and 22.9 against 26.2 us); short rows of few slabs, long rows (28672 columns), batch 3-8 and the
+  // shared-codebook formats are faster in the cluster kernels, whose K-split meets in distributed
+  // shared memory instead of the workspace.
+  bool stream_first = g.b == 4 && g.d == 2 && g.N >= 8192 && g.stride <= 2048 && (batch <= 2 || batch > 8);
+#ifdef VQ_TUNING
+  if (path == 1) stream_first = true;
+#endif
+  if (ws && stream_first) {   // (the persistent kernel needs the workspace)
     StreamCall call = {};
     call.g = g;
     call.n_seg = 1;
@@ -106,10 +121,28 @@ vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half*
     call.ws_bytes = ws_bytes;
     st = launch_gemm_stream(call, s);
     if (st != VQ_ERR_UNSUPPORTED) return st;
+#ifdef VQ_TUNING
+    if (path == 1) return st;
+#endif
   }
   st = launch_gemm_blockcb(g, p, X, Y, batch, s);
   if (st != VQ_ERR_UNSUPPORTED) return st;
-  return launch_gemm_rowcb(g, p, X, Y, batch, s);
+  st = launch_gemm_rowcb(g, p, X, Y, batch, s);
+  if (st != VQ_ERR_UNSUPPORTED || !ws || stream_first) return st;
+  // shapes the cluster kernels do not take: the persistent kernel if it does
+  StreamCall call = {};
+  call.g = g;
+  call.n_seg = 1;
+  call.idx[0] = p.idx;
+  call.cb[0] = p.cb;
+  call.scale[0] = p.scale;
+  call.Y[0] = Y;
+  call.N[0] = g.N;
+  call.X = X;
+  call.batch = batch;
+  call.ws = ws;
+  call.ws_bytes = ws_bytes;
+  return launch_gemm_stream(call, s);
 }
 
 

@@ -23,8 +23,31 @@ def draw(spec: vq_synth.LayerSpec, seed: int, layer_id: int = 0) -> vq_synth.Lay
     return vq_synth.make_layer(spec, oracle_fmt(spec).stride, seed, layer_id)
 
 
+CANARY = 0xA5          # byte pattern of the guard bands
+GUARD = 256            # bytes on either side of every output buffer
+
+
+def guarded(shape, dtype, device, fill=float("nan")):
+    """An output tensor with GUARD bytes of a known pattern on both sides: (view, raw buffer)."""
+    import torch
+    n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+    raw = torch.full((GUARD + n + GUARD,), CANARY, dtype=torch.uint8, device=device)
+    view = raw[GUARD:GUARD + n].view(dtype).view(*shape)
+    if fill is not None:
+        view.fill_(fill)
+    return view, raw
+
+
+def assert_guards_intact(raw, what=""):
+    """Nothing wrote before the start or past the end of the buffer."""
+    import torch
+    lo, hi = raw[:GUARD], raw[-GUARD:]
+    assert bool((lo == CANARY).all()) and bool((hi == CANARY).all()), f"{what}: write outside the output buffer"
+
+
 class DeviceLayer:
-    """Device copies of one layer + workspace, made with torch (memory plumbing only)."""
+    """Device copies of one layer + workspace, made with torch (memory plumbing only).  Outputs are
+    allocated with guard bands that are checked after every call."""
 
     def __init__(self, spec, layer, max_batch=16, device="cuda:0"):
         import torch
@@ -43,20 +66,25 @@ class DeviceLayer:
         X = np.ascontiguousarray(np.atleast_2d(X))
         batch = X.shape[0]
         dX = torch.from_numpy(X).to(self.device)
-        dY = torch.full((batch, self.spec.N), float("nan"), dtype=torch.float16, device=self.device)
+        dY, raw = guarded((batch, self.spec.N), torch.float16, self.device)
         if impl is None:
             vq.vq_gemm_small_batch(self.fmt, self.idx, self.cb, self.scale, dX, dY, batch, self.ws)
+        elif impl == "gemv":
+            assert batch == 1
+            vq.vq_gemv(self.fmt, self.idx, self.cb, self.scale, dX, dY, self.ws)
         else:
             vq.vq_gemm_small_batch_impl(self.fmt, self.idx, self.cb, self.scale, dX, dY, batch, self.ws, impl)
         torch.cuda.synchronize()
+        assert_guards_intact(raw, f"{self.spec.name} gemm batch {batch} impl {impl}")
         return dY.cpu().numpy()
 
     def decode(self):
         import torch
         import paper_2402_15319_b200 as vq
-        dW = torch.full((self.spec.N, self.spec.K), float("nan"), dtype=torch.float16, device=self.device)
+        dW, raw = guarded((self.spec.N, self.spec.K), torch.float16, self.device)
         vq.vq_decode_weights(self.fmt, self.idx, self.cb, self.scale, dW)
         torch.cuda.synchronize()
+        assert_guards_intact(raw, f"{self.spec.name} decode")
         return dW.cpu().numpy()
 
 

@@ -22,6 +22,13 @@ from tests.helpers import TOL, DeviceLayer, draw, oracle_fmt
 import paper_2402_15319_b200 as vq
 
 
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2402_15319_b200 import build as vq_build
+    vq_build.build()
+    vq.load()
+
+
 def test_oversized_problem_is_refused_on_the_host():
     # 16 x (65536 + 65536) x 2 bytes = 4 MiB > 2 MiB: refused by size alone, no pointer is touched
     fmt = vq.VQFormat(65536, 65536, 2, 4, 1, 2048, vq.VQ_CB_INT8_SCALED)
@@ -59,5 +66,11 @@ def test_static_scratch_variant_matches_workspace_variant_twice(spec):
         torch.cuda.synchronize()
         got, want = hY.numpy().astype(np.float64), hY_ref.numpy().astype(np.float64)
         assert np.isfinite(got).all()
-        _, A = orc.gemm(f, L.idx, L.cb, L.scale, X, threads=4)
+        Y, A = orc.gemm(f, L.idx, L.cb, L.scale, X, threads=4)
         assert (np.abs(got - want) <= TOL * A).all(), f"{spec.name} call {call}: differs from the workspace variant"
+        assert (np.abs(got - Y) <= TOL * A).all(), f"{spec.name} call {call}: differs from the oracle"
+        # a further call allocates nothing: neither the driver's free memory nor torch's pool moves
+        free0, alloc0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+        vq.vq_gemm_small_batch_host_static(dev.fmt, dev.idx, dev.cb, dev.scale, hX, hY, batch)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == alloc0
