@@ -3,9 +3,11 @@
 
 A step = one pass of the whole hot path (stream indices, stage codebooks, unpack, look up,
 multiply-accumulate, reduce + store) over one batch of synthetic activations for every layer
-of one benchmark configuration (default: the Llama-2-7B-shaped layer set, 2-D VQ with 6-bit
-indices, batch 1).  Metric: compressed bytes (indices + codebooks + scales + activations +
-outputs) moved per second, i.e. achieved HBM bandwidth on the compressed representation.
+of one benchmark configuration (default: the Llama-2-70B-shaped layer set, 2-D VQ with 4-bit
+indices and int8 codebooks, batch 1: the largest single-GPU workload).  Layers that read the same
+activations in a transformer block (q/k/v, gate/up) go through one grouped call.  Metric:
+compressed bytes (indices + codebooks + scales + activations + outputs) moved per second, i.e.
+achieved HBM bandwidth on the compressed representation.
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
 """
@@ -108,6 +110,28 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------
 # the CUDA arm
 # ------------------------------------------------------------------------------------------
+GROUPS = (("q", "k", "v"), ("gate", "up"))   # projections of a transformer block that read the same activations
+
+
+def call_groups(specs):
+    """Layer indices per library call: adjacent q/k/v and gate/up layers of one format and K form a
+    group (at most 4 members), everything else is a call of its own."""
+    out, i = [], 0
+    while i < len(specs):
+        name = specs[i].name.split(".")[-1]
+        grp = next((g for g in GROUPS if name == g[0]), None)
+        members = [i]
+        if grp:
+            for j, want in enumerate(grp[1:], start=1):
+                if i + j < len(specs) and specs[i + j].name.split(".")[-1] == want and specs[i + j].K == specs[i].K:
+                    members.append(i + j)
+                else:
+                    break
+        out.append(members)
+        i += len(members)
+    return out
+
+
 class DeviceSet:
     """R distinct device copies of every layer of a configuration, so that a layer's bytes have
     been evicted from L2 by the time its copy is read again."""
@@ -118,6 +142,7 @@ class DeviceSet:
         self.vq, self.torch = vq, torch
         conf = vq_synth.CONFIGS[cfg_name]
         self.cfg_name, self.batch, self.device = cfg_name, batch, device
+        self.batch_built = batch
         self.specs = conf["layers"]
         self.fmts, self.host, self.bytes_per_layer = [], [], []
         for lid, spec in enumerate(self.specs):
@@ -128,7 +153,10 @@ class DeviceSet:
             self.fmts.append(fmt)
             self.host.append((L, X))
             self.bytes_per_layer.append(layer_bytes(spec, info.row_stride_bytes, batch))
-        self.step_bytes = int(sum(self.bytes_per_layer))
+        self.groups = call_groups(self.specs)
+        # a group's members read ONE activation tensor (the first member's): count it once
+        shared_x = sum(2 * batch * self.specs[i].K for g in self.groups for i in g[1:])
+        self.step_bytes = int(sum(self.bytes_per_layer)) - shared_x
         self.n_weights = sum(s.n_weights for s in self.specs)
         self.copies = max(2, -(-2 * L2_BYTES // self.step_bytes))
         if max_copies:
@@ -144,6 +172,13 @@ class DeviceSet:
         self.X = [torch.from_numpy(X).to(device) for (_, X) in self.host]
         self.Y = [torch.empty((batch, s.N), dtype=torch.float16, device=device) for s in self.specs]
         self.ws = [torch.zeros(vq.vq_workspace_bytes(f, batch), dtype=torch.uint8, device=device) for f in self.fmts]
+        self.group_fmt, self.group_ws = {}, {}
+        for g in self.groups:
+            if len(g) > 1:
+                sp = self.specs[g[0]]
+                gf = vq.VQFormat(sum(self.specs[i].N for i in g), sp.K, sp.d, sp.b, sp.Br, sp.Bc, int(sp.int8))
+                self.group_fmt[g[0]] = gf
+                self.group_ws[g[0]] = torch.zeros(vq.vq_workspace_bytes(gf, batch), dtype=torch.uint8, device=device)
         # host side of the end-to-end path
         self.hX = [torch.from_numpy(X).pin_memory() for (_, X) in self.host]
         self.hY = [torch.empty((batch, s.N), dtype=torch.float16).pin_memory() for s in self.specs]
@@ -153,9 +188,28 @@ class DeviceSet:
 
     def step(self, copy: int):
         vq = self.vq
-        for i, fmt in enumerate(self.fmts):
-            idx, cb, sc = self.dev[copy][i]
-            vq.vq_gemm_small_batch(fmt, idx, cb, sc, self.X[i], self.Y[i], self.batch, self.ws[i])
+        for g in self.groups:
+            i = g[0]
+            if len(g) == 1:
+                idx, cb, sc = self.dev[copy][i]
+                vq.vq_gemm_small_batch(self.fmts[i], idx, cb, sc, self.X[i], self.Y[i], self.batch, self.ws[i])
+            else:
+                members = [(self.dev[copy][j][0], self.dev[copy][j][1], self.dev[copy][j][2], self.Y[j], self.specs[j].N) for j in g]
+                vq.vq_gemm_small_batch_grouped(self.group_fmt[i], members, self.X[i], self.batch, self.group_ws[i])
+
+    def set_batch(self, batch: int):
+        """Same weights, another batch size (activations, outputs and workspaces are remade)."""
+        torch, vq = self.torch, self.vq
+        conf = vq_synth.CONFIGS[self.cfg_name]
+        self.batch = batch
+        self.X = [torch.from_numpy(vq_synth.make_x(s, conf["seed"], batch, lid)).to(self.device) for lid, s in enumerate(self.specs)]
+        self.Y = [torch.empty((batch, s.N), dtype=torch.float16, device=self.device) for s in self.specs]
+        self.ws = [torch.zeros(vq.vq_workspace_bytes(f, batch), dtype=torch.uint8, device=self.device) for f in self.fmts]
+        for i in list(self.group_fmt):
+            self.group_ws[i] = torch.zeros(vq.vq_workspace_bytes(self.group_fmt[i], batch), dtype=torch.uint8, device=self.device)
+        per_layer = [b - 2 * self.batch_built * (s.K + s.N) + 2 * batch * (s.K + s.N) for b, s in zip(self.bytes_per_layer, self.specs)]
+        self.bytes_per_layer, self.batch_built = per_layer, batch
+        self.step_bytes = int(sum(per_layer)) - sum(2 * batch * self.specs[i].K for g in self.groups for i in g[1:])
 
     def step_host(self, copy: int):
         vq = self.vq
@@ -165,7 +219,53 @@ class DeviceSet:
         self.torch.cuda.synchronize()
 
     def launches_per_step(self) -> int:
-        return len(self.fmts) * self.vq.vq_kernel_launches() if hasattr(self.vq, "vq_kernel_launches") else len(self.fmts)
+        """Library kernels one step launches (a grouped call launches one kernel, or one per member)."""
+        n = 0
+        for g in self.groups:
+            n += 1 if len(g) == 1 else self.vq.vq_grouped_kernel_launches(self.group_fmt[g[0]], len(g), self.batch)
+        return n
+
+    def call_names(self):
+        return ["+".join(self.specs[i].name.split(".")[-1] for i in g) for g in self.groups]
+
+    def call_bytes(self, gi: int) -> int:
+        g = self.groups[gi]
+        return int(sum(self.bytes_per_layer[i] for i in g) - sum(2 * self.batch * self.specs[i].K for i in g[1:]))
+
+    def time_calls(self, reps: int = 10):
+        """Every library call of the step alone in a graph (its copies round-robin, cold cache):
+        [(name, us, bytes, GB/s)]."""
+        torch, vq = self.torch, self.vq
+        out = []
+        for gi, g in enumerate(self.groups):
+            def one(copy, g=g):
+                i = g[0]
+                if len(g) == 1:
+                    idx, cb, sc = self.dev[copy][i]
+                    vq.vq_gemm_small_batch(self.fmts[i], idx, cb, sc, self.X[i], self.Y[i], self.batch, self.ws[i])
+                else:
+                    members = [(self.dev[copy][j][0], self.dev[copy][j][1], self.dev[copy][j][2], self.Y[j], self.specs[j].N) for j in g]
+                    vq.vq_gemm_small_batch_grouped(self.group_fmt[i], members, self.X[i], self.batch, self.group_ws[i])
+            nbytes = self.call_bytes(gi)
+            rounds = max(1, -(-2 * L2_BYTES // max(1, nbytes * self.copies)))   # enough calls to outrun the L2
+            one(0)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                for _ in range(rounds):
+                    for c in range(self.copies):
+                        one(c)
+            graph.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) * 1e3 / (reps * rounds * self.copies)
+            out.append((self.call_names()[gi], us, nbytes, nbytes / us / 1e3))
+        return out
 
     def graph(self, n_steps: int, first_copy: int = 0):
         torch = self.torch
@@ -295,9 +395,10 @@ def dram_traffic_note(cfg_name: str):
         return None
 
 
-KERNEL_OF = {"cfg1": "rowcb_kernel<LdsTbl<false>,1>", "cfg2": "rowcb_kernel<PrmtI8,1>", "cfg3": "blockcb_kernel<2,6,1>",
-             "cfg4": "blockcb_kernel<4,8,NB>", "cfg5": "rowcb_kernel<LdsTbl<true>,NB>",
-             "llama3_8b": "blockcb_kernel<2,6,NB,warp-private tables>"}
+KERNEL_OF = {"cfg1": "rowcb_kernel<LdsTbl<false>,1>", "cfg2": "rowcb_kernel<PrmtI8,1>",
+             "cfg3": "blockcb_kernel<2,6,1> / stream_kernel<BlkD2B6> (groups)",
+             "cfg4": "blockcb_kernel<4,8,NB>", "cfg5": "stream_kernel<RowD2B4<int8>,NB,R,4> (groups, 8192-column layers) / rowcb_kernel<LdsTbl<true>,NB>",
+             "llama3_8b": "blockcb_kernel<2,6,NB,warp-private tables> / stream_kernel<BlkD2B6> (groups)"}
 
 
 def max_over_ranks(value: float, dist=None, device=None) -> float:
@@ -313,6 +414,52 @@ def max_over_ranks(value: float, dist=None, device=None) -> float:
 def whole_job_gbs(step_bytes_per_rank: int, world: int, ms_per_step: float) -> float:
     """Replicas only: every rank moves step_bytes_per_rank per step; value = all ranks' bytes / slowest time."""
     return world * step_bytes_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
+PROBE_POLICY = {"cfg1": 0, "cfg2": 1, "cfg3": 3, "cfg5": 0}   # decode-loop probe that matches a configuration's kernel
+
+
+def measure_ceilings(device, torch, vq, sm_mhz: float):
+    """What this GPU allows before any kernel design: a plain read of 1 GiB, and the look-up +
+    multiply-accumulate loops of the kernels on data that already sits in shared memory (8 warps per
+    SM, no global traffic).  The decode-loop rates are turned into GB/s of compressed bytes with each
+    configuration's stored bytes per weight and the SM clock `sm_mhz`."""
+    out = {"sm_mhz_used": sm_mhz}
+    buf = torch.empty(1 << 30, dtype=torch.uint8, device=device)
+    buf.random_(0, 255)
+    sink = torch.zeros(4, dtype=torch.uint8, device=device)
+    for _ in range(2):
+        vq.vq_probe_read(buf, sink)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(5):
+        vq.vq_probe_read(buf, sink)
+    e1.record()
+    torch.cuda.synchronize()
+    out["read_peak_GBps"] = 5 * buf.numel() / (e0.elapsed_time(e1) * 1e-3) / 1e9
+    del buf
+    sms = torch.cuda.get_device_properties(device).multi_processor_count
+    scratch = torch.zeros(8 * sms + 128 * sms * 8 + 1024, dtype=torch.uint8, device=device)
+    names = {0: "2-D 4-bit per-row codebooks (two row tiles per warp)", 1: "1-D 4-bit int8 codebooks (register look-up)",
+             2: "uniform INT4 g128", 3: "2-D 6-bit shared codebooks (two row tiles per warp)"}
+    loops = {}
+    for pol in (0, 1, 2, 3):
+        vq.vq_probe_decode_loop(pol, 8, 1, 50, scratch)
+        clocks, weights = vq.vq_probe_decode_loop(pol, 8, 1, 2000, scratch)
+        loops[pol] = {"policy": names[pol], "weights_per_clk_per_sm": weights / clocks,
+                      "Tweights_per_s": weights / clocks * sms * sm_mhz * 1e6 / 1e12}
+    out["decode_loop"] = loops
+    per_cfg = {}
+    for cfg, pol in PROBE_POLICY.items():
+        conf = vq_synth.CONFIGS[cfg]
+        nbytes = sum(layer_bytes(sp, vq.vq_pack_info(vq.VQFormat(sp.N, sp.K, sp.d, sp.b, sp.Br, sp.Bc, int(sp.int8))).row_stride_bytes, 1)
+                     for sp in conf["layers"])
+        nw = sum(sp.n_weights for sp in conf["layers"])
+        per_cfg[cfg] = {"bytes_per_weight": nbytes / nw, "decode_loop_GBps": loops[pol]["Tweights_per_s"] * 1e3 * nbytes / nw}
+    per_cfg["int4g128"] = {"bytes_per_weight": 4.125 / 8, "decode_loop_GBps": loops[2]["Tweights_per_s"] * 1e3 * 4.125 / 8}
+    out["per_config"] = per_cfg
+    return out
 
 
 def time_int4g128(cfg_name: str, batch: int, device, torch, vq):
@@ -413,7 +560,7 @@ def time_transfer_decode(device, torch, vq, N: int = 11008, K: int = 4096, reps:
 def time_assign(device, torch, vq, cfg_name: str = "cfg3", N: int = 11008, K: int = 4096, reps: int = 5):
     """E-step (Eq. 5) on a gate_proj-shaped dense matrix against the codebooks of a configuration's
     format: us per call, vectors per second, and the arithmetic rate against the fp32 lanes of the
-    GPU (148 SMs x 128 lanes x SM clock, one operation per lane and clock)."""
+    GPU (SM count x 128 lanes x SM clock, one operation per lane and clock)."""
     t = vq_synth.CONFIGS[cfg_name]["layers"][0]
     spec = vq_synth.LayerSpec("assign", N, K, t.d, t.b, t.Br, t.Bc, t.int8, cb_sigma=t.cb_sigma)
     fmt = vq.VQFormat(N, K, spec.d, spec.b, spec.Br, spec.Bc, vq.VQ_CB_INT8_SCALED if spec.int8 else vq.VQ_CB_FP16)
@@ -441,8 +588,9 @@ def time_assign(device, torch, vq, cfg_name: str = "cfg3", N: int = 11008, K: in
     sqnr = 10.0 * np.log10(d_W.double().pow(2).mean().item() / err)
     vectors = N * K // spec.d
     ops = vectors * (1 << spec.b) * (4 * spec.d + 2)   # per (vector, centroid): d sub, 2d mul, d-1 add, compare, 2 selects
-    sm_mhz = torch.cuda.get_device_properties(device).clock_rate / 1e3 if hasattr(torch.cuda.get_device_properties(device), "clock_rate") else 1965.0
-    peak = 148 * 128 * sm_mhz * 1e6
+    props = torch.cuda.get_device_properties(device)
+    sm_mhz = props.clock_rate / 1e3 if hasattr(props, "clock_rate") else 1965.0
+    peak = props.multi_processor_count * 128 * sm_mhz * 1e6
     return {"layer": f"{N}x{K}", "format": f"d={spec.d} b={spec.b} {spec.Br}x{spec.Bc}", "us": us,
             "Gvectors_per_s": vectors / us / 1e3, "alu_ops_per_s": ops / us * 1e6, "alu_peak_ops_per_s": peak,
             "alu_frac": ops / us * 1e6 / peak, "sqnr_db_random_codebook": sqnr}
@@ -499,6 +647,18 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     peak, peak_src = measured_peaks()
+    if args.ceilings:   # the micro-benchmarks alone; the SM clock is the median polled while they run
+        if rank == 0:
+            sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
+            sampler.start()
+            t_end = time.time() + 1.0
+            while time.time() < t_end:
+                measure_ceilings(dev, torch, vq, 1965.0)
+            sampler.stop()
+            clocks = sampler.summary("polled during the micro-benchmarks")
+            print(json.dumps({"metric": "ceilings", "peak_GBps": peak, "peak_source": peak_src, "clocks": clocks,
+                              **measure_ceilings(dev, torch, vq, float(clocks.get("sm_mhz") or 1965.0))}))
+        return
     ds = DeviceSet(args.config, args.batch, dev)
     if args.decode_only:   # vq_decode_weights alone on the configuration's largest layer (profiling runs)
         dec = time_decode(ds)
@@ -527,35 +687,44 @@ def run_ours(args):
     ms_e2e = max_over_ranks(ms_e2e, dist, dev)
     e2e_val = whole_job_gbs(ds.step_bytes, world, ms_e2e / e2e_steps)
 
-    launches = len(ds.fmts) * args.steps
-    per_launch_gbs = ds.step_bytes / (ms_per_step * 1e-3) / 1e9  # one GPU's kernels
+    launches_per_step = ds.launches_per_step()
+    step_gbs = ds.step_bytes / (ms_per_step * 1e-3) / 1e9  # one GPU's kernels
+    # the dominant kernel: every library call of the step timed alone (CUDA events, graph replay, cold cache)
+    calls = ds.time_calls()
+    dom = max(calls, key=lambda c: c[1])
     traffic = dram_traffic_note(args.config)
+    clocks = sampler.summary(clock_src)
+    sp0 = ds.specs[0]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {
-            "workload": f"{args.config}: {ds.specs[0].name.split('.')[0]} layer set ({len(ds.specs)} layers, "
-                        f"{ds.n_weights} weights), d={ds.specs[0].d}, {ds.specs[0].b}-bit indices, "
-                        f"{'int8+scale' if ds.specs[0].int8 else 'fp16'} codebook per "
-                        f"{ds.specs[0].Br}x{ds.specs[0].Bc} block, batch {args.batch}",
+            "workload": f"{args.config}: {sp0.name.split('.')[0]} layer set ({len(ds.specs)} layers, "
+                        f"{ds.n_weights} weights), d={sp0.d}, {sp0.b}-bit indices, "
+                        f"{'int8+scale' if sp0.int8 else 'fp16'} codebook per {sp0.Br}x{sp0.Bc} block, batch {args.batch}",
+            "calls_per_step": ds.call_names(),
+            "grouping": "q/k/v and gate/up read one activation tensor each (the first member's) through vq_gemm_small_batch_grouped; "
+                        "that tensor is counted once in bytes_per_step",
             "bytes_per_step": ds.step_bytes, "us_per_layer_set": ms_per_step * 1e3,
             "cold_cache": f"{ds.copies} distinct device copies of every layer visited round-robin "
                           f"({ds.copies * ds.step_bytes / 2**20:.0f} MiB > 2 x L2); inputs larger than L2, no flush",
             "launch": "CUDA graph of one round over all copies, replayed",
-            "pct_of_nominal_8TBps": 100 * per_launch_gbs / NOMINAL_HBM_GBS,
+            "pct_of_nominal_8TBps": 100 * step_gbs / NOMINAL_HBM_GBS,
+            "frac_of_measured_whole_step": step_gbs / peak,
             "parallelism": "replicas only (one GPU per process, no collective)" if world > 1 else "single GPU",
         },
-        "clocks": sampler.summary(clock_src),
+        "clocks": clocks,
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": ds.h2d, "d2h_bytes_per_step": ds.d2h,
                 "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps,
                 "what": "vq_gemm_small_batch_host per layer: activations read from pinned host memory, kernel, outputs written back to pinned host memory, stream synchronised every step; compressed weights resident in HBM"},
-        "gpu_launches": launches,
+        "gpu_launches": launches_per_step * args.steps,
         "roofline": {
-            "bound": "hbm", "kernel": KERNEL_OF.get(args.config, "vq gemm kernel") + " (one launch per layer)", "achieved": per_launch_gbs, "peak": peak,
-            "unit": "GB/s", "frac": per_launch_gbs / peak, "peak_source": peak_src,
-            "algorithmic_bytes_per_launch": ds.step_bytes / len(ds.fmts),
-            "avg_launch_us": ms_per_step * 1e3 / len(ds.fmts), "traffic": traffic,
+            "bound": "hbm", "kernel": f"{KERNEL_OF.get(args.config, 'vq gemm kernel')}: call '{dom[0]}' (largest share of the step: "
+                                      f"{100 * dom[1] / sum(c[1] for c in calls):.0f}% of the summed call times)",
+            "achieved": dom[3], "peak": peak, "unit": "GB/s", "frac": dom[3] / peak, "peak_source": peak_src,
+            "algorithmic_bytes_per_launch": dom[2], "avg_launch_us": dom[1], "traffic": traffic,
+            "calls_alone": [{"call": c[0], "us": c[1], "bytes": c[2], "GBps": c[3], "frac": c[3] / peak} for c in calls],
         },
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -565,33 +734,47 @@ def run_ours(args):
         dt, nbytes, desc = OracleWork(args.config, args.batch).run(12.0 * ORACLE_WEIGHTS_PER_SEC_PER_THREAD * threads, threads)
         line["cpu_baseline"] = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
                                 "sample": desc, "seconds": dt}
-    if rank == 0 and args.all_configs and world == 1:
-        per = {}
+    if rank == 0 and world == 1 and not args.no_per_config:
         del ds
         torch.cuda.empty_cache()
-        for cfg in vq_synth.CONFIGS:
+        sm_mhz = clocks.get("sm_mhz") or 1965.0
+        ceil = measure_ceilings(dev, torch, vq, float(sm_mhz))
+        line["ceilings"] = ceil
+        per, i4 = {}, {}
+        cfgs = list(vq_synth.CONFIGS) if args.all_configs else ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"]
+        for cfg in cfgs:
+            d2 = None
             for b in vq_synth.CONFIGS[cfg]["batches"]:
-                d2 = DeviceSet(cfg, b, dev)
-                st = max(d2.copies * 20, 200)
+                if d2 is None:
+                    d2 = DeviceSet(cfg, b, dev)
+                else:
+                    d2.set_batch(b)
+                st = max(d2.copies * 10, 100)
                 m = time_steps(d2, st, d2.copies * 3) / st
-                g = d2.step_bytes / (m * 1e-3) / 1e9
-                per[f"{cfg}.b{b}"] = {"us_per_step": m * 1e3, "GBps": g, "frac_of_measured": g / peak,
-                                      "pct_of_nominal_8TBps": 100 * g / NOMINAL_HBM_GBS, "bytes": d2.step_bytes}
-                if b == vq_synth.CONFIGS[cfg]["batches"][0]:
+                gbs = d2.step_bytes / (m * 1e-3) / 1e9
+                row = {"us": round(m * 1e3, 2), "GBps": round(gbs, 1), "frac": round(gbs / peak, 4), "launches": d2.launches_per_step()}
+                lim = ceil["per_config"].get(cfg)
+                if lim and b <= 8:
+                    row["ceilings_GBps"] = {"hbm": round(peak, 1), "read": round(ceil["read_peak_GBps"], 1),
+                                            "decode_loop": round(lim["decode_loop_GBps"], 1)}
+                per[f"{cfg}.b{b}"] = row
+                if args.all_configs and b == vq_synth.CONFIGS[cfg]["batches"][0]:
                     dec = time_decode(d2)
                     dec["frac_of_measured"] = dec["GBps"] / peak
                     per[f"{cfg}.decode_weights"] = dec
-                del d2
-                torch.cuda.empty_cache()
-            for b in vq_synth.CONFIGS[cfg]["batches"][:1]:
-                r = time_int4g128(cfg, b, dev, torch, vq)
-                if r:
-                    r["frac_of_measured"] = r["GBps"] / peak
-                    per[f"{cfg}.int4g128_yardstick.b{b}"] = r
-                torch.cuda.empty_cache()
+            del d2
+            torch.cuda.empty_cache()
+            r = time_int4g128(cfg, vq_synth.CONFIGS[cfg]["batches"][0], dev, torch, vq)
+            if r:
+                i4[cfg] = {"us": round(r["us_per_step"], 2), "GBps": round(r["GBps"], 1), "frac": round(r["GBps"] / peak, 4)}
+            torch.cuda.empty_cache()
         line["per_config"] = per
-        line["transfer_decode"] = time_transfer_decode(dev, torch, vq)
-        line["assign"] = time_assign(dev, torch, vq)
+        line["int4g128"] = {"what": "uniform INT4 group-128 GEMV (4.125 bits per weight) on each configuration's layer shapes, "
+                                    "one call per layer, batch = the configuration's first", "decode_loop_ceiling_GBps":
+                            round(ceil["per_config"]["int4g128"]["decode_loop_GBps"], 1), **i4}
+        if args.all_configs:
+            line["transfer_decode"] = time_transfer_decode(dev, torch, vq)
+            line["assign"] = time_assign(dev, torch, vq)
     if rank == 0:
         print(json.dumps(line))
     if dist:
@@ -599,15 +782,29 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def spawn_replicas(args):
+    """`--gpus N` without a launcher: start N local ranks (one per GPU) of this same command."""
+    import socket
+    import subprocess
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=4000)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=40)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="cfg3", choices=sorted(vq_synth.CONFIGS))
+    ap.add_argument("--config", default="cfg5", choices=sorted(vq_synth.CONFIGS))
     ap.add_argument("--batch", type=int, default=1)
-    ap.add_argument("--all-configs", action="store_true", help="also time every configuration and batch (adds per_config)")
+    ap.add_argument("--all-configs", action="store_true", help="per_config also covers llama3_8b and vq_decode_weights; adds transfer_decode and assign")
+    ap.add_argument("--no-per-config", action="store_true", help="skip per_config, int4g128 and ceilings (profiling runs)")
+    ap.add_argument("--ceilings", action="store_true", help="run the ceiling micro-benchmarks alone and print them")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode-only", action="store_true", help="time vq_decode_weights on the configuration's largest layer and exit")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end loop (profiling runs)")
@@ -616,6 +813,8 @@ def main():
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_replicas(args))
     else:
         run_ours(args)
 

@@ -168,6 +168,9 @@ typedef struct {
 } vq_group_member;
 vq_status vq_gemm_small_batch_grouped(const vq_format* fmt, const vq_group_member* members, int n_members,
                                       const void* d_X, int batch, void* d_ws, size_t ws_bytes, void* stream);
+/* Kernels a grouped call of this format launches: 1 (one persistent kernel for the group) or n_members.
+ * Host only; 0 for invalid arguments. */
+int vq_grouped_kernel_launches(const vq_format* fmt, int n_members, int batch);
 
 /* Same computation with HOST activations and outputs: copies h_X (binary16 [batch][K]) to the
  * device, runs vq_gemm_small_batch, copies Y back into h_Y (binary16 [batch][N]); all three
@@ -252,6 +255,21 @@ vq_status vq_assign_indices(const vq_format* fmt, const void* d_W, const void* d
 typedef enum { VQ_UNPACK_FP16 = 0, VQ_UNPACK_INT8_ROW = 1, VQ_UNPACK_INT4_G128 = 2 } vq_unpack_kind;
 vq_status vq_unpack_uniform(int kind, int32_t n_rows, int32_t k_cols, const void* d_src,
                             const void* d_scale, void* d_W, void* stream);
+
+/* Probes behind the ceilings bench.py prints beside the achieved bandwidth (paper Sec. 3.2: the decode
+ * must keep up with DRAM; these measure what the decode loop and a plain read can do on this GPU).
+ * vq_probe_decode_loop: `iters` passes of the look-up + multiply-accumulate loop of one kernel policy
+ *   over a stage that stays in shared memory (no global traffic), on every SM, `warps` (1..8) warps per
+ *   SM, batch 1..8.  policy 0: 2-D 4-bit per-row codebooks, 1: 1-D 4-bit int8 codebooks, 2: uniform
+ *   INT4 g128, 3: 2-D 6-bit shared codebooks.  d_scratch: device memory of at least
+ *   8*SMs + 128*SMs*warps bytes.  Returns the average clocks per pass and the weights one pass decodes
+ *   on one SM; synchronises `stream`.
+ * vq_probe_read: reads every byte of d_buf once with streaming 128-bit loads; asynchronous on `stream`,
+ *   the caller times it.  d_out4: 4 writable device bytes.
+ * Errors: NULL, SHAPE, ALIGN, WORKSPACE, UNSUPPORTED, CUDA. */
+vq_status vq_probe_decode_loop(int policy, int warps, int batch, int iters, void* d_scratch, size_t scratch_bytes,
+                               double* h_clocks, double* h_weights_per_pass, void* stream);
+vq_status vq_probe_read(const void* d_buf, size_t bytes, void* d_out4, void* stream);
 
 /* Diagnostics.  The tuned kernels wait for their asynchronous copies (Sec. 3.2 index stream) with a
  * bounded number of polls; a wait that runs out increments a per-device counter and the kernel

@@ -82,6 +82,7 @@ _SIGNATURES = {
     "vq_gemm_small_batch_impl": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_int]),
     "vq_gemm_small_batch_grouped": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int,
                                                    ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
+    "vq_grouped_kernel_launches": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int, ctypes.c_int]),
     "vq_gemm_small_batch_host": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
     "vq_gemm_small_batch_host_static": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p]),
     "vq_static_scratch_bytes": (ctypes.c_size_t, []),
@@ -90,6 +91,9 @@ _SIGNATURES = {
     "vq_assign_indices": (ctypes.c_int, [ctypes.c_void_p] * 7),
     "vq_unpack_uniform": (ctypes.c_int, [ctypes.c_int, ctypes.c_int32, ctypes.c_int32] + [ctypes.c_void_p] * 4),
     "vq_device_wait_failures": (ctypes.c_int, [ctypes.c_void_p]),
+    "vq_probe_decode_loop": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t,
+                                            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "vq_probe_read": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p]),
     "vq_status_string": (ctypes.c_char_p, [ctypes.c_int]),
 }
 
@@ -187,6 +191,11 @@ def vq_gemm_small_batch_grouped(fmt: VQFormat, members, d_X, batch: int, d_ws, s
            "vq_gemm_small_batch_grouped")
 
 
+def vq_grouped_kernel_launches(fmt: VQFormat, n_members: int, batch: int) -> int:
+    c = fmt.c()
+    return load().vq_grouped_kernel_launches(ctypes.byref(c), int(n_members), int(batch))
+
+
 def vq_gemm_small_batch_impl(fmt: VQFormat, d_idx, d_cb, d_scale, d_X, d_Y, batch: int, d_ws, impl: int,
                              stream=None) -> None:
     c = fmt.c()
@@ -218,6 +227,19 @@ def vq_gemm_small_batch_host_static(fmt: VQFormat, d_idx, d_cb, d_scale, h_X, h_
 
 def vq_static_scratch_bytes() -> int:
     return load().vq_static_scratch_bytes()
+
+
+def vq_probe_decode_loop(policy: int, warps: int, batch: int, iters: int, d_scratch, stream=None):
+    """(clocks per pass, weights decoded per pass and SM) of one policy's decode loop on resident data."""
+    clocks, weights = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    _check(load().vq_probe_decode_loop(int(policy), int(warps), int(batch), int(iters), _ptr(d_scratch),
+                                       d_scratch.numel() * d_scratch.element_size(), ctypes.byref(clocks), ctypes.byref(weights),
+                                       _stream(stream)), "vq_probe_decode_loop")
+    return clocks.value, weights.value
+
+
+def vq_probe_read(d_buf, d_out4, stream=None) -> None:
+    _check(load().vq_probe_read(_ptr(d_buf), d_buf.numel() * d_buf.element_size(), _ptr(d_out4), _stream(stream)), "vq_probe_read")
 
 
 def vq_device_wait_failures() -> int:

@@ -177,6 +177,12 @@ vq_status vq_gemm_small_batch_impl(const vq_format* fmt, const void* d_idx, cons
   return launch_gemm_generic(g, p, X, Y, batch, s);
 }
 
+int vq_grouped_kernel_launches(const vq_format* fmt, int n_members, int batch) {
+  Geometry g;
+  if (make_geometry(fmt, &g) != VQ_OK || n_members < 1 || n_members > VQ_MAX_GROUP || batch < 1 || batch > 16) return 0;
+  return (n_members > 1 && (batch <= 2 || batch > 8) && stream_covers(g)) ? 1 : n_members;
+}
+
 vq_status vq_gemm_small_batch_grouped(const vq_format* fmt, const vq_group_member* members, int n_members,
                                       const void* d_X, int batch, void* d_ws, size_t ws_bytes, void* stream) {
   if (!fmt || !members) return VQ_ERR_NULL;

@@ -63,6 +63,7 @@ struct StreamCall {
 size_t stream_workspace_bytes(long long rows, int batch);
 size_t stream_ticket_bytes(long long rows);   // the counters at the start of the workspace
 vq_status launch_gemm_stream(const StreamCall& call, cudaStream_t s);
+bool stream_covers(const Geometry& g);
 vq_status launch_int4g128_stream(int N, int K, const uint8_t* q, const __half* scale, const __half* X, __half* Y, int batch,
                                  void* ws, size_t ws_bytes, cudaStream_t s);
 vq_status launch_gemm_blockcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,

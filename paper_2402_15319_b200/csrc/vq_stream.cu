@@ -1354,7 +1354,103 @@ vq_status launch_tiles(const StreamCall& call, int chunks_per_block, cudaStream_
   return VQ_ERR_UNSUPPORTED;
 }
 
+
+// =============================================================================================
+// Probes: the consumers' decode loops on a stage that stays in shared memory (no global traffic,
+// no pipeline), and a plain read of a buffer.  bench.py turns their rates into the ceilings it
+// prints beside the achieved numbers.
+// =============================================================================================
+template <class P, int NB, int R>
+__global__ void __launch_bounds__(256, 1) probe_decode_kernel(int iters, int batch, long long* cycles, float* sink) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  const uint32_t sbase = (smem_u32(smem_raw) + (P::BASE_ALIGN - 1)) & ~static_cast<uint32_t>(P::BASE_ALIGN - 1);
+  unsigned char* smem = smem_raw + (sbase - smem_u32(smem_raw));
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, W = blockDim.x / 32;
+  const int g = lane >> 2, t = lane & 3;
+  // [stage table | per-warp tables | index rows of every warp | activations]
+  const int tbl_words = (P::STAGE_TABLE_BYTES + W * R * P::TILE_TABLE_BYTES) / 4;
+  const int idx_words = W * R * 16 * P::CHUNK_BYTES / 4;
+  const int x_words = P::X_ROWS * batch * P::X_ROW_BYTES / 4;
+  uint32_t* words = reinterpret_cast<uint32_t*>(smem);
+  uint32_t seed = 1234567u + tid * 7919u + blockIdx.x;
+  for (int i = tid; i < tbl_words + idx_words + x_words; i += blockDim.x) {
+    seed = seed * 1664525u + 1013904223u;
+    // small finite fp16 pairs for tables and activations, anything for indices
+    words[i] = i < tbl_words ? (0x2C002C00u | (seed & 0x03FF03FFu)) : i < tbl_words + idx_words ? seed : (0x34003400u | (seed & 0x83FF83FFu));
+  }
+  __syncthreads();
+  typename P::template State<NB, R> st;
+  st.init(sbase + P::STAGE_TABLE_BYTES + warp * (R * P::TILE_TABLE_BYTES), lane);
+  float total[R][NB][4];
+#pragma unroll
+  for (int r = 0; r < R; ++r)
+#pragma unroll
+    for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) total[r][nb][e] = 0.f;
+  int xm[NB];
+#pragma unroll
+  for (int nb = 0; nb < NB; ++nb) xm[nb] = min(nb * 8 + g, batch - 1);
+  const unsigned char* idx = smem + tbl_words * 4 + (warp * R * 16 + g) * P::CHUNK_BYTES + t * P::LANE_BYTES;
+  const unsigned char* xpart = smem + (tbl_words + idx_words) * 4;
+  const long long c0 = clock64();
+  for (int it = 0; it < iters; ++it) {
+    st.compute(idx, xpart, xm, batch, sbase, lane, total);
+    asm volatile("" ::: "memory");
+  }
+  const long long c1 = clock64();
+  st.flush(total);
+  float sum = 0.f;
+#pragma unroll
+  for (int r = 0; r < R; ++r)
+#pragma unroll
+    for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) sum += total[r][nb][e];
+  sink[blockIdx.x * blockDim.x + tid] = sum;
+  if (tid == 0) cycles[blockIdx.x] = c1 - c0;
+}
+
+template <class P, int R>
+vq_status run_probe(int warps, int batch, int iters, int sms, long long* d_cycles, float* d_sink, cudaStream_t s,
+                    double* weights_per_stage) {
+  auto kern = probe_decode_kernel<P, 1, R>;
+  const size_t smem = P::BASE_ALIGN + P::STAGE_TABLE_BYTES + static_cast<size_t>(warps) * R * (P::TILE_TABLE_BYTES + 16 * P::CHUNK_BYTES) +
+                      static_cast<size_t>(P::X_ROWS) * batch * P::X_ROW_BYTES + 1024;
+  if (smem > kSmemMax) return VQ_ERR_UNSUPPORTED;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemMax)) != cudaSuccess) return VQ_ERR_CUDA;
+  kern<<<sms, warps * 32, smem, s>>>(iters, batch, d_cycles, d_sink);
+  *weights_per_stage = static_cast<double>(warps) * R * 16 * P::CHUNK_COLS;
+  return check_launch();
+}
+
+__global__ void __launch_bounds__(256) probe_read_kernel(const uint4* __restrict__ src, long long n16, uint32_t* __restrict__ out) {
+  uint32_t acc = 0u;
+  const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+  long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  for (; i + 3 * stride < n16; i += 4 * stride) {   // four independent 128-bit loads in flight per thread
+    const uint4 a = ldg128_stream(src + i), b = ldg128_stream(src + i + stride), c = ldg128_stream(src + i + 2 * stride),
+                d = ldg128_stream(src + i + 3 * stride);
+    acc ^= a.x ^ a.y ^ a.z ^ a.w ^ b.x ^ b.y ^ b.z ^ b.w ^ c.x ^ c.y ^ c.z ^ c.w ^ d.x ^ d.y ^ d.z ^ d.w;
+  }
+  for (; i < n16; i += stride) {
+    const uint4 a = ldg128_stream(src + i);
+    acc ^= a.x ^ a.y ^ a.z ^ a.w;
+  }
+  if (acc == 0x9e3779b9u) out[0] = acc;   // (keeps the loads alive; practically never true)
+}
+
 }  // namespace
+
+// Does the persistent kernel have a policy for this format (the launch may still decline a shape)?
+bool stream_covers(const Geometry& g) {
+  if (g.cb_int4) return false;
+  if (g.b == 4 && g.Br >= 1 && g.stride % 128 == 0 && g.stride * 8 == static_cast<long long>(g.J) * 4) {
+    if (g.d == 2) return g.Bc % 512 == 0;
+    if (g.d == 1 && g.cb_int8) return g.Bc % 256 == 0;
+  }
+  return g.d == 2 && g.b == 6 && g.K % 256 == 0 && g.Bc % 128 == 0 && g.Br % 32 == 0 && g.stride * 8 == static_cast<long long>(g.J) * 6;
+}
 
 vq_status launch_gemm_stream(const StreamCall& call, cudaStream_t s) {
   const Geometry& g = call.g;
@@ -1402,3 +1498,52 @@ vq_status launch_int4g128_stream(int N, int K, const uint8_t* q, const __half* s
 }
 
 }  // namespace vq
+
+using namespace vq;
+
+// Decode-loop probe: `iters` passes of the inner loop of one policy over a stage that stays in shared
+// memory, on every SM.  policy 0: 2-D 4-bit (two row tiles per warp), 1: 1-D 4-bit int8, 2: INT4 g128,
+// 3: 2-D 6-bit shared codebooks (two row tiles per warp).  d_scratch: device memory of at least
+// 8 * sms + 4 * sms * 32 * warps bytes.  Writes the average clocks of the loop and the weights one
+// pass decodes per SM; synchronises the stream.
+extern "C" vq_status vq_probe_decode_loop(int policy, int warps, int batch, int iters, void* d_scratch, size_t scratch_bytes,
+                                          double* h_clocks, double* h_weights_per_pass, void* stream) {
+  if (!d_scratch || !h_clocks || !h_weights_per_pass) return VQ_ERR_NULL;
+  if (warps < 1 || warps > 8 || batch < 1 || batch > 8 || iters < 1) return VQ_ERR_SHAPE;
+  int sms = 0;
+  if (device_sms(&sms) != VQ_OK) return VQ_ERR_CUDA;
+  const size_t need = static_cast<size_t>(sms) * 8 + static_cast<size_t>(sms) * 32 * warps * 4;
+  if (scratch_bytes < need) return VQ_ERR_WORKSPACE;
+  long long* d_cycles = static_cast<long long*>(d_scratch);
+  float* d_sink = reinterpret_cast<float*>(static_cast<char*>(d_scratch) + static_cast<size_t>(sms) * 8);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  double wps = 0.0;
+  vq_status st = VQ_ERR_UNSUPPORTED;
+  if (policy == 0) st = run_probe<RowD2B4<true>, 2>(warps, batch, iters, sms, d_cycles, d_sink, s, &wps);
+  else if (policy == 1) st = run_probe<RowD1B4I8, 1>(warps, batch, iters, sms, d_cycles, d_sink, s, &wps);
+  else if (policy == 2) st = run_probe<RowInt4G128, 1>(warps, batch, iters, sms, d_cycles, d_sink, s, &wps);
+  else if (policy == 3) st = run_probe<BlkD2B6, 2>(warps, batch, iters, sms, d_cycles, d_sink, s, &wps);
+  if (st != VQ_OK) return st;
+  long long h[1024];
+  if (sms > 1024) return VQ_ERR_UNSUPPORTED;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return VQ_ERR_CUDA;
+  if (cudaMemcpy(h, d_cycles, static_cast<size_t>(sms) * 8, cudaMemcpyDeviceToHost) != cudaSuccess) return VQ_ERR_CUDA;
+  double sum = 0.0;
+  for (int i = 0; i < sms; ++i) sum += static_cast<double>(h[i]);
+  *h_clocks = sum / sms / iters;
+  *h_weights_per_pass = wps;
+  return VQ_OK;
+}
+
+// Read probe: every byte of d_buf once with streaming 128-bit loads (nothing is written unless a
+// checksum happens to match a constant).  Enqueued on `stream`; the caller times it.
+extern "C" vq_status vq_probe_read(const void* d_buf, size_t bytes, void* d_out4, void* stream) {
+  if (!d_buf || !d_out4) return VQ_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(d_buf) & 15u) || bytes < 16) return VQ_ERR_ALIGN;
+  int sms = 0;
+  if (device_sms(&sms) != VQ_OK) return VQ_ERR_CUDA;
+  probe_read_kernel<<<sms * 8, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const uint4*>(d_buf),
+                                                                            static_cast<long long>(bytes / 16),
+                                                                            static_cast<uint32_t*>(d_out4));
+  return check_launch();
+}
