@@ -11,15 +11,17 @@
  *   (1) packed VQ indices, (2) its codebook / LUT, (3) an optional scale factor.
  * One index of `index_bits` bits selects one of k = 2^index_bits codebook entries;
  * an entry holds `vq_dim` values which are `vq_dim` ADJACENT COLUMNS of one row
- * (Sec. 4, "we quantize d columns at a time").  Bits per value follow the paper's
- * formula  log2(k)/d + k*d*b_c/l  (Sec. 4, "Total bits per value").
+ * (Sec. 4: the quantizer walks the matrix d columns at a time).  Bits per value follow the
+ * paper's formula  log2(k)/d + k*d*b_c/l  (Sec. 4, the paragraph on total bits per value).
  *
- * Memory layout fixed by this library (the paper only says "packed tightly"):
+ * Memory layout fixed by this library (the paper fixes no bit order or row pitch):
  *   indices : N rows; row n is a little-endian bitstream: index j (covering columns
  *             j*d .. j*d+d-1) occupies bits [j*b, (j+1)*b) where bit t of the stream is
  *             bit (t mod 8) of byte (t div 8).  Rows start at n*row_stride_bytes;
  *             row_stride_bytes = ceil(K/d*b/8) rounded up to a multiple of 16.
- *             Padding bits/bytes are ignored.
+ *             The CALLER lays the rows out at that pitch: the buffer holds N * row_stride_bytes
+ *             bytes (vq_pack_info().index_bytes), all of them readable.  The value of padding
+ *             bits/bytes is ignored, but the kernels' bulk copies do read them.
  *   codebook: cb[blk][entry][t], t < d; blk = (n / block_rows)*(K / block_cols) + (k / block_cols).
  *             VQ_CB_FP16: IEEE binary16.  VQ_CB_INT8_SCALED: signed 8-bit.
  *   scale   : VQ_CB_INT8_SCALED only: one binary16 per block, w = scale * int8.
@@ -32,6 +34,19 @@
  *     h_* are HOST pointers; `stream` is a cudaStream_t passed as void* (NULL = default stream).
  *   - The caller owns all buffers.  Inputs are read-only.  The library allocates nothing,
  *     frees nothing, never synchronises: work is enqueued on `stream` and the call returns.
+ *   - WEIGHT buffers (indices, codebooks, scales) must be complete and visible to the device
+ *     BEFORE a GEMV/GEMM call is enqueued: the kernels are launched with programmatic dependent
+ *     launch and start fetching weights while the previous kernel on `stream` may still be
+ *     running; only activations, outputs and workspace are ordered after that kernel.  Weights
+ *     produced on the device (vq_assign_indices, a copy, the caller's own kernel) therefore need
+ *     a host-side stream or event synchronisation before the first call that reads them; stream
+ *     order alone is not enough.
+ *   - WORKSPACE (d_ws): the first vq_workspace_bytes()-defined counter region of a workspace must
+ *     read as zero the first time it is used: zero-fill a workspace once after allocating it
+ *     (cudaMemsetAsync on the same stream is enough).  Every call leaves the counters zero again,
+ *     so the workspace can be reused by later calls of any format and batch without clearing.
+ *     The rest of its contents is scratch (ignored on entry, unspecified on exit).  Calls that
+ *     may overlap on the GPU (different streams) need different workspaces.
  *   - All argument checks run on the host before any launch; on error nothing is launched.
  *   - Same inputs give bit-identical outputs (no floating-point atomics).
  */
@@ -57,7 +72,7 @@ typedef enum {
   VQ_ERR_CUDA = 8         /* a CUDA runtime call or the launch itself reported an error                 */
 } vq_status;
 
-/* VQ_CB_INT4_G128 (paper Sec. 4.2, "INT4 codebooks" with codebook quantization groups of 128 values):
+/* VQ_CB_INT4_G128 (paper Sec. 4.2: codebooks held as 4-bit integers, one scale per group of 128 values):
  *   d_cb    : per block 2^index_bits * vq_dim signed 4-bit integers (-8..7), two per byte, value
  *             v = entry * vq_dim + t in nibble v mod 2 (low nibble first) of byte v / 2;
  *   d_scale : binary16 [N][K/128]; w[n][k] = scale[n][k/128] * c.  K % 128 == 0.
@@ -92,30 +107,31 @@ typedef struct {
 /* Library-filled sizes for a format. */
 typedef struct {
   int32_t entries;                  /* k = 2^b                                              */
-  int32_t codebook_bits;            /* b_c: 16 (fp16) or 8 (int8)                           */
+  int32_t codebook_bits;            /* b_c: 16 (fp16), 8 (int8) or 4 (INT4_G128)            */
   int64_t indices_per_row;          /* K/d                                                  */
   int64_t row_stride_bytes;         /* bytes between consecutive rows of the index stream   */
   int64_t index_bytes;              /* N * row_stride_bytes                                 */
   int64_t n_blocks;                 /* (N/block_rows) * (K/block_cols)                      */
   int64_t codebook_bytes_per_block; /* k * d * b_c/8                                        */
   int64_t codebook_bytes;           /* n_blocks * codebook_bytes_per_block                  */
-  int64_t scale_bytes;              /* 2*n_blocks for INT8_SCALED, else 0                   */
+  int64_t scale_bytes;              /* INT8_SCALED 2*n_blocks; INT4_G128 2*N*K/128; FP16 0  */
   int64_t total_bytes;              /* index + codebook + scale bytes                       */
   double bpv_paper;                 /* log2(k)/d + k*d*b_c/l  (no scale term)               */
   double bpv_stored;                /* 8*total_bytes/(N*K), everything stored               */
 } vq_pack_info_t;
 
-/* Sizes and bits-per-value of a format (paper Sec. 4 "Total bits per value"; Sec. 3.1 tuple).
+/* Sizes and bits-per-value of a format (paper Sec. 4, total bits per value; Sec. 3.1 tuple).
  * Host only, no CUDA call.  Errors: NULL, FORMAT, SHAPE. */
 vq_status vq_pack_info(const vq_format* fmt, vq_pack_info_t* out);
 
-/* Bytes of device scratch the GEMV/GEMM entry points need for (fmt, batch): room for the
- * fp32 split-K partial sums (Sec. 3.2 mat-vec; the split is this library's).  Host only.
- * Returns 0 for an invalid format or batch. */
+/* Bytes of device scratch the GEMV/GEMM entry points need for (fmt, batch): arrival counters
+ * (one 32-bit word per 16 rows, at the start) and room for the fp32 partial sums of column
+ * ranges handled by different thread blocks (Sec. 3.2 mat-vec; the split is this library's).
+ * Host only.  Returns 0 for an invalid format or batch.  See WORKSPACE above for the zero rule. */
 size_t vq_workspace_bytes(const vq_format* fmt, int batch);
 
-/* Materialise W: unpack every index and look its entry up (paper App. A: "Q is constructed by
- * looking up values of C"; Sec. 3.2 decode step; App. B transfer+decode experiment).
+/* Materialise W: unpack every index and look its entry up (paper App. A: the quantized matrix Q
+ * is the codebook C read through the index array; Sec. 3.2 decode step; App. B transfer+decode).
  *   d_idx, d_cb, d_scale : device, layouts above; d_scale NULL iff cb_type == VQ_CB_FP16.
  *   d_W   : device, binary16 [N][K] row-major, written completely.
  * FP16 codebooks are copied bit-exactly; INT8_SCALED values are fp32(scale)*int8 rounded once
@@ -126,7 +142,7 @@ vq_status vq_decode_weights(const vq_format* fmt, const void* d_idx, const void*
 /* y = W x for one token (paper Sec. 3.2: indices -> LUT -> values -> matrix-vector product).
  *   d_x : device binary16 [K];  d_y : device binary16 [N], written completely.
  *   d_ws / ws_bytes : device scratch of at least vq_workspace_bytes(fmt, 1) bytes, 16-byte
- *                     aligned; contents on entry are ignored, contents on exit unspecified.
+ *                     aligned, zero-filled once before its first use (WORKSPACE above).
  * Errors: NULL, FORMAT, SHAPE, ALIGN, WORKSPACE, CUDA. */
 vq_status vq_gemv(const vq_format* fmt, const void* d_idx, const void* d_cb, const void* d_scale,
                   const void* d_x, void* d_y, void* d_ws, size_t ws_bytes, void* stream);
@@ -216,12 +232,14 @@ vq_status vq_gemm_small_batch_host_static(const vq_format* fmt, const void* d_id
 size_t vq_static_scratch_bytes(void);
 
 /* Uniform INT4 group-128 reference GEMV used as the bandwidth yard-stick beside the VQ
- * kernels (paper Sec. 2.1 symmetric uniform quantiser x ~ s*x_int; Sec. 5 "INT4 g128", 4.125 bpv).
+ * kernels (paper Sec. 2.1 symmetric uniform quantiser x ~ s*x_int; Sec. 5 compares against uniform
+ * 4-bit weights with one scale per 128 columns, 4.125 bits per value).
  *   d_q     : device, N rows of K/2 bytes; column k of row n is nibble (k mod 2) of byte k/2
  *             (low nibble first); stored value q in 0..15 means integer q-8.
  *   d_scale : device binary16 [N][K/128];  w[n][k] = scale[n][k/128] * (q-8).
  *   d_X binary16 [batch][K], d_Y binary16 [batch][N], batch 1..16.  K % 128 == 0, K/2 % 16 == 0.
- * Errors: NULL, SHAPE, ALIGN, BATCH, CUDA. */
+ *   d_ws / ws_bytes : at least vq_int4g128_workspace_bytes(n_rows, batch) bytes, rules as WORKSPACE above.
+ * Errors: NULL, SHAPE, ALIGN, BATCH, WORKSPACE, CUDA. */
 vq_status vq_int4g128_gemm_small_batch(int32_t n_rows, int32_t k_cols, const void* d_q,
                                        const void* d_scale, const void* d_X, void* d_Y,
                                        int batch, void* d_ws, size_t ws_bytes, void* stream);

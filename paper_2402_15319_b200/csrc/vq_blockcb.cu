@@ -594,16 +594,14 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
   using P = Policy<D, B>;
   using T = Tile<D, B>;
   auto kern = blockcb_kernel<D, B, NB, PRIV>;
-  static int sms_of[kMaxDevices] = {};
-  int dev = 0;
+  static int attr_set[kMaxDevices] = {};
+  int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VQ_ERR_CUDA;
-  if (sms_of[dev] == 0) {
-    int n = 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return VQ_ERR_CUDA;
+  if (device_sms(&sms) != VQ_OK) return VQ_ERR_CUDA;
+  if (!__atomic_load_n(&attr_set[dev], __ATOMIC_ACQUIRE)) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess) return VQ_ERR_CUDA;
-    sms_of[dev] = n;
+    __atomic_store_n(&attr_set[dev], 1, __ATOMIC_RELEASE);
   }
-  const int sms = sms_of[dev];
   int* error_flag = nullptr;
   if (device_error_counter(&error_flag) != VQ_OK) return VQ_ERR_CUDA;
 

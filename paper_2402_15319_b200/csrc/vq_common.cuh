@@ -80,6 +80,8 @@ vq_status launch_assign(const Geometry& g, const LayerPtrs& p, const __half* W, 
 // Device address of this device's counter of bounded waits that ran out inside a kernel (a copy
 // that never completed); looked up once per device.
 vq_status device_error_counter(int** d_counter);
+// SM count of the current device (looked up once per device).
+vq_status device_sms(int* out);
 
 // Tensor map of the packed index stream seen as a 2-D byte tensor (N rows of `stride` bytes) with
 // boxes of box_rows rows x box_bytes bytes, for tiled TMA loads without swizzle or multicast.

@@ -191,13 +191,13 @@ vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, 
   const size_t smem = static_cast<size_t>(a.br_per_tile) * a.bc_per_tile * g.entries * g.d * sizeof(__half);
   if (smem > 96 * 1024) return VQ_ERR_UNSUPPORTED;
   const dim3 grid((g.K + a.tile_cols - 1) / a.tile_cols, (g.N + kTileRows - 1) / kTileRows, 1);
-  static bool attr_set[kMaxDevices][3] = {};
+  static int attr_set[kMaxDevices][3] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VQ_ERR_CUDA;
   auto launch = [&](auto kern, int slot) {
-    if (!attr_set[dev][slot]) {
+    if (!__atomic_load_n(&attr_set[dev][slot], __ATOMIC_ACQUIRE)) {
       if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024) != cudaSuccess) return VQ_ERR_CUDA;
-      attr_set[dev][slot] = true;
+      __atomic_store_n(&attr_set[dev][slot], 1, __ATOMIC_RELEASE);
     }
     kern<<<grid, 32 * kWarps, smem, s>>>(a);
     return check_launch();

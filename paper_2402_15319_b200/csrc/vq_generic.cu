@@ -156,7 +156,9 @@ vq_status launch_decode_generic(const Geometry& g, const LayerPtrs& p, __half* W
   if (g.J % 8 == 0 && !g.cb_int4) {   // K % 8 == 0 follows: every 128-bit store is aligned
     const long long total = static_cast<long long>(g.N) * (g.J / 8);
     long long blocks = (total + 255) / 256;
-    if (blocks > 148LL * 32) blocks = 148LL * 32;
+    int sms = 0;
+    if (device_sms(&sms) != VQ_OK) return VQ_ERR_CUDA;
+    if (blocks > static_cast<long long>(sms) * 32) blocks = static_cast<long long>(sms) * 32;
     const unsigned nb = static_cast<unsigned>(blocks);
     if (g.d == 1) decode_vec_kernel<1><<<nb, 256, 0, s>>>(g, p, W);
     else if (g.d == 2) decode_vec_kernel<2><<<nb, 256, 0, s>>>(g, p, W);
@@ -165,7 +167,9 @@ vq_status launch_decode_generic(const Geometry& g, const LayerPtrs& p, __half* W
   }
   const long long total = static_cast<long long>(g.N) * ((g.J + 7) / 8);
   long long blocks = (total + 255) / 256;
-  if (blocks > 148LL * 64) blocks = 148LL * 64;
+  int sms = 0;
+  if (device_sms(&sms) != VQ_OK) return VQ_ERR_CUDA;
+  if (blocks > static_cast<long long>(sms) * 64) blocks = static_cast<long long>(sms) * 64;
   decode_generic_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(g, p, W);
   return check_launch();
 }
@@ -173,7 +177,9 @@ vq_status launch_decode_generic(const Geometry& g, const LayerPtrs& p, __half* W
 vq_status launch_gemm_generic(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
                               cudaStream_t s) {
   long long blocks = (g.N + 7) / 8;
-  if (blocks > 148LL * 8) blocks = 148LL * 8;
+  int sms = 0;
+  if (device_sms(&sms) != VQ_OK) return VQ_ERR_CUDA;
+  if (blocks > static_cast<long long>(sms) * 8) blocks = static_cast<long long>(sms) * 8;
   const unsigned nb = static_cast<unsigned>(blocks);
   if (batch == 1) gemm_generic_kernel<1><<<nb, 256, 0, s>>>(g, p, X, Y, batch);
   else if (batch == 2) gemm_generic_kernel<2><<<nb, 256, 0, s>>>(g, p, X, Y, batch);

@@ -115,7 +115,9 @@ extern "C" vq_status vq_int4g128_gemm_small_batch(int32_t N, int32_t K, const vo
     if (st != VQ_ERR_UNSUPPORTED) return st;
   }
   long long blocks = (N + 7) / 8;
-  if (blocks > 148LL * 8) blocks = 148LL * 8;
+  int sms = 0;
+  if (device_sms(&sms) != VQ_OK) return VQ_ERR_CUDA;
+  if (blocks > static_cast<long long>(sms) * 8) blocks = static_cast<long long>(sms) * 8;
   const unsigned nb = static_cast<unsigned>(blocks);
   const uint32_t* q = static_cast<const uint32_t*>(d_q);
   const __half* sc = static_cast<const __half*>(d_scale);
@@ -140,7 +142,9 @@ extern "C" vq_status vq_unpack_uniform(int kind, int32_t N, int32_t K, const voi
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const long long groups8 = static_cast<long long>(N) * (K / 8);
   long long blocks = (groups8 + 255) / 256;
-  if (blocks > 148LL * 64) blocks = 148LL * 64;
+  int sms = 0;
+  if (device_sms(&sms) != VQ_OK) return VQ_ERR_CUDA;
+  if (blocks > static_cast<long long>(sms) * 64) blocks = static_cast<long long>(sms) * 64;
   const unsigned nb = static_cast<unsigned>(blocks);
   const __half* sc = static_cast<const __half*>(d_scale);
   uint4* W = static_cast<uint4*>(d_W);

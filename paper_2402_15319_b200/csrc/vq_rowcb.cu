@@ -639,15 +639,14 @@ template <class P, int NB, bool XS = false>
 vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch, cudaStream_t s) {
   if (g.K % P::STEP_COLS || g.Bc % P::STEP_COLS) return VQ_ERR_UNSUPPORTED;
   // per device, once: SM count and the opt-in to large dynamic shared memory
-  static int sms_of[kMaxDevices] = {};
+  static int attr_set[kMaxDevices] = {};
   auto kern = rowcb_kernel<P, NB, XS>;
-  int dev = 0;
+  int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VQ_ERR_CUDA;
-  if (sms_of[dev] == 0) {
-    int n = 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return VQ_ERR_CUDA;
+  if (device_sms(&sms) != VQ_OK) return VQ_ERR_CUDA;
+  if (!__atomic_load_n(&attr_set[dev], __ATOMIC_ACQUIRE)) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024) != cudaSuccess) return VQ_ERR_CUDA;
-    sms_of[dev] = n;
+    __atomic_store_n(&attr_set[dev], 1, __ATOMIC_RELEASE);
   }
   RowArgs a;
   a.idx = p.idx;
@@ -665,7 +664,7 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
   a.blocks_per_row = g.blocks_per_row;
   a.Br = g.Br;
   constexpr size_t kSmemBudget = 200 * 1024;
-  const Plan pl = make_plan(g.N, a.n_steps, P::STEP_COLS, batch, sms_of[dev], P::TABLE_BYTES_PER_WARP, NB, kSmemBudget, XS);
+  const Plan pl = make_plan(g.N, a.n_steps, P::STEP_COLS, batch, sms, P::TABLE_BYTES_PER_WARP, NB, kSmemBudget, XS);
   const int T = pl.S * pl.WK;
   if (pl.WR < 1 || pl.WK < 1 || pl.WR * pl.WK > 8 || pl.S < 1 || pl.S > 8 || T > a.n_steps) return VQ_ERR_UNSUPPORTED;
   a.WR = pl.WR;

@@ -239,11 +239,12 @@ struct RowD2B4 {
     float acc[R][NB][4];
     float sc[R][2], sc_raw[R][2];
     uint32_t raw[R][2][RAW];
-    uint32_t tbl, fill;
+    uint32_t tbl, fill, pat;
     int cur_key, pend_key;
 
     __device__ __forceinline__ void init(uint32_t warp_tbl, int lane) {
       tbl = warp_tbl + lane * 4;
+      pat = ((warp_tbl >> 12) & 0xFu) * 0x10101010u;   // address bits 12..15 of the tables, in every byte's high half
       fill = warp_tbl + (4 * (lane >> 3)) * 256 + (lane & 7) * 16;   // entries 4tb..4tb+3, the quad of row gb
       cur_key = pend_key = -1;
 #pragma unroll
@@ -337,11 +338,14 @@ struct RowD2B4 {
       }
     }
 
+    // Index I of a word whose even indices lie one per byte in `we` and odd ones in `wo`, each byte already
+    // carrying address bits 12..15 in its high half: one byte permute puts the byte into bits 8..15 of the
+    // lane's table address (a shift and a logic op per look-up otherwise; the integer pipe issues half as
+    // many instructions per clock as the four schedulers can).
     template <int I, int OFF>
-    __device__ __forceinline__ uint32_t gather(uint32_t w) const {
-      constexpr int p = 4 * I;
-      const uint32_t x = p < 8 ? w << (8 - p) : w >> (p - 8);
-      return lds32_off<OFF>((x & 0xF00u) | tbl);
+    __device__ __forceinline__ uint32_t gather(uint32_t we, uint32_t wo) const {
+      constexpr uint32_t sel = 0x3200u | ((4u + I / 2) << 4);
+      return lds32_off<OFF>(prmt(tbl, (I & 1) ? wo : we, sel));
     }
 
     template <int RR>
@@ -349,11 +353,13 @@ struct RowD2B4 {
       uint32_t wl, wh;
       load_words(idx + RR * 2048, ww, sw, wl, wh);
       constexpr int T0 = RR * TILE_TABLE_BYTES, T1 = T0 + 128;
+      const uint32_t le = (wl & 0x0F0F0F0Fu) | pat, lo = ((wl >> 4) & 0x0F0F0F0Fu) | pat;
+      const uint32_t he = (wh & 0x0F0F0F0Fu) | pat, ho = ((wh >> 4) & 0x0F0F0F0Fu) | pat;
       uint32_t af[4][4];
-      af[0][0] = gather<0, T0>(wl); af[0][1] = gather<0, T1>(wh); af[0][2] = gather<1, T0>(wl); af[0][3] = gather<1, T1>(wh);
-      af[1][0] = gather<2, T0>(wl); af[1][1] = gather<2, T1>(wh); af[1][2] = gather<3, T0>(wl); af[1][3] = gather<3, T1>(wh);
-      af[2][0] = gather<4, T0>(wl); af[2][1] = gather<4, T1>(wh); af[2][2] = gather<5, T0>(wl); af[2][3] = gather<5, T1>(wh);
-      af[3][0] = gather<6, T0>(wl); af[3][1] = gather<6, T1>(wh); af[3][2] = gather<7, T0>(wl); af[3][3] = gather<7, T1>(wh);
+      af[0][0] = gather<0, T0>(le, lo); af[0][1] = gather<0, T1>(he, ho); af[0][2] = gather<1, T0>(le, lo); af[0][3] = gather<1, T1>(he, ho);
+      af[1][0] = gather<2, T0>(le, lo); af[1][1] = gather<2, T1>(he, ho); af[1][2] = gather<3, T0>(le, lo); af[1][3] = gather<3, T1>(he, ho);
+      af[2][0] = gather<4, T0>(le, lo); af[2][1] = gather<4, T1>(he, ho); af[2][2] = gather<5, T0>(le, lo); af[2][3] = gather<5, T1>(he, ho);
+      af[3][0] = gather<6, T0>(le, lo); af[3][1] = gather<6, T1>(he, ho); af[3][2] = gather<7, T0>(le, lo); af[3][3] = gather<7, T1>(he, ho);
 #pragma unroll
       for (int nb = 0; nb < NB; ++nb) {
         mma16816(acc[RR][nb], af[0][0], af[0][1], af[0][2], af[0][3], b[nb][0].x, b[nb][0].y);
@@ -1119,19 +1125,6 @@ int env_int(const char* name, int dflt) {
 }
 
 size_t round_up(size_t v, size_t al) { return (v + al - 1) / al * al; }
-
-vq_status device_sms(int* out) {
-  static int sms_of[kMaxDevices] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VQ_ERR_CUDA;
-  int n = __atomic_load_n(&sms_of[dev], __ATOMIC_ACQUIRE);
-  if (n == 0) {
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return VQ_ERR_CUDA;
-    __atomic_store_n(&sms_of[dev], n, __ATOMIC_RELEASE);
-  }
-  *out = n;
-  return VQ_OK;
-}
 
 constexpr size_t kSmemMax = 224 * 1024;
 

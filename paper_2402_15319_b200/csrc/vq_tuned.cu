@@ -66,16 +66,33 @@ vq_status encode_tensor_map(CUtensorMap* tm, const void* base, int elem_bytes, i
   return VQ_OK;
 }
 
+// Per-device values looked up on first use.  Two host threads may make that first call together: both
+// then compute the same value and publish it with a release store, readers use an acquire load.
 vq_status device_error_counter(int** d_counter) {
   static int* addr_of[kMaxDevices] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VQ_ERR_CUDA;
-  if (!addr_of[dev]) {
+  int* addr = __atomic_load_n(&addr_of[dev], __ATOMIC_ACQUIRE);
+  if (!addr) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_wait_failures) != cudaSuccess || !p) return VQ_ERR_CUDA;
-    addr_of[dev] = static_cast<int*>(p);
+    addr = static_cast<int*>(p);
+    __atomic_store_n(&addr_of[dev], addr, __ATOMIC_RELEASE);
   }
-  *d_counter = addr_of[dev];
+  *d_counter = addr;
+  return VQ_OK;
+}
+
+vq_status device_sms(int* out) {
+  static int sms_of[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VQ_ERR_CUDA;
+  int n = __atomic_load_n(&sms_of[dev], __ATOMIC_ACQUIRE);
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return VQ_ERR_CUDA;
+    __atomic_store_n(&sms_of[dev], n, __ATOMIC_RELEASE);
+  }
+  *out = n;
   return VQ_OK;
 }
 
