@@ -1,5 +1,6 @@
 // C-ABI entry points: host-side validation and kernel dispatch.  No kernel lives here.
 #include <math.h>
+#include <stdlib.h>
 
 #include "vq_common.cuh"
 
@@ -177,10 +178,22 @@ vq_status vq_gemm_small_batch_impl(const vq_format* fmt, const void* d_idx, cons
   return launch_gemm_generic(g, p, X, Y, batch, s);
 }
 
+// Which kernel family serves a group in one launch: 2 = the cluster kernels of the shared-codebook
+// formats (their K-split meets in distributed shared memory: lowest latency on the small layers those
+// formats come with), 1 = the persistent kernel (per-row formats at batch 1-2 and 9-16, where one launch
+// beat the members' separate launches: q/k/v of the 70B-shaped set 12.9 us against 19.5 us at batch 1,
+// a tie at batch 4), 0 = member by member.
+static int group_family(const Geometry& g, int batch) {
+  if (g.cb_int4) return 0;
+  if (blockcb_covers(g)) return 2;
+  return (batch <= 2 || batch > 8) ? 1 : 0;
+}
+
 int vq_grouped_kernel_launches(const vq_format* fmt, int n_members, int batch) {
   Geometry g;
   if (make_geometry(fmt, &g) != VQ_OK || n_members < 1 || n_members > VQ_MAX_GROUP || batch < 1 || batch > 16) return 0;
-  return (n_members > 1 && (batch <= 2 || batch > 8) && stream_covers(g)) ? 1 : n_members;
+  if (n_members > 1 && blockcb_covers(g) && group_family(g, batch) == 2) return 1;
+  return (n_members > 1 && group_family(g, batch) == 1 && stream_covers(g)) ? 1 : n_members;
 }
 
 vq_status vq_gemm_small_batch_grouped(const vq_format* fmt, const vq_group_member* members, int n_members,
@@ -219,10 +232,15 @@ vq_status vq_gemm_small_batch_grouped(const vq_format* fmt, const vq_group_membe
   call.ws = d_ws;
   call.ws_bytes = ws_bytes;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  // one persistent kernel for the group where it is the faster way (measured: q/k/v of the 70B-shaped
-  // set 12.9 us against 19.5 us for three launches at batch 1, a tie at batch 4)
   vq_status st = VQ_ERR_UNSUPPORTED;
-  if (!call.g.cb_int4 && n_members > 1 && (batch <= 2 || batch > 8)) st = launch_gemm_stream(call, s);
+  if (n_members > 1) {
+    int fam = group_family(call.g, batch);
+#ifdef VQ_TUNING
+    if (getenv("VQ_GROUP_FAMILY")) fam = atoi(getenv("VQ_GROUP_FAMILY"));
+#endif
+    if (fam == 2) st = launch_gemm_blockcb_group(call, s);
+    if (fam == 1 || (fam == 2 && st == VQ_ERR_UNSUPPORTED && (batch <= 2 || batch > 8))) st = launch_gemm_stream(call, s);
+  }
   if (st != VQ_ERR_UNSUPPORTED) return st;
   for (int i = 0; i < n_members; ++i) {   // formats the persistent kernel does not take: member by member
     one.n_rows = members[i].n_rows;

@@ -67,6 +67,20 @@ struct BlockArgs {
   int compact_off, ring_off, bar_off, x_off, recv_off;
 };
 
+// Layers of one call (same format and K, their own rows): row tiles [tile0, next tile0) of the grid
+// belong to layer i.
+struct BlockGroup {
+  const void* cb[kMaxSegments];
+  const __half* scale[kMaxSegments];
+  __half* Y[kMaxSegments];
+  int N[kMaxSegments];
+  int tile0[kMaxSegments];
+  int n_seg;
+};
+struct BlockMaps {
+  CUtensorMap m[kMaxSegments];   // the layers' index streams
+};
+
 // ---- format policies -----------------------------------------------------------------------
 template <int D, int B>
 struct Policy;
@@ -314,7 +328,7 @@ __device__ __forceinline__ void write_private(uint32_t table, const PrivateRegs<
 // PRIV: every warp keeps its own pair of tables (block rows a multiple of 32, 2-D only).
 template <int D, int B, int NB, bool PRIV>
 __global__ void __launch_bounds__(Tile<D, B>::THREADS)
-blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
+blockcb_kernel(const __grid_constant__ BlockMaps maps, const BlockArgs a_in, const BlockGroup grp) {
   static_assert(!PRIV || D == 2, "warp-private tables exist for 2-D codebooks only");
   constexpr int ST = kStagesOf<D, PRIV>;   // ring stages per warp
   using P = Policy<D, B>;
@@ -328,6 +342,17 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int S = gridDim.x, rank = blockIdx.x;
+  // the layer of this row tile
+  int sgi = 0;
+#pragma unroll
+  for (int i = 1; i < kMaxSegments; ++i)
+    if (i < grp.n_seg && static_cast<int>(blockIdx.y) >= grp.tile0[i]) sgi = i;
+  BlockArgs a = a_in;
+  a.cb = grp.cb[sgi];
+  a.scale = grp.scale[sgi];
+  a.Y = grp.Y[sgi];
+  a.N = grp.N[sgi];
+  const CUtensorMap* tm = &maps.m[sgi];
   // Receive barrier of the K-part reduction: S * rpo * batch values of 4 bytes arrive through
   // asynchronous remote stores.  Initialised before the start-up arrive so that every CTA of the
   // cluster sees it once its start-up wait (in front of the first remote store) returns.
@@ -344,7 +369,7 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
   pdl_launch_dependents();
 
   const int c0 = a.n_chunks * rank / S, c1 = a.n_chunks * (rank + 1) / S, n = c1 - c0;
-  const int row0 = blockIdx.y * T::CTA_ROWS;
+  const int row0 = (static_cast<int>(blockIdx.y) - grp.tile0[sgi]) * T::CTA_ROWS;
   // first block of the block row the CTA's (PRIV: the warp's) rows lie in
   const long long blk_row = static_cast<long long>((row0 + (PRIV ? 32 * warp : 0)) / a.Br) * a.blocks_per_row;
   const int cpt = D == 2 ? 1 : a.Bc / 256;   // chunks that share one table
@@ -361,7 +386,7 @@ blockcb_kernel(const __grid_constant__ CUtensorMap tm, const BlockArgs a) {
   auto issue = [&](int i) {   // lane 0 only
     const int st = i % ST;
     mbar_arrive_expect_tx(bars + 8 * st, T::STAGE_BYTES);
-    tma_box_2d(ring + st * T::STAGE_BYTES, &tm, (c0 + i) * P::SEG, row0 + 32 * warp, bars + 8 * st);
+    tma_box_2d(ring + st * T::STAGE_BYTES, tm, (c0 + i) * P::SEG, row0 + 32 * warp, bars + 8 * st);
   };
   if (lane == 0)
     for (int i = 0; i < ST && i < n; ++i) issue(i);
@@ -590,7 +615,10 @@ int env_int(const char* name, int dflt) {
 size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 template <int D, int B, int NB, bool PRIV = false>
-vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch, cudaStream_t s) {
+vq_status launch(const StreamCall& call, cudaStream_t s) {
+  const Geometry& g = call.g;
+  const __half* X = call.X;
+  const int batch = call.batch;
   using P = Policy<D, B>;
   using T = Tile<D, B>;
   auto kern = blockcb_kernel<D, B, NB, PRIV>;
@@ -606,19 +634,34 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
   if (device_error_counter(&error_flag) != VQ_OK) return VQ_ERR_CUDA;
 
   BlockArgs a;
-  a.cb = p.cb;
-  a.scale = g.cb_int8 ? p.scale : nullptr;
+  a.cb = nullptr;      // (per layer: the kernel takes them from the group)
+  a.scale = nullptr;
   a.X = X;
-  a.Y = Y;
+  a.Y = nullptr;
   a.error_flag = error_flag;
-  a.N = g.N;
+  a.N = 0;
   a.K = g.K;
   a.batch = batch;
   a.n_chunks = g.K / 256;
   a.blocks_per_row = g.blocks_per_row;
   a.Br = g.Br;
   a.Bc = g.Bc;
-  const int row_blocks = g.N / T::CTA_ROWS;
+  BlockGroup grp = {};
+  BlockMaps maps;
+  grp.n_seg = call.n_seg;
+  int row_blocks = 0;
+  for (int i = 0; i < call.n_seg; ++i) {
+    if (call.N[i] <= 0 || call.N[i] % T::CTA_ROWS) return VQ_ERR_UNSUPPORTED;
+    grp.cb[i] = call.cb[i];
+    grp.scale[i] = g.cb_int8 ? call.scale[i] : nullptr;
+    grp.Y[i] = call.Y[i];
+    grp.N[i] = call.N[i];
+    grp.tile0[i] = row_blocks;
+    row_blocks += call.N[i] / T::CTA_ROWS;
+    // index stream as a 2-D byte tensor: rows of `stride` bytes; one box = 32 rows x SEG bytes
+    if (encode_index_map(&maps.m[i], call.idx[i], g.stride, call.N[i], P::SEG, 32) != VQ_OK) return VQ_ERR_CUDA;
+  }
+  for (int i = call.n_seg; i < kMaxSegments; ++i) maps.m[i] = maps.m[0];
 
   // Shared memory of a CTA whose column range is `chunks` long.
   auto smem_for = [&](int chunks, BlockArgs* out) {
@@ -659,10 +702,6 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
   const size_t smem_bytes = smem_for((a.n_chunks + best - 1) / best, &a);
   if (smem_bytes > 220 * 1024) return VQ_ERR_UNSUPPORTED;
 
-  // index stream as a 2-D byte tensor: rows of `stride` bytes; one box = 32 rows x SEG bytes
-  CUtensorMap tm;
-  if (encode_index_map(&tm, p.idx, g.stride, g.N, P::SEG, 32) != VQ_OK) return VQ_ERR_CUDA;
-
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(best, row_blocks, 1);
   cfg.blockDim = dim3(T::THREADS, 1, 1);
@@ -684,7 +723,7 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
   }
   cfg.attrs = attr;
   cfg.numAttrs = na;
-  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tm, a);
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, maps, a, grp);
   if (e != cudaSuccess) {
 #ifdef VQ_TUNING
     fprintf(stderr, "blockcb launch failed: %s (S %d smem %zu)\n", cudaGetErrorString(e), best, smem_bytes);
@@ -697,28 +736,54 @@ vq_status launch(const Geometry& g, const LayerPtrs& p, const __half* X, __half*
 }  // namespace
 
 // Shared-codebook families: fp16 or int8 codebooks, block rows a multiple of the CTA's rows, block columns
-// a multiple of 128 (2-D) / 256 (4-D), K a multiple of the 256-column chunk.
-vq_status launch_gemm_blockcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
-                              cudaStream_t s) {
+// a multiple of 128 (2-D) / 256 (4-D), K a multiple of the 256-column chunk.  One launch serves every
+// layer of the call (same format and K; rows per layer in call.N).
+bool blockcb_covers(const Geometry& g) {
+  if (g.cb_int4 || g.K % 256) return false;
+  if (g.d == 2 && (g.b == 6 || g.b == 5)) return g.Bc % 128 == 0 && (g.Br % 128 == 0 || (g.Br % 32 == 0 && 128 % g.Br == 0));
+  if (g.d == 4 && g.b == 8) return g.Br % Tile<4, 8>::CTA_ROWS == 0 && g.Bc % 256 == 0;
+  return false;
+}
+
+vq_status launch_gemm_blockcb_group(const StreamCall& call, cudaStream_t s) {
+  const Geometry& g = call.g;
+  const int batch = call.batch;
   if (g.K % 256) return VQ_ERR_UNSUPPORTED;
   if (g.d == 2 && (g.b == 6 || g.b == 5)) {
     if (g.Bc % 128) return VQ_ERR_UNSUPPORTED;
     // blocks of 128 rows or more: one pair of tables per CTA; 32 or 64 rows (the CTA's 128 rows must
     // consist of whole blocks): a pair per warp
     const bool shared_tables = g.Br % 128 == 0;
-    if (!shared_tables && (g.Br % 32 || 128 % g.Br || g.N % 128)) return VQ_ERR_UNSUPPORTED;
+    if (!shared_tables && (g.Br % 32 || 128 % g.Br)) return VQ_ERR_UNSUPPORTED;
+    for (int i = 0; i < call.n_seg; ++i)
+      if (call.N[i] % 128) return VQ_ERR_UNSUPPORTED;
     if (g.b == 6) {
-      if (shared_tables) return batch <= 8 ? launch<2, 6, 1>(g, p, X, Y, batch, s) : launch<2, 6, 2>(g, p, X, Y, batch, s);
-      return batch <= 8 ? launch<2, 6, 1, true>(g, p, X, Y, batch, s) : launch<2, 6, 2, true>(g, p, X, Y, batch, s);
+      if (shared_tables) return batch <= 8 ? launch<2, 6, 1>(call, s) : launch<2, 6, 2>(call, s);
+      return batch <= 8 ? launch<2, 6, 1, true>(call, s) : launch<2, 6, 2, true>(call, s);
     }
-    if (shared_tables) return batch <= 8 ? launch<2, 5, 1>(g, p, X, Y, batch, s) : launch<2, 5, 2>(g, p, X, Y, batch, s);
-    return batch <= 8 ? launch<2, 5, 1, true>(g, p, X, Y, batch, s) : launch<2, 5, 2, true>(g, p, X, Y, batch, s);
+    if (shared_tables) return batch <= 8 ? launch<2, 5, 1>(call, s) : launch<2, 5, 2>(call, s);
+    return batch <= 8 ? launch<2, 5, 1, true>(call, s) : launch<2, 5, 2, true>(call, s);
   }
   if (g.d == 4 && g.b == 8) {
     if (g.Br % Tile<4, 8>::CTA_ROWS || g.Bc % 256) return VQ_ERR_UNSUPPORTED;
-    return batch <= 8 ? launch<4, 8, 1>(g, p, X, Y, batch, s) : launch<4, 8, 2>(g, p, X, Y, batch, s);
+    return batch <= 8 ? launch<4, 8, 1>(call, s) : launch<4, 8, 2>(call, s);
   }
   return VQ_ERR_UNSUPPORTED;
+}
+
+vq_status launch_gemm_blockcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
+                              cudaStream_t s) {
+  StreamCall call = {};
+  call.g = g;
+  call.n_seg = 1;
+  call.idx[0] = p.idx;
+  call.cb[0] = p.cb;
+  call.scale[0] = p.scale;
+  call.Y[0] = Y;
+  call.N[0] = g.N;
+  call.X = X;
+  call.batch = batch;
+  return launch_gemm_blockcb_group(call, s);
 }
 
 }  // namespace vq

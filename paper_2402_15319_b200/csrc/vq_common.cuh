@@ -68,6 +68,10 @@ vq_status launch_int4g128_stream(int N, int K, const uint8_t* q, const __half* s
                                  void* ws, size_t ws_bytes, cudaStream_t s);
 vq_status launch_gemm_blockcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
                               cudaStream_t s);
+// The same kernels over several layers of one format and K in one launch (rows per layer in call.N;
+// call.ws is not used), and whether they take the format (member rows must be multiples of 128 too).
+vq_status launch_gemm_blockcb_group(const StreamCall& call, cudaStream_t s);
+bool blockcb_covers(const Geometry& g);
 vq_status launch_gemm_rowcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
                             cudaStream_t s);
 vq_status launch_int4g128_rowcb(int N, int K, const uint8_t* q, const __half* scale, const __half* X, __half* Y, int batch,

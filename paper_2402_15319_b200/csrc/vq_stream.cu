@@ -39,12 +39,6 @@ namespace {
 
 using namespace dev;
 
-#ifndef VQ_UNROLL_D2
-#define VQ_UNROLL_D2 2   // index-word steps of the 2-D loop emitted back to back (the loop body must stay small: the
-#endif                  // kernel is sensitive to instruction-cache misses)
-#ifndef VQ_UNROLL_D1
-#define VQ_UNROLL_D1 4
-#endif
 // Index-word steps of the decode loops that are emitted back to back (8 = the whole chunk; measured
 // on B200: 1, 2, 4, 8 steps give 32.3 / 31.4 / 30.7 / 30.0 us on a 28672 x 8192 layer).
 #ifndef VQ_UNROLL_D2
@@ -143,6 +137,11 @@ __device__ __forceinline__ void fence_acc(float (&acc)[NB][4]) {
 constexpr uint32_t kMagic = 0x64646464u;      // high byte of fp16 1024.0
 constexpr uint32_t kBias2 = 0x64806480u;      // fp16 pair (1152, 1152) = 1024 + 128
 // (1024 + u) - 1152 = u - 128, exact in fp16
+__device__ __forceinline__ uint32_t mul_f16x2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
 __device__ __forceinline__ uint32_t sub_bias(uint32_t h) {
   uint32_t r;
   asm("sub.f16x2 %0, %1, %2;" : "=r"(r) : "r"(h), "r"(kBias2));
@@ -237,32 +236,31 @@ struct RowD2B4 {
   template <int NB, int R>
   struct State {
     float acc[R][NB][4];
-    float sc[R][2], sc_raw[R][2];
+    uint32_t sc_raw[R][2];      // the block scale of the rows this lane FILLS, twice (an fp16 pair)
     uint32_t raw[R][2][RAW];
     uint32_t tbl, fill, pat;
     int cur_key, pend_key;
 
+    __device__ __forceinline__ void probe_fill(const uint32_t*) {}
     __device__ __forceinline__ void init(uint32_t warp_tbl, int lane) {
       tbl = warp_tbl + lane * 4;
       pat = ((warp_tbl >> 12) & 0xFu) * 0x10101010u;   // address bits 12..15 of the tables, in every byte's high half
       fill = warp_tbl + (4 * (lane >> 3)) * 256 + (lane & 7) * 16;   // entries 4tb..4tb+3, the quad of row gb
       cur_key = pend_key = -1;
 #pragma unroll
-      for (int r = 0; r < R; ++r) {
-        sc[r][0] = sc[r][1] = 1.f;
+      for (int r = 0; r < R; ++r)
 #pragma unroll
         for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
           for (int e = 0; e < 4; ++e) acc[r][nb][e] = 0.f;
-      }
     }
 
     // Request the entries (and scales) of the block of `w`; lane l takes entries 4*(l/8)..+3 of rows
-    // l%8 and l%8+8 of every tile (the mapping the table is WRITTEN with), the scales of its own rows.
+    // l%8 and l%8+8 of every tile (the mapping the table is WRITTEN with) and those rows' scales.
     __device__ __forceinline__ void fetch(const StreamArgs& a, const Where& w, int lane) {
       const Segment& sg = a.seg[w.seg];
       const int blk = w.ch >> a.cpb_shift;
-      const int gb = lane & 7, tb = lane >> 3, g = lane >> 2;
+      const int gb = lane & 7, tb = lane >> 3;
 #pragma unroll
       for (int r = 0; r < R; ++r)
 #pragma unroll
@@ -273,8 +271,8 @@ struct RowD2B4 {
           if constexpr (INT8) {
             const uint2 v = ldg64_nc(p);
             raw[r][h][0] = v.x; raw[r][h][1] = v.y;
-            const int rr = min(w.row0 + 16 * r + g + 8 * h, sg.N - 1);
-            sc_raw[r][h] = __half2float(__ldg(sg.scale + static_cast<long long>(rr >> a.br_shift) * a.blocks_per_row + blk));
+            const uint32_t s16 = __ldg(reinterpret_cast<const unsigned short*>(sg.scale) + static_cast<long long>(rb >> a.br_shift) * a.blocks_per_row + blk);
+            sc_raw[r][h] = s16 * 0x10001u;
           } else {
             const uint4 v = ldg128_nc(p);
             raw[r][h][0] = v.x; raw[r][h][1] = v.y; raw[r][h][2] = v.z; raw[r][h][3] = v.w;
@@ -290,12 +288,11 @@ struct RowD2B4 {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           uint32_t e[4];
-          if constexpr (INT8) {
-            e[0] = sub_bias(prmt(raw[r][h][0] ^ 0x80808080u, kMagic, 0x4140));
-            e[1] = sub_bias(prmt(raw[r][h][0] ^ 0x80808080u, kMagic, 0x4342));
-            e[2] = sub_bias(prmt(raw[r][h][1] ^ 0x80808080u, kMagic, 0x4140));
-            e[3] = sub_bias(prmt(raw[r][h][1] ^ 0x80808080u, kMagic, 0x4342));
-            sc[r][h] = sc_raw[r][h];
+          if constexpr (INT8) {   // the table holds fp16(scale * c), the values vq_decode_weights writes
+            e[0] = mul_f16x2(sub_bias(prmt(raw[r][h][0] ^ 0x80808080u, kMagic, 0x4140)), sc_raw[r][h]);
+            e[1] = mul_f16x2(sub_bias(prmt(raw[r][h][0] ^ 0x80808080u, kMagic, 0x4342)), sc_raw[r][h]);
+            e[2] = mul_f16x2(sub_bias(prmt(raw[r][h][1] ^ 0x80808080u, kMagic, 0x4140)), sc_raw[r][h]);
+            e[3] = mul_f16x2(sub_bias(prmt(raw[r][h][1] ^ 0x80808080u, kMagic, 0x4342)), sc_raw[r][h]);
           } else {
 #pragma unroll
             for (int i = 0; i < 4; ++i) e[i] = raw[r][h][i];
@@ -307,19 +304,18 @@ struct RowD2B4 {
       fence_value(tbl);   // gathers of the new block stay behind the rewrite
     }
 
-    // Close the current block: its scale multiplies its fp32 partial sums.
+    // Hand the slab's sums over (the scales are already inside the tables: one accumulator runs
+    // across the blocks of a row).
     __device__ __forceinline__ void flush(float (&total)[R][NB][4]) {
 #pragma unroll
       for (int r = 0; r < R; ++r)
 #pragma unroll
-        for (int nb = 0; nb < NB; ++nb) {
-          total[r][nb][0] = fmaf(sc[r][0], acc[r][nb][0], total[r][nb][0]);
-          total[r][nb][1] = fmaf(sc[r][0], acc[r][nb][1], total[r][nb][1]);
-          total[r][nb][2] = fmaf(sc[r][1], acc[r][nb][2], total[r][nb][2]);
-          total[r][nb][3] = fmaf(sc[r][1], acc[r][nb][3], total[r][nb][3]);
+        for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-          for (int e = 0; e < 4; ++e) acc[r][nb][e] = 0.f;
-        }
+          for (int e = 0; e < 4; ++e) {
+            total[r][nb][e] = acc[r][nb][e];
+            acc[r][nb][e] = 0.f;
+          }
     }
 
     __device__ __forceinline__ void prefetch(const StreamArgs& a, const Where& next, int lane) {
@@ -329,9 +325,6 @@ struct RowD2B4 {
     // Make the block of `w` the current one (its tables must be complete before the stage's look-ups).
     __device__ __forceinline__ void begin(const StreamArgs& a, const Where& w, int lane, float (&total)[R][NB][4]) {
       if (w.key != cur_key) {
-#pragma unroll
-        for (int r = 0; r < R; ++r) fence_acc(acc[r]);
-        flush(total);
         if (pend_key != w.key) fetch(a, w, lane);
         install();
         cur_key = w.key;
@@ -416,6 +409,15 @@ struct RowD1B4I8 {
     uint4 raw[R][2];
     int cur_key, pend_key;
 
+    // (decode-loop probe) register tables from arbitrary values: w must not be a compile-time constant
+    __device__ __forceinline__ void probe_fill(const uint32_t* w) {
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) T[r][h][i] = w[r * 8 + h * 4 + i];
+    }
     __device__ __forceinline__ void init(uint32_t, int) {
       cur_key = pend_key = -1;
 #pragma unroll
@@ -535,6 +537,7 @@ struct RowInt4G128 {
     uint32_t sc_cur[R][2], sc_next[R][2];   // two fp16 scales (the chunk's two groups) per row
     int cur_key, pend_key;
 
+    __device__ __forceinline__ void probe_fill(const uint32_t*) {}
     __device__ __forceinline__ void init(uint32_t, int) { cur_key = pend_key = -1; }
     __device__ __forceinline__ void fetch(const StreamArgs& a, const Where& w, int lane) {
       const Segment& sg = a.seg[w.seg];
@@ -704,6 +707,7 @@ struct BlkD2B6 {
   template <int NB, int R>
   struct State {
     float acc[R][NB][4];
+    __device__ __forceinline__ void probe_fill(const uint32_t*) {}
     __device__ __forceinline__ void init(uint32_t, int) {
 #pragma unroll
       for (int r = 0; r < R; ++r)
@@ -1360,16 +1364,20 @@ __global__ void __launch_bounds__(256, 1) probe_decode_kernel(int iters, int bat
   unsigned char* smem = smem_raw + (sbase - smem_u32(smem_raw));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, W = blockDim.x / 32;
   const int g = lane >> 2, t = lane & 3;
-  // [stage table | per-warp tables | index rows of every warp | activations]
+  // [stage table | per-warp tables | two stages of (index rows of every warp | activations)]: the passes
+  // alternate between the stages as the pipeline of the real kernel does, so that no load of one pass
+  // can be kept for the next
   const int tbl_words = (P::STAGE_TABLE_BYTES + W * R * P::TILE_TABLE_BYTES) / 4;
   const int idx_words = W * R * 16 * P::CHUNK_BYTES / 4;
   const int x_words = P::X_ROWS * batch * P::X_ROW_BYTES / 4;
+  const int stage_words = idx_words + x_words;
   uint32_t* words = reinterpret_cast<uint32_t*>(smem);
   uint32_t seed = 1234567u + tid * 7919u + blockIdx.x;
-  for (int i = tid; i < tbl_words + idx_words + x_words; i += blockDim.x) {
+  for (int i = tid; i < tbl_words + 2 * stage_words; i += blockDim.x) {
     seed = seed * 1664525u + 1013904223u;
     // small finite fp16 pairs for tables and activations, anything for indices
-    words[i] = i < tbl_words ? (0x2C002C00u | (seed & 0x03FF03FFu)) : i < tbl_words + idx_words ? seed : (0x34003400u | (seed & 0x83FF83FFu));
+    const int j = i < tbl_words ? -1 : (i - tbl_words) % stage_words;
+    words[i] = j < 0 ? (0x2C002C00u | (seed & 0x03FF03FFu)) : j < idx_words ? seed : (0x34003400u | (seed & 0x83FF83FFu));
   }
   __syncthreads();
   typename P::template State<NB, R> st;
@@ -1386,9 +1394,11 @@ __global__ void __launch_bounds__(256, 1) probe_decode_kernel(int iters, int bat
   for (int nb = 0; nb < NB; ++nb) xm[nb] = min(nb * 8 + g, batch - 1);
   const unsigned char* idx = smem + tbl_words * 4 + (warp * R * 16 + g) * P::CHUNK_BYTES + t * P::LANE_BYTES;
   const unsigned char* xpart = smem + (tbl_words + idx_words) * 4;
+  st.probe_fill(words + tbl_words + (tid * 41) % (idx_words - 64));
   const long long c0 = clock64();
   for (int it = 0; it < iters; ++it) {
-    st.compute(idx, xpart, xm, batch, sbase, lane, total);
+    const int off = (it & 1) * stage_words * 4;
+    st.compute(idx + off, xpart + off, xm, batch, sbase, lane, total);
     asm volatile("" ::: "memory");
   }
   const long long c1 = clock64();
@@ -1408,8 +1418,8 @@ template <class P, int R>
 vq_status run_probe(int warps, int batch, int iters, int sms, long long* d_cycles, float* d_sink, cudaStream_t s,
                     double* weights_per_stage) {
   auto kern = probe_decode_kernel<P, 1, R>;
-  const size_t smem = P::BASE_ALIGN + P::STAGE_TABLE_BYTES + static_cast<size_t>(warps) * R * (P::TILE_TABLE_BYTES + 16 * P::CHUNK_BYTES) +
-                      static_cast<size_t>(P::X_ROWS) * batch * P::X_ROW_BYTES + 1024;
+  const size_t smem = P::BASE_ALIGN + P::STAGE_TABLE_BYTES + static_cast<size_t>(warps) * R * (P::TILE_TABLE_BYTES + 2 * 16 * P::CHUNK_BYTES) +
+                      2 * static_cast<size_t>(P::X_ROWS) * batch * P::X_ROW_BYTES + 1024;
   if (smem > kSmemMax) return VQ_ERR_UNSUPPORTED;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemMax)) != cudaSuccess) return VQ_ERR_CUDA;
   kern<<<sms, warps * 32, smem, s>>>(iters, batch, d_cycles, d_sink);

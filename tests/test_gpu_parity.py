@@ -156,6 +156,8 @@ GROUPS = [
     (vq_synth.LayerSpec("g_row", N=0, K=4096, d=2, b=4, Br=1, Bc=2048, int8=True), [2048, 264, 256]),
     (vq_synth.LayerSpec("g_row16", N=0, K=2048, d=2, b=4, Br=1, Bc=1024, int8=False), [300, 1000]),
     (vq_synth.LayerSpec("g_blk", N=0, K=1024, d=2, b=6, Br=128, Bc=128, int8=False), [512, 128, 128, 256]),
+    (vq_synth.LayerSpec("g_blk32", N=0, K=1024, d=2, b=6, Br=32, Bc=256, int8=True), [256, 128, 384]),
+    (vq_synth.LayerSpec("g_d4b8", N=0, K=1024, d=4, b=8, Br=256, Bc=512, int8=False), [256, 512]),
     (vq_synth.LayerSpec("g_generic", N=0, K=312, d=1, b=5, Br=1, Bc=156, int8=False), [37, 5]),
 ]
 
