@@ -521,11 +521,13 @@ struct RowD1B4I8 {
 };
 
 // ---- uniform INT4 with an fp16 scale per 128 columns (paper Sec. 2.1 symmetric uniform quantiser;
-// Sec. 5 "INT4 g128"), the bandwidth yard-stick: no table.  Byte j of an index word holds columns
-// 2j (low nibble) and 2j+1 (high nibble): the byte is copied into both halves of a register, masked
-// to (q_lo, 16*q_hi) and merged with the fp16 exponent of 1024, giving the pair (1024 + q_lo,
-// 1024 + 16*q_hi); one fused multiply-add by (1, 1/16) and (-1032, -72) makes it (q_lo - 8, q_hi - 8),
-// exactly.
+// Sec. 5, the uniform 4-bit group-128 rows of the tables), the bandwidth yard-stick: no table.  Nibble i
+// of an index word is column i of the lane's 8 columns.  Masking the word with 0x000F000F leaves nibbles
+// 0 and 4 in the two halves of a register, 0x00F000F0 nibbles 1 and 5 (times 16); merged with the fp16
+// exponent of 1024 they are the pairs (1024 + q0, 1024 + q4) and (1024 + 16 q1, 1024 + 16 q5), and one
+// fused multiply-add by (1, -1032) or (1/16, -72) makes them (q - 8), exactly.  The tensor-core step sums
+// over its 16 columns in any order, so the activations are paired the same way (one byte permute per
+// pair, shared by the row tiles): five integer-pipe operations per 8 weights instead of eight.
 struct RowInt4G128 {
   static constexpr int CHUNK_BYTES = 128, CHUNK_COLS = 256, X_ROW_BYTES = 64, X_ROWS = 8, LANE_BYTES = 4;
   static constexpr bool X_SWIZZLE = false, IDX_SWIZZLE = true, X_BATCH_INNER = true;
@@ -572,8 +574,8 @@ struct RowInt4G128 {
 #pragma unroll
       for (int nb = 0; nb < NB; ++nb) xrow[nb] = xpart + xm[nb] * X_ROW_BYTES;
       const uint32_t xstep = batch * X_ROW_BYTES;
-      constexpr uint32_t kMul = 0x2C003C00u;    // fp16 pair (1, 1/16)
-      constexpr uint32_t kAdd = 0xD480E408u;    // fp16 pair (-1032, -72)
+      constexpr uint32_t kOne = 0x3C003C00u, kLoAdd = 0xE408E408u;         // (1, 1), (-1032, -1032)
+      constexpr uint32_t kSixteenth = 0x2C002C00u, kHiAdd = 0xD480D480u;   // (1/16, 1/16), (-72, -72)
       const uint32_t sw = static_cast<uint32_t>(lane >> 2) << 4;
       const uint32_t t16 = static_cast<uint32_t>(lane & 3) << 4;
       uint4 b[NB];
@@ -590,24 +592,33 @@ struct RowInt4G128 {
         for (int w4 = 0; w4 < 4; ++w4) {
           const int ww = 4 * grp + w4;
 #pragma unroll
-          for (int nb = 0; nb < NB; ++nb) b[nb] = *reinterpret_cast<const uint4*>(xrow[nb] + ww * xstep + t16);
+          for (int nb = 0; nb < NB; ++nb) {
+            // the lane's 8 activations x0..x7, paired as the nibbles pair below: (x0,x4) (x1,x5) (x2,x6) (x3,x7);
+            // one permute per pair, shared by every row tile
+            const uint4 v = *reinterpret_cast<const uint4*>(xrow[nb] + ww * xstep + t16);
+            b[nb] = make_uint4(prmt(v.x, v.z, 0x5410u), prmt(v.x, v.z, 0x7632u), prmt(v.y, v.w, 0x5410u), prmt(v.y, v.w, 0x7632u));
+          }
 #pragma unroll
           for (int r = 0; r < R; ++r) {
             uint32_t wd[2];
             load_words(idx + r * 2048, ww, sw, wd[0], wd[1]);
+            // nibbles n0..n7 of a word are columns 0..7: one logic op takes (n0, n4) or (16 n1, 16 n5) into
+            // the mantissas of the pair (1024, 1024); the word shifted by 8 gives (n2, n6) and (16 n3, 16 n7)
             uint32_t q[2][4];
 #pragma unroll
-            for (int h = 0; h < 2; ++h)
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const uint32_t both = prmt(wd[h], 0u, 0x4040u + 0x0101u * i);      // byte i in bits 0..7 and 16..23
-                const uint32_t m = (both & 0x00F0000Fu) | 0x64006400u;             // (1024 + q_lo, 1024 + 16 q_hi)
-                asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(q[h][i]) : "r"(m), "r"(kMul), "r"(kAdd));
-              }
+            for (int h = 0; h < 2; ++h) {
+              const uint32_t w0 = wd[h], w8 = wd[h] >> 8;
+              const uint32_t m0 = (w0 & 0x000F000Fu) | 0x64006400u, m1 = (w0 & 0x00F000F0u) | 0x64006400u;
+              const uint32_t m2 = (w8 & 0x000F000Fu) | 0x64006400u, m3 = (w8 & 0x00F000F0u) | 0x64006400u;
+              asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(q[h][0]) : "r"(m0), "r"(kOne), "r"(kLoAdd));
+              asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(q[h][1]) : "r"(m1), "r"(kSixteenth), "r"(kHiAdd));
+              asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(q[h][2]) : "r"(m2), "r"(kOne), "r"(kLoAdd));
+              asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(q[h][3]) : "r"(m3), "r"(kSixteenth), "r"(kHiAdd));
+            }
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb) {
-              mma16816(acc[r][nb], q[0][0], q[1][0], q[0][1], q[1][1], b[nb].x, b[nb].y);   // columns 0,1 | 2,3
-              mma16816(acc[r][nb], q[0][2], q[1][2], q[0][3], q[1][3], b[nb].z, b[nb].w);   // columns 4,5 | 6,7
+              mma16816(acc[r][nb], q[0][0], q[1][0], q[0][1], q[1][1], b[nb].x, b[nb].y);   // columns 0,4 | 1,5
+              mma16816(acc[r][nb], q[0][2], q[1][2], q[0][3], q[1][3], b[nb].z, b[nb].w);   // columns 2,6 | 3,7
             }
           }
         }
