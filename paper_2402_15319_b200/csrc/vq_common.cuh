@@ -29,7 +29,7 @@ struct LayerPtrs {
 
 // Workspace of the persistent kernel (vq_stream.cu): one ticket counter per 16 rows at most, and
 // two slabs (at most 256 rows each) of fp32 partial sums per persistent CTA.
-constexpr int kMaxStreamCtas = 320;
+constexpr int kMaxStreamCtas = 448;
 constexpr int kMaxSlabRows = 256;
 // Layers of one grouped call (they share the activations).
 constexpr int kMaxSegments = 4;

@@ -1,5 +1,5 @@
 // Uniform INT4 group-128 GEMV/skinny GEMM: the bandwidth yard-stick reported beside the VQ
-// kernels (paper Sec. 2.1 symmetric uniform quantiser; Sec. 5 "INT4 g128", 4.125 bits per value).
+// kernels (paper Sec. 2.1 symmetric uniform quantiser; Sec. 5: uniform 4-bit weights, one scale per 128 columns, 4.125 bits per value).
 #include "vq_common.cuh"
 
 namespace vq {

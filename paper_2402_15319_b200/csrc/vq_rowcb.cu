@@ -1,5 +1,5 @@
 // Tuned skinny-GEMM kernels for formats whose codebooks belong to ONE row (block_rows == 1) and
-// are indexed by 4-bit indices: the "mobile LUT" layouts (16-entry int8 codebook + fp16 scale per
+// are indexed by 4-bit indices: the layouts of the mobile LUT decode (16-entry int8 codebook + fp16 scale per
 // row segment) and the 16-entry fp16 2-D codebooks.
 //
 // Work decomposition.  A CTA owns WR tiles of 16 rows and a column range; warp (wr, wk) walks part
@@ -239,7 +239,7 @@ struct LdsTbl {
 
 // ---------------------------------------------------------------------------------------------
 // Int4G128: the uniform INT4 group-128 yard-stick run through the same skeleton (paper Sec. 2.1
-// symmetric uniform quantiser x ~ s*x_int; Sec. 5 "INT4 g128").  No table: a nibble q becomes the
+// symmetric uniform quantiser x ~ s*x_int; Sec. 5: uniform 4-bit weights with a scale per 128 columns).  No table: a nibble q becomes the
 // fp16 value q - 8 by the exponent trick, (1024 + q) - 1032; a "block" is one 128-column group whose
 // fp16 scale multiplies the group's fp32 partial sum.  The two nibbles that share a mask
 // (columns c and c+4 of an 8-column word) land in one fp16 pair, so the activations are staged in

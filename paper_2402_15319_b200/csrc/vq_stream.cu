@@ -74,8 +74,11 @@ struct StreamArgs {
   int cpb_shift;         // row policies: log2 of the chunks that share one codebook block
   int br_shift;          // log2 of the rows that share one codebook block
   int sr_shift;          // log2 of the rows of a slab (16*WR)
-  // byte offsets from the 4096-byte aligned start of dynamic shared memory
+  // byte offsets from the tables' boundary (the first BASE_ALIGN boundary that leaves front_bytes of
+  // dynamic shared memory in front of it): the slab hand-over buffers and the barriers lie in front
+  // (negative offsets), tables and stages behind
   int red_off, bar_off, stage_off;
+  int front_bytes, after_bytes;
   int stage_bytes;       // a stage: WK index boxes, then WK activation boxes
   int x_off;             // activations inside a stage
   int idx_part_bytes, x_part_bytes;
@@ -806,20 +809,29 @@ struct BlkD2B6 {
 // (one thread), warp W+1 writes the results.  CW = the most consumer warps a launch may use (4: two
 // CTAs per SM, 8: one), which fixes the registers a thread may take.
 // =============================================================================================
-template <class P, int NB, int R, int CW>
-__global__ void __launch_bounds__((CW + 3) * 32, CW <= 4 ? 2 : 1)
+// CPS = CTAs per SM the kernel is compiled for (it bounds the registers of a thread).
+template <class P, int NB, int R, int CW, int CPS>
+__global__ void __launch_bounds__((CW + (P::STAGE_TABLE_BYTES ? 3 : 2)) * 32, CPS)
 stream_kernel(const __grid_constant__ Maps maps, const StreamArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  const uint32_t sbase = (smem_u32(smem_raw) + (P::BASE_ALIGN - 1)) & ~static_cast<uint32_t>(P::BASE_ALIGN - 1);
+  const uint32_t sbase = (smem_u32(smem_raw) + a.front_bytes + (P::BASE_ALIGN - 1)) & ~static_cast<uint32_t>(P::BASE_ALIGN - 1);
   unsigned char* smem = smem_raw + (sbase - smem_u32(smem_raw));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  {   // the host sized the launch for dynamic shared memory that starts 1024 bytes into the CTA's window
+    uint32_t dyn;
+    asm("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn));
+    if (sbase - smem_u32(smem_raw) + static_cast<uint32_t>(a.after_bytes) > dyn) {   // (the same for every thread)
+      if (tid == 0) atomicAdd(a.error_flag, 1);
+      return;
+    }
+  }
   const int W = a.WR * a.WK;
   const int D = a.D;
   // barriers: full[D], empty[D] (pipeline stages); out_full[2], out_empty[2] (results of a slab)
   const uint32_t full0 = sbase + a.bar_off, empty0 = full0 + 8 * D;
   const uint32_t out_full0 = empty0 + 8 * D, out_empty0 = out_full0 + 16;
   constexpr int NBT = 8 * NB;
-  const int red_floats = W * R * 16 * NBT;   // one buffer of the slab's partial sums: [wk][16*R*WR rows][NBT]
+  const int red_floats = W * R * 16 * a.batch;   // one buffer of the slab's partial sums: [wk][16*R*WR rows][batch]
 
   if (tid == 0) {
     for (int i = 0; i < D; ++i) {
@@ -950,7 +962,7 @@ stream_kernel(const __grid_constant__ Maps maps, const StreamArgs a) {
         for (int o = lane; o < n_out; o += 32) {
           const int n = o >> a.sr_shift, rr = o & (slab_rows - 1);
           float sum = 0.f;
-          for (int p = 0; p < a.WK; ++p) sum += red[(p * slab_rows + rr) * NBT + n];
+          for (int p = 0; p < a.WK; ++p) sum += red[(p * slab_rows + rr) * a.batch + n];
           if (complete) {
             if (srow0 + rr < sg.N) sg.Y[static_cast<long long>(n) * sg.N + srow0 + rr] = __float2half_rn(sum);
           } else {
@@ -1109,14 +1121,15 @@ stream_kernel(const __grid_constant__ Maps maps, const StreamArgs a) {
       }
       dead = __any_sync(0xffffffffu, dead);
       // total[r][nb][e]: row 16r + g + 8*(e/2) of the warp's rows, batch row nb*8 + 2t + (e&1)
-      float* mine = reinterpret_cast<float*>(smem + a.red_off) + buf * red_floats + ((wk * a.WR + wr) * (16 * R) + g) * NBT + 2 * t;
+      // (only batch rows that exist are kept)
+      float* mine = reinterpret_cast<float*>(smem + a.red_off) + buf * red_floats + ((wk * a.WR + wr) * (16 * R) + g) * a.batch + 2 * t;
 #pragma unroll
       for (int r = 0; r < R; ++r)
 #pragma unroll
         for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            mine[(r * 16 + (e >> 1) * 8) * NBT + nb * 8 + (e & 1)] = total[r][nb][e];
+            if (nb * 8 + 2 * t + (e & 1) < a.batch) mine[(r * 16 + (e >> 1) * 8) * a.batch + nb * 8 + (e & 1)] = total[r][nb][e];
             total[r][nb][e] = 0.f;
           }
       __syncwarp();
@@ -1143,9 +1156,9 @@ size_t round_up(size_t v, size_t al) { return (v + al - 1) / al * al; }
 
 constexpr size_t kSmemMax = 224 * 1024;
 
-template <class P, int NB, int R, int CW>
+template <class P, int NB, int R, int CW, int CPS>
 vq_status launch(const StreamCall& call, int chunks_per_block, cudaStream_t s, int want_wk, int min_depth) {
-  auto kern = stream_kernel<P, NB, R, CW>;
+  auto kern = stream_kernel<P, NB, R, CW, CPS>;
   static int attr_set[kMaxDevices] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VQ_ERR_CUDA;
@@ -1177,7 +1190,7 @@ vq_status launch(const StreamCall& call, int chunks_per_block, cudaStream_t s, i
 
   // ---- CTA shape: W = WR row tiles x WK column parts (WK divides the chunks of a row); D stages ----
   int W = CW;
-  int ctas_per_sm = env_int("VQ_CTAS", CW <= 4 ? 2 : 1);
+  int ctas_per_sm = CPS;
   int WK = n_chunks % 4 == 0 ? 4 : n_chunks % 2 == 0 ? 2 : 1;
   if (P::STAGE_TABLE_BYTES) {   // shared tables: as many row tiles of the block as the CTA has warps, then column parts
     const int tiles = g.Br / (16 * R);
@@ -1211,33 +1224,45 @@ vq_status launch(const StreamCall& call, int chunks_per_block, cudaStream_t s, i
     return VQ_ERR_UNSUPPORTED;
 
   const size_t tbl_bytes = static_cast<size_t>(P::TILE_TABLE_BYTES) * R * W;
-  const size_t red_bytes = 2 * static_cast<size_t>(W) * R * 16 * 8 * NB * sizeof(float);   // two buffers
+  const size_t red_bytes = round_up(2 * static_cast<size_t>(W) * R * 16 * batch * sizeof(float), 16);   // two buffers
   const size_t idx_part = static_cast<size_t>(slab_rows) * P::CHUNK_BYTES;       // multiple of 512
   const size_t x_part = static_cast<size_t>(P::X_ROWS) * batch * P::X_ROW_BYTES;
   const size_t x_off = round_up(idx_part * WK, 1024);
   const size_t tbl_off = round_up(x_off + x_part * WK, P::STAGE_TABLE_BYTES ? P::STAGE_TABLE_BYTES : 1024);
   const size_t stage_bytes = round_up(tbl_off + static_cast<size_t>(P::STAGE_TABLE_BYTES) * WK, P::STAGE_TABLE_BYTES ? P::STAGE_TABLE_BYTES : 1024);
-  const size_t red_off = tbl_bytes;
-  const size_t bar_off = round_up(red_off + red_bytes, 16);
-  const size_t stage_off = round_up(bar_off + 16 * 16 + 32, P::STAGE_TABLE_BYTES ? P::STAGE_TABLE_BYTES : 1024);
-  // shared memory of a CTA: the SM's 227 KB minus 1 KB per resident CTA, shared by the resident CTAs
-  size_t budget = (227 * 1024 - 1024 * ctas_per_sm) / ctas_per_sm;
+  // In front of the tables: the slab hand-over buffers and the barriers.  Dynamic shared memory starts
+  // 1024 bytes into the CTA's window (the first 1024 are the system's; the kernel checks what it gets), so
+  // the tables' boundary lies `lead` bytes in and the front region fills bytes that alignment would waste.
+  const size_t front = round_up(red_bytes + 16 * 16 + 32, 16);
+  const size_t lead = round_up(1024 + front, P::BASE_ALIGN) - 1024;
+  const size_t stage_off = round_up(tbl_bytes, P::STAGE_TABLE_BYTES ? P::STAGE_TABLE_BYTES : 1024);
+  // shared memory of a CTA: the SM's 228 KB shared by the resident CTAs, 1 KB of each for the system
+  size_t budget = (228 * 1024) / ctas_per_sm - 1024;
   if (budget > kSmemMax) budget = kSmemMax;
-  if (budget < stage_off + P::BASE_ALIGN + static_cast<size_t>(min_depth) * stage_bytes) {   // does not fit twice
+  const size_t kSlack = lead;
+  if (budget < stage_off + kSlack + static_cast<size_t>(min_depth) * stage_bytes) {   // does not fit CPS times
     if (CW <= 4) return VQ_ERR_UNSUPPORTED;   // (a 4-warp CTA alone on an SM would leave it half empty)
     ctas_per_sm = 1;
     budget = kSmemMax;
   }
-  if (budget < stage_off + P::BASE_ALIGN + 2 * stage_bytes) return VQ_ERR_UNSUPPORTED;
-  int D = static_cast<int>((budget - P::BASE_ALIGN - stage_off) / stage_bytes);
+  if (budget < stage_off + kSlack + 2 * stage_bytes) return VQ_ERR_UNSUPPORTED;
+  int D = static_cast<int>((budget - kSlack - stage_off) / stage_bytes);
   if (D > 8) D = 8;
   D = env_int("VQ_D", D);
   if (D < min_depth || D > 16) return VQ_ERR_UNSUPPORTED;
-  const size_t smem_bytes = stage_off + static_cast<size_t>(D) * stage_bytes + P::BASE_ALIGN;
+  const size_t smem_bytes = stage_off + static_cast<size_t>(D) * stage_bytes + kSlack;
   if (smem_bytes > kSmemMax) return VQ_ERR_UNSUPPORTED;
   a.D = D;
-  a.red_off = static_cast<int>(red_off);
-  a.bar_off = static_cast<int>(bar_off);
+  a.front_bytes = static_cast<int>(front);
+  a.after_bytes = static_cast<int>(stage_off + static_cast<size_t>(D) * stage_bytes);
+  a.red_off = -static_cast<int>(front);
+  a.bar_off = -static_cast<int>(front) + static_cast<int>(red_bytes);
+  if (CPS > 2) {   // three CTAs per SM only if the device agrees that they fit
+    int resident = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kern, (W + (P::STAGE_TABLE_BYTES ? 3 : 2)) * 32, smem_bytes) != cudaSuccess)
+      return VQ_ERR_CUDA;
+    if (resident < CPS) return VQ_ERR_UNSUPPORTED;
+  }
   a.stage_off = static_cast<int>(stage_off);
   a.stage_bytes = static_cast<int>(stage_bytes);
   a.x_off = static_cast<int>(x_off);
@@ -1319,6 +1344,10 @@ vq_status launch(const StreamCall& call, int chunks_per_block, cudaStream_t s, i
   }
   cfg.attrs = attr;
   cfg.numAttrs = na;
+#ifdef VQ_TUNING
+  if (env_int("VQ_VERBOSE", 0))
+    fprintf(stderr, "stream launch: CPS %d grid %d block %d depth %d smem %zu WR %d WK %d R %d\n", CPS, Pn, (int)cfg.blockDim.x, D, smem_bytes, WR, WK, R);
+#endif
   const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, maps, a);
   if (e != cudaSuccess) {
 #ifdef VQ_TUNING
@@ -1345,17 +1374,32 @@ vq_status launch_tiles(const StreamCall& call, int chunks_per_block, cudaStream_
   // can start beside one of this kernel) with as many column parts as fit, then one 8-warp CTA;
   // first with at least three pipeline stages, then with two.
   static const int kShapes[][2] = {{4, 4}, {4, 2}, {8, 4}, {8, 2}, {4, 1}, {8, 1}};
+  // Three 4-warp CTAs per SM (12 consumer warps, two pipeline stages) where a CTA still gets eight
+  // stages or more: measured on B200 at batch 1, 28672 x 8192 26.7 against 27.9 us with two CTAs per
+  // SM, but 8192 x 8192 12.4 against 9.9 us (2.3 stages per CTA: all start-up and workspace reduction).
+  if constexpr (NB == 1 && P::STAGE_TABLE_BYTES == 0) {
+    int sms = 0;
+    if (device_sms(&sms) != VQ_OK) return VQ_ERR_CUDA;
+    const long long stages = rows * static_cast<long long>(call.g.stride / P::CHUNK_BYTES) / (16 * R * 4);
+    // (and where every CTA gets whole slabs: with fewer slabs than CTAs every output goes through the
+    // workspace, 8192 x 28672: 34.1 against 30.3 us)
+    if (stages >= 8LL * 3 * sms && rows / (16 * R) >= 3LL * sms && env_int("VQ_CTAS", 3) == 3 && (only_w == 0 || only_w == 4))
+      for (int wk = 4; wk >= 2; wk /= 2) {
+        const vq_status st = R == 2 ? launch<P, 1, 2, 4, 3>(call, chunks_per_block, s, wk, 2) : launch<P, 1, 1, 4, 3>(call, chunks_per_block, s, wk, 2);
+        if (st != VQ_ERR_UNSUPPORTED) return st;
+      }
+  }
   for (int min_depth = 3; min_depth >= 2; --min_depth)
     for (const auto& sh : kShapes) {
       const int cw = sh[0], wk = sh[1];
       if (only_w && cw != only_w) continue;
       vq_status st;
       if (cw == 8) {
-        st = (NB == 1 && R == 2) ? launch<P, NB, 2, 8>(call, chunks_per_block, s, wk, min_depth)
-                                 : launch<P, NB, 1, 8>(call, chunks_per_block, s, wk, min_depth);
+        st = (NB == 1 && R == 2) ? launch<P, NB, 2, 8, 1>(call, chunks_per_block, s, wk, min_depth)
+                                 : launch<P, NB, 1, 8, 1>(call, chunks_per_block, s, wk, min_depth);
       } else {
-        st = (NB == 1 && R == 2) ? launch<P, NB, 2, 4>(call, chunks_per_block, s, wk, min_depth)
-                                 : launch<P, NB, 1, 4>(call, chunks_per_block, s, wk, min_depth);
+        st = (NB == 1 && R == 2) ? launch<P, NB, 2, 4, 2>(call, chunks_per_block, s, wk, min_depth)
+                                 : launch<P, NB, 1, 4, 2>(call, chunks_per_block, s, wk, min_depth);
       }
       if (st != VQ_ERR_UNSUPPORTED) return st;
     }

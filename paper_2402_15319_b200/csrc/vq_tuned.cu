@@ -114,12 +114,12 @@ vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half*
   if (path == 2) ws = nullptr;
 #endif
   // Which family serves a single layer (measured on B200, both families on every benchmark shape at
-  // batch 1 / 4 / 16): the persistent kernel wins on the large per-row 4-bit 2-D layers (28672 x 8192:
-  // 30.6 against 37.8 us at batch 1, 68.6 against 77.6 us at batch 16; 8192 x 8192: 10.8 against 11.0 us
-  // and 22.9 against 26.2 us); short rows of few slabs, long rows (28672 columns), batch 3-8 and the
-  // shared-codebook formats are faster in the cluster kernels, whose K-split meets in distributed
-  // shared memory instead of the workspace.
-  bool stream_first = g.b == 4 && g.d == 2 && g.N >= 8192 && g.stride <= 2048 && (batch <= 2 || batch > 8);
+  // batch 1 / 4 / 16): the persistent kernel wins on the per-row 4-bit 2-D layers of 8192 rows or more
+  // (28672 x 8192: 26.7 against 37.8 us at batch 1, 66.5 against 77.6 us at batch 16; 8192 x 8192: 9.9
+  // against 11.0 us and 22.9 against 26.2 us; 8192 x 28672: 30.3 against 32.5 us and 72.2 against 76.7 us);
+  // short layers of few slabs, batch 3-8 and the shared-codebook formats are faster in the cluster
+  // kernels, whose K-split meets in distributed shared memory instead of the workspace.
+  bool stream_first = g.b == 4 && g.d == 2 && g.N >= 8192 && (batch <= 2 || batch > 8);
 #ifdef VQ_TUNING
   if (path == 1) stream_first = true;
 #endif
