@@ -180,13 +180,13 @@ vq_status vq_gemm_small_batch_impl(const vq_format* fmt, const void* d_idx, cons
 
 // Which kernel family serves a group in one launch: 2 = the cluster kernels of the shared-codebook
 // formats (their K-split meets in distributed shared memory: lowest latency on the small layers those
-// formats come with), 1 = the persistent kernel (per-row formats at batch 1-2 and 9-16, where one launch
-// beat the members' separate launches: q/k/v of the 70B-shaped set 12.9 us against 19.5 us at batch 1,
-// a tie at batch 4), 0 = member by member.
-static int group_family(const Geometry& g, int batch) {
+// formats come with), 1 = the persistent kernel (per-row formats: q/k/v of the 70B-shaped set in one
+// launch 11.4 us against 19.5 us for three launches at batch 1, 20.3 against 37.4 us at batch 8),
+// 0 = member by member.
+static int group_family(const Geometry& g, int) {
   if (g.cb_int4) return 0;
   if (blockcb_covers(g)) return 2;
-  return (batch <= 2 || batch > 8) ? 1 : 0;
+  return 1;
 }
 
 int vq_grouped_kernel_launches(const vq_format* fmt, int n_members, int batch) {
@@ -239,7 +239,7 @@ vq_status vq_gemm_small_batch_grouped(const vq_format* fmt, const vq_group_membe
     if (getenv("VQ_GROUP_FAMILY")) fam = atoi(getenv("VQ_GROUP_FAMILY"));
 #endif
     if (fam == 2) st = launch_gemm_blockcb_group(call, s);
-    if (fam == 1 || (fam == 2 && st == VQ_ERR_UNSUPPORTED && (batch <= 2 || batch > 8))) st = launch_gemm_stream(call, s);
+    if (fam == 1 || (fam == 2 && st == VQ_ERR_UNSUPPORTED)) st = launch_gemm_stream(call, s);
   }
   if (st != VQ_ERR_UNSUPPORTED) return st;
   for (int i = 0; i < n_members; ++i) {   // formats the persistent kernel does not take: member by member

@@ -117,9 +117,10 @@ vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half*
   // batch 1 / 4 / 16): the persistent kernel wins on the per-row 4-bit 2-D layers of 8192 rows or more
   // (28672 x 8192: 26.7 against 37.8 us at batch 1, 66.5 against 77.6 us at batch 16; 8192 x 8192: 9.9
   // against 11.0 us and 22.9 against 26.2 us; 8192 x 28672: 30.3 against 32.5 us and 72.2 against 76.7 us);
-  // short layers of few slabs, batch 3-8 and the shared-codebook formats are faster in the cluster
+  // at batch 8: 34.7 against 52.5, 13.8 against 17.8, 35.2 against 54.3 us); short layers of few slabs
+  // (1024 x 8192: 6.8 against 5.2 us at batch 3) and the shared-codebook formats are faster in the cluster
   // kernels, whose K-split meets in distributed shared memory instead of the workspace.
-  bool stream_first = g.b == 4 && g.d == 2 && g.N >= 8192 && (batch <= 2 || batch > 8);
+  bool stream_first = g.b == 4 && g.d == 2 && g.N >= 8192;
 #ifdef VQ_TUNING
   if (path == 1) stream_first = true;
 #endif
