@@ -164,3 +164,42 @@ def test_pack_info_int4_codebook_with_group_scales():
         vq.vq_pack_info(vq.VQFormat(256, 1024 + 64, 2, 3, 32, 32, vq.VQ_CB_INT4_G128))
     assert e.value.code == 3
 
+
+
+def test_grouped_call_argument_errors_and_launch_counts():
+    """vq_gemm_small_batch_grouped validates on the host (member pointers, row sums, workspace) before
+    any launch, and vq_grouped_kernel_launches tells one kernel for the formats a kernel family takes
+    as a group (per-row 4-bit formats, shared-codebook formats), n_members for the rest."""
+    from paper_2402_15319_b200.binding import _CGroupMember
+    lib = vq.load()
+    total = _replace(GOOD, n_rows=16)
+    c = total.c()
+
+    def call(members, n=None, X=FAKE, batch=1, ws=FAKE, ws_bytes=1 << 30, fmt=c):
+        arr = (_CGroupMember * max(1, len(members)))()
+        for i, m in enumerate(members):
+            arr[i] = _CGroupMember(*m)
+        return lib.vq_gemm_small_batch_grouped(ctypes.byref(fmt), arr, len(members) if n is None else n, X, batch, ws, ws_bytes, None)
+
+    two = [(FAKE, FAKE, None, FAKE, 8), (FAKE, FAKE, None, FAKE, 8)]
+    assert lib.vq_gemm_small_batch_grouped(ctypes.byref(c), None, 2, FAKE, 1, FAKE, 1 << 30, None) == 1
+    assert call(two, n=0) == 3 and call(two, n=5) == 3                     # 1..VQ_MAX_GROUP members
+    assert call(two, batch=0) == 6 and call(two, batch=17) == 6
+    assert call(two, X=None) == 1 and call(two, X=ODD) == 4
+    assert call(two, ws=None) == 5 and call(two, ws_bytes=16) == 5 and call(two, ws=ODD) == 4
+    assert call([(FAKE, FAKE, None, None, 8), two[1]]) == 1                # member without an output
+    assert call([(FAKE, FAKE, None, ODD, 8), two[1]]) == 4
+    assert call([(None, FAKE, None, FAKE, 8), two[1]]) == 1
+    assert call([(FAKE, FAKE, FAKE, FAKE, 8), two[1]]) == 1                # fp16 codebook must not carry a scale
+    assert call([(FAKE, FAKE, None, FAKE, 8), (FAKE, FAKE, None, FAKE, 4)]) == 3   # rows do not add up to fmt.n_rows
+    # launch counts (host only)
+    row4 = vq.VQFormat(10240, 8192, 2, 4, 1, 2048, vq.VQ_CB_INT8_SCALED)
+    blk6 = vq.VQFormat(12288, 4096, 2, 6, 128, 128, vq.VQ_CB_FP16)
+    odd5 = vq.VQFormat(42, 312, 1, 5, 1, 156, vq.VQ_CB_FP16)
+    for batch in (1, 4, 16):
+        assert vq.vq_grouped_kernel_launches(row4, 3, batch) == 1
+        assert vq.vq_grouped_kernel_launches(blk6, 3, batch) == 1
+        assert vq.vq_grouped_kernel_launches(odd5, 2, batch) == 2
+        assert vq.vq_grouped_kernel_launches(row4, 1, batch) == 1
+    assert vq.vq_grouped_kernel_launches(row4, 0, 1) == 0 and vq.vq_grouped_kernel_launches(row4, 5, 1) == 0
+    assert vq.vq_grouped_kernel_launches(row4, 2, 17) == 0
