@@ -11,6 +11,7 @@ beyond the fixed size are refused before anything is launched.
 The file name sorts last on purpose: a run that stops at the first failure has then already run
 every other test."""
 import ctypes
+import gc
 
 import numpy as np
 import pytest
@@ -70,7 +71,10 @@ def test_static_scratch_variant_matches_workspace_variant_twice(spec):
         assert (np.abs(got - want) <= TOL * A).all(), f"{spec.name} call {call}: differs from the workspace variant"
         assert (np.abs(got - Y) <= TOL * A).all(), f"{spec.name} call {call}: differs from the oracle"
         # a further call allocates nothing: neither the driver's free memory nor torch's pool moves
+        # (garbage of earlier tests is collected first, so that nothing but this call can move the numbers)
+        gc.collect()
+        torch.cuda.synchronize()
         free0, alloc0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
         vq.vq_gemm_small_batch_host_static(dev.fmt, dev.idx, dev.cb, dev.scale, hX, hY, batch)
         torch.cuda.synchronize()
-        assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == alloc0
+        assert torch.cuda.mem_get_info()[0] >= free0 and torch.cuda.memory_allocated() <= alloc0
