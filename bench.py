@@ -46,8 +46,12 @@ def measured_peaks():
 def layer_bytes(spec: vq_synth.LayerSpec, stride: int, batch: int) -> int:
     """Algorithmic bytes of one layer call: everything stored for W plus activations and outputs."""
     idx = spec.N * stride
-    cb = spec.n_blocks * spec.entries * spec.d * (1 if spec.int8 else 2)
-    sc = spec.n_blocks * 2 if spec.int8 else 0
+    if int(spec.int8) == 2:   # int4 codebooks: two entries' values per byte, one fp16 scale per row and 128 columns
+        cb = spec.n_blocks * spec.entries * spec.d // 2
+        sc = spec.N * (spec.K // 128) * 2
+    else:
+        cb = spec.n_blocks * spec.entries * spec.d * (1 if spec.int8 else 2)
+        sc = spec.n_blocks * 2 if spec.int8 else 0
     return idx + cb + sc + 2 * batch * (spec.K + spec.N)
 
 
@@ -396,9 +400,10 @@ def dram_traffic_note(cfg_name: str):
 
 
 KERNEL_OF = {"cfg1": "rowcb_kernel<LdsTbl<false>,1>", "cfg2": "rowcb_kernel<PrmtI8,1>",
-             "cfg3": "blockcb_kernel<2,6,1> / stream_kernel<BlkD2B6> (groups)",
-             "cfg4": "blockcb_kernel<4,8,NB>", "cfg5": "stream_kernel<RowD2B4<int8>,NB,R,4> (groups, 8192-column layers) / rowcb_kernel<LdsTbl<true>,NB>",
-             "llama3_8b": "blockcb_kernel<2,6,NB,warp-private tables> / stream_kernel<BlkD2B6> (groups)"}
+             "cfg3": "blockcb_kernel<2,6,1> (q/k/v and gate/up as grouped launches)",
+             "cfg4": "blockcb_kernel<4,8,NB>", "cfg5": "stream_kernel<RowD2B4<int8>,NB,R,CW,CPS>",
+             "llama3_8b": "blockcb_kernel<2,6,NB,warp-private tables>",
+             "llama3_8b_int4cb": "blockcb_kernel<2,6,NB,warp-private tables, int4 codebooks>"}
 
 
 def max_over_ranks(value: float, dist=None, device=None) -> float:
@@ -702,7 +707,7 @@ def run_ours(args):
         "config": {
             "workload": f"{args.config}: {sp0.name.split('.')[0]} layer set ({len(ds.specs)} layers, "
                         f"{ds.n_weights} weights), d={sp0.d}, {sp0.b}-bit indices, "
-                        f"{'int8+scale' if sp0.int8 else 'fp16'} codebook per {sp0.Br}x{sp0.Bc} block, batch {args.batch}",
+                        f"{'int4 (+scale per row and 128 columns)' if int(sp0.int8) == 2 else 'int8+scale' if sp0.int8 else 'fp16'} codebook per {sp0.Br}x{sp0.Bc} block, batch {args.batch}",
             "calls_per_step": ds.call_names(),
             "grouping": "q/k/v and gate/up read one activation tensor each (the first member's) through vq_gemm_small_batch_grouped; "
                         "that tensor is counted once in bytes_per_step",

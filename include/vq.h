@@ -76,8 +76,11 @@ typedef enum {
  *   d_cb    : per block 2^index_bits * vq_dim signed 4-bit integers (-8..7), two per byte, value
  *             v = entry * vq_dim + t in nibble v mod 2 (low nibble first) of byte v / 2;
  *   d_scale : binary16 [N][K/128]; w[n][k] = scale[n][k/128] * c.  K % 128 == 0.
- * vq_decode_weights decodes it with its tile kernel; the skinny GEMM runs in the format-generic
- * kernel (VQ_IMPL_TUNED returns VQ_ERR_UNSUPPORTED); vq_assign_indices does not take it. */
+ * vq_decode_weights decodes it with its tile kernel; the skinny GEMM runs in the tuned shared-codebook
+ * kernels for 2-D formats with 5- or 6-bit indices (blocks of 32, 64 or a multiple of 128 rows and a
+ * multiple of 128 columns, K a multiple of 256), where a looked-up pair is fp16(scale * c), the value
+ * vq_decode_weights writes; other formats of this codebook type run in the format-generic kernel
+ * (VQ_IMPL_TUNED returns VQ_ERR_UNSUPPORTED for them); vq_assign_indices does not take it. */
 typedef enum {
   VQ_CB_FP16 = 0,         /* binary16 entries                                                        */
   VQ_CB_INT8_SCALED = 1,  /* signed 8-bit entries, one binary16 scale per block                       */

@@ -56,6 +56,7 @@ constexpr int kWaitTries = 1 << 18;   // mbarrier polls before a warp gives up a
 struct BlockArgs {
   const void* cb;
   const __half* scale;   // one per block for int8 codebooks, else null
+  const __half* gscale;  // int4 codebooks (Sec. 4.2): one per row and group of 128 columns, [N][K/128]; else null
   const __half* X;
   __half* Y;
   int* error_flag;       // device counter of waits that ran out
@@ -175,12 +176,29 @@ __device__ __forceinline__ void gather_steps(uint32_t (&a)[NSTEPS][4], const uin
 
 // Both 16-row tiles of a warp for NSTEPS steps: their accumulator chains are independent, so the
 // look-ups are issued together and the mmas alternate.
-template <int D, int B, int NB, int STEP0, int NSTEPS>
+// I4 (int4 codebooks): the table holds the signed 4-bit entries as fp16; sc[q] is the fp16 scale (twice)
+// of row 8q + g of the warp's rows for the lane's group of 128 columns, and every looked-up pair is
+// multiplied by it: fp16(scale * c), the value vq_decode_weights writes (one rounding of an exact product).
+__device__ __forceinline__ uint32_t mul_f16x2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+template <int D, int B, int NB, int STEP0, int NSTEPS, bool I4 = false>
 __device__ __forceinline__ void chunk_steps(float (&acc)[2][NB][4], const uint32_t (&w)[4][Policy<D, B>::LANE_WORDS],
-                                            const uint32_t (&xr)[NB][32], uint32_t tbl) {
+                                            const uint32_t (&xr)[NB][32], uint32_t tbl, const uint32_t (&sc)[4]) {
   uint32_t a0[NSTEPS][4], a1[NSTEPS][4];
   gather_steps<D, B, STEP0, NSTEPS>(a0, w[0], w[1], tbl);
   gather_steps<D, B, STEP0, NSTEPS>(a1, w[2], w[3], tbl);
+  if constexpr (I4) {
+#pragma unroll
+    for (int s = 0; s < NSTEPS; ++s) {
+      a0[s][0] = mul_f16x2(a0[s][0], sc[0]); a0[s][1] = mul_f16x2(a0[s][1], sc[1]);
+      a0[s][2] = mul_f16x2(a0[s][2], sc[0]); a0[s][3] = mul_f16x2(a0[s][3], sc[1]);
+      a1[s][0] = mul_f16x2(a1[s][0], sc[2]); a1[s][1] = mul_f16x2(a1[s][1], sc[3]);
+      a1[s][2] = mul_f16x2(a1[s][2], sc[2]); a1[s][3] = mul_f16x2(a1[s][3], sc[3]);
+    }
+  }
 #pragma unroll
   for (int s = 0; s < NSTEPS; ++s)
 #pragma unroll
@@ -218,7 +236,10 @@ __device__ __forceinline__ uint2 fetch_entry(const BlockArgs& a, long long blk_r
     const int e = tid % P::ENTRIES, h = tid / P::ENTRIES;
     if (h >= 2) return v;
     const long long blk = blk_row + (chunk * 256 + h * 128) / a.Bc;
-    if (a.scale == nullptr) {
+    if (a.gscale != nullptr) {   // int4 entries: one byte per 2-D entry, low nibble = first value; exact in fp16
+      const uint32_t byte = __ldg(static_cast<const uint8_t*>(a.cb) + blk * P::ENTRIES + e);
+      v.x = pair(1.f, (static_cast<int>(byte & 15u) ^ 8) - 8, (static_cast<int>(byte >> 4) ^ 8) - 8);
+    } else if (a.scale == nullptr) {
       v.x = __ldg(static_cast<const uint32_t*>(a.cb) + blk * P::ENTRIES + e);
     } else {
       const uint16_t raw = __ldg(static_cast<const uint16_t*>(a.cb) + blk * P::ENTRIES + e);
@@ -280,7 +301,12 @@ __device__ __forceinline__ void load_private(PrivateRegs<B>& r, const BlockArgs&
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     const long long blk = blk_row + (chunk * 256 + h * 128) / a.Bc;
-    if (a.scale == nullptr) {
+    if (a.gscale != nullptr) {   // int4 entries: EPL bytes
+      const uint8_t* src = static_cast<const uint8_t*>(a.cb) + blk * E + lane * EPL;
+      if constexpr (EPL == 2) r.raw[h][0] = __ldg(reinterpret_cast<const uint16_t*>(src));
+      else r.raw[h][0] = __ldg(src);
+      r.scale[h] = 1.f;
+    } else if (a.scale == nullptr) {
       const uint32_t* src = static_cast<const uint32_t*>(a.cb) + blk * E + lane * EPL;
       if constexpr (EPL == 2) {
         const uint2 q = ldg64_nc(src);
@@ -299,15 +325,19 @@ __device__ __forceinline__ void load_private(PrivateRegs<B>& r, const BlockArgs&
   }
 }
 template <int B>
-__device__ __forceinline__ void write_private(uint32_t table, const PrivateRegs<B>& r, bool int8, int lane) {
+__device__ __forceinline__ void write_private(uint32_t table, const PrivateRegs<B>& r, int mode, int lane) {   // mode 0 fp16, 1 int8, 2 int4
   constexpr int EPL = PrivateRegs<B>::EPL;
 #pragma unroll
   for (int i = 0; i < EPL; ++i) {
     uint32_t e[2];
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      if (!int8) {
+      if (mode == 0) {
         e[h] = r.raw[h][i];
+      } else if (mode == 2) {
+        const uint32_t byte = (r.raw[h][0] >> (8 * i)) & 0xffu;
+        const __half2 hv = __halves2half2(__int2half_rn((static_cast<int>(byte & 15u) ^ 8) - 8), __int2half_rn((static_cast<int>(byte >> 4) ^ 8) - 8));
+        e[h] = *reinterpret_cast<const uint32_t*>(&hv);
       } else {
         const uint32_t two = r.raw[h][0] >> (16 * i);
         const __half2 hv = __halves2half2(__float2half_rn(r.scale[h] * static_cast<float>(static_cast<int8_t>(two & 0xff))),
@@ -326,10 +356,13 @@ __device__ __forceinline__ void write_private(uint32_t table, const PrivateRegs<
 // boundary: two tables, two compact codebooks, the warps' index rings, their barriers, the
 // activations, the receive buffer of the reduction.
 // PRIV: every warp keeps its own pair of tables (block rows a multiple of 32, 2-D only).
-template <int D, int B, int NB, bool PRIV>
+// I4: int4 codebooks with a scale per row and group of 128 columns (2-D only; a lane's 64 columns of a
+// chunk lie inside one group).
+template <int D, int B, int NB, bool PRIV, bool I4>
 __global__ void __launch_bounds__(Tile<D, B>::THREADS)
 blockcb_kernel(const __grid_constant__ BlockMaps maps, const BlockArgs a_in, const BlockGroup grp) {
   static_assert(!PRIV || D == 2, "warp-private tables exist for 2-D codebooks only");
+  static_assert(!I4 || D == 2, "int4 codebooks are served for 2-D formats only");
   constexpr int ST = kStagesOf<D, PRIV>;   // ring stages per warp
   using P = Policy<D, B>;
   using T = Tile<D, B>;
@@ -349,7 +382,8 @@ blockcb_kernel(const __grid_constant__ BlockMaps maps, const BlockArgs a_in, con
     if (i < grp.n_seg && static_cast<int>(blockIdx.y) >= grp.tile0[i]) sgi = i;
   BlockArgs a = a_in;
   a.cb = grp.cb[sgi];
-  a.scale = grp.scale[sgi];
+  a.scale = I4 ? nullptr : grp.scale[sgi];
+  a.gscale = I4 ? grp.scale[sgi] : nullptr;
   a.Y = grp.Y[sgi];
   a.N = grp.N[sgi];
   const CUtensorMap* tm = &maps.m[sgi];
@@ -423,7 +457,7 @@ blockcb_kernel(const __grid_constant__ BlockMaps maps, const BlockArgs a_in, con
       }
     }
     if constexpr (PRIV) {
-      if (n > 0) write_private<B>(my_tables, mine, a.scale != nullptr, lane);
+      if (n > 0) write_private<B>(my_tables, mine, I4 ? 2 : a.scale != nullptr ? 1 : 0, lane);
       if (n > 1) load_private<B>(mine, a, blk_row, c0 + 1, lane);
     } else {
       if (nt > 0) store_compact<D, B>(compact, cb0, tid);
@@ -472,6 +506,18 @@ blockcb_kernel(const __grid_constant__ BlockMaps maps, const BlockArgs a_in, con
   const uint32_t xstride = a.batch * 64;
   const uint32_t lane_off = D == 2 ? lane * 4 : (lane & 15) * 8;
   const uint32_t row_off = t * (LW * 4) + g * P::SEG;
+  // int4 codebooks: the scales of the lane's four rows (8q + g of the warp's 32) for its group of 128
+  // columns (lanes t < 2: the chunk's first group, t >= 2: the second), requested one chunk ahead
+  uint32_t sc[4] = {0u, 0u, 0u, 0u}, sc_next[4] = {0u, 0u, 0u, 0u};
+  auto load_scales = [&](int chunk, uint32_t (&o)[4]) {
+    const unsigned short* base_sc = reinterpret_cast<const unsigned short*>(a.gscale) + chunk * 2 + (t >> 1);
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      o[q] = __ldg(base_sc + static_cast<long long>(row0 + 32 * warp + 8 * q + g) * (a.K / 128)) * 0x10001u;
+  };
+  if constexpr (I4) {
+    if (n > 0) load_scales(c0, sc_next);
+  }
 
   for (int i = 0; i < n; ++i) {
     const int c = c0 + i;
@@ -487,6 +533,11 @@ blockcb_kernel(const __grid_constant__ BlockMaps maps, const BlockArgs a_in, con
         replicate<D, B>(base + ((k + 1) & 1) * P::TABLE_BYTES, compact + ((k + 1) & 1) * P::COMPACT_BYTES, tid);
     }
 
+    if constexpr (I4) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) sc[q] = sc_next[q];
+      if (i + 1 < n) load_scales(c + 1, sc_next);
+    }
     // ---- this warp's indices of the chunk ----
     const int st = i % ST;
     if (!mbar_wait(bars + 8 * st, (i / ST) & 1, kWaitTries) && lane == 0) atomicAdd(a.error_flag, 1);
@@ -529,10 +580,10 @@ blockcb_kernel(const __grid_constant__ BlockMaps maps, const BlockArgs a_in, con
     uint32_t tbl = (my_tables + (PRIV || kTableBuffers<D> == 1 ? 0 : (k & 1) * P::TABLE_BYTES)) | lane_off;
     if constexpr (!PRIV && kTableBuffers<D> == 1) fence_value(tbl);
     if constexpr (PRIV) fence_value(tbl);   // the gathers stay behind the warp's own table writes
-    chunk_steps<D, B, NB, 0, 4>(acc, w, xr, tbl);
-    chunk_steps<D, B, NB, 4, 4>(acc, w, xr, tbl);
-    chunk_steps<D, B, NB, 8, 4>(acc, w, xr, tbl);
-    chunk_steps<D, B, NB, 12, 4>(acc, w, xr, tbl);
+    chunk_steps<D, B, NB, 0, 4, I4>(acc, w, xr, tbl, sc);
+    chunk_steps<D, B, NB, 4, 4, I4>(acc, w, xr, tbl, sc);
+    chunk_steps<D, B, NB, 8, 4, I4>(acc, w, xr, tbl, sc);
+    chunk_steps<D, B, NB, 12, 4, I4>(acc, w, xr, tbl, sc);
 
     if constexpr (PRIV) {
       // the warp's table for the next chunk replaces the one it has just finished with (only this
@@ -540,7 +591,7 @@ blockcb_kernel(const __grid_constant__ BlockMaps maps, const BlockArgs a_in, con
       if (i + 1 < n) {
         fence_acc(acc);   // this chunk's gathers are emitted before the writes
         __syncwarp();     // ... by every lane of the warp
-        write_private<B>(my_tables, mine, a.scale != nullptr, lane);
+        write_private<B>(my_tables, mine, I4 ? 2 : a.scale != nullptr ? 1 : 0, lane);
         if (i + 2 < n) load_private<B>(mine, a, blk_row, c + 2, lane);
         __syncwarp();
       }
@@ -621,14 +672,20 @@ vq_status launch(const StreamCall& call, cudaStream_t s) {
   const int batch = call.batch;
   using P = Policy<D, B>;
   using T = Tile<D, B>;
-  auto kern = blockcb_kernel<D, B, NB, PRIV>;
-  static int attr_set[kMaxDevices] = {};
+  auto kern = blockcb_kernel<D, B, NB, PRIV, false>;
+  if constexpr (D == 2) {
+    if (call.g.cb_int4) kern = blockcb_kernel<D, B, NB, PRIV, true>;
+  } else {
+    if (call.g.cb_int4) return VQ_ERR_UNSUPPORTED;
+  }
+  static int attr_set[kMaxDevices][2] = {};   // [device][fp16 / int8 kernel, int4 kernel]
+  const int which = call.g.cb_int4 ? 1 : 0;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VQ_ERR_CUDA;
   if (device_sms(&sms) != VQ_OK) return VQ_ERR_CUDA;
-  if (!__atomic_load_n(&attr_set[dev], __ATOMIC_ACQUIRE)) {
+  if (!__atomic_load_n(&attr_set[dev][which], __ATOMIC_ACQUIRE)) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess) return VQ_ERR_CUDA;
-    __atomic_store_n(&attr_set[dev], 1, __ATOMIC_RELEASE);
+    __atomic_store_n(&attr_set[dev][which], 1, __ATOMIC_RELEASE);
   }
   int* error_flag = nullptr;
   if (device_error_counter(&error_flag) != VQ_OK) return VQ_ERR_CUDA;
@@ -636,6 +693,7 @@ vq_status launch(const StreamCall& call, cudaStream_t s) {
   BlockArgs a;
   a.cb = nullptr;      // (per layer: the kernel takes them from the group)
   a.scale = nullptr;
+  a.gscale = nullptr;
   a.X = X;
   a.Y = nullptr;
   a.error_flag = error_flag;
@@ -653,7 +711,7 @@ vq_status launch(const StreamCall& call, cudaStream_t s) {
   for (int i = 0; i < call.n_seg; ++i) {
     if (call.N[i] <= 0 || call.N[i] % T::CTA_ROWS) return VQ_ERR_UNSUPPORTED;
     grp.cb[i] = call.cb[i];
-    grp.scale[i] = g.cb_int8 ? call.scale[i] : nullptr;
+    grp.scale[i] = (g.cb_int8 || g.cb_int4) ? call.scale[i] : nullptr;   // per block (int8) or per row and 128 columns (int4)
     grp.Y[i] = call.Y[i];
     grp.N[i] = call.N[i];
     grp.tile0[i] = row_blocks;
@@ -739,7 +797,8 @@ vq_status launch(const StreamCall& call, cudaStream_t s) {
 // a multiple of 128 (2-D) / 256 (4-D), K a multiple of the 256-column chunk.  One launch serves every
 // layer of the call (same format and K; rows per layer in call.N).
 bool blockcb_covers(const Geometry& g) {
-  if (g.cb_int4 || g.K % 256) return false;
+  if (g.K % 256) return false;
+  if (g.cb_int4 && g.d != 2) return false;   // int4 codebooks: the 2-D policies only
   if (g.d == 2 && (g.b == 6 || g.b == 5)) return g.Bc % 128 == 0 && (g.Br % 128 == 0 || (g.Br % 32 == 0 && 128 % g.Br == 0));
   if (g.d == 4 && g.b == 8) return g.Br % Tile<4, 8>::CTA_ROWS == 0 && g.Bc % 256 == 0;
   return false;

@@ -106,7 +106,7 @@ size_t stream_workspace_bytes(long long rows, int batch) {
 
 vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch, void* ws,
                             size_t ws_bytes, cudaStream_t s) {
-  if (g.cb_int4) return VQ_ERR_UNSUPPORTED;   // int4 codebooks: format-generic kernels only
+  if (g.cb_int4) return launch_gemm_blockcb(g, p, X, Y, batch, s);   // int4 codebooks: the 2-D shared-codebook kernels only
   vq_status st = VQ_ERR_UNSUPPORTED;
 #ifdef VQ_TUNING
   const char* path_env = getenv("VQ_PATH");

@@ -158,6 +158,7 @@ GROUPS = [
     (vq_synth.LayerSpec("g_blk", N=0, K=1024, d=2, b=6, Br=128, Bc=128, int8=False), [512, 128, 128, 256]),
     (vq_synth.LayerSpec("g_blk32", N=0, K=1024, d=2, b=6, Br=32, Bc=256, int8=True), [256, 128, 384]),
     (vq_synth.LayerSpec("g_d4b8", N=0, K=1024, d=4, b=8, Br=256, Bc=512, int8=False), [256, 512]),
+    (vq_synth.LayerSpec("g_i4cb", N=0, K=1024, d=2, b=6, Br=32, Bc=128, int8=2), [256, 128]),
     (vq_synth.LayerSpec("g_generic", N=0, K=312, d=1, b=5, Br=1, Bc=156, int8=False), [37, 5]),
 ]
 
@@ -195,7 +196,7 @@ def test_tall_block_kernel_extra_formats(spec):
     _check_layer(spec, seed=91, batches=(1, 3, 8, 16), impls=[vq.VQ_IMPL_TUNED, vq.VQ_IMPL_GENERIC], decode=True)
 
 
-@pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "llama3_8b"])
+@pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "llama3_8b", "llama3_8b_int4cb"])
 def test_tuned_kernels_cover_every_benchmark_format(cfg):
     """VQ_IMPL_TUNED never falls back: it must run (not VQ_ERR_UNSUPPORTED) on every layer shape of
     the five configurations, at every batch of the configuration (row count cut to two tiles)."""
@@ -337,7 +338,7 @@ def _decode_slab_check(spec, L, dev_W, block_row):
     assert np.array_equal(dev_W[r0:r0 + spec.Br].view(np.uint16), W16), f"{spec.name}: decode rows {r0}.."
 
 
-@pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "llama3_8b"])
+@pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "llama3_8b", "llama3_8b_int4cb"])
 def test_benchmark_configs_full_size(cfg):
     conf = vq_synth.CONFIGS[cfg]
     seen = set()
@@ -475,14 +476,31 @@ INT4_CODEBOOK_CASES = [
 @pytest.mark.parametrize("spec", INT4_CODEBOOK_CASES, ids=lambda s: s.name)
 def test_int4_codebooks_with_group_scales(spec):
     """INT4 codebooks decoded with a scale per row and group of 128 columns (Sec. 4.2): bit-exact
-    decode, mat-vec within the tolerance, through the format-generic kernels (the only ones that take
-    this codebook type: VQ_IMPL_TUNED must refuse it)."""
+    decode, mat-vec within the tolerance, through the format-generic kernels; VQ_IMPL_TUNED must refuse
+    these shapes (it takes this codebook type for the 2-D 5/6-bit tall-block formats only, tested below)."""
     _check_layer(spec, seed=55, batches=(1, 5, 16), impls=[vq.VQ_IMPL_GENERIC, vq.VQ_IMPL_AUTO])
     L = draw(spec, 55)
     dev = DeviceLayer(spec, L)
     with pytest.raises(vq.VQError) as err:
         dev.gemm(vq_synth.make_x(spec, 1, 1), vq.VQ_IMPL_TUNED)
     assert err.value.code == 7
+
+
+INT4_CODEBOOK_TUNED = [
+    # 2-D, 3 bits per dimension, blocks of 4096 weights: the setting of the paper's INT4-codebook table (Sec. 4.2)
+    vq_synth.LayerSpec("i4cb_tb_d2b6_32x128", N=256, K=1024, d=2, b=6, Br=32, Bc=128, int8=2),
+    vq_synth.LayerSpec("i4cb_tb_d2b6_128x128", N=384, K=2816, d=2, b=6, Br=128, Bc=128, int8=2),
+    vq_synth.LayerSpec("i4cb_tb_d2b5_64x256", N=128, K=1280, d=2, b=5, Br=64, Bc=256, int8=2),
+    vq_synth.LayerSpec("i4cb_tb_d2b5_256x128", N=256, K=768, d=2, b=5, Br=256, Bc=128, int8=2),
+]
+
+
+@pytest.mark.parametrize("spec", INT4_CODEBOOK_TUNED, ids=lambda s: s.name)
+def test_int4_codebooks_in_the_tall_block_kernel(spec):
+    """The tuned shared-codebook kernels with INT4 codebooks (Sec. 4.2): entries enter the look-up tables
+    as exact fp16 integers, every looked-up pair is multiplied by the fp16 scale of its row and group of
+    128 columns; no fallback (VQ_IMPL_TUNED), every batch class, against the oracle."""
+    _check_layer(spec, seed=77, batches=(1, 3, 8, 16), impls=[vq.VQ_IMPL_TUNED, vq.VQ_IMPL_AUTO, vq.VQ_IMPL_GENERIC], decode=True)
 
 
 def test_host_buffer_entry_point():

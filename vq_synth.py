@@ -151,6 +151,12 @@ CONFIGS = {
                  ("q", 4096, 4096), ("k", 1024, 4096), ("v", 1024, 4096), ("o", 4096, 4096),
                  ("gate", 14336, 4096), ("up", 14336, 4096), ("down", 4096, 14336)],
                  d=2, b=6, Br=32, Bc=256, int8=True)),
+    # the same shapes with INT4 codebooks (Sec. 4.2: 2-D, 3 bits per dimension, blocks of 4096 weights,
+    # entries quantized to 4 bits, one scale per row and group of 128 columns)
+    "llama3_8b_int4cb": dict(seed=6, batches=(1, 8), layers=_set("llama3_8b_i4", [
+                 ("q", 4096, 4096), ("k", 1024, 4096), ("v", 1024, 4096), ("o", 4096, 4096),
+                 ("gate", 14336, 4096), ("up", 14336, 4096), ("down", 4096, 14336)],
+                 d=2, b=6, Br=32, Bc=128, int8=2)),
 }
 
 
