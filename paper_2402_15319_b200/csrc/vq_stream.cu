@@ -3,31 +3,40 @@
 // codebook).  The tiling, the pipeline and the reduction are this library's.
 //
 // Work.  The rows of every layer of a call ("segment": layers that share the activations, e.g. the
-// q/k/v or gate/up projections) are cut into slabs of 16*WR rows, a row's index stream into chunks
-// of CHUNK_BYTES.  A slab takes S = chunks / WK pipeline stages; in stage s consumer warp (wr, wk)
-// multiplies its 16 rows by chunk wk*S + s.  Every persistent CTA (one per SM) first takes q =
+// q/k/v or gate/up projections) are cut into slabs of 16*R*WR rows (R row tiles of 16 rows per consumer
+// warp, WR row groups per CTA), a row's index stream into WK column parts of S chunks of CHUNK_BYTES.
+// A slab takes S pipeline stages; in stage s consumer warp (wr, wk) multiplies its 16*R rows by chunk
+// wk*S + s.  The grid is persistent: 1, 2 or 3 CTAs per SM (the kernel is compiled per occupancy, which
+// bounds its registers), each with a static share computed from its index alone.  Every CTA takes q =
 // slabs / P whole slabs; the stages of the slabs left over form one sequence that is cut into equal
-// contiguous pieces, one per CTA, so that every SM streams the same number of bytes whatever the
-// layer shape.
+// contiguous pieces, one per CTA, and a CTA walks its piece FIRST, so that the slabs shared with other
+// CTAs are summed while everyone still computes whole slabs.
 //
-// Pipeline.  One elected producer thread walks the CTA's stages D deep ahead of the consumers with
-// two tiled TMA loads per stage, both counted on the stage's "full" mbarrier: a box {CHUNK_BYTES,
-// 16*WR rows, WK parts} of the index stream and a box of the activations of the same columns, laid
-// out [part][w][batch row][row bytes] so that the B fragments of mma.sync m16n8k16 (batch row =
-// lane / 4) are read without bank conflicts.  Consumers wait on "full", expand indices to fp16
-// weights (A fragments), run the tensor-core steps with fp32 accumulation, and release the stage
-// through its "empty" mbarrier.
+// Roles.  Warps 0..W-1 consume (W = WR*WK); warp W (one thread) produces; warp W+1 writes results; warp
+// W+2 exists for shared-codebook policies only and builds every stage's look-up tables.
 //
-// Reduction.  The partial sums of the WK column parts meet in shared memory and are added in part
-// order.  A slab whose stages all belong to one CTA is rounded to fp16 and stored.  A left-over
-// slab spans several CTAs: each writes its fp32 partial sums into the workspace; at the end of the
-// kernel it draws a ticket from the slab's counter, and the CTA that draws the last ticket adds
-// the partial sums in CTA order (fixed order: results do not depend on timing), stores the outputs
-// and resets the counter to 0.
+// Pipeline.  The producer thread walks the CTA's stages D deep ahead of the consumers with two tiled TMA
+// loads per stage, both counted on the stage's "full" mbarrier: a box {CHUNK_BYTES, slab rows, WK parts}
+// of the index stream and a box of the activations of the same columns, laid out so that the B
+// fragments of mma.sync m16n8k16 (batch row = lane / 4) are read without bank conflicts.  Index boxes
+// are issued before the programmatic-dependency wait (weights must be complete before the call is
+// enqueued), activation boxes after it.  Consumers wait on "full", expand indices to fp16 weights (A
+// fragments; the R row tiles share one activation fragment), run the tensor-core steps with fp32
+// accumulation, and release the stage through its "empty" mbarrier.
+//
+// Reduction.  At the end of a slab the consumers hand their fp32 sums to the results warp through a
+// double-buffered shared-memory area; it adds the WK column parts in part order.  A slab whose stages all
+// belong to one CTA is rounded to fp16 and stored.  A left-over slab spans several CTAs: each writes
+// its partial sums into the workspace and, when its piece is done, draws a ticket from the slab's
+// counter; the CTA that draws the last ticket adds the partial sums in CTA order (fixed order: results
+// do not depend on timing), stores the outputs and resets the counter to 0.
+//
+// Shared memory.  Dynamic shared memory starts 1024 bytes into the CTA's window; the hand-over buffers
+// and the barriers fill the bytes up to the tables' 4096-byte boundary, tables and stages follow.  The
+// kernel checks the size it was given against what the host planned and leaves if they disagree.
 //
 // Every wait is bounded; a wait that runs out increments a device counter, and the warp stops
-// waiting for anything else but still takes part in every block-level barrier, so that the kernel
-// ends.
+// waiting for anything else but still arrives on every barrier it owes, so that the kernel ends.
 #include <cstdio>
 #include <cstdlib>
 
