@@ -88,12 +88,12 @@ vq_status device_error_counter(int** d_counter);
 vq_status device_sms(int* out);
 
 // Tensor map of the packed index stream seen as a 2-D byte tensor (N rows of `stride` bytes) with
-// boxes of box_rows rows x box_bytes bytes, for tiled TMA loads without swizzle or multicast.
+// boxes of box_rows rows x box_bytes bytes, for tiled TMA loads without swizzle, into the issuing CTA only.
 // swizzle128: rows of the box (box_bytes == 128) land with the 128-byte swizzle pattern.
 vq_status encode_index_map(CUtensorMap* tm, const uint8_t* idx, long long stride, int N, int box_bytes, int box_rows,
                            bool swizzle128 = false);
 
-// General tiled tensor map (no multicast is ever used with it): elements of 1 or 2 bytes, rank <= 5,
+// General tiled tensor map (loads with it always target the issuing CTA alone): elements of 1 or 2 bytes, rank <= 5,
 // dims / box in elements, strides of dimensions 1.. in bytes; swizzle 0 none, 1 64-byte, 2 128-byte.
 vq_status encode_tensor_map(CUtensorMap* tm, const void* base, int elem_bytes, int rank, const uint64_t* dims,
                             const uint64_t* strides, const uint32_t* box, int swizzle);

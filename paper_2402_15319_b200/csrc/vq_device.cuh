@@ -118,7 +118,7 @@ __device__ __forceinline__ void st_async_f32(uint32_t cluster_addr, float v, uin
                ::"r"(cluster_addr), "f"(v), "r"(cluster_bar) : "memory");
 }
 
-// ---- bulk asynchronous copies (TMA, untiled, no multicast) tracked by an mbarrier ----------------
+// ---- bulk asynchronous copies (TMA, untiled, into the issuing CTA only) tracked by an mbarrier ----------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t arrivals) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(arrivals) : "memory");
 }
