@@ -1403,7 +1403,13 @@ vq_status launch_tiles(const StreamCall& call, int chunks_per_block, cudaStream_
   // Batch 3-8: a stage's activations are as large as its indices, so one 8-warp CTA per SM with four
   // column parts and two stages comes first (28672 x 8192 at batch 8: 34.5 us against 39.5 us for two
   // 4-warp CTAs with two parts and 79 us for eight row tiles without column parts).
+  // While two 4-warp CTAs with four parts still fit an SM with two stages (batch 3-4) they are faster
+  // still (28672 x 8192 at batch 4: 28.8 against 32.0 us, 8192 x 8192 10.5 against 12.3).
   if constexpr (NB == 1 && P::STAGE_TABLE_BYTES == 0) {
+    if (call.batch > 2 && (only_w == 0 || only_w == 4)) {
+      const vq_status st = R == 2 ? launch<P, 1, 2, 4, 2>(call, chunks_per_block, s, 4, 2) : launch<P, 1, 1, 4, 2>(call, chunks_per_block, s, 4, 2);
+      if (st != VQ_ERR_UNSUPPORTED) return st;
+    }
     if (call.batch > 2 && (only_w == 0 || only_w == 8)) {
       const vq_status st = R == 2 ? launch<P, 1, 2, 8, 1>(call, chunks_per_block, s, 4, 2) : launch<P, 1, 1, 8, 1>(call, chunks_per_block, s, 4, 2);
       if (st != VQ_ERR_UNSUPPORTED) return st;
