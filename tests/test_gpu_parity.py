@@ -370,6 +370,49 @@ def test_benchmark_configs_full_size(cfg):
                 assert_outputs_close(Yg[:, rows], Y, A, f"{spec.name} batch={batch}")
 
 
+@pytest.mark.parametrize("cfg,names", [("cfg5", ("q", "k", "v")), ("cfg5", ("gate", "up")),
+                                       ("cfg3", ("q", "k", "v")), ("cfg3", ("gate", "up"))],
+                         ids=lambda v: v if isinstance(v, str) else "+".join(v))
+def test_benchmark_groups_full_size(cfg, names):
+    """The grouped calls bench.py times, at full size and in its launch configuration (one launch per
+    group): every output row of every member at the configuration's first batch, sampled rows at the
+    others; twice on one workspace."""
+    import torch
+    conf = vq_synth.CONFIGS[cfg]
+    ids = [i for i, sp in enumerate(conf["layers"]) if sp.name.split(".")[-1] in names]
+    specs = [conf["layers"][i] for i in ids]
+    assert len(specs) == len(names)
+    layers = [draw(sp, conf["seed"], i) for sp, i in zip(specs, ids)]
+    t = specs[0]
+    total = vq_synth.LayerSpec("sum", N=sum(sp.N for sp in specs), K=t.K, d=t.d, b=t.b, Br=t.Br, Bc=t.Bc, int8=t.int8)
+    fmt = lib_fmt(total)
+    dev = [(torch.from_numpy(L.idx).cuda(), torch.from_numpy(L.cb).cuda(), None if L.scale is None else torch.from_numpy(L.scale).cuda())
+           for L in layers]
+    batches = conf["batches"] if cfg != "cfg5" else (1, 4, 8, 16)
+    for batch in batches:
+        assert vq.vq_grouped_kernel_launches(fmt, len(specs), batch) == 1
+        X = vq_synth.make_x(specs[0], conf["seed"], batch, ids[0])
+        dX = torch.from_numpy(X).cuda()
+        ws = torch.zeros(vq.vq_workspace_bytes(fmt, batch), dtype=torch.uint8, device="cuda")
+        outs = [guarded((batch, sp.N), torch.float16, "cuda") for sp in specs]
+        members = [(d[0], d[1], d[2], o[0], sp.N) for d, o, sp in zip(dev, outs, specs)]
+        for _ in range(2):
+            vq.vq_gemm_small_batch_grouped(fmt, members, dX, batch, ws)
+        torch.cuda.synchronize()
+        assert vq.vq_device_wait_failures() == 0
+        for sp, L, (Y, raw), lid in zip(specs, layers, outs, ids):
+            assert_guards_intact(raw, sp.name)
+            Yg = Y.cpu().numpy()
+            assert np.isfinite(Yg.astype(np.float64)).all()
+            if batch == batches[0]:
+                Yr, A = orc.gemm(oracle_fmt(sp), L.idx, L.cb, L.scale, X, threads=THREADS)
+                assert_outputs_close(Yg, Yr, A, f"{sp.name} grouped batch={batch} all rows")
+            else:
+                rows = _sample_rows(sp.N, sp.Br, seed=lid)
+                Yr, A = orc.gemm(oracle_fmt(sp), L.idx, L.cb, L.scale, X, rows=rows, threads=THREADS)
+                assert_outputs_close(Yg[:, rows], Yr, A, f"{sp.name} grouped batch={batch}")
+
+
 # ---- INT4 g128 yard-stick ---------------------------------------------------------------------
 @pytest.mark.parametrize("N,K", [(100, 256), (64, 4096), (37, 11008 - 11008 % 128)])
 def test_int4g128(N, K):
