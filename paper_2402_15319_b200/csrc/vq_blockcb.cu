@@ -64,8 +64,11 @@ struct BlockArgs {
   int n_chunks;          // K / 256
   int blocks_per_row;    // K / block_cols
   int Br, Bc;
-  // byte offsets from the aligned start of dynamic shared memory
+  // byte offsets from the tables' boundary (the first TABLE_BYTES boundary that leaves front_bytes of
+  // dynamic shared memory in front of it): parts that fit lie in front of the tables (negative
+  // offsets), in bytes that alignment would otherwise waste; the rest follows the tables
   int compact_off, ring_off, bar_off, x_off, recv_off;
+  int front_bytes, after_bytes;
 };
 
 // Layers of one call (same format and K, their own rows): row tiles [tile0, next tile0) of the grid
@@ -370,8 +373,16 @@ blockcb_kernel(const __grid_constant__ BlockMaps maps, const BlockArgs a_in, con
   constexpr int NBT = 8 * NB;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const uint32_t raw_u32 = smem_u32(smem_raw);
-  const uint32_t base = (raw_u32 + P::TABLE_BYTES - 1) & ~static_cast<uint32_t>(P::TABLE_BYTES - 1);
+  const uint32_t base = (raw_u32 + a_in.front_bytes + P::TABLE_BYTES - 1) & ~static_cast<uint32_t>(P::TABLE_BYTES - 1);
   unsigned char* smem = smem_raw + (base - raw_u32);
+  {   // the host sized the launch for dynamic shared memory that starts 1024 bytes into the CTA's window
+    uint32_t dyn;
+    asm("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn));
+    if (base - raw_u32 + static_cast<uint32_t>(a_in.after_bytes) > dyn) {   // (the same for every thread of the cluster)
+      if (threadIdx.x == 0) atomicAdd(a_in.error_flag, 1);
+      return;
+    }
+  }
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int S = gridDim.x, rank = blockIdx.x;
@@ -722,19 +733,49 @@ vq_status launch(const StreamCall& call, cudaStream_t s) {
   for (int i = call.n_seg; i < kMaxSegments; ++i) maps.m[i] = maps.m[0];
 
   // Shared memory of a CTA whose column range is `chunks` long.
+  // The tables start on a TABLE_BYTES boundary of the CTA's shared-memory window (their address bits
+  // merge with the index bits); dynamic shared memory starts 1024 bytes into the window (the first 1024
+  // are the system's; the kernel checks what it gets).  Parts that fit into the bytes in front of that
+  // boundary go there, largest first; the others follow the tables.
   auto smem_for = [&](int chunks, BlockArgs* out) {
     constexpr int ST = kStagesOf<D, PRIV>;
-    size_t off = (PRIV ? P::WARPS : kTableBuffers<D>) * static_cast<size_t>(P::TABLE_BYTES);
-    const size_t compact_off = off; off += 2 * P::COMPACT_BYTES;
-    const size_t ring_off = round_up(off, 128); off = ring_off + static_cast<size_t>(P::WARPS) * ST * T::STAGE_BYTES;
-    const size_t bar_off = off; off += static_cast<size_t>(P::WARPS) * ST * 8 + 8;   // rings + receive barrier
-    const size_t x_off = round_up(off, 16); off = x_off + static_cast<size_t>(chunks) * 512 * batch;
-    const size_t recv_off = round_up(off, 16); off = recv_off + static_cast<size_t>(T::CTA_ROWS) * 8 * NB * sizeof(float);
-    if (out) {
-      out->compact_off = static_cast<int>(compact_off); out->ring_off = static_cast<int>(ring_off);
-      out->bar_off = static_cast<int>(bar_off); out->x_off = static_cast<int>(x_off); out->recv_off = static_cast<int>(recv_off);
+    const size_t tables = (PRIV ? P::WARPS : kTableBuffers<D>) * static_cast<size_t>(P::TABLE_BYTES);
+    struct Part { size_t bytes, align; long long off; };
+    Part ring = {static_cast<size_t>(P::WARPS) * ST * T::STAGE_BYTES, 128, 0};
+    Part x = {static_cast<size_t>(chunks) * 512 * batch, 16, 0};
+    Part recv = {static_cast<size_t>(T::CTA_ROWS) * 8 * NB * sizeof(float), 16, 0};
+    Part compact = {2 * static_cast<size_t>(P::COMPACT_BYTES), 16, 0};
+    Part bars = {static_cast<size_t>(P::WARPS) * ST * 8 + 8, 8, 0};   // rings + receive barrier
+    Part* order[5] = {&ring, &x, &recv, &compact, &bars};
+    for (int i = 0; i < 5; ++i)   // largest first
+      for (int j = i + 1; j < 5; ++j)
+        if (order[j]->bytes > order[i]->bytes) { Part* t = order[i]; order[i] = order[j]; order[j] = t; }
+    const size_t room = P::TABLE_BYTES - 1024;
+    size_t front = 0, after = tables;
+    bool in_front[5];
+    for (int i = 0; i < 5; ++i) {
+      const size_t at = round_up(front, order[i]->align);
+      in_front[i] = at + order[i]->bytes <= room;
+      if (in_front[i]) {
+        order[i]->off = static_cast<long long>(at);
+        front = at + order[i]->bytes;
+      } else {
+        const size_t pos = round_up(after, order[i]->align);
+        order[i]->off = static_cast<long long>(pos);
+        after = pos + order[i]->bytes;
+      }
     }
-    return off + P::TABLE_BYTES;   // + room to align the tables
+    front = round_up(front, 128);   // the front region ends at the tables' boundary
+    for (int i = 0; i < 5; ++i)
+      if (in_front[i]) order[i]->off -= static_cast<long long>(front);
+    const size_t lead = round_up(1024 + front, P::TABLE_BYTES) - 1024;
+    if (out) {
+      out->compact_off = static_cast<int>(compact.off); out->ring_off = static_cast<int>(ring.off);
+      out->bar_off = static_cast<int>(bars.off); out->x_off = static_cast<int>(x.off); out->recv_off = static_cast<int>(recv.off);
+      out->front_bytes = static_cast<int>(front);
+      out->after_bytes = static_cast<int>(after);
+    }
+    return lead + after;
   };
   // K split: waves of co-resident CTAs times (chunks per CTA + fixed overhead, in chunk times); ties
   // go to the larger split.
@@ -745,7 +786,7 @@ vq_status launch(const StreamCall& call, cudaStream_t s) {
     const int chunks = (a.n_chunks + S - 1) / S;
     const size_t smem = smem_for(chunks, nullptr);
     if (smem > 220 * 1024) continue;
-    const int per_sm = static_cast<int>((227 * 1024) / (smem + 1024));
+    const int per_sm = static_cast<int>((228 * 1024) / (smem + 1024));
     const long long ctas = static_cast<long long>(row_blocks) * S;
     const long long slots = static_cast<long long>(per_sm < 1 ? 1 : per_sm) * sms;
     const double waves = static_cast<double>((ctas + slots - 1) / slots);
