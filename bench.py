@@ -147,6 +147,7 @@ class DeviceSet:
         conf = vq_synth.CONFIGS[cfg_name]
         self.cfg_name, self.batch, self.device = cfg_name, batch, device
         self.batch_built = batch
+        self.batch_host = batch   # the host-side buffers keep the constructor's batch
         self.specs = conf["layers"]
         self.fmts, self.host, self.bytes_per_layer = [], [], []
         for lid, spec in enumerate(self.specs):
@@ -187,7 +188,10 @@ class DeviceSet:
         self.hX = [torch.from_numpy(X).pin_memory() for (_, X) in self.host]
         self.hY = [torch.empty((batch, s.N), dtype=torch.float16).pin_memory() for s in self.specs]
         self.ws_host = [torch.zeros(vq.vq_workspace_bytes_host(f, batch), dtype=torch.uint8, device=device) for f in self.fmts]
-        self.h2d = sum(int(x.numel()) * 2 for x in self.hX)
+        self.group_ws_host = {i: torch.zeros(vq.vq_workspace_bytes_grouped_host(gf, len(g), batch), dtype=torch.uint8, device=device)
+                              for g in self.groups if len(g) > 1 for i, gf in [(g[0], self.group_fmt[g[0]])]}
+        # a group's activations cross the host boundary once
+        self.h2d = sum(int(self.hX[g[0]].numel()) * 2 for g in self.groups)
         self.d2h = sum(int(y.numel()) * 2 for y in self.hY)
 
     def step(self, copy: int):
@@ -216,10 +220,16 @@ class DeviceSet:
         self.step_bytes = int(sum(per_layer)) - sum(2 * batch * self.specs[i].K for g in self.groups for i in g[1:])
 
     def step_host(self, copy: int):
+        """The same calls as step() with host activations and outputs (built for the batch of the constructor)."""
         vq = self.vq
-        for i, fmt in enumerate(self.fmts):
-            idx, cb, sc = self.dev[copy][i]
-            vq.vq_gemm_small_batch_host(fmt, idx, cb, sc, self.hX[i], self.hY[i], self.batch, self.ws_host[i])
+        for g in self.groups:
+            i = g[0]
+            if len(g) == 1:
+                idx, cb, sc = self.dev[copy][i]
+                vq.vq_gemm_small_batch_host(self.fmts[i], idx, cb, sc, self.hX[i], self.hY[i], self.batch_host, self.ws_host[i])
+            else:
+                members = [(self.dev[copy][j][0], self.dev[copy][j][1], self.dev[copy][j][2], self.hY[j], self.specs[j].N) for j in g]
+                vq.vq_gemm_small_batch_grouped_host(self.group_fmt[i], members, self.hX[i], self.batch_host, self.group_ws_host[i])
         self.torch.cuda.synchronize()
 
     def launches_per_step(self) -> int:
@@ -722,7 +732,7 @@ def run_ours(args):
         "clocks": clocks,
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": ds.h2d, "d2h_bytes_per_step": ds.d2h,
                 "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps,
-                "what": "vq_gemm_small_batch_host per layer: activations read from pinned host memory, kernel, outputs written back to pinned host memory, stream synchronised every step; compressed weights resident in HBM"},
+                "what": "the step's calls with host buffers (vq_gemm_small_batch_grouped_host for q/k/v and gate/up, vq_gemm_small_batch_host for o and down): activations read from pinned host memory, kernels, outputs written back to pinned host memory, stream synchronised every step; compressed weights resident in HBM"},
         "gpu_launches": launches_per_step * args.steps,
         "roofline": {
             "bound": "hbm", "kernel": f"{KERNEL_OF.get(args.config, 'vq gemm kernel')}: call '{dom[0]}' (largest share of the step: "

@@ -208,6 +208,18 @@ vq_status vq_gemm_small_batch_host(const vq_format* fmt, const void* d_idx, cons
                                    void* d_ws, size_t ws_bytes, void* stream);
 size_t vq_workspace_bytes_host(const vq_format* fmt, int batch);
 
+/* vq_gemm_small_batch_grouped with HOST activations and outputs: h_X (binary16 [batch][K]) is brought to
+ * the device once for the whole group, every member's result goes back to the HOST buffer its d_Y field
+ * names (binary16 [batch][n_rows]; in this call d_Y is a host pointer).  Steps are enqueued on `stream`, the
+ * call returns without synchronising; pinned buffers take the same direct path as
+ * vq_gemm_small_batch_host (paper Sec. 1 / Sec. 3.2: per generated token only activations cross the host
+ * boundary, the weights stay on the device).
+ *   d_ws : at least vq_workspace_bytes_grouped_host(fmt, n_members, batch) bytes, rules as WORKSPACE above.
+ * Errors: as vq_gemm_small_batch_grouped. */
+vq_status vq_gemm_small_batch_grouped_host(const vq_format* fmt, const vq_group_member* members, int n_members,
+                                           const void* h_X, int batch, void* d_ws, size_t ws_bytes, void* stream);
+size_t vq_workspace_bytes_grouped_host(const vq_format* fmt, int n_members, int batch);
+
 /* The same computation as vq_gemm_small_batch_host for callers that cannot allocate device memory
  * at all: code that runs where cudaMalloc is forbidden or unavailable - inside a region whose
  * memory is owned and budgeted by another allocator (an inference server's arena, a real-time

@@ -6,7 +6,7 @@ from .binding import (  # noqa: F401
     VQError, VQFormat, PackInfo, lib_path, load, exported_symbols,
     vq_pack_info, vq_workspace_bytes, vq_workspace_bytes_host, vq_decode_weights, vq_gemv,
     vq_gemm_small_batch, vq_gemm_small_batch_grouped, vq_grouped_kernel_launches, vq_gemm_small_batch_impl, vq_gemm_small_batch_host,
-    vq_gemm_small_batch_host_static, vq_static_scratch_bytes,
+    vq_gemm_small_batch_host_static, vq_static_scratch_bytes, vq_gemm_small_batch_grouped_host, vq_workspace_bytes_grouped_host,
     vq_int4g128_gemm_small_batch, vq_int4g128_workspace_bytes, vq_status_string, vq_device_wait_failures,
     vq_assign_indices, vq_unpack_uniform, vq_probe_decode_loop, vq_probe_read, VQ_UNPACK_FP16, VQ_UNPACK_INT8_ROW, VQ_UNPACK_INT4_G128,
 )

@@ -83,6 +83,9 @@ _SIGNATURES = {
     "vq_gemm_small_batch_grouped": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int,
                                                    ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
     "vq_grouped_kernel_launches": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int, ctypes.c_int]),
+    "vq_gemm_small_batch_grouped_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int,
+                                                        ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
+    "vq_workspace_bytes_grouped_host": (ctypes.c_size_t, [ctypes.c_void_p, ctypes.c_int, ctypes.c_int]),
     "vq_gemm_small_batch_host": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
     "vq_gemm_small_batch_host_static": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p]),
     "vq_static_scratch_bytes": (ctypes.c_size_t, []),
@@ -189,6 +192,23 @@ def vq_gemm_small_batch_grouped(fmt: VQFormat, members, d_X, batch: int, d_ws, s
     _check(load().vq_gemm_small_batch_grouped(ctypes.byref(c), arr, len(members), _ptr(d_X), int(batch), _ptr(d_ws),
                                               d_ws.numel() * d_ws.element_size(), _stream(stream)),
            "vq_gemm_small_batch_grouped")
+
+
+def vq_gemm_small_batch_grouped_host(fmt: VQFormat, members, h_X, batch: int, d_ws, stream=None) -> None:
+    """members: sequence of (d_idx, d_cb, d_scale, h_Y, n_rows) with HOST outputs; h_X a host tensor (pinned for
+    the direct path).  Synchronise before reading the outputs."""
+    arr = (_CGroupMember * len(members))()
+    for i, (idx, cb, sc, Y, n) in enumerate(members):
+        arr[i] = _CGroupMember(_ptr(idx), _ptr(cb), _ptr(sc), _ptr(Y), int(n))
+    c = fmt.c()
+    _check(load().vq_gemm_small_batch_grouped_host(ctypes.byref(c), arr, len(members), _ptr(h_X), int(batch), _ptr(d_ws),
+                                                   d_ws.numel() * d_ws.element_size(), _stream(stream)),
+           "vq_gemm_small_batch_grouped_host")
+
+
+def vq_workspace_bytes_grouped_host(fmt: VQFormat, n_members: int, batch: int) -> int:
+    c = fmt.c()
+    return load().vq_workspace_bytes_grouped_host(ctypes.byref(c), int(n_members), int(batch))
 
 
 def vq_grouped_kernel_launches(fmt: VQFormat, n_members: int, batch: int) -> int:

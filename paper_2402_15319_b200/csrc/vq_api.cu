@@ -306,6 +306,72 @@ vq_status vq_gemm_small_batch_host(const vq_format* fmt, const void* d_idx, cons
   return VQ_OK;
 }
 
+// Grouped call with host activations and outputs (see vq.h).  The members' d_Y fields are HOST pointers here.
+vq_status vq_gemm_small_batch_grouped_host(const vq_format* fmt, const vq_group_member* members, int n_members,
+                                           const void* h_X, int batch, void* d_ws, size_t ws_bytes, void* stream) {
+  if (!fmt || !members || !h_X) return VQ_ERR_NULL;
+  if (n_members < 1 || n_members > VQ_MAX_GROUP) return VQ_ERR_SHAPE;
+  if (batch < 1 || batch > 16) return VQ_ERR_BATCH;
+  const size_t base = vq_workspace_bytes(fmt, batch);
+  if (!base) return VQ_ERR_FORMAT;
+  // device copies: X, then every member's Y on a 256-byte boundary
+  const size_t x_bytes = static_cast<size_t>(batch) * fmt->k_cols * 2;
+  size_t need = base + round256(x_bytes);
+  long long rows = 0;
+  for (int i = 0; i < n_members; ++i) {
+    if (!members[i].d_Y) return VQ_ERR_NULL;
+    if (members[i].n_rows <= 0) return VQ_ERR_SHAPE;
+    need += round256(static_cast<size_t>(batch) * members[i].n_rows * 2);
+    rows += members[i].n_rows;
+  }
+  if (rows != fmt->n_rows) return VQ_ERR_SHAPE;
+  if (!d_ws || ws_bytes < need) return VQ_ERR_WORKSPACE;
+  if (!aligned16(d_ws)) return VQ_ERR_ALIGN;
+  char* ws = static_cast<char*>(d_ws);
+  void* d_X = ws + base;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  vq_group_member dev[VQ_MAX_GROUP];
+  // pinned (mapped) buffers: one small kernel fetches X, the mat-vec kernel stores every Y straight
+  // into host memory (as vq_gemm_small_batch_host does)
+  bool mapped = x_bytes % 16 == 0;
+  const void* dx = mapped ? mapped_device_pointer(h_X) : nullptr;
+  mapped = mapped && dx && aligned16(dx);
+  for (int i = 0; i < n_members && mapped; ++i) {
+    dev[i] = members[i];
+    dev[i].d_Y = const_cast<void*>(mapped_device_pointer(members[i].d_Y));
+    mapped = dev[i].d_Y && aligned16(dev[i].d_Y);
+  }
+  if (mapped) {
+    const int n16 = static_cast<int>(x_bytes / 16);
+    int blocks = (n16 + 255) / 256;
+    if (blocks > 8) blocks = 8;
+    fetch_kernel<<<blocks, 256, 0, s>>>(static_cast<const uint4*>(dx), static_cast<uint4*>(d_X), n16);
+    if (check_launch() != VQ_OK) return VQ_ERR_CUDA;
+    return vq_gemm_small_batch_grouped(fmt, dev, n_members, d_X, batch, d_ws, base, stream);
+  }
+  size_t off = base + round256(x_bytes);
+  for (int i = 0; i < n_members; ++i) {
+    dev[i] = members[i];
+    dev[i].d_Y = ws + off;
+    off += round256(static_cast<size_t>(batch) * members[i].n_rows * 2);
+  }
+  if (cudaMemcpyAsync(d_X, h_X, x_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return VQ_ERR_CUDA;
+  const vq_status st = vq_gemm_small_batch_grouped(fmt, dev, n_members, d_X, batch, d_ws, base, stream);
+  if (st != VQ_OK) return st;
+  for (int i = 0; i < n_members; ++i)
+    if (cudaMemcpyAsync(members[i].d_Y, dev[i].d_Y, static_cast<size_t>(batch) * members[i].n_rows * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+      return VQ_ERR_CUDA;
+  return VQ_OK;
+}
+
+size_t vq_workspace_bytes_grouped_host(const vq_format* fmt, int n_members, int batch) {
+  const size_t base = vq_workspace_bytes(fmt, batch);
+  if (!base || n_members < 1 || n_members > VQ_MAX_GROUP) return 0;
+  // every member's Y on its own 256-byte boundary: at most 256 bytes of padding each
+  return base + round256(static_cast<size_t>(batch) * fmt->k_cols * 2) + round256(static_cast<size_t>(batch) * fmt->n_rows * 2) +
+         256 * static_cast<size_t>(n_members);
+}
+
 const char* vq_status_string(vq_status s) {
   switch (s) {
     case VQ_OK: return "VQ_OK";

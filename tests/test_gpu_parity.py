@@ -546,6 +546,41 @@ def test_int4_codebooks_in_the_tall_block_kernel(spec):
     _check_layer(spec, seed=77, batches=(1, 3, 8, 16), impls=[vq.VQ_IMPL_TUNED, vq.VQ_IMPL_AUTO, vq.VQ_IMPL_GENERIC], decode=True)
 
 
+@pytest.mark.parametrize("pinned", [True, False], ids=["pinned", "pageable"])
+def test_grouped_host_buffer_entry_point(pinned):
+    """vq_gemm_small_batch_grouped_host: activations from host memory once for the group, every member's
+    result in its own host buffer; pinned buffers (direct path) and pageable ones (copies) against the
+    oracle, and bit-identical to the device-pointer grouped call."""
+    import torch
+    rows = [512, 136, 128]
+    tmpl = dict(K=4096, d=2, b=4, Br=1, Bc=2048, int8=True)
+    specs = [vq_synth.LayerSpec(f"gh{i}", N=n, **tmpl) for i, n in enumerate(rows)]
+    layers = [draw(sp, 61, i) for i, sp in enumerate(specs)]
+    fmt = lib_fmt(vq_synth.LayerSpec("gh", N=sum(rows), **tmpl))
+    dev = [(torch.from_numpy(L.idx).cuda(), torch.from_numpy(L.cb).cuda(), torch.from_numpy(L.scale).cuda()) for L in layers]
+    for batch in (1, 6):
+        X = vq_synth.make_x(specs[0], 62, batch)
+        hX = torch.from_numpy(X)
+        hYs = [torch.full((batch, n), float("nan"), dtype=torch.float16) for n in rows]
+        if pinned:
+            hX, hYs = hX.pin_memory(), [y.pin_memory() for y in hYs]
+        ws = torch.zeros(vq.vq_workspace_bytes_grouped_host(fmt, len(rows), batch), dtype=torch.uint8, device="cuda")
+        vq.vq_gemm_small_batch_grouped_host(fmt, [(d[0], d[1], d[2], y, n) for d, y, n in zip(dev, hYs, rows)], hX, batch, ws)
+        torch.cuda.synchronize()
+        dYs = [torch.empty((batch, n), dtype=torch.float16, device="cuda") for n in rows]
+        ws2 = torch.zeros(vq.vq_workspace_bytes(fmt, batch), dtype=torch.uint8, device="cuda")
+        vq.vq_gemm_small_batch_grouped(fmt, [(d[0], d[1], d[2], y, n) for d, y, n in zip(dev, dYs, rows)], torch.from_numpy(X).cuda(), batch, ws2)
+        torch.cuda.synchronize()
+        for sp, L, hY, dY in zip(specs, layers, hYs, dYs):
+            Yr, A = orc.gemm(oracle_fmt(sp), L.idx, L.cb, L.scale, X, threads=4)
+            assert_outputs_close(hY.numpy(), Yr, A, f"{sp.name} batch {batch}")
+            assert np.array_equal(hY.numpy().view(np.uint16), dY.cpu().numpy().view(np.uint16))
+    with pytest.raises(vq.VQError) as err:   # workspace too small
+        vq.vq_gemm_small_batch_grouped_host(fmt, [(d[0], d[1], d[2], y, n) for d, y, n in zip(dev, hYs, rows)], hX, 6,
+                                            torch.zeros(64, dtype=torch.uint8, device="cuda"))
+    assert err.value.code == 5
+
+
 def test_host_buffer_entry_point():
     import torch
     spec = vq_synth.LayerSpec("host", N=256, K=1024, d=2, b=6, Br=128, Bc=128, int8=False)
