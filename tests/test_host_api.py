@@ -203,3 +203,24 @@ def test_grouped_call_argument_errors_and_launch_counts():
         assert vq.vq_grouped_kernel_launches(row4, 1, batch) == 1
     assert vq.vq_grouped_kernel_launches(row4, 0, 1) == 0 and vq.vq_grouped_kernel_launches(row4, 5, 1) == 0
     assert vq.vq_grouped_kernel_launches(row4, 2, 17) == 0
+
+
+def test_grouped_host_call_argument_errors():
+    from paper_2402_15319_b200.binding import _CGroupMember
+    lib = vq.load()
+    total = _replace(GOOD, n_rows=16)
+    c = total.c()
+    arr = (_CGroupMember * 2)(_CGroupMember(FAKE, FAKE, None, FAKE, 8), _CGroupMember(FAKE, FAKE, None, FAKE, 8))
+    big = vq.vq_workspace_bytes_grouped_host(total, 2, 1)
+    assert big > vq.vq_workspace_bytes(total, 1)
+    assert vq.vq_workspace_bytes_grouped_host(total, 0, 1) == 0 and vq.vq_workspace_bytes_grouped_host(total, 2, 17) == 0
+    call = lambda n=2, X=FAKE, batch=1, ws=FAKE, nbytes=big: lib.vq_gemm_small_batch_grouped_host(
+        ctypes.byref(c), arr, n, X, batch, ws, nbytes, None)
+    assert call(X=None) == 1 and call(n=0) == 3 and call(n=5) == 3
+    assert call(batch=0) == 6 and call(batch=17) == 6
+    assert call(ws=None) == 5 and call(nbytes=big - 600) == 5 and call(ws=ODD) == 4
+    arr[1].n_rows = 4       # rows no longer add up
+    assert call() == 3
+    arr[1].n_rows = 8
+    arr[0].d_Y = None
+    assert call() == 1
