@@ -736,8 +736,8 @@ vq_status launch(const StreamCall& call, cudaStream_t s) {
   // The tables start on a TABLE_BYTES boundary of the CTA's shared-memory window (their address bits
   // merge with the index bits); dynamic shared memory starts 1024 bytes into the window (the first 1024
   // are the system's; the kernel checks what it gets).  Parts that fit into the bytes in front of that
-  // boundary go there, largest first; the others follow the tables.
-  auto smem_for = [&](int chunks, BlockArgs* out) {
+  // boundary go there, largest first (`compact`); the others follow the tables.
+  auto smem_for = [&](int chunks, BlockArgs* out, bool use_front) {
     constexpr int ST = kStagesOf<D, PRIV>;
     const size_t tables = (PRIV ? P::WARPS : kTableBuffers<D>) * static_cast<size_t>(P::TABLE_BYTES);
     struct Part { size_t bytes, align; long long off; };
@@ -750,12 +750,12 @@ vq_status launch(const StreamCall& call, cudaStream_t s) {
     for (int i = 0; i < 5; ++i)   // largest first
       for (int j = i + 1; j < 5; ++j)
         if (order[j]->bytes > order[i]->bytes) { Part* t = order[i]; order[i] = order[j]; order[j] = t; }
-    const size_t room = P::TABLE_BYTES - 1024;
+    const size_t room = use_front ? P::TABLE_BYTES - 1024 : 0;
     size_t front = 0, after = tables;
     bool in_front[5];
     for (int i = 0; i < 5; ++i) {
       const size_t at = round_up(front, order[i]->align);
-      in_front[i] = at + order[i]->bytes <= room;
+      in_front[i] = room > 0 && at + order[i]->bytes <= room;
       if (in_front[i]) {
         order[i]->off = static_cast<long long>(at);
         front = at + order[i]->bytes;
@@ -779,26 +779,39 @@ vq_status launch(const StreamCall& call, cudaStream_t s) {
   };
   // K split: waves of co-resident CTAs times (chunks per CTA + fixed overhead, in chunk times); ties
   // go to the larger split.
-  int best = 0;
-  double best_cost = -1.0;
-  for (int S = 1; S <= 8; S *= 2) {
-    if (S > a.n_chunks) break;
-    const int chunks = (a.n_chunks + S - 1) / S;
-    const size_t smem = smem_for(chunks, nullptr);
-    if (smem > 220 * 1024) continue;
-    const int per_sm = static_cast<int>((228 * 1024) / (smem + 1024));
-    const long long ctas = static_cast<long long>(row_blocks) * S;
-    const long long slots = static_cast<long long>(per_sm < 1 ? 1 : per_sm) * sms;
-    const double waves = static_cast<double>((ctas + slots - 1) / slots);
-    const double cost = waves * (chunks + (S > 1 ? 2.0 : 1.5));
-    if (best_cost < 0.0 || cost <= best_cost) {
-      best_cost = cost;
-      best = S;
+  auto plan = [&](bool compact, double* cost_out) {
+    int best = 0;
+    double best_cost = -1.0;
+    for (int S = 1; S <= 8; S *= 2) {
+      if (S > a.n_chunks) break;
+      const int chunks = (a.n_chunks + S - 1) / S;
+      const size_t smem = smem_for(chunks, nullptr, compact);
+      if (smem > 220 * 1024) continue;
+      const int per_sm = static_cast<int>((228 * 1024) / (smem + 1024));
+      const long long ctas = static_cast<long long>(row_blocks) * S;
+      const long long slots = static_cast<long long>(per_sm < 1 ? 1 : per_sm) * sms;
+      const double waves = static_cast<double>((ctas + slots - 1) / slots);
+      const double cost = waves * (chunks + (S > 1 ? 2.0 : 1.5));
+      if (best_cost < 0.0 || cost <= best_cost) {
+        best_cost = cost;
+        best = S;
+      }
     }
-  }
+    *cost_out = best_cost;
+    return best;
+  };
+  // The compact layout lets more CTAs share an SM.  It is taken from batch 3 on, where the staged
+  // activations make a CTA large (4-D format at batch 8: one 128 KB CTA per SM becomes two of 96 KB, 106 ->
+  // 88 us per 13B-shaped layer set; 2-D 6-bit 32 x 256 blocks at batch 8: 94 -> 87 us).  At batch 1-2 the
+  // grids are less than a wave and the plain layout stays: once an extra CTA fits, such a grid spreads
+  // unevenly over the SMs (224 CTAs on 148 SMs: 37 against 31 us alone, 67 against 63 us per layer set).
+  double cost = -1.0;
+  bool compact = batch > 2;
+  int best = plan(compact, &cost);
+  compact = env_int("VQ_COMPACT", compact ? 1 : 0) != 0;
   best = env_int("VQ_SPLIT", best);
   if (best < 1 || best > 8 || (best & (best - 1)) || best > a.n_chunks) return VQ_ERR_UNSUPPORTED;
-  const size_t smem_bytes = smem_for((a.n_chunks + best - 1) / best, &a);
+  const size_t smem_bytes = smem_for((a.n_chunks + best - 1) / best, &a, compact);
   if (smem_bytes > 220 * 1024) return VQ_ERR_UNSUPPORTED;
 
   cudaLaunchConfig_t cfg = {};
@@ -822,6 +835,10 @@ vq_status launch(const StreamCall& call, cudaStream_t s) {
   }
   cfg.attrs = attr;
   cfg.numAttrs = na;
+#ifdef VQ_TUNING
+  if (env_int("VQ_VERBOSE", 0))
+    fprintf(stderr, "blockcb launch: split %d row tiles %d smem %zu front %d after %d\n", best, row_blocks, smem_bytes, a.front_bytes, a.after_bytes);
+#endif
   const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, maps, a, grp);
   if (e != cudaSuccess) {
 #ifdef VQ_TUNING
