@@ -173,9 +173,9 @@ struct Walk {
 
   __device__ __forceinline__ void init(const StreamArgs& a, int c, int P) {
     t0 = t1 = 0;
-    if (c < a.tail_ctas) {
-      t0 = static_cast<int>(static_cast<long long>(a.tail_units) * c / a.tail_ctas);
-      t1 = static_cast<int>(static_cast<long long>(a.tail_units) * (c + 1) / a.tail_ctas);
+    if (c < a.tail_ctas) {   // (the host keeps tail_units * tail_ctas below 2^31: 32-bit arithmetic)
+      t0 = static_cast<int>(static_cast<unsigned>(a.tail_units) * static_cast<unsigned>(c) / static_cast<unsigned>(a.tail_ctas));
+      t1 = static_cast<int>(static_cast<unsigned>(a.tail_units) * static_cast<unsigned>(c + 1) / static_cast<unsigned>(a.tail_ctas));
     }
     n_tail = t1 - t0;
     n = n_tail + a.q * a.S;
@@ -1293,6 +1293,7 @@ vq_status launch(const StreamCall& call, int chunks_per_block, cudaStream_t s, i
   const long long tail = static_cast<long long>(left) * a.S;
   a.tail_units = static_cast<int>(tail);
   a.tail_ctas = static_cast<int>(tail < Pn ? tail : Pn);
+  if (tail * (a.tail_ctas + 1) >= (1LL << 31)) return VQ_ERR_UNSUPPORTED;   // the kernel splits the tail in 32-bit arithmetic
   // Left-over slabs are either cut into stages shared evenly by all CTAs (their partial sums then meet
   // through the workspace, which costs about two stage times at the end of the kernel) or handed out
   // whole, one per CTA, whichever ends earlier.
