@@ -74,6 +74,11 @@ vq_status launch_gemm_blockcb_group(const StreamCall& call, cudaStream_t s);
 bool blockcb_covers(const Geometry& g);
 vq_status launch_gemm_rowcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
                             cudaStream_t s);
+// Warp-private pair tables: small codebook blocks (1, 2, 4, 8 or a multiple of 16 rows), 2-D indices of
+// any width, 1-D indices of up to 4 bits, fp16 / int8 codebooks, K and block columns multiples of 64.
+vq_status launch_gemm_warptab(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
+                              cudaStream_t s);
+bool warptab_covers(const Geometry& g);
 vq_status launch_int4g128_rowcb(int N, int K, const uint8_t* q, const __half* scale, const __half* X, __half* Y, int batch,
                                 cudaStream_t s);
 vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s);

@@ -146,21 +146,25 @@ vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half*
   st = launch_gemm_blockcb(g, p, X, Y, batch, s);
   if (st != VQ_ERR_UNSUPPORTED) return st;
   st = launch_gemm_rowcb(g, p, X, Y, batch, s);
-  if (st != VQ_ERR_UNSUPPORTED || !ws || stream_first) return st;
-  // shapes the cluster kernels do not take: the persistent kernel if it does
-  StreamCall call = {};
-  call.g = g;
-  call.n_seg = 1;
-  call.idx[0] = p.idx;
-  call.cb[0] = p.cb;
-  call.scale[0] = p.scale;
-  call.Y[0] = Y;
-  call.N[0] = g.N;
-  call.X = X;
-  call.batch = batch;
-  call.ws = ws;
-  call.ws_bytes = ws_bytes;
-  return launch_gemm_stream(call, s);
+  if (st != VQ_ERR_UNSUPPORTED) return st;
+  if (ws && !stream_first) {   // shapes the cluster kernels do not take: the persistent kernel if it does
+    StreamCall call = {};
+    call.g = g;
+    call.n_seg = 1;
+    call.idx[0] = p.idx;
+    call.cb[0] = p.cb;
+    call.scale[0] = p.scale;
+    call.Y[0] = Y;
+    call.N[0] = g.N;
+    call.X = X;
+    call.batch = batch;
+    call.ws = ws;
+    call.ws_bytes = ws_bytes;
+    st = launch_gemm_stream(call, s);
+    if (st != VQ_ERR_UNSUPPORTED) return st;
+  }
+  // small codebook blocks and the index widths no other family takes: warp-private pair tables
+  return launch_gemm_warptab(g, p, X, Y, batch, s);
 }
 
 

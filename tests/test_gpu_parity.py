@@ -196,6 +196,45 @@ def test_tall_block_kernel_extra_formats(spec):
     _check_layer(spec, seed=91, batches=(1, 3, 8, 16), impls=[vq.VQ_IMPL_TUNED, vq.VQ_IMPL_GENERIC], decode=True)
 
 
+# the rows of the paper's table of VQ configurations (App. on VQ configurations) that no other tuned family
+# takes, and formats around them: small codebook blocks, 5-bit and 8-bit 2-D indices, 1-D indices looked up
+# two at a time; ragged row counts, K parts that do not divide among the warps, block columns of 64..256
+PAIR_TABLE_CASES = [
+    vq_synth.LayerSpec("pt_d1b2_1x256_i8", N=200, K=1024, d=1, b=2, Br=1, Bc=256, int8=True),
+    vq_synth.LayerSpec("pt_d1b2_1x128_i8", N=48, K=1152, d=1, b=2, Br=1, Bc=128, int8=True),
+    vq_synth.LayerSpec("pt_d2b5_4x256_i8", N=212, K=2048, d=2, b=5, Br=4, Bc=256, int8=True),
+    vq_synth.LayerSpec("pt_d2b5_2x256_i8", N=130, K=1280, d=2, b=5, Br=2, Bc=256, int8=True),
+    vq_synth.LayerSpec("pt_d2b5_1x256", N=77, K=768, d=2, b=5, Br=1, Bc=256, int8=False),
+    vq_synth.LayerSpec("pt_d1b3_32x256_i8", N=96, K=2304, d=1, b=3, Br=32, Bc=256, int8=True),
+    vq_synth.LayerSpec("pt_d2b8_256x256_i8", N=512, K=1024, d=2, b=8, Br=256, Bc=256, int8=True),
+    vq_synth.LayerSpec("pt_d2b7_16x64", N=64, K=4480, d=2, b=7, Br=16, Bc=64, int8=False),
+    vq_synth.LayerSpec("pt_d2b3_8x128_i8", N=72, K=640, d=2, b=3, Br=8, Bc=128, int8=True),
+    vq_synth.LayerSpec("pt_d2b6_4x256", N=100, K=11008, d=2, b=6, Br=4, Bc=256, int8=False),
+    vq_synth.LayerSpec("pt_d1b4_8x64", N=40, K=704, d=1, b=4, Br=8, Bc=64, int8=False),
+    vq_synth.LayerSpec("pt_d2b1_1x64_i8", N=33, K=320, d=2, b=1, Br=1, Bc=64, int8=True),
+    vq_synth.LayerSpec("pt_d1b1_2x192", N=34, K=1344, d=1, b=1, Br=2, Bc=192, int8=False),
+    vq_synth.LayerSpec("pt_d2b2_48x64_i8", N=96, K=64, d=2, b=2, Br=48, Bc=64, int8=True),
+]
+
+
+@pytest.mark.parametrize("spec", PAIR_TABLE_CASES, ids=lambda s: s.name)
+def test_pair_table_kernel_formats(spec):
+    # tuned kernel only (no fallback), every batch size class, against the oracle
+    _check_layer(spec, seed=113, batches=(1, 3, 8, 9, 16), impls=[vq.VQ_IMPL_TUNED, vq.VQ_IMPL_AUTO], decode=False)
+
+
+@pytest.mark.parametrize("spec", [
+    vq_synth.LayerSpec("pt_full_d2b5_4x256_i8", N=4096, K=4096, d=2, b=5, Br=4, Bc=256, int8=True),
+    vq_synth.LayerSpec("pt_full_d1b2_1x256_i8", N=14336, K=4096, d=1, b=2, Br=1, Bc=256, int8=True),
+    vq_synth.LayerSpec("pt_full_d2b8_256x256_i8", N=4096, K=14336, d=2, b=8, Br=256, Bc=256, int8=True),
+], ids=lambda s: s.name)
+def test_pair_table_kernel_layer_sizes(spec):
+    """Llama-3-8B-sized layers in the paper's small-block configurations: sampled output rows against the
+    oracle in the launch shapes that full-size layers get (fewer warps per CTA as the row count grows)."""
+    rows = _sample_rows(spec.N, spec.Br, n=128, seed=5)
+    _check_layer(spec, seed=7, batches=(1, 8, 16), impls=[vq.VQ_IMPL_TUNED], decode=False, rows=rows)
+
+
 @pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "llama3_8b", "llama3_8b_int4cb"])
 def test_tuned_kernels_cover_every_benchmark_format(cfg):
     """VQ_IMPL_TUNED never falls back: it must run (not VQ_ERR_UNSUPPORTED) on every layer shape of
