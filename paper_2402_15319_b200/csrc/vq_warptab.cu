@@ -17,8 +17,12 @@
 // them as A fragments to four m16n8k16 tensor-core steps whose B fragments are the activations of the
 // same columns (batch rows 0..7, and 8..15 in a second accumulator when NB == 2); fp32 accumulation.
 // Tables are private to the warp: one table per codebook block row that the 16 rows touch (16 / Br
-// tables, one if Br >= 16), rebuilt whenever the walk enters a new block column.  The warps' partial
-// sums meet in shared memory in a fixed order (bit-identical results run to run).
+// tables, one if Br >= 16), rebuilt whenever the walk enters a new block column.  The index stream
+// reaches the lanes through warp-private shared-memory stages filled with 16-byte asynchronous copies,
+// a chunk of 8 steps (32 * EB contiguous bytes of each of the 16 rows) at a time, kStages chunks deep:
+// HBM sees row segments of 32..256 bytes instead of the 4 * EB bytes a step needs, and the copies of
+// the next chunks run under the look-ups of this one.  Nothing in the loop synchronises beyond the warp.
+// The warps' partial sums meet in shared memory in a fixed order (bit-identical results run to run).
 #include "vq_common.cuh"
 #include "vq_device.cuh"
 
@@ -28,6 +32,15 @@ namespace {
 using namespace dev;
 
 constexpr int kMaxWarps = 8;   // per CTA; three CTAs of that size fit an SM's registers
+constexpr int kChunkSteps = 8;   // steps per staged chunk of the index stream
+constexpr int kStages = 2;
+constexpr int kBuildGroup = 8;   // table words per lane whose loads are in flight together
+// Bytes between the rows of a staged chunk: 32 * EB of indices + 16, an odd number of 16-byte units, so
+// that the eight rows one look-up instruction reads start in different banks.
+__host__ __device__ constexpr int stage_pitch(int eb) { return 32 * eb + 16; }
+__host__ __device__ constexpr int stage_bytes(int eb) { return 16 * stage_pitch(eb); }
+// Alignment of a warp's region: the size of one table (tables start on multiples of their size), 16 at least.
+__host__ __device__ constexpr int region_align(int eb) { return (4 << eb) < 16 ? 16 : (4 << eb); }
 
 struct WarpTabArgs {
   const uint8_t* idx;
@@ -43,63 +56,74 @@ struct WarpTabArgs {
   int blocks_per_row;
   int steps_total, steps_per_warp;
   int tbl_words;                  // words of one warp's tables (tables << EB)
-  int red_off;                    // byte offset of the reduction buffer in shared memory
+  int tbl_bytes;                  // the same in bytes, rounded up to 16
+  int warp_bytes;                 // shared memory of one warp: tables, then kStages chunk stages
+  int red_off;                    // byte offset of the reduction buffer in shared memory (it reuses the warps' regions)
 };
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 __device__ __forceinline__ void fence_acc4(float (&c)[4]) {
   asm volatile("" : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])::"memory");
 }
 
-// Byte address offset (entry * 4) of pair P of a lane's 8 pairs; (lo, hi, top) hold the lane's EB bytes
-// from bit 0 of lo upwards.
+// Shared-memory address of the table word of pair P of a lane's 8 pairs; (lo, hi) hold the lane's EB bytes
+// from bit 0 of lo upwards.  The table starts on a multiple of its size, so base | entry * 4 == base + entry * 4
+// and one logic operation masks the field and merges the base.
 template <int EB, int P>
-__device__ __forceinline__ uint32_t pair_offset(uint32_t lo, uint32_t hi) {
+__device__ __forceinline__ uint32_t pair_address(uint32_t lo, uint32_t hi, uint32_t table) {
   constexpr int SH = P * EB;
   constexpr uint32_t M4 = ((1u << EB) - 1u) << 2;
   if constexpr (SH + EB <= 32) {
-    if constexpr (SH >= 2) return (lo >> (SH - 2)) & M4;
-    else return (lo << (2 - SH)) & M4;
+    if constexpr (SH >= 2) return ((lo >> (SH - 2)) & M4) | table;
+    else return ((lo << (2 - SH)) & M4) | table;
   } else if constexpr (SH >= 32) {
-    if constexpr (SH - 32 >= 2) return (hi >> (SH - 34)) & M4;
-    else return (hi << (34 - SH)) & M4;
+    if constexpr (SH - 32 >= 2) return ((hi >> (SH - 34)) & M4) | table;
+    else return ((hi << (34 - SH)) & M4) | table;
   } else {
-    return __funnelshift_r(lo, hi, SH - 2) & M4;   // SH >= 25 here
+    return (__funnelshift_r(lo, hi, SH - 2) & M4) | table;   // SH >= 25 here
   }
 }
 
-// The EB bytes at byte offset `o` of a row as (lo, hi): aligned 32-bit loads of the words that hold them.
-// Every word read lies inside the row pitch: the last byte needed is o + EB - 1 < row bytes <= pitch,
-// and both are multiples of 4 past the word's start.
+// The EB bytes at byte offset `o` of a staged row as (lo, hi): aligned 32-bit loads of the words that hold
+// them.  Every word read lies inside the row's slot: the last byte needed is o + EB - 1 < 32 * EB.
 template <int EB>
-__device__ __forceinline__ void load_bits(const uint8_t* row, int o, uint32_t& lo, uint32_t& hi) {
+__device__ __forceinline__ void load_bits(uint32_t row_s, int o, uint32_t& lo, uint32_t& hi) {
   const int sh = (o & 3) * 8;
-  const uint32_t* w = reinterpret_cast<const uint32_t*>(row + (o & ~3));
-  const uint32_t w0 = __ldg(w);
-  uint32_t w1 = 0, w2 = 0;
-  if ((o & 3) + EB > 4) w1 = __ldg(w + 1);
+  const uint32_t at = row_s + (o & ~3);
+  uint32_t w0, w1 = 0, w2 = 0;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w0) : "r"(at));
+  if ((o & 3) + EB > 4) asm volatile("ld.shared.b32 %0, [%1+4];" : "=r"(w1) : "r"(at));
   if constexpr (EB == 7) {
-    if ((o & 3) + EB > 8) w2 = __ldg(w + 2);
+    if ((o & 3) + EB > 8) asm volatile("ld.shared.b32 %0, [%1+8];" : "=r"(w2) : "r"(at));
   }
   lo = __funnelshift_r(w0, w1, sh);
   hi = __funnelshift_r(w1, w2, sh);
 }
 
 template <int EB, int NB>
-__global__ void __launch_bounds__(kMaxWarps * 32, 3) warptab_kernel(const WarpTabArgs a) {
+__global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kernel(const WarpTabArgs a) {
   extern __shared__ __align__(16) uint8_t smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int row0 = blockIdx.x * 16;
   const int rA = min(row0 + g, a.N - 1), rB = min(row0 + g + 8, a.N - 1);   // rows past N: computed, not written
   const int brow0 = a.Br >= 16 ? row0 / a.Br : row0 >> a.br_shift;
-  uint32_t* tbl = reinterpret_cast<uint32_t*>(smem) + warp * a.tbl_words;
+  // warp regions start on a multiple of the table size (the host adds that much slack)
+  uint8_t* mine = smem + ((0u - smem_u32(smem)) & static_cast<uint32_t>(region_align(EB) - 1)) + warp * a.warp_bytes;
+  uint32_t* tbl = reinterpret_cast<uint32_t*>(mine);
   uint32_t tA = smem_u32(tbl), tB = tA;
   if (a.Br < 16) {
     tA += static_cast<uint32_t>((rA >> a.br_shift) - brow0) << (EB + 2);
     tB += static_cast<uint32_t>((rB >> a.br_shift) - brow0) << (EB + 2);
   }
-  const uint8_t* rowA = a.idx + rA * a.stride;
-  const uint8_t* rowB = a.idx + rB * a.stride;
+  constexpr int PITCH = stage_pitch(EB);
+  const uint32_t stage_s = smem_u32(mine) + a.tbl_bytes;
 
   float acc[NB][4];
 #pragma unroll
@@ -108,94 +132,169 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 3) warptab_kernel(const WarpTa
     for (int c = 0; c < 4; ++c) acc[nb][c] = 0.f;
 
   // One table word per (table j, pair entry e): the two fp16 weights that the EB index bits stand for.
+  // Offsets into the codebook fit 32 bits (checked on the host).  The loads of kBuildGroup words per lane are
+  // issued together and converted afterwards, so that a build waits for memory once per group, not once
+  // per word.  (Asking L2 for the next block columns' entries at each build, prefetch.global.L2, was
+  // measured and is slower on every shape: 72 against 68 us on 28672 x 8192, 22 against 11 us on 4096 x 4096
+  // with 8-bit indices.)
+  const uint32_t cb_shift = static_cast<uint32_t>(a.b);   // entries per block = 1 << b
   auto build = [&](int col_blk) {
-    for (int i = lane; i < a.tbl_words; i += 32) {
-      const int j = i >> EB, e = i & ((1 << EB) - 1);
-      const int brow = min(brow0 + j, a.block_rows - 1);
-      const long long blk = static_cast<long long>(brow) * a.blocks_per_row + col_blk;
-      long long at0, at1;
-      if (a.d == 2) {
-        at0 = (blk * a.entries + e) * 2;
-        at1 = at0 + 1;
-      } else {
-        at0 = blk * a.entries + (e & (a.entries - 1));
-        at1 = blk * a.entries + (e >> a.b);
+#pragma unroll 1
+    for (int i0 = lane; i0 < a.tbl_words; i0 += 32 * kBuildGroup) {
+      uint32_t raw[kBuildGroup];
+      __half sc[kBuildGroup];
+#pragma unroll
+      for (int k = 0; k < kBuildGroup; ++k) {
+        const int i = i0 + 32 * k;
+        raw[k] = 0u;
+        sc[k] = __ushort_as_half(0);
+        if (i < a.tbl_words) {
+          const uint32_t e = static_cast<uint32_t>(i) & ((1u << EB) - 1u);
+          const uint32_t blk = static_cast<uint32_t>(min(brow0 + (i >> EB), a.block_rows - 1)) * static_cast<uint32_t>(a.blocks_per_row) +
+                               static_cast<uint32_t>(col_blk);
+          if (a.cb_int8) {
+            sc[k] = __ldg(a.scale + blk);
+          }
+          if (a.d == 2) {
+            const uint32_t at = (blk << cb_shift) + e;   // in entries of two values
+            if (a.cb_int8) {
+              const uint16_t* c = static_cast<const uint16_t*>(a.cb) + at;
+              raw[k] = __ldg(c);
+            } else {
+              const uint32_t* c = static_cast<const uint32_t*>(a.cb) + at;
+              raw[k] = __ldg(c);
+            }
+          } else {   // two 1-D entries: the first column's in the low half
+            const uint32_t at0 = (blk << cb_shift) + (e & ((1u << cb_shift) - 1u)), at1 = (blk << cb_shift) + (e >> cb_shift);
+            if (a.cb_int8) {
+              const uint8_t* c = static_cast<const uint8_t*>(a.cb);
+              raw[k] = static_cast<uint32_t>(__ldg(c + at0)) | (static_cast<uint32_t>(__ldg(c + at1)) << 8);
+            } else {
+              const uint16_t* c = static_cast<const uint16_t*>(a.cb);
+              raw[k] = static_cast<uint32_t>(__ldg(c + at0)) | (static_cast<uint32_t>(__ldg(c + at1)) << 16);
+            }
+          }
+        }
       }
-      __half h0, h1;
-      if (a.cb_int8) {
-        const float sc = __half2float(__ldg(a.scale + blk));
-        const int8_t* c = static_cast<const int8_t*>(a.cb);
-        h0 = __float2half_rn(sc * static_cast<float>(__ldg(c + at0)));   // exact product, one rounding
-        h1 = __float2half_rn(sc * static_cast<float>(__ldg(c + at1)));
-      } else {
-        const __half* c = static_cast<const __half*>(a.cb);
-        h0 = __ldg(c + at0);
-        h1 = __ldg(c + at1);
+#pragma unroll
+      for (int k = 0; k < kBuildGroup; ++k) {
+        const int i = i0 + 32 * k;
+        if (i < a.tbl_words) {
+          uint32_t word = raw[k];
+          if (a.cb_int8) {   // exact products of the block scale and the 8-bit entries, one rounding each
+            const float f = __half2float(sc[k]);
+            const __half2 hv = __floats2half2_rn(f * static_cast<float>(static_cast<int8_t>(raw[k] & 0xffu)),
+                                                 f * static_cast<float>(static_cast<int8_t>((raw[k] >> 8) & 0xffu)));
+            word = *reinterpret_cast<const uint32_t*>(&hv);
+          }
+          tbl[i] = word;
+        }
       }
-      tbl[i] = static_cast<uint32_t>(__half_as_ushort(h0)) | (static_cast<uint32_t>(__half_as_ushort(h1)) << 16);
     }
   };
 
-  constexpr int U = NB == 1 ? 4 : 2;   // steps whose index words and activations are fetched ahead
+  // Chunk c of this warp (steps s_begin + 8c ..) into stage c % kStages: 2 * EB pieces of 16 bytes per row,
+  // EB pieces per lane.  Pieces that start past the row pitch (last chunk of a row) are left out; the
+  // steps that would read them lie past K and are never computed.  One commit per call, even if empty.
   const int s_begin = warp * a.steps_per_warp;
   const int s_end = min(a.steps_total, s_begin + a.steps_per_warp);
-  int until_rebuild = 0;   // steps left in the current codebook block column
-  for (int s0 = s_begin; s0 < s_end; s0 += U) {
-    uint32_t lo[U][2], hi[U][2];
-    uint4 xv[U][NB][2];
+  const int n_chunks = (s_end - s_begin + kChunkSteps - 1) / kChunkSteps;
+  // lane = 2 * row + y copies pieces y, y + 2, y + 4, ... of its row: a lane pair moves 32 contiguous bytes
+  const int fr = lane >> 1, fy = lane & 1;
+  const int off0 = s_begin * (4 * EB) + fy * 16;   // byte offset inside the row of this lane's first piece of chunk 0
+  const uint8_t* src0 = a.idx + min(row0 + fr, a.N - 1) * a.stride + off0;
+  const uint32_t dst0 = stage_s + fr * PITCH + fy * 16;
+  const int row_bytes = static_cast<int>(a.stride);
+  auto fetch = [&](int c) {
+    if (c < n_chunks) {
+      const int adv = c * (kChunkSteps * 4 * EB);
+      const uint32_t dst = dst0 + (c % kStages) * stage_bytes(EB);
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int s = min(s0 + u, s_end - 1);   // (steps past the range are loaded again, not used)
-      const int o = (s * 4 + t) * EB;
-      load_bits<EB>(rowA, o, lo[u][0], hi[u][0]);
-      load_bits<EB>(rowB, o, lo[u][1], hi[u][1]);
+      for (int q = 0; q < EB; ++q)
+        if (off0 + adv + 32 * q < row_bytes) cp_async16(dst + 32 * q, src0 + adv + 32 * q);
+    }
+    cp_async_commit();
+  };
+
+  // Activations of one step: columns 16t .. 16t+15 of batch row g (+ 8 for the second accumulator).  Lanes
+  // whose batch row does not exist read the last row instead: their accumulator columns are never written.
+  const __half* xp[NB];
+#pragma unroll
+  for (int nb = 0; nb < NB; ++nb)
+    xp[nb] = a.X + static_cast<long long>(min(nb * 8 + g, a.batch - 1)) * a.K + s_begin * 64 + t * 16;
+  uint4 xn[NB][2];   // the next step's activations, fetched one step ahead
+#pragma unroll
+  for (int nb = 0; nb < NB; ++nb) {
+    xn[nb][0] = ldg128_nc(xp[nb]);
+    xn[nb][1] = ldg128_nc(xp[nb] + 8);
+  }
+
+#pragma unroll
+  for (int c = 0; c < kStages - 1; ++c) fetch(c);
+  // the first tables, while the first chunk is on its way
+  int until_rebuild;   // steps left in the current codebook block column
+  {
+    const int col_blk = s_begin / a.bsteps;
+    until_rebuild = a.bsteps - (s_begin - col_blk * a.bsteps);
+    build(col_blk);
+    __syncwarp();
+    fence_value(tA);
+    fence_value(tB);
+  }
+  for (int c = 0; c < n_chunks; ++c) {
+    cp_async_wait<kStages - 2>();   // chunk c has landed (this lane's pieces; the warp barrier covers the others')
+    __syncwarp();                   // ... and every lane is done reading the stage that chunk c + kStages - 1 overwrites
+    fetch(c + kStages - 1);
+    const uint32_t rowA_s = stage_s + (c % kStages) * stage_bytes(EB) + g * PITCH;
+    const uint32_t rowB_s = rowA_s + 8 * PITCH;
+    const int sc0 = s_begin + c * kChunkSteps;
+    const int nst = min(kChunkSteps, s_end - sc0);
+#pragma unroll 2
+    for (int u = 0; u < nst; ++u) {
+      const int s = sc0 + u;
+      if (until_rebuild == 0) {
+        const int col_blk = s / a.bsteps;
+        until_rebuild = a.bsteps - (s - col_blk * a.bsteps);
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) fence_acc4(acc[nb]);   // the gathers of the old tables are done
+        __syncwarp();
+        build(col_blk);
+        __syncwarp();
+        fence_value(tA);
+        fence_value(tB);
+      }
+      --until_rebuild;
+      uint4 x[NB][2];
 #pragma unroll
       for (int nb = 0; nb < NB; ++nb) {
-        const int m = nb * 8 + g;
-        if (m < a.batch) {
-          const __half* x = a.X + static_cast<long long>(m) * a.K + s * 64 + t * 16;
-          xv[u][nb][0] = ldg128_nc(x);
-          xv[u][nb][1] = ldg128_nc(x + 8);
-        } else {
-          xv[u][nb][0] = make_uint4(0u, 0u, 0u, 0u);
-          xv[u][nb][1] = make_uint4(0u, 0u, 0u, 0u);
-        }
+        x[nb][0] = xn[nb][0];
+        x[nb][1] = xn[nb][1];
+        if (s + 1 < s_end) xp[nb] += 64;   // (the warp's last step is read twice)
+        xn[nb][0] = ldg128_nc(xp[nb]);
+        xn[nb][1] = ldg128_nc(xp[nb] + 8);
       }
-    }
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int s = s0 + u;
-      if (s < s_end) {
-        if (until_rebuild == 0) {
-          const int col_blk = s / a.bsteps;
-          until_rebuild = a.bsteps - (s - col_blk * a.bsteps);
-#pragma unroll
-          for (int nb = 0; nb < NB; ++nb) fence_acc4(acc[nb]);   // the gathers of the old tables are done
-          __syncwarp();
-          build(col_blk);
-          __syncwarp();
-          fence_value(tA);
-          fence_value(tB);
-        }
-        --until_rebuild;
-        uint32_t wa[8], wb[8];
-#define VQ_WT_PAIR(P)                                                     \
-  wa[P] = lds32(tA + pair_offset<EB, P>(lo[u][0], hi[u][0]));            \
-  wb[P] = lds32(tB + pair_offset<EB, P>(lo[u][1], hi[u][1]));
-        VQ_WT_PAIR(0) VQ_WT_PAIR(1) VQ_WT_PAIR(2) VQ_WT_PAIR(3)
-        VQ_WT_PAIR(4) VQ_WT_PAIR(5) VQ_WT_PAIR(6) VQ_WT_PAIR(7)
+      const int o = (u * 4 + t) * EB;
+      uint32_t loA, hiA, loB, hiB;
+      load_bits<EB>(rowA_s, o, loA, hiA);
+      load_bits<EB>(rowB_s, o, loB, hiB);
+      uint32_t wa[8], wb[8];
+#define VQ_WT_PAIR(P)                                    \
+  wa[P] = lds32(pair_address<EB, P>(loA, hiA, tA));     \
+  wb[P] = lds32(pair_address<EB, P>(loB, hiB, tB));
+      VQ_WT_PAIR(0) VQ_WT_PAIR(1) VQ_WT_PAIR(2) VQ_WT_PAIR(3)
+      VQ_WT_PAIR(4) VQ_WT_PAIR(5) VQ_WT_PAIR(6) VQ_WT_PAIR(7)
 #undef VQ_WT_PAIR
 #pragma unroll
-        for (int nb = 0; nb < NB; ++nb) {
-          const uint4 x0 = xv[u][nb][0], x1 = xv[u][nb][1];
-          mma16816(acc[nb], wa[0], wb[0], wa[1], wb[1], x0.x, x0.y);
-          mma16816(acc[nb], wa[2], wb[2], wa[3], wb[3], x0.z, x0.w);
-          mma16816(acc[nb], wa[4], wb[4], wa[5], wb[5], x1.x, x1.y);
-          mma16816(acc[nb], wa[6], wb[6], wa[7], wb[7], x1.z, x1.w);
-        }
+      for (int nb = 0; nb < NB; ++nb) {
+        mma16816(acc[nb], wa[0], wb[0], wa[1], wb[1], x[nb][0].x, x[nb][0].y);
+        mma16816(acc[nb], wa[2], wb[2], wa[3], wb[3], x[nb][0].z, x[nb][0].w);
+        mma16816(acc[nb], wa[4], wb[4], wa[5], wb[5], x[nb][1].x, x[nb][1].y);
+        mma16816(acc[nb], wa[6], wb[6], wa[7], wb[7], x[nb][1].z, x[nb][1].w);
       }
     }
   }
+  cp_async_wait<0>();
+  __syncthreads();   // the reduction buffer lies over the warps' tables and stages
 
   // K parts of the warps meet in shared memory; thread i then owns output (batch row i / 16, row i % 16).
   float* red = reinterpret_cast<float*>(smem + a.red_off);
@@ -224,11 +323,51 @@ int pair_bits(const Geometry& g) {
 
 int tables_per_tile(const Geometry& g) { return g.Br >= 16 ? 1 : 16 / g.Br; }
 
-template <int EB>
-vq_status launch_eb(const WarpTabArgs& a, int nb, unsigned grid, unsigned threads, size_t smem_bytes, cudaStream_t s) {
-  if (nb == 1) warptab_kernel<EB, 1><<<grid, threads, smem_bytes, s>>>(a);
-  else warptab_kernel<EB, 2><<<grid, threads, smem_bytes, s>>>(a);
+constexpr size_t kSmemLimit = 100 * 1024;   // dynamic shared memory a CTA may ask for (fewer warps per CTA beyond it)
+constexpr size_t kSmemPerSm = 228 * 1024;   // shared memory of an SM; every resident CTA also costs 1 KB of it
+
+// Picks the K split, finishes the arguments and launches.  The dynamic shared-memory limit is raised and the
+// kernel's register count read once per device and instantiation.
+template <int EB, int NB>
+vq_status launch_one(WarpTabArgs a, long long tiles, int sms, cudaStream_t s) {
+  static int regs_of[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VQ_ERR_CUDA;
+  int regs = __atomic_load_n(&regs_of[dev], __ATOMIC_ACQUIRE);
+  if (!regs) {
+    cudaFuncAttributes fa;
+    if (cudaFuncSetAttribute(warptab_kernel<EB, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemLimit)) !=
+            cudaSuccess ||
+        cudaFuncGetAttributes(&fa, warptab_kernel<EB, NB>) != cudaSuccess || fa.numRegs < 1)
+      return VQ_ERR_CUDA;
+    regs = fa.numRegs;
+    __atomic_store_n(&regs_of[dev], regs, __ATOMIC_RELEASE);
+  }
+  // CTAs of w warps that one SM holds: registers (allocated per warp in units of 256), shared memory, 32 CTAs
+  const int warps_by_regs = 65536 / ((regs * 32 + 255) / 256 * 256);
+  auto resident = [&](int w) {
+    long long c = warps_by_regs / w;
+    c = c < 32 ? c : 32;
+    const long long by_smem = static_cast<long long>(kSmemPerSm / (static_cast<size_t>(w) * a.warp_bytes + region_align(EB) + 1024));
+    return c < by_smem ? c : by_smem;
+  };
+  // K split: the most warps per CTA (at most kMaxWarps, at most one per chunk of the row) with which every
+  // CTA of the grid is resident at once.  A grid one CTA larger than that costs a second pass over the
+  // device, which weighs more than the longer walk of fewer, longer-running warps.
+  const int chunks_total = (a.steps_total + kChunkSteps - 1) / kChunkSteps;
+  int wk = kMaxWarps < chunks_total ? kMaxWarps : chunks_total;
+  while (wk > 1 && (static_cast<size_t>(wk) * a.warp_bytes + region_align(EB) > kSmemLimit || tiles > resident(wk) * sms)) --wk;
+  a.steps_per_warp = ((a.steps_total + wk - 1) / wk + kChunkSteps - 1) / kChunkSteps * kChunkSteps;   // whole chunks
+  wk = (a.steps_total + a.steps_per_warp - 1) / a.steps_per_warp;   // no warp without work
+  const size_t smem_bytes = static_cast<size_t>(wk) * a.warp_bytes + region_align(EB);
+  if (smem_bytes > kSmemLimit) return VQ_ERR_UNSUPPORTED;
+  warptab_kernel<EB, NB><<<static_cast<unsigned>(tiles), static_cast<unsigned>(wk) * 32u, smem_bytes, s>>>(a);
   return check_launch();
+}
+
+template <int EB>
+vq_status launch_eb(const WarpTabArgs& a, int nb, long long tiles, int sms, cudaStream_t s) {
+  return nb == 1 ? launch_one<EB, 1>(a, tiles, sms, s) : launch_one<EB, 2>(a, tiles, sms, s);
 }
 
 }  // namespace
@@ -239,6 +378,9 @@ bool warptab_covers(const Geometry& g) {
   if (eb < 1 || eb > 8) return false;
   if (g.K % 64 || g.Bc % 64) return false;
   if (!(g.Br == 1 || g.Br == 2 || g.Br == 4 || g.Br == 8 || g.Br % 16 == 0)) return false;
+  // the kernel addresses codebook entries and index bytes of a row with 32-bit offsets
+  const long long cb_values = static_cast<long long>(g.N / g.Br) * g.blocks_per_row * g.entries * g.d;
+  if (cb_values >= (1LL << 31) || g.stride >= (1LL << 30)) return false;
   return (tables_per_tile(g) << eb) <= 1024;
 }
 
@@ -268,31 +410,23 @@ vq_status launch_gemm_warptab(const Geometry& g, const LayerPtrs& p, const __hal
   a.blocks_per_row = g.blocks_per_row;
   a.steps_total = g.K / 64;
   a.tbl_words = tables_per_tile(g) << eb;
-  // K split: enough warps to fill the device (about 32 per SM), at most kMaxWarps per CTA, each at least one step
-  // and, where the layer is large enough for that, at least one whole codebook block column
+  // per warp: tables + chunk stages; the reduction buffer (nb * 512 bytes per warp) reuses that space
+  a.tbl_bytes = (a.tbl_words * 4 + 15) / 16 * 16;
+  const int tbl_align = region_align(eb);
+  a.warp_bytes = (a.tbl_bytes + kStages * stage_bytes(eb) + tbl_align - 1) / tbl_align * tbl_align;
+  a.red_off = 0;
   int sms = 0;
   if (device_sms(&sms) != VQ_OK) return VQ_ERR_CUDA;
   const long long tiles = (static_cast<long long>(g.N) + 15) / 16;
-  int wk = kMaxWarps;
-  while (wk > 1 && tiles * wk > 32LL * sms && tiles * (wk / 2) >= 24LL * sms) wk /= 2;
-  if (wk > a.steps_total) wk = a.steps_total;
-  auto smem_for = [&](int w) { return static_cast<size_t>(w) * (a.tbl_words * 4 + nb * 4 * 32 * 4); };
-  while (wk > 1 && smem_for(wk) > 48 * 1024) --wk;
-  a.steps_per_warp = (a.steps_total + wk - 1) / wk;
-  wk = (a.steps_total + a.steps_per_warp - 1) / a.steps_per_warp;   // no warp without work
-  a.red_off = wk * a.tbl_words * 4;
-  const size_t smem_bytes = smem_for(wk);
-  if (smem_bytes > 48 * 1024) return VQ_ERR_UNSUPPORTED;
-  const unsigned grid = static_cast<unsigned>(tiles), threads = static_cast<unsigned>(wk) * 32u;
   switch (eb) {
-    case 1: return launch_eb<1>(a, nb, grid, threads, smem_bytes, s);
-    case 2: return launch_eb<2>(a, nb, grid, threads, smem_bytes, s);
-    case 3: return launch_eb<3>(a, nb, grid, threads, smem_bytes, s);
-    case 4: return launch_eb<4>(a, nb, grid, threads, smem_bytes, s);
-    case 5: return launch_eb<5>(a, nb, grid, threads, smem_bytes, s);
-    case 6: return launch_eb<6>(a, nb, grid, threads, smem_bytes, s);
-    case 7: return launch_eb<7>(a, nb, grid, threads, smem_bytes, s);
-    default: return launch_eb<8>(a, nb, grid, threads, smem_bytes, s);
+    case 1: return launch_eb<1>(a, nb, tiles, sms, s);
+    case 2: return launch_eb<2>(a, nb, tiles, sms, s);
+    case 3: return launch_eb<3>(a, nb, tiles, sms, s);
+    case 4: return launch_eb<4>(a, nb, tiles, sms, s);
+    case 5: return launch_eb<5>(a, nb, tiles, sms, s);
+    case 6: return launch_eb<6>(a, nb, tiles, sms, s);
+    case 7: return launch_eb<7>(a, nb, tiles, sms, s);
+    default: return launch_eb<8>(a, nb, tiles, sms, s);
   }
 }
 
