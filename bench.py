@@ -413,7 +413,8 @@ KERNEL_OF = {"cfg1": "rowcb_kernel<LdsTbl<false>,1>", "cfg2": "rowcb_kernel<Prmt
              "cfg3": "blockcb_kernel<2,6,1> (q/k/v and gate/up as grouped launches)",
              "cfg4": "blockcb_kernel<4,8,NB>", "cfg5": "stream_kernel<RowD2B4<int8>,NB,R,CW,CPS>",
              "llama3_8b": "blockcb_kernel<2,6,NB,warp-private tables>",
-             "llama3_8b_int4cb": "blockcb_kernel<2,6,NB,warp-private tables, int4 codebooks>"}
+             "llama3_8b_int4cb": "blockcb_kernel<2,6,NB,warp-private tables, int4 codebooks>",
+             "llama3_8b_d2b5_4x256": "warptab_kernel<5,NB>"}
 
 
 def max_over_ranks(value: float, dist=None, device=None) -> float:

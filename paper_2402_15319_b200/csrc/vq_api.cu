@@ -182,10 +182,13 @@ vq_status vq_gemm_small_batch_impl(const vq_format* fmt, const void* d_idx, cons
 // formats (their K-split meets in distributed shared memory: lowest latency on the small layers those
 // formats come with), 1 = the persistent kernel (per-row formats: q/k/v of the 70B-shaped set in one
 // launch 11.4 us against 19.5 us for three launches at batch 1, 20.3 against 37.4 us at batch 8),
-// 0 = member by member.
+// 3 = the pair-table kernel (small codebook blocks; index widths other than 4 bits, which the row kernels
+// or the persistent kernel take: q/k/v of the Llama-3-8B-shaped set with 5-bit indices and 4 x 256 blocks in
+// one launch instead of three), 0 = member by member.
 static int group_family(const Geometry& g, int) {
   if (blockcb_covers(g)) return 2;
   if (g.cb_int4) return 0;
+  if (g.b != 4 && !stream_covers(g) && warptab_covers(g)) return 3;
   return 1;
 }
 
@@ -193,6 +196,7 @@ int vq_grouped_kernel_launches(const vq_format* fmt, int n_members, int batch) {
   Geometry g;
   if (make_geometry(fmt, &g) != VQ_OK || n_members < 1 || n_members > VQ_MAX_GROUP || batch < 1 || batch > 16) return 0;
   if (n_members > 1 && blockcb_covers(g) && group_family(g, batch) == 2) return 1;
+  if (n_members > 1 && group_family(g, batch) == 3) return 1;
   return (n_members > 1 && group_family(g, batch) == 1 && stream_covers(g)) ? 1 : n_members;
 }
 
@@ -238,6 +242,7 @@ vq_status vq_gemm_small_batch_grouped(const vq_format* fmt, const vq_group_membe
 #ifdef VQ_TUNING
     if (getenv("VQ_GROUP_FAMILY")) fam = atoi(getenv("VQ_GROUP_FAMILY"));
 #endif
+    if (fam == 3) st = launch_gemm_warptab_group(call, s);
     if (fam == 2) st = launch_gemm_blockcb_group(call, s);
     if (fam == 1 || (fam == 2 && st == VQ_ERR_UNSUPPORTED)) st = launch_gemm_stream(call, s);
   }

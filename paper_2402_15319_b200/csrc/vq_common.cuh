@@ -78,6 +78,8 @@ vq_status launch_gemm_rowcb(const Geometry& g, const LayerPtrs& p, const __half*
 // any width, 1-D indices of up to 4 bits, fp16 / int8 codebooks, K and block columns multiples of 64.
 vq_status launch_gemm_warptab(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
                               cudaStream_t s);
+// ... over several layers of one format and K in one launch (rows per layer in call.N; call.ws is not used)
+vq_status launch_gemm_warptab_group(const StreamCall& call, cudaStream_t s);
 bool warptab_covers(const Geometry& g);
 vq_status launch_int4g128_rowcb(int N, int K, const uint8_t* q, const __half* scale, const __half* X, __half* Y, int batch,
                                 cudaStream_t s);

@@ -43,15 +43,19 @@ __host__ __device__ constexpr int stage_bytes(int eb) { return 16 * stage_pitch(
 __host__ __device__ constexpr int region_align(int eb) { return (4 << eb) < 16 ? 16 : (4 << eb); }
 
 struct WarpTabArgs {
-  const uint8_t* idx;
-  const void* cb;
-  const __half* scale;
+  // the layers of the call (same format and K, one activation tensor); tile0 = first 16-row tile of each
+  const uint8_t* idx[kMaxSegments];
+  const void* cb[kMaxSegments];
+  const __half* scale[kMaxSegments];
+  __half* Y[kMaxSegments];
+  int N[kMaxSegments];
+  int tile0[kMaxSegments];
+  int n_seg;
   const __half* X;
-  __half* Y;
   long long stride;
-  int N, K, batch;
+  int K, batch;
   int d, b, entries, cb_int8;
-  int Br, br_shift, block_rows;   // br_shift: log2(Br) when Br < 16
+  int Br, br_shift;               // br_shift: log2(Br) when Br < 16
   int bsteps;                     // 64-column steps per codebook block (Bc / 64)
   int blocks_per_row;
   int steps_total, steps_per_warp;
@@ -111,9 +115,27 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
   extern __shared__ __align__(16) uint8_t smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
-  const int row0 = blockIdx.x * 16;
-  const int rA = min(row0 + g, a.N - 1), rB = min(row0 + g + 8, a.N - 1);   // rows past N: computed, not written
+  // the layer this CTA's tile belongs to (selects, not indexed loads: the arguments stay in constant memory)
+  int seg = 0;
+#pragma unroll
+  for (int i = 1; i < kMaxSegments; ++i)
+    if (i < a.n_seg && static_cast<int>(blockIdx.x) >= a.tile0[i]) seg = i;
+  auto pick = [&](const auto& arr) {
+    auto v = arr[0];
+#pragma unroll
+    for (int i = 1; i < kMaxSegments; ++i)
+      if (seg == i) v = arr[i];
+    return v;
+  };
+  const uint8_t* const seg_idx = pick(a.idx);
+  const void* const seg_cb = pick(a.cb);
+  const __half* const seg_scale = pick(a.scale);
+  __half* const seg_Y = pick(a.Y);
+  const int seg_N = pick(a.N);
+  const int row0 = (static_cast<int>(blockIdx.x) - pick(a.tile0)) * 16;
+  const int rA = min(row0 + g, seg_N - 1), rB = min(row0 + g + 8, seg_N - 1);   // rows past N: computed, not written
   const int brow0 = a.Br >= 16 ? row0 / a.Br : row0 >> a.br_shift;
+  const int block_rows = a.Br >= 16 ? seg_N / a.Br : seg_N >> a.br_shift;
   // warp regions start on a multiple of the table size (the host adds that much slack)
   uint8_t* mine = smem + ((0u - smem_u32(smem)) & static_cast<uint32_t>(region_align(EB) - 1)) + warp * a.warp_bytes;
   uint32_t* tbl = reinterpret_cast<uint32_t*>(mine);
@@ -150,27 +172,27 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
         sc[k] = __ushort_as_half(0);
         if (i < a.tbl_words) {
           const uint32_t e = static_cast<uint32_t>(i) & ((1u << EB) - 1u);
-          const uint32_t blk = static_cast<uint32_t>(min(brow0 + (i >> EB), a.block_rows - 1)) * static_cast<uint32_t>(a.blocks_per_row) +
+          const uint32_t blk = static_cast<uint32_t>(min(brow0 + (i >> EB), block_rows - 1)) * static_cast<uint32_t>(a.blocks_per_row) +
                                static_cast<uint32_t>(col_blk);
           if (a.cb_int8) {
-            sc[k] = __ldg(a.scale + blk);
+            sc[k] = __ldg(seg_scale + blk);
           }
           if (a.d == 2) {
             const uint32_t at = (blk << cb_shift) + e;   // in entries of two values
             if (a.cb_int8) {
-              const uint16_t* c = static_cast<const uint16_t*>(a.cb) + at;
+              const uint16_t* c = static_cast<const uint16_t*>(seg_cb) + at;
               raw[k] = __ldg(c);
             } else {
-              const uint32_t* c = static_cast<const uint32_t*>(a.cb) + at;
+              const uint32_t* c = static_cast<const uint32_t*>(seg_cb) + at;
               raw[k] = __ldg(c);
             }
           } else {   // two 1-D entries: the first column's in the low half
             const uint32_t at0 = (blk << cb_shift) + (e & ((1u << cb_shift) - 1u)), at1 = (blk << cb_shift) + (e >> cb_shift);
             if (a.cb_int8) {
-              const uint8_t* c = static_cast<const uint8_t*>(a.cb);
+              const uint8_t* c = static_cast<const uint8_t*>(seg_cb);
               raw[k] = static_cast<uint32_t>(__ldg(c + at0)) | (static_cast<uint32_t>(__ldg(c + at1)) << 8);
             } else {
-              const uint16_t* c = static_cast<const uint16_t*>(a.cb);
+              const uint16_t* c = static_cast<const uint16_t*>(seg_cb);
               raw[k] = static_cast<uint32_t>(__ldg(c + at0)) | (static_cast<uint32_t>(__ldg(c + at1)) << 16);
             }
           }
@@ -202,7 +224,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
   // lane = 2 * row + y copies pieces y, y + 2, y + 4, ... of its row: a lane pair moves 32 contiguous bytes
   const int fr = lane >> 1, fy = lane & 1;
   const int off0 = s_begin * (4 * EB) + fy * 16;   // byte offset inside the row of this lane's first piece of chunk 0
-  const uint8_t* src0 = a.idx + min(row0 + fr, a.N - 1) * a.stride + off0;
+  const uint8_t* src0 = seg_idx + min(row0 + fr, seg_N - 1) * a.stride + off0;
   const uint32_t dst0 = stage_s + fr * PITCH + fy * 16;
   const int row_bytes = static_cast<int>(a.stride);
   auto fetch = [&](int c) {
@@ -215,6 +237,19 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
     }
     cp_async_commit();
   };
+
+#pragma unroll
+  for (int c = 0; c < kStages - 1; ++c) fetch(c);
+  // the first tables, while the first chunk is on its way
+  int until_rebuild;   // steps left in the current codebook block column
+  {
+    const int col_blk = s_begin / a.bsteps;
+    until_rebuild = a.bsteps - (s_begin - col_blk * a.bsteps);
+    build(col_blk);
+    __syncwarp();
+    fence_value(tA);
+    fence_value(tB);
+  }
 
   // Activations of one step: columns 16t .. 16t+15 of batch row g (+ 8 for the second accumulator).  Lanes
   // whose batch row does not exist read the last row instead: their accumulator columns are never written.
@@ -229,18 +264,6 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
     xn[nb][1] = ldg128_nc(xp[nb] + 8);
   }
 
-#pragma unroll
-  for (int c = 0; c < kStages - 1; ++c) fetch(c);
-  // the first tables, while the first chunk is on its way
-  int until_rebuild;   // steps left in the current codebook block column
-  {
-    const int col_blk = s_begin / a.bsteps;
-    until_rebuild = a.bsteps - (s_begin - col_blk * a.bsteps);
-    build(col_blk);
-    __syncwarp();
-    fence_value(tA);
-    fence_value(tB);
-  }
   for (int c = 0; c < n_chunks; ++c) {
     cp_async_wait<kStages - 2>();   // chunk c has landed (this lane's pieces; the warp barrier covers the others')
     __syncwarp();                   // ... and every lane is done reading the stage that chunk c + kStages - 1 overwrites
@@ -311,7 +334,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
     const int src_lane = (r & 7) * 4 + (mm >> 1);
     float sum = 0.f;
     for (int w = 0; w < warps; ++w) sum += red[(w * NB * 4 + nb * 4 + c) * 32 + src_lane];
-    if (m < a.batch && row0 + r < a.N) a.Y[static_cast<long long>(m) * a.N + row0 + r] = __float2half_rn(sum);
+    if (m < a.batch && row0 + r < seg_N) seg_Y[static_cast<long long>(m) * seg_N + row0 + r] = __float2half_rn(sum);
   }
 }
 
@@ -361,6 +384,9 @@ vq_status launch_one(WarpTabArgs a, long long tiles, int sms, cudaStream_t s) {
   wk = (a.steps_total + a.steps_per_warp - 1) / a.steps_per_warp;   // no warp without work
   const size_t smem_bytes = static_cast<size_t>(wk) * a.warp_bytes + region_align(EB);
   if (smem_bytes > kSmemLimit) return VQ_ERR_UNSUPPORTED;
+  // A plain launch, in stream order.  (With programmatic dependent launch the next launch's CTAs take the
+  // SM slots this grid leaves free and stay where they land: two such layers back to back then run with
+  // 3 CTAs on some SMs and 1 on others; measured 31.5 against 23.2 us on 4096 x 14336.)
   warptab_kernel<EB, NB><<<static_cast<unsigned>(tiles), static_cast<unsigned>(wk) * 32u, smem_bytes, s>>>(a);
   return check_launch();
 }
@@ -378,34 +404,41 @@ bool warptab_covers(const Geometry& g) {
   if (eb < 1 || eb > 8) return false;
   if (g.K % 64 || g.Bc % 64) return false;
   if (!(g.Br == 1 || g.Br == 2 || g.Br == 4 || g.Br == 8 || g.Br % 16 == 0)) return false;
-  // the kernel addresses codebook entries and index bytes of a row with 32-bit offsets
-  const long long cb_values = static_cast<long long>(g.N / g.Br) * g.blocks_per_row * g.entries * g.d;
-  if (cb_values >= (1LL << 31) || g.stride >= (1LL << 30)) return false;
+  if (g.stride >= (1LL << 30)) return false;   // byte offsets inside a row are 32-bit in the kernel
   return (tables_per_tile(g) << eb) <= 1024;
 }
 
-vq_status launch_gemm_warptab(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
-                              cudaStream_t s) {
-  if (!warptab_covers(g)) return VQ_ERR_UNSUPPORTED;
+vq_status launch_gemm_warptab_group(const StreamCall& call, cudaStream_t s) {
+  const Geometry& g = call.g;
+  if (!warptab_covers(g) || call.n_seg < 1 || call.n_seg > kMaxSegments) return VQ_ERR_UNSUPPORTED;
   const int eb = pair_bits(g);
-  const int nb = batch <= 8 ? 1 : 2;
+  const int nb = call.batch <= 8 ? 1 : 2;
   WarpTabArgs a = {};
-  a.idx = p.idx;
-  a.cb = p.cb;
-  a.scale = p.scale;
-  a.X = X;
-  a.Y = Y;
+  long long tiles = 0;
+  for (int i = 0; i < call.n_seg; ++i) {
+    if (call.N[i] <= 0 || call.N[i] % g.Br) return VQ_ERR_UNSUPPORTED;
+    // the kernel addresses codebook entries with 32-bit offsets
+    if (static_cast<long long>(call.N[i] / g.Br) * g.blocks_per_row * g.entries * g.d >= (1LL << 31)) return VQ_ERR_UNSUPPORTED;
+    a.idx[i] = call.idx[i];
+    a.cb[i] = call.cb[i];
+    a.scale[i] = call.scale[i];
+    a.Y[i] = call.Y[i];
+    a.N[i] = call.N[i];
+    a.tile0[i] = static_cast<int>(tiles);
+    tiles += (call.N[i] + 15) / 16;
+  }
+  if (tiles >= (1LL << 31)) return VQ_ERR_UNSUPPORTED;
+  a.n_seg = call.n_seg;
+  a.X = call.X;
   a.stride = g.stride;
-  a.N = g.N;
   a.K = g.K;
-  a.batch = batch;
+  a.batch = call.batch;
   a.d = g.d;
   a.b = g.b;
   a.entries = g.entries;
   a.cb_int8 = g.cb_int8;
   a.Br = g.Br;
   a.br_shift = g.Br == 1 ? 0 : g.Br == 2 ? 1 : g.Br == 4 ? 2 : 3;
-  a.block_rows = g.N / g.Br;
   a.bsteps = g.Bc / 64;
   a.blocks_per_row = g.blocks_per_row;
   a.steps_total = g.K / 64;
@@ -417,7 +450,6 @@ vq_status launch_gemm_warptab(const Geometry& g, const LayerPtrs& p, const __hal
   a.red_off = 0;
   int sms = 0;
   if (device_sms(&sms) != VQ_OK) return VQ_ERR_CUDA;
-  const long long tiles = (static_cast<long long>(g.N) + 15) / 16;
   switch (eb) {
     case 1: return launch_eb<1>(a, nb, tiles, sms, s);
     case 2: return launch_eb<2>(a, nb, tiles, sms, s);
@@ -428,6 +460,21 @@ vq_status launch_gemm_warptab(const Geometry& g, const LayerPtrs& p, const __hal
     case 7: return launch_eb<7>(a, nb, tiles, sms, s);
     default: return launch_eb<8>(a, nb, tiles, sms, s);
   }
+}
+
+vq_status launch_gemm_warptab(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
+                              cudaStream_t s) {
+  StreamCall call = {};
+  call.g = g;
+  call.n_seg = 1;
+  call.idx[0] = p.idx;
+  call.cb[0] = p.cb;
+  call.scale[0] = p.scale;
+  call.Y[0] = Y;
+  call.N[0] = g.N;
+  call.X = X;
+  call.batch = batch;
+  return launch_gemm_warptab_group(call, s);
 }
 
 }  // namespace vq

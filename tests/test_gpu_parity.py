@@ -160,6 +160,10 @@ GROUPS = [
     (vq_synth.LayerSpec("g_d4b8", N=0, K=1024, d=4, b=8, Br=256, Bc=512, int8=False), [256, 512]),
     (vq_synth.LayerSpec("g_i4cb", N=0, K=1024, d=2, b=6, Br=32, Bc=128, int8=2), [256, 128]),
     (vq_synth.LayerSpec("g_generic", N=0, K=312, d=1, b=5, Br=1, Bc=156, int8=False), [37, 5]),
+    # the pair-table kernel over several layers in one launch: ragged member heights (row tails inside the group)
+    (vq_synth.LayerSpec("g_pt_d2b5", N=0, K=1280, d=2, b=5, Br=4, Bc=256, int8=True), [212, 64, 36, 100]),
+    (vq_synth.LayerSpec("g_pt_d1b2", N=0, K=1024, d=1, b=2, Br=1, Bc=256, int8=True), [33, 200]),
+    (vq_synth.LayerSpec("g_pt_d2b8", N=0, K=768, d=2, b=8, Br=256, Bc=256, int8=False), [256, 512]),
 ]
 
 
@@ -235,7 +239,7 @@ def test_pair_table_kernel_layer_sizes(spec):
     _check_layer(spec, seed=7, batches=(1, 8, 16), impls=[vq.VQ_IMPL_TUNED], decode=False, rows=rows)
 
 
-@pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "llama3_8b", "llama3_8b_int4cb"])
+@pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "llama3_8b", "llama3_8b_int4cb", "llama3_8b_d2b5_4x256"])
 def test_tuned_kernels_cover_every_benchmark_format(cfg):
     """VQ_IMPL_TUNED never falls back: it must run (not VQ_ERR_UNSUPPORTED) on every layer shape of
     the five configurations, at every batch of the configuration (row count cut to two tiles)."""
@@ -377,7 +381,7 @@ def _decode_slab_check(spec, L, dev_W, block_row):
     assert np.array_equal(dev_W[r0:r0 + spec.Br].view(np.uint16), W16), f"{spec.name}: decode rows {r0}.."
 
 
-@pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "llama3_8b", "llama3_8b_int4cb"])
+@pytest.mark.parametrize("cfg", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "llama3_8b", "llama3_8b_int4cb", "llama3_8b_d2b5_4x256"])
 def test_benchmark_configs_full_size(cfg):
     conf = vq_synth.CONFIGS[cfg]
     seen = set()
@@ -410,7 +414,8 @@ def test_benchmark_configs_full_size(cfg):
 
 
 @pytest.mark.parametrize("cfg,names", [("cfg5", ("q", "k", "v")), ("cfg5", ("gate", "up")),
-                                       ("cfg3", ("q", "k", "v")), ("cfg3", ("gate", "up"))],
+                                       ("cfg3", ("q", "k", "v")), ("cfg3", ("gate", "up")),
+                                       ("llama3_8b_d2b5_4x256", ("q", "k", "v")), ("llama3_8b_d2b5_4x256", ("gate", "up"))],
                          ids=lambda v: v if isinstance(v, str) else "+".join(v))
 def test_benchmark_groups_full_size(cfg, names):
     """The grouped calls bench.py times, at full size and in its launch configuration (one launch per

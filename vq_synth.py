@@ -157,6 +157,12 @@ CONFIGS = {
                  ("q", 4096, 4096), ("k", 1024, 4096), ("v", 1024, 4096), ("o", 4096, 4096),
                  ("gate", 14336, 4096), ("up", 14336, 4096), ("down", 4096, 14336)],
                  d=2, b=6, Br=32, Bc=128, int8=2)),
+    # the same shapes at the 2.75-bit row of the paper's table of VQ configurations (App. on VQ
+    # configurations): 2-D, 2.5 bits per dimension (5-bit indices), 8-bit codebooks, blocks of 4 x 256
+    "llama3_8b_d2b5_4x256": dict(seed=7, batches=(1, 8), layers=_set("llama3_8b_b5", [
+                 ("q", 4096, 4096), ("k", 1024, 4096), ("v", 1024, 4096), ("o", 4096, 4096),
+                 ("gate", 14336, 4096), ("up", 14336, 4096), ("down", 4096, 14336)],
+                 d=2, b=5, Br=4, Bc=256, int8=True)),
 }
 
 
