@@ -23,6 +23,8 @@
 // HBM sees row segments of 32..256 bytes instead of the 4 * EB bytes a step needs, and the copies of
 // the next chunks run under the look-ups of this one.  Nothing in the loop synchronises beyond the warp.
 // The warps' partial sums meet in shared memory in a fixed order (bit-identical results run to run).
+#include <type_traits>
+
 #include "vq_common.cuh"
 #include "vq_device.cuh"
 
@@ -34,7 +36,7 @@ using namespace dev;
 constexpr int kMaxWarps = 8;   // per CTA; three CTAs of that size fit an SM's registers
 constexpr int kChunkSteps = 8;   // steps per staged chunk of the index stream
 constexpr int kStages = 2;
-constexpr int kBuildGroup = 8;   // table words per lane whose loads are in flight together
+constexpr int kBuildGroup = 4;   // table words per lane whose loads are in flight together
 // Bytes between the rows of a staged chunk: 32 * EB of indices + 16, an odd number of 16-byte units, so
 // that the eight rows one look-up instruction reads start in different banks.
 __host__ __device__ constexpr int stage_pitch(int eb) { return 32 * eb + 16; }
@@ -94,17 +96,17 @@ __device__ __forceinline__ uint32_t pair_address(uint32_t lo, uint32_t hi, uint3
   }
 }
 
-// The EB bytes at byte offset `o` of a staged row as (lo, hi): aligned 32-bit loads of the words that hold
-// them.  Every word read lies inside the row's slot: the last byte needed is o + EB - 1 < 32 * EB.
-template <int EB>
-__device__ __forceinline__ void load_bits(uint32_t row_s, int o, uint32_t& lo, uint32_t& hi) {
-  const int sh = (o & 3) * 8;
-  const uint32_t at = row_s + (o & ~3);
+// The EB bytes of a lane at byte (base + IMM) + r of a staged row as (lo, hi), r = 0..3 being the lane's
+// constant misalignment (sh = 8r): aligned 32-bit loads of the words that hold them.  two / three: whether
+// the bytes reach into a second / third word (r + EB > 4 / > 8).  Every word read lies inside the row's
+// slot: the last byte needed is the last one of the lane's field.
+template <int EB, int IMM>
+__device__ __forceinline__ void load_bits(uint32_t base, int sh, bool two, bool three, uint32_t& lo, uint32_t& hi) {
   uint32_t w0, w1 = 0, w2 = 0;
-  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w0) : "r"(at));
-  if ((o & 3) + EB > 4) asm volatile("ld.shared.b32 %0, [%1+4];" : "=r"(w1) : "r"(at));
+  asm volatile("ld.shared.b32 %0, [%1+%2];" : "=r"(w0) : "r"(base), "n"(IMM));
+  if (two) asm volatile("ld.shared.b32 %0, [%1+%2];" : "=r"(w1) : "r"(base), "n"(IMM + 4));
   if constexpr (EB == 7) {
-    if ((o & 3) + EB > 8) asm volatile("ld.shared.b32 %0, [%1+8];" : "=r"(w2) : "r"(at));
+    if (three) asm volatile("ld.shared.b32 %0, [%1+%2];" : "=r"(w2) : "r"(base), "n"(IMM + 8));
   }
   lo = __funnelshift_r(w0, w1, sh);
   hi = __funnelshift_r(w1, w2, sh);
@@ -170,7 +172,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
         const int i = i0 + 32 * k;
         raw[k] = 0u;
         sc[k] = __ushort_as_half(0);
-        if (i < a.tbl_words) {
+        if (i - lane < a.tbl_words && i < a.tbl_words) {   // (the first test is the same for the whole warp: unused slots are jumped over)
           const uint32_t e = static_cast<uint32_t>(i) & ((1u << EB) - 1u);
           const uint32_t blk = static_cast<uint32_t>(min(brow0 + (i >> EB), block_rows - 1)) * static_cast<uint32_t>(a.blocks_per_row) +
                                static_cast<uint32_t>(col_blk);
@@ -201,7 +203,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
 #pragma unroll
       for (int k = 0; k < kBuildGroup; ++k) {
         const int i = i0 + 32 * k;
-        if (i < a.tbl_words) {
+        if (i - lane < a.tbl_words && i < a.tbl_words) {
           uint32_t word = raw[k];
           if (a.cb_int8) {   // exact products of the block scale and the 8-bit entries, one rounding each
             const float f = __half2float(sc[k]);
@@ -264,17 +266,22 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
     xn[nb][1] = ldg128_nc(xp[nb] + 8);
   }
 
+  // a lane's EB bytes of a step start t * EB bytes after the step's: the same misalignment in every step
+  const int bit_sh = ((t * EB) & 3) * 8;
+  const bool two_words = ((t * EB) & 3) + EB > 4, three_words = ((t * EB) & 3) + EB > 8;
+  static_assert(kChunkSteps == 8, "the chunk loop below is written out for 8 steps");
   for (int c = 0; c < n_chunks; ++c) {
     cp_async_wait<kStages - 2>();   // chunk c has landed (this lane's pieces; the warp barrier covers the others')
     __syncwarp();                   // ... and every lane is done reading the stage that chunk c + kStages - 1 overwrites
     fetch(c + kStages - 1);
-    const uint32_t rowA_s = stage_s + (c % kStages) * stage_bytes(EB) + g * PITCH;
+    // this lane's first word of step 0 in rows g and g + 8 of the stage
+    const uint32_t rowA_s = stage_s + (c % kStages) * stage_bytes(EB) + g * PITCH + ((t * EB) & ~3);
     const uint32_t rowB_s = rowA_s + 8 * PITCH;
     const int sc0 = s_begin + c * kChunkSteps;
     const int nst = min(kChunkSteps, s_end - sc0);
-#pragma unroll 2
-    for (int u = 0; u < nst; ++u) {
-      const int s = sc0 + u;
+    auto step = [&](auto uc) {
+      constexpr int UU = decltype(uc)::value;
+      const int s = sc0 + UU;
       if (until_rebuild == 0) {
         const int col_blk = s / a.bsteps;
         until_rebuild = a.bsteps - (s - col_blk * a.bsteps);
@@ -296,10 +303,9 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
         xn[nb][0] = ldg128_nc(xp[nb]);
         xn[nb][1] = ldg128_nc(xp[nb] + 8);
       }
-      const int o = (u * 4 + t) * EB;
       uint32_t loA, hiA, loB, hiB;
-      load_bits<EB>(rowA_s, o, loA, hiA);
-      load_bits<EB>(rowB_s, o, loB, hiB);
+      load_bits<EB, UU * 4 * EB>(rowA_s, bit_sh, two_words, three_words, loA, hiA);
+      load_bits<EB, UU * 4 * EB>(rowB_s, bit_sh, two_words, three_words, loB, hiB);
       uint32_t wa[8], wb[8];
 #define VQ_WT_PAIR(P)                                    \
   wa[P] = lds32(pair_address<EB, P>(loA, hiA, tA));     \
@@ -314,7 +320,16 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
         mma16816(acc[nb], wa[4], wb[4], wa[5], wb[5], x[nb][1].x, x[nb][1].y);
         mma16816(acc[nb], wa[6], wb[6], wa[7], wb[7], x[nb][1].z, x[nb][1].w);
       }
-    }
+    };
+    // the chunk's steps, unrolled: every shared-memory offset of a step is then an immediate
+    if (0 < nst) step(std::integral_constant<int, 0>{});
+    if (1 < nst) step(std::integral_constant<int, 1>{});
+    if (2 < nst) step(std::integral_constant<int, 2>{});
+    if (3 < nst) step(std::integral_constant<int, 3>{});
+    if (4 < nst) step(std::integral_constant<int, 4>{});
+    if (5 < nst) step(std::integral_constant<int, 5>{});
+    if (6 < nst) step(std::integral_constant<int, 6>{});
+    if (7 < nst) step(std::integral_constant<int, 7>{});
   }
   cp_async_wait<0>();
   __syncthreads();   // the reduction buffer lies over the warps' tables and stages
