@@ -87,7 +87,13 @@ typedef enum {
   VQ_CB_INT4_G128 = 2     /* signed 4-bit entries, one binary16 scale per row and group of 128 columns */
 } vq_cb_type;
 
-/* Kernel selection for the *_impl entry points.  VQ_IMPL_AUTO is what the plain entry points use. */
+/* Kernel selection for the *_impl entry points.  VQ_IMPL_AUTO is what the plain entry points use.
+ * Tuned kernels exist for: 4-bit indices with per-row codebooks or blocks of a few rows (2-D, and 1-D
+ * with int8 codebooks); 2-D 5- and 6-bit and 4-D 8-bit indices with tall blocks (32, 64 or a multiple of
+ * 128 rows; 256 for 4-D); and, through tables of fp16 PAIRS private to a warp, every other 2-D format
+ * and every 1-D format of up to 4 index bits (two indices per look-up) whose blocks have 1, 2, 4, 8 or
+ * a multiple of 16 rows and whose block columns and K are multiples of 64 (fp16 or int8 codebooks) -
+ * the remaining rows of the paper's table of VQ configurations (its appendix on VQ configurations). */
 typedef enum {
   VQ_IMPL_AUTO = 0,     /* tuned kernel when one covers the format/shape, else the generic one   */
   VQ_IMPL_GENERIC = 1,  /* format-generic fp32-FMA kernel (any valid format)                     */
@@ -174,8 +180,9 @@ vq_status vq_gemm_small_batch_impl(const vq_format* fmt, const void* d_idx, cons
  *               pointers (layouts as for vq_gemm_small_batch), its output d_Y (binary16
  *               [batch][n_rows]) and its row count (a multiple of block_rows).
  *   d_X       : device binary16 [batch][K], shared by all members.
- * One kernel serves the whole group where the tuned persistent kernel covers the format; otherwise
- * the members run one after the other on `stream`.  Results are the same as n_members separate calls.
+ * One kernel serves the whole group where the persistent kernel, the shared-codebook kernels or the
+ * pair-table kernel cover the format (vq_grouped_kernel_launches tells); otherwise the members run one
+ * after the other on `stream`.  Results are the same as n_members separate calls.
  * Errors: as vq_gemm_small_batch; SHAPE also if the rows do not add up to fmt->n_rows. */
 #define VQ_MAX_GROUP 4
 typedef struct {
@@ -187,7 +194,7 @@ typedef struct {
 } vq_group_member;
 vq_status vq_gemm_small_batch_grouped(const vq_format* fmt, const vq_group_member* members, int n_members,
                                       const void* d_X, int batch, void* d_ws, size_t ws_bytes, void* stream);
-/* Kernels a grouped call of this format launches: 1 (one persistent kernel for the group) or n_members.
+/* Kernels a grouped call of this format launches: 1 (one kernel for the group) or n_members.
  * Host only; 0 for invalid arguments. */
 int vq_grouped_kernel_launches(const vq_format* fmt, int n_members, int batch);
 
