@@ -90,10 +90,11 @@ typedef enum {
 /* Kernel selection for the *_impl entry points.  VQ_IMPL_AUTO is what the plain entry points use.
  * Tuned kernels exist for: 4-bit indices with per-row codebooks or blocks of a few rows (2-D, and 1-D
  * with int8 codebooks); 2-D 5- and 6-bit and 4-D 8-bit indices with tall blocks (32, 64 or a multiple of
- * 128 rows; 256 for 4-D); and, through tables of fp16 PAIRS private to a warp, every other 2-D format
- * and every 1-D format of up to 4 index bits (two indices per look-up) whose blocks have 1, 2, 4, 8 or
- * a multiple of 16 rows and whose block columns and K are multiples of 64 (fp16 or int8 codebooks) -
- * the remaining rows of the paper's table of VQ configurations (its appendix on VQ configurations). */
+ * 128 rows; 256 for 4-D); and, through tables of fp16 PAIRS private to a warp, every other 2-D format,
+ * every 1-D format of up to 4 index bits (two indices per look-up) and 4-D 8-bit indices (four weights
+ * per look-up) whose blocks have 1, 2, 4, 8 (4-D: 8) or a multiple of 16 rows and whose block columns
+ * and K are multiples of 64 (fp16 or int8 codebooks) - the remaining rows of the paper's table of VQ
+ * configurations (its appendix on VQ configurations). */
 typedef enum {
   VQ_IMPL_AUTO = 0,     /* tuned kernel when one covers the format/shape, else the generic one   */
   VQ_IMPL_GENERIC = 1,  /* format-generic fp32-FMA kernel (any valid format)                     */

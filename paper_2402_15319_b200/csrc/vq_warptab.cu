@@ -1,15 +1,18 @@
-// warptab_kernel<EB, NB>: formats with SMALL codebook blocks (1, 2, 4, 8 rows, or any multiple of 16
+// warptab_kernel<EB, NB, QUAD>: formats with SMALL codebook blocks (1, 2, 4, 8 rows, or any multiple of 16
 // rows) and any index width the other tuned families do not take: 2-D indices of 1..8 bits, 1-D indices
 // of 1..4 bits; fp16 or scaled-int8 codebooks; block columns and K multiples of 64.  These are the
 // remaining rows of the paper's configuration table (App. on VQ configurations: 1-D 2-bit 1x256 and
-// 1x128, 2-D 2.5 bits per dimension on 2x256 and 4x256, 1-D 3-bit 32x256, 2-D 8-bit indices 256x256).
+// 1x128, 2-D 2.5 bits per dimension on 2x256 and 4x256, 1-D 3-bit 32x256, 2-D 8-bit indices 256x256,
+// 4-D 8-bit indices 128x256).
 //
 // Everything is expressed as PAIR look-ups: EB bits of the index stream select one 32-bit table word
 // holding the two fp16 weights of two adjacent columns.  For d = 2 that is the codebook entry itself
 // (EB = index_bits); for d = 1 two consecutive indices are looked up at once in the product table
 // word[e] = (c[e mod k], c[e div k]) with EB = 2 * index_bits (the decode of Sec. 3.2 / App. A, two values
 // per look-up as the paper's LUT instructions do).  Scales of int8 codebooks are folded into the table
-// (w = fp16(scale * c), Sec. 3.1).
+// (w = fp16(scale * c), Sec. 3.1).  QUAD variant (d = 4, 8-bit indices): one stream byte selects four weights,
+// two adjacent table words fetched by one 64-bit gather; everything else is the pair kernel at 4 stream
+// bytes per lane and step.
 //
 // Work: a CTA owns 16 output rows; its warps split K.  A warp walks its column range in steps of 64
 // columns.  In a step, lane (g = lane / 4, t = lane % 4) takes 8 consecutive pairs (EB bytes of the
@@ -41,8 +44,9 @@ constexpr int kBuildGroup = 4;   // table words per lane whose loads are in flig
 // that the eight rows one look-up instruction reads start in different banks.
 __host__ __device__ constexpr int stage_pitch(int eb) { return 32 * eb + 16; }
 __host__ __device__ constexpr int stage_bytes(int eb) { return 16 * stage_pitch(eb); }
-// Alignment of a warp's region: the size of one table (tables start on multiples of their size), 16 at least.
-__host__ __device__ constexpr int region_align(int eb) { return (4 << eb) < 16 ? 16 : (4 << eb); }
+// Alignment of a warp's region: the size of one table of 2^tb words (tables start on multiples of their
+// size), 16 at least.
+__host__ __device__ constexpr int region_align(int tb) { return (4 << tb) < 16 ? 16 : (4 << tb); }
 
 struct WarpTabArgs {
   // the layers of the call (same format and K, one activation tensor); tile0 = first 16-row tile of each
@@ -112,8 +116,10 @@ __device__ __forceinline__ void load_bits(uint32_t base, int sh, bool two, bool 
   hi = __funnelshift_r(w1, w2, sh);
 }
 
-template <int EB, int NB>
+template <int EB, int NB, bool QUAD>
 __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kernel(const WarpTabArgs a) {
+  static_assert(!QUAD || EB == 4, "4-D entries: one 8-bit index per 4 columns = 4 stream bytes per lane and step");
+  constexpr int TB = QUAD ? 9 : EB;   // log2 of the words of one table
   extern __shared__ __align__(16) uint8_t smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
@@ -139,12 +145,12 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
   const int brow0 = a.Br >= 16 ? row0 / a.Br : row0 >> a.br_shift;
   const int block_rows = a.Br >= 16 ? seg_N / a.Br : seg_N >> a.br_shift;
   // warp regions start on a multiple of the table size (the host adds that much slack)
-  uint8_t* mine = smem + ((0u - smem_u32(smem)) & static_cast<uint32_t>(region_align(EB) - 1)) + warp * a.warp_bytes;
+  uint8_t* mine = smem + ((0u - smem_u32(smem)) & static_cast<uint32_t>(region_align(TB) - 1)) + warp * a.warp_bytes;
   uint32_t* tbl = reinterpret_cast<uint32_t*>(mine);
   uint32_t tA = smem_u32(tbl), tB = tA;
   if (a.Br < 16) {
-    tA += static_cast<uint32_t>((rA >> a.br_shift) - brow0) << (EB + 2);
-    tB += static_cast<uint32_t>((rB >> a.br_shift) - brow0) << (EB + 2);
+    tA += static_cast<uint32_t>((rA >> a.br_shift) - brow0) << (TB + 2);
+    tB += static_cast<uint32_t>((rB >> a.br_shift) - brow0) << (TB + 2);
   }
   constexpr int PITCH = stage_pitch(EB);
   const uint32_t stage_s = smem_u32(mine) + a.tbl_bytes;
@@ -173,8 +179,8 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
         raw[k] = 0u;
         sc[k] = __ushort_as_half(0);
         if (i - lane < a.tbl_words && i < a.tbl_words) {   // (the first test is the same for the whole warp: unused slots are jumped over)
-          const uint32_t e = static_cast<uint32_t>(i) & ((1u << EB) - 1u);
-          const uint32_t blk = static_cast<uint32_t>(min(brow0 + (i >> EB), block_rows - 1)) * static_cast<uint32_t>(a.blocks_per_row) +
+          const uint32_t e = static_cast<uint32_t>(i) & ((1u << TB) - 1u);
+          const uint32_t blk = static_cast<uint32_t>(min(brow0 + (i >> TB), block_rows - 1)) * static_cast<uint32_t>(a.blocks_per_row) +
                                static_cast<uint32_t>(col_blk);
           if (a.cb_int8) {
             sc[k] = __ldg(seg_scale + blk);
@@ -307,12 +313,22 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
       load_bits<EB, UU * 4 * EB>(rowA_s, bit_sh, two_words, three_words, loA, hiA);
       load_bits<EB, UU * 4 * EB>(rowB_s, bit_sh, two_words, three_words, loB, hiB);
       uint32_t wa[8], wb[8];
+      if constexpr (QUAD) {   // one byte selects four weights: a 64-bit gather fills pairs 2q and 2q + 1
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint2 va = lds64((((loA >> (8 * q)) & 0xffu) << 3) | tA);
+          const uint2 vb = lds64((((loB >> (8 * q)) & 0xffu) << 3) | tB);
+          wa[2 * q] = va.x; wa[2 * q + 1] = va.y;
+          wb[2 * q] = vb.x; wb[2 * q + 1] = vb.y;
+        }
+      } else {
 #define VQ_WT_PAIR(P)                                    \
   wa[P] = lds32(pair_address<EB, P>(loA, hiA, tA));     \
   wb[P] = lds32(pair_address<EB, P>(loB, hiB, tB));
-      VQ_WT_PAIR(0) VQ_WT_PAIR(1) VQ_WT_PAIR(2) VQ_WT_PAIR(3)
-      VQ_WT_PAIR(4) VQ_WT_PAIR(5) VQ_WT_PAIR(6) VQ_WT_PAIR(7)
+        VQ_WT_PAIR(0) VQ_WT_PAIR(1) VQ_WT_PAIR(2) VQ_WT_PAIR(3)
+        VQ_WT_PAIR(4) VQ_WT_PAIR(5) VQ_WT_PAIR(6) VQ_WT_PAIR(7)
 #undef VQ_WT_PAIR
+      }
 #pragma unroll
       for (int nb = 0; nb < NB; ++nb) {
         mma16816(acc[nb], wa[0], wb[0], wa[1], wb[1], x[nb][0].x, x[nb][0].y);
@@ -353,11 +369,19 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
   }
 }
 
+// 4-D entries selected by 8-bit indices: one look-up returns four weights (two table words).
+bool quad_format(const Geometry& g) { return g.d == 4 && g.b == 8; }
+
+// Stream bits per pair of columns: what a lane consumes is 8 of them = that many bytes per step.
 int pair_bits(const Geometry& g) {
   if (g.d == 2) return g.b;
   if (g.d == 1 && g.b <= 4) return 2 * g.b;
+  if (quad_format(g)) return 4;
   return 0;
 }
+
+// log2 of the 32-bit words of one table.
+int table_bits(const Geometry& g) { return quad_format(g) ? 9 : pair_bits(g); }
 
 int tables_per_tile(const Geometry& g) { return g.Br >= 16 ? 1 : 16 / g.Br; }
 
@@ -366,17 +390,18 @@ constexpr size_t kSmemPerSm = 228 * 1024;   // shared memory of an SM; every res
 
 // Picks the K split, finishes the arguments and launches.  The dynamic shared-memory limit is raised and the
 // kernel's register count read once per device and instantiation.
-template <int EB, int NB>
+template <int EB, int NB, bool QUAD>
 vq_status launch_one(WarpTabArgs a, long long tiles, int sms, cudaStream_t s) {
+  constexpr int TB = QUAD ? 9 : EB;
   static int regs_of[kMaxDevices] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VQ_ERR_CUDA;
   int regs = __atomic_load_n(&regs_of[dev], __ATOMIC_ACQUIRE);
   if (!regs) {
     cudaFuncAttributes fa;
-    if (cudaFuncSetAttribute(warptab_kernel<EB, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemLimit)) !=
+    if (cudaFuncSetAttribute(warptab_kernel<EB, NB, QUAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemLimit)) !=
             cudaSuccess ||
-        cudaFuncGetAttributes(&fa, warptab_kernel<EB, NB>) != cudaSuccess || fa.numRegs < 1)
+        cudaFuncGetAttributes(&fa, warptab_kernel<EB, NB, QUAD>) != cudaSuccess || fa.numRegs < 1)
       return VQ_ERR_CUDA;
     regs = fa.numRegs;
     __atomic_store_n(&regs_of[dev], regs, __ATOMIC_RELEASE);
@@ -386,7 +411,7 @@ vq_status launch_one(WarpTabArgs a, long long tiles, int sms, cudaStream_t s) {
   auto resident = [&](int w) {
     long long c = warps_by_regs / w;
     c = c < 32 ? c : 32;
-    const long long by_smem = static_cast<long long>(kSmemPerSm / (static_cast<size_t>(w) * a.warp_bytes + region_align(EB) + 1024));
+    const long long by_smem = static_cast<long long>(kSmemPerSm / (static_cast<size_t>(w) * a.warp_bytes + region_align(TB) + 1024));
     return c < by_smem ? c : by_smem;
   };
   // K split: the most warps per CTA (at most kMaxWarps, at most one per chunk of the row) with which every
@@ -394,21 +419,21 @@ vq_status launch_one(WarpTabArgs a, long long tiles, int sms, cudaStream_t s) {
   // device, which weighs more than the longer walk of fewer, longer-running warps.
   const int chunks_total = (a.steps_total + kChunkSteps - 1) / kChunkSteps;
   int wk = kMaxWarps < chunks_total ? kMaxWarps : chunks_total;
-  while (wk > 1 && (static_cast<size_t>(wk) * a.warp_bytes + region_align(EB) > kSmemLimit || tiles > resident(wk) * sms)) --wk;
+  while (wk > 1 && (static_cast<size_t>(wk) * a.warp_bytes + region_align(TB) > kSmemLimit || tiles > resident(wk) * sms)) --wk;
   a.steps_per_warp = ((a.steps_total + wk - 1) / wk + kChunkSteps - 1) / kChunkSteps * kChunkSteps;   // whole chunks
   wk = (a.steps_total + a.steps_per_warp - 1) / a.steps_per_warp;   // no warp without work
-  const size_t smem_bytes = static_cast<size_t>(wk) * a.warp_bytes + region_align(EB);
+  const size_t smem_bytes = static_cast<size_t>(wk) * a.warp_bytes + region_align(TB);
   if (smem_bytes > kSmemLimit) return VQ_ERR_UNSUPPORTED;
   // A plain launch, in stream order.  (With programmatic dependent launch the next launch's CTAs take the
   // SM slots this grid leaves free and stay where they land: two such layers back to back then run with
   // 3 CTAs on some SMs and 1 on others; measured 31.5 against 23.2 us on 4096 x 14336.)
-  warptab_kernel<EB, NB><<<static_cast<unsigned>(tiles), static_cast<unsigned>(wk) * 32u, smem_bytes, s>>>(a);
+  warptab_kernel<EB, NB, QUAD><<<static_cast<unsigned>(tiles), static_cast<unsigned>(wk) * 32u, smem_bytes, s>>>(a);
   return check_launch();
 }
 
-template <int EB>
+template <int EB, bool QUAD = false>
 vq_status launch_eb(const WarpTabArgs& a, int nb, long long tiles, int sms, cudaStream_t s) {
-  return nb == 1 ? launch_one<EB, 1>(a, tiles, sms, s) : launch_one<EB, 2>(a, tiles, sms, s);
+  return nb == 1 ? launch_one<EB, 1, QUAD>(a, tiles, sms, s) : launch_one<EB, 2, QUAD>(a, tiles, sms, s);
 }
 
 }  // namespace
@@ -420,7 +445,7 @@ bool warptab_covers(const Geometry& g) {
   if (g.K % 64 || g.Bc % 64) return false;
   if (!(g.Br == 1 || g.Br == 2 || g.Br == 4 || g.Br == 8 || g.Br % 16 == 0)) return false;
   if (g.stride >= (1LL << 30)) return false;   // byte offsets inside a row are 32-bit in the kernel
-  return (tables_per_tile(g) << eb) <= 1024;
+  return (tables_per_tile(g) << table_bits(g)) <= 1024;
 }
 
 vq_status launch_gemm_warptab_group(const StreamCall& call, cudaStream_t s) {
@@ -448,19 +473,20 @@ vq_status launch_gemm_warptab_group(const StreamCall& call, cudaStream_t s) {
   a.stride = g.stride;
   a.K = g.K;
   a.batch = call.batch;
-  a.d = g.d;
-  a.b = g.b;
-  a.entries = g.entries;
+  // (a 4-D codebook of 256 entries lies in memory like a 2-D one of 512: the table build treats it as such)
+  a.d = quad_format(g) ? 2 : g.d;
+  a.b = quad_format(g) ? 9 : g.b;
+  a.entries = quad_format(g) ? 512 : g.entries;
   a.cb_int8 = g.cb_int8;
   a.Br = g.Br;
   a.br_shift = g.Br == 1 ? 0 : g.Br == 2 ? 1 : g.Br == 4 ? 2 : 3;
   a.bsteps = g.Bc / 64;
   a.blocks_per_row = g.blocks_per_row;
   a.steps_total = g.K / 64;
-  a.tbl_words = tables_per_tile(g) << eb;
+  a.tbl_words = tables_per_tile(g) << table_bits(g);
   // per warp: tables + chunk stages; the reduction buffer (nb * 512 bytes per warp) reuses that space
   a.tbl_bytes = (a.tbl_words * 4 + 15) / 16 * 16;
-  const int tbl_align = region_align(eb);
+  const int tbl_align = region_align(table_bits(g));
   a.warp_bytes = (a.tbl_bytes + kStages * stage_bytes(eb) + tbl_align - 1) / tbl_align * tbl_align;
   a.red_off = 0;
   int sms = 0;
@@ -469,7 +495,7 @@ vq_status launch_gemm_warptab_group(const StreamCall& call, cudaStream_t s) {
     case 1: return launch_eb<1>(a, nb, tiles, sms, s);
     case 2: return launch_eb<2>(a, nb, tiles, sms, s);
     case 3: return launch_eb<3>(a, nb, tiles, sms, s);
-    case 4: return launch_eb<4>(a, nb, tiles, sms, s);
+    case 4: return quad_format(g) ? launch_eb<4, true>(a, nb, tiles, sms, s) : launch_eb<4>(a, nb, tiles, sms, s);
     case 5: return launch_eb<5>(a, nb, tiles, sms, s);
     case 6: return launch_eb<6>(a, nb, tiles, sms, s);
     case 7: return launch_eb<7>(a, nb, tiles, sms, s);

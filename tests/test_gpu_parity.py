@@ -164,6 +164,7 @@ GROUPS = [
     (vq_synth.LayerSpec("g_pt_d2b5", N=0, K=1280, d=2, b=5, Br=4, Bc=256, int8=True), [212, 64, 36, 100]),
     (vq_synth.LayerSpec("g_pt_d1b2", N=0, K=1024, d=1, b=2, Br=1, Bc=256, int8=True), [33, 200]),
     (vq_synth.LayerSpec("g_pt_d2b8", N=0, K=768, d=2, b=8, Br=256, Bc=256, int8=False), [256, 512]),
+    (vq_synth.LayerSpec("g_pt_d4b8", N=0, K=1024, d=4, b=8, Br=128, Bc=256, int8=True), [128, 384]),
 ]
 
 
@@ -218,6 +219,11 @@ PAIR_TABLE_CASES = [
     vq_synth.LayerSpec("pt_d2b1_1x64_i8", N=33, K=320, d=2, b=1, Br=1, Bc=64, int8=True),
     vq_synth.LayerSpec("pt_d1b1_2x192", N=34, K=1344, d=1, b=1, Br=2, Bc=192, int8=False),
     vq_synth.LayerSpec("pt_d2b2_48x64_i8", N=96, K=64, d=2, b=2, Br=48, Bc=64, int8=True),
+    # 4-D, 8-bit indices with blocks of fewer than 256 rows (128 x 256: the 2.25-bit 4-D row of the paper's
+    # table): one byte looks up four weights
+    vq_synth.LayerSpec("pt_d4b8_128x256_i8", N=256, K=1024, d=4, b=8, Br=128, Bc=256, int8=True),
+    vq_synth.LayerSpec("pt_d4b8_16x64", N=48, K=704, d=4, b=8, Br=16, Bc=64, int8=False, cb_sigma=0.015),
+    vq_synth.LayerSpec("pt_d4b8_8x128_i8", N=40, K=640, d=4, b=8, Br=8, Bc=128, int8=True),
 ]
 
 
@@ -231,6 +237,7 @@ def test_pair_table_kernel_formats(spec):
     vq_synth.LayerSpec("pt_full_d2b5_4x256_i8", N=4096, K=4096, d=2, b=5, Br=4, Bc=256, int8=True),
     vq_synth.LayerSpec("pt_full_d1b2_1x256_i8", N=14336, K=4096, d=1, b=2, Br=1, Bc=256, int8=True),
     vq_synth.LayerSpec("pt_full_d2b8_256x256_i8", N=4096, K=14336, d=2, b=8, Br=256, Bc=256, int8=True),
+    vq_synth.LayerSpec("pt_full_d4b8_128x256_i8", N=14336, K=4096, d=4, b=8, Br=128, Bc=256, int8=True),
 ], ids=lambda s: s.name)
 def test_pair_table_kernel_layer_sizes(spec):
     """Llama-3-8B-sized layers in the paper's small-block configurations: sampled output rows against the
