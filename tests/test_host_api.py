@@ -169,7 +169,7 @@ def test_pack_info_int4_codebook_with_group_scales():
 def test_grouped_call_argument_errors_and_launch_counts():
     """vq_gemm_small_batch_grouped validates on the host (member pointers, row sums, workspace) before
     any launch, and vq_grouped_kernel_launches tells one kernel for the formats a kernel family takes
-    as a group (per-row 4-bit formats, shared-codebook formats), n_members for the rest."""
+    as a group (per-row 4-bit formats, shared-codebook formats, pair-table formats), n_members for the rest."""
     from paper_2402_15319_b200.binding import _CGroupMember
     lib = vq.load()
     total = _replace(GOOD, n_rows=16)
@@ -196,9 +196,15 @@ def test_grouped_call_argument_errors_and_launch_counts():
     row4 = vq.VQFormat(10240, 8192, 2, 4, 1, 2048, vq.VQ_CB_INT8_SCALED)
     blk6 = vq.VQFormat(12288, 4096, 2, 6, 128, 128, vq.VQ_CB_FP16)
     odd5 = vq.VQFormat(42, 312, 1, 5, 1, 156, vq.VQ_CB_FP16)
+    # small blocks / index widths only the pair-table kernel takes: 2-D 5-bit 4x256, 1-D 2-bit 1x256, 4-D 8-bit 128x256
+    pair = [vq.VQFormat(6144, 4096, 2, 5, 4, 256, vq.VQ_CB_INT8_SCALED), vq.VQFormat(6144, 4096, 1, 2, 1, 256, vq.VQ_CB_INT8_SCALED),
+            vq.VQFormat(6144, 4096, 4, 8, 128, 256, vq.VQ_CB_FP16)]
+    i4 = vq.VQFormat(6144, 4096, 2, 5, 4, 256, vq.VQ_CB_INT4_G128)   # INT4 codebooks on small blocks: generic kernel, member by member
     for batch in (1, 4, 16):
         assert vq.vq_grouped_kernel_launches(row4, 3, batch) == 1
         assert vq.vq_grouped_kernel_launches(blk6, 3, batch) == 1
+        assert all(vq.vq_grouped_kernel_launches(f, 3, batch) == 1 for f in pair)
+        assert vq.vq_grouped_kernel_launches(i4, 3, batch) == 3
         assert vq.vq_grouped_kernel_launches(odd5, 2, batch) == 2
         assert vq.vq_grouped_kernel_launches(row4, 1, batch) == 1
     assert vq.vq_grouped_kernel_launches(row4, 0, 1) == 0 and vq.vq_grouped_kernel_launches(row4, 5, 1) == 0
