@@ -78,9 +78,10 @@ typedef enum {
  *   d_scale : binary16 [N][K/128]; w[n][k] = scale[n][k/128] * c.  K % 128 == 0.
  * vq_decode_weights decodes it with its tile kernel; the skinny GEMM runs in the tuned shared-codebook
  * kernels for 2-D formats with 5- or 6-bit indices (blocks of 32, 64 or a multiple of 128 rows and a
- * multiple of 128 columns, K a multiple of 256), where a looked-up pair is fp16(scale * c), the value
- * vq_decode_weights writes; other formats of this codebook type run in the format-generic kernel
- * (VQ_IMPL_TUNED returns VQ_ERR_UNSUPPORTED for them); vq_assign_indices does not take it. */
+ * multiple of 128 columns, K a multiple of 256) and in the pair-table kernel for the block shapes that
+ * one takes (see vq_impl); in both a looked-up pair is fp16(scale * c), the value vq_decode_weights
+ * writes; other formats of this codebook type run in the format-generic kernel (VQ_IMPL_TUNED returns
+ * VQ_ERR_UNSUPPORTED for them); vq_assign_indices does not take it. */
 typedef enum {
   VQ_CB_FP16 = 0,         /* binary16 entries                                                        */
   VQ_CB_INT8_SCALED = 1,  /* signed 8-bit entries, one binary16 scale per block                       */
@@ -93,7 +94,7 @@ typedef enum {
  * 128 rows; 256 for 4-D); and, through tables of fp16 PAIRS private to a warp, every other 2-D format,
  * every 1-D format of up to 4 index bits (two indices per look-up) and 4-D 8-bit indices (four weights
  * per look-up) whose blocks have 1, 2, 4, 8 (4-D: 8) or a multiple of 16 rows and whose block columns
- * and K are multiples of 64 (fp16 or int8 codebooks) - the remaining rows of the paper's table of VQ
+ * and K are multiples of 64 (any codebook type) - the remaining rows of the paper's table of VQ
  * configurations (its appendix on VQ configurations). */
 typedef enum {
   VQ_IMPL_AUTO = 0,     /* tuned kernel when one covers the format/shape, else the generic one   */

@@ -187,7 +187,7 @@ vq_status vq_gemm_small_batch_impl(const vq_format* fmt, const void* d_idx, cons
 // one launch instead of three), 0 = member by member.
 static int group_family(const Geometry& g, int) {
   if (blockcb_covers(g)) return 2;
-  if (g.cb_int4) return 0;
+  if (g.cb_int4) return warptab_covers(g) ? 3 : 0;
   if (g.b != 4 && !stream_covers(g) && warptab_covers(g)) return 3;
   return 1;
 }

@@ -75,7 +75,7 @@ bool blockcb_covers(const Geometry& g);
 vq_status launch_gemm_rowcb(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
                             cudaStream_t s);
 // Warp-private pair tables: small codebook blocks (1, 2, 4, 8 or a multiple of 16 rows), 2-D indices of
-// any width, 1-D indices of up to 4 bits, 4-D 8-bit indices, fp16 / int8 codebooks, K and block columns
+// any width, 1-D indices of up to 4 bits, 4-D 8-bit indices, every codebook type, K and block columns
 // multiples of 64.
 vq_status launch_gemm_warptab(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,
                               cudaStream_t s);

@@ -106,8 +106,11 @@ size_t stream_workspace_bytes(long long rows, int batch) {
 
 vq_status launch_gemm_tuned(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch, void* ws,
                             size_t ws_bytes, cudaStream_t s) {
-  if (g.cb_int4) return launch_gemm_blockcb(g, p, X, Y, batch, s);   // int4 codebooks: the 2-D shared-codebook kernels only
   vq_status st = VQ_ERR_UNSUPPORTED;
+  if (g.cb_int4) {   // int4 codebooks: the 2-D shared-codebook kernels, else warp-private pair tables
+    st = launch_gemm_blockcb(g, p, X, Y, batch, s);
+    return st != VQ_ERR_UNSUPPORTED ? st : launch_gemm_warptab(g, p, X, Y, batch, s);
+  }
 #ifdef VQ_TUNING
   const char* path_env = getenv("VQ_PATH");
   const int path = path_env ? atoi(path_env) : 0;   // 1: persistent kernel only, 2: cluster kernels only

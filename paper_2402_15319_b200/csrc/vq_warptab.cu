@@ -1,6 +1,6 @@
-// warptab_kernel<EB, NB, QUAD>: formats with SMALL codebook blocks (1, 2, 4, 8 rows, or any multiple of 16
+// warptab_kernel<EB, NB, QUAD, I4>: formats with SMALL codebook blocks (1, 2, 4, 8 rows, or any multiple of 16
 // rows) and any index width the other tuned families do not take: 2-D indices of 1..8 bits, 1-D indices
-// of 1..4 bits; fp16 or scaled-int8 codebooks; block columns and K multiples of 64.  These are the
+// of 1..4 bits; fp16, scaled-int8 or int4 codebooks; block columns and K multiples of 64.  These are the
 // remaining rows of the paper's configuration table (App. on VQ configurations: 1-D 2-bit 1x256 and
 // 1x128, 2-D 2.5 bits per dimension on 2x256 and 4x256, 1-D 3-bit 32x256, 2-D 8-bit indices 256x256,
 // 4-D 8-bit indices 128x256).
@@ -12,7 +12,9 @@
 // per look-up as the paper's LUT instructions do).  Scales of int8 codebooks are folded into the table
 // (w = fp16(scale * c), Sec. 3.1).  QUAD variant (d = 4, 8-bit indices): one stream byte selects four weights,
 // two adjacent table words fetched by one 64-bit gather; everything else is the pair kernel at 4 stream
-// bytes per lane and step.
+// bytes per lane and step.  I4 variant (INT4 codebooks, Sec. 4.2): tables hold the 4-bit entries as exact
+// fp16 integers and every gathered pair is multiplied (one fp16x2 multiply, rounded once) by the fp16
+// scale of its row and group of 128 columns, which gives fp16(scale * c), the value vq_decode_weights writes.
 //
 // Work: a CTA owns 16 output rows; its warps split K.  A warp walks its column range in steps of 64
 // columns.  In a step, lane (g = lane / 4, t = lane % 4) takes 8 consecutive pairs (EB bytes of the
@@ -61,6 +63,7 @@ struct WarpTabArgs {
   long long stride;
   int K, batch;
   int d, b, entries, cb_int8;
+  int cb_int4;                    // 4-bit entries (tables hold them as exact fp16 integers) + a scale per row and 128 columns
   int Br, br_shift;               // br_shift: log2(Br) when Br < 16
   int bsteps;                     // 64-column steps per codebook block (Bc / 64)
   int blocks_per_row;
@@ -71,6 +74,11 @@ struct WarpTabArgs {
   int red_off;                    // byte offset of the reduction buffer in shared memory (it reuses the warps' regions)
 };
 
+__device__ __forceinline__ uint32_t mul_f16x2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
@@ -116,7 +124,7 @@ __device__ __forceinline__ void load_bits(uint32_t base, int sh, bool two, bool 
   hi = __funnelshift_r(w1, w2, sh);
 }
 
-template <int EB, int NB, bool QUAD>
+template <int EB, int NB, bool QUAD, bool I4>
 __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kernel(const WarpTabArgs a) {
   static_assert(!QUAD || EB == 4, "4-D entries: one 8-bit index per 4 columns = 4 stream bytes per lane and step");
   constexpr int TB = QUAD ? 9 : EB;   // log2 of the words of one table
@@ -182,10 +190,19 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
           const uint32_t e = static_cast<uint32_t>(i) & ((1u << TB) - 1u);
           const uint32_t blk = static_cast<uint32_t>(min(brow0 + (i >> TB), block_rows - 1)) * static_cast<uint32_t>(a.blocks_per_row) +
                                static_cast<uint32_t>(col_blk);
-          if (a.cb_int8) {
+          if (!I4 && a.cb_int8) {
             sc[k] = __ldg(seg_scale + blk);
           }
-          if (a.d == 2) {
+          if (I4) {   // two 4-bit values per byte, low nibble first
+            const uint8_t* c = static_cast<const uint8_t*>(seg_cb);
+            if (a.d == 2) {
+              raw[k] = __ldg(c + (blk << cb_shift) + e);   // one byte = the entry's two values
+            } else {
+              const uint32_t v0 = (blk << cb_shift) + (e & ((1u << cb_shift) - 1u)), v1 = (blk << cb_shift) + (e >> cb_shift);
+              const uint32_t n0 = (__ldg(c + (v0 >> 1)) >> (4 * (v0 & 1u))) & 15u, n1 = (__ldg(c + (v1 >> 1)) >> (4 * (v1 & 1u))) & 15u;
+              raw[k] = n0 | (n1 << 4);
+            }
+          } else if (a.d == 2) {
             const uint32_t at = (blk << cb_shift) + e;   // in entries of two values
             if (a.cb_int8) {
               const uint16_t* c = static_cast<const uint16_t*>(seg_cb) + at;
@@ -211,7 +228,11 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
         const int i = i0 + 32 * k;
         if (i - lane < a.tbl_words && i < a.tbl_words) {
           uint32_t word = raw[k];
-          if (a.cb_int8) {   // exact products of the block scale and the 8-bit entries, one rounding each
+          if (I4) {   // signed nibbles as fp16 integers (exact); the row-group scale multiplies after the look-up
+            const int lo4 = static_cast<int>(raw[k] << 28) >> 28, hi4 = static_cast<int>(raw[k] << 24) >> 28;
+            const __half2 hv = __floats2half2_rn(static_cast<float>(lo4), static_cast<float>(hi4));
+            word = *reinterpret_cast<const uint32_t*>(&hv);
+          } else if (a.cb_int8) {   // exact products of the block scale and the 8-bit entries, one rounding each
             const float f = __half2float(sc[k]);
             const __half2 hv = __floats2half2_rn(f * static_cast<float>(static_cast<int8_t>(raw[k] & 0xffu)),
                                                  f * static_cast<float>(static_cast<int8_t>((raw[k] >> 8) & 0xffu)));
@@ -272,6 +293,9 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
     xn[nb][1] = ldg128_nc(xp[nb] + 8);
   }
 
+  // INT4 codebooks: the scales of rows g and g + 8, one per group of 128 columns
+  const __half* const scA = seg_scale + static_cast<long long>(rA) * (a.K / 128);
+  const __half* const scB = seg_scale + static_cast<long long>(rB) * (a.K / 128);
   // a lane's EB bytes of a step start t * EB bytes after the step's: the same misalignment in every step
   const int bit_sh = ((t * EB) & 3) * 8;
   const bool two_words = ((t * EB) & 3) + EB > 4, three_words = ((t * EB) & 3) + EB > 8;
@@ -328,6 +352,16 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
         VQ_WT_PAIR(0) VQ_WT_PAIR(1) VQ_WT_PAIR(2) VQ_WT_PAIR(3)
         VQ_WT_PAIR(4) VQ_WT_PAIR(5) VQ_WT_PAIR(6) VQ_WT_PAIR(7)
 #undef VQ_WT_PAIR
+      }
+      if constexpr (I4) {   // w = fp16(scale of the row's group of 128 columns * c): the value vq_decode_weights writes
+        const int grp = s >> 1;   // a step's 64 columns lie inside one group
+        const __half2 sA = __half2half2(__ldg(scA + grp)), sB = __half2half2(__ldg(scB + grp));
+        const uint32_t uA = *reinterpret_cast<const uint32_t*>(&sA), uB = *reinterpret_cast<const uint32_t*>(&sB);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          wa[q] = mul_f16x2(wa[q], uA);
+          wb[q] = mul_f16x2(wb[q], uB);
+        }
       }
 #pragma unroll
       for (int nb = 0; nb < NB; ++nb) {
@@ -390,7 +424,7 @@ constexpr size_t kSmemPerSm = 228 * 1024;   // shared memory of an SM; every res
 
 // Picks the K split, finishes the arguments and launches.  The dynamic shared-memory limit is raised and the
 // kernel's register count read once per device and instantiation.
-template <int EB, int NB, bool QUAD>
+template <int EB, int NB, bool QUAD, bool I4>
 vq_status launch_one(WarpTabArgs a, long long tiles, int sms, cudaStream_t s) {
   constexpr int TB = QUAD ? 9 : EB;
   static int regs_of[kMaxDevices] = {};
@@ -399,9 +433,9 @@ vq_status launch_one(WarpTabArgs a, long long tiles, int sms, cudaStream_t s) {
   int regs = __atomic_load_n(&regs_of[dev], __ATOMIC_ACQUIRE);
   if (!regs) {
     cudaFuncAttributes fa;
-    if (cudaFuncSetAttribute(warptab_kernel<EB, NB, QUAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemLimit)) !=
+    if (cudaFuncSetAttribute(warptab_kernel<EB, NB, QUAD, I4>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemLimit)) !=
             cudaSuccess ||
-        cudaFuncGetAttributes(&fa, warptab_kernel<EB, NB, QUAD>) != cudaSuccess || fa.numRegs < 1)
+        cudaFuncGetAttributes(&fa, warptab_kernel<EB, NB, QUAD, I4>) != cudaSuccess || fa.numRegs < 1)
       return VQ_ERR_CUDA;
     regs = fa.numRegs;
     __atomic_store_n(&regs_of[dev], regs, __ATOMIC_RELEASE);
@@ -427,19 +461,19 @@ vq_status launch_one(WarpTabArgs a, long long tiles, int sms, cudaStream_t s) {
   // A plain launch, in stream order.  (With programmatic dependent launch the next launch's CTAs take the
   // SM slots this grid leaves free and stay where they land: two such layers back to back then run with
   // 3 CTAs on some SMs and 1 on others; measured 31.5 against 23.2 us on 4096 x 14336.)
-  warptab_kernel<EB, NB, QUAD><<<static_cast<unsigned>(tiles), static_cast<unsigned>(wk) * 32u, smem_bytes, s>>>(a);
+  warptab_kernel<EB, NB, QUAD, I4><<<static_cast<unsigned>(tiles), static_cast<unsigned>(wk) * 32u, smem_bytes, s>>>(a);
   return check_launch();
 }
 
 template <int EB, bool QUAD = false>
 vq_status launch_eb(const WarpTabArgs& a, int nb, long long tiles, int sms, cudaStream_t s) {
-  return nb == 1 ? launch_one<EB, 1, QUAD>(a, tiles, sms, s) : launch_one<EB, 2, QUAD>(a, tiles, sms, s);
+  if (a.cb_int4) return nb == 1 ? launch_one<EB, 1, QUAD, true>(a, tiles, sms, s) : launch_one<EB, 2, QUAD, true>(a, tiles, sms, s);
+  return nb == 1 ? launch_one<EB, 1, QUAD, false>(a, tiles, sms, s) : launch_one<EB, 2, QUAD, false>(a, tiles, sms, s);
 }
 
 }  // namespace
 
 bool warptab_covers(const Geometry& g) {
-  if (g.cb_int4) return false;
   const int eb = pair_bits(g);
   if (eb < 1 || eb > 8) return false;
   if (g.K % 64 || g.Bc % 64) return false;
@@ -478,6 +512,7 @@ vq_status launch_gemm_warptab_group(const StreamCall& call, cudaStream_t s) {
   a.b = quad_format(g) ? 9 : g.b;
   a.entries = quad_format(g) ? 512 : g.entries;
   a.cb_int8 = g.cb_int8;
+  a.cb_int4 = g.cb_int4;
   a.Br = g.Br;
   a.br_shift = g.Br == 1 ? 0 : g.Br == 2 ? 1 : g.Br == 4 ? 2 : 3;
   a.bsteps = g.Bc / 64;

@@ -165,6 +165,7 @@ GROUPS = [
     (vq_synth.LayerSpec("g_pt_d1b2", N=0, K=1024, d=1, b=2, Br=1, Bc=256, int8=True), [33, 200]),
     (vq_synth.LayerSpec("g_pt_d2b8", N=0, K=768, d=2, b=8, Br=256, Bc=256, int8=False), [256, 512]),
     (vq_synth.LayerSpec("g_pt_d4b8", N=0, K=1024, d=4, b=8, Br=128, Bc=256, int8=True), [128, 384]),
+    (vq_synth.LayerSpec("g_pt_i4cb", N=0, K=1280, d=2, b=5, Br=4, Bc=256, int8=2), [100, 36, 64]),
 ]
 
 
@@ -558,21 +559,30 @@ def test_assign_indices_rejects_what_it_does_not_cover():
 
 
 INT4_CODEBOOK_CASES = [
-    vq_synth.LayerSpec("i4cb_d2b3", N=64, K=1024, d=2, b=3, Br=32, Bc=256, int8=2),
-    vq_synth.LayerSpec("i4cb_d2b6", N=37, K=256, d=2, b=6, Br=37, Bc=128, int8=2),
-    vq_synth.LayerSpec("i4cb_d1b4", N=20, K=384, d=1, b=4, Br=4, Bc=96, int8=2),
-    vq_synth.LayerSpec("i4cb_d4b8", N=16, K=1280, d=4, b=8, Br=16, Bc=640, int8=2),
-    vq_synth.LayerSpec("i4cb_d4b8_tile", N=96, K=2560, d=4, b=8, Br=32, Bc=512, int8=2),   # tile decode kernel
-    vq_synth.LayerSpec("i4cb_d1b4_tile", N=40, K=512, d=1, b=4, Br=8, Bc=128, int8=2),
+    # (layer, whether a tuned kernel takes it: the pair-table kernel does when blocks have 1/2/4/8 or a multiple
+    # of 16 rows and block columns are multiples of 64)
+    (vq_synth.LayerSpec("i4cb_d2b3", N=64, K=1024, d=2, b=3, Br=32, Bc=256, int8=2), True),
+    (vq_synth.LayerSpec("i4cb_d2b6", N=37, K=256, d=2, b=6, Br=37, Bc=128, int8=2), False),
+    (vq_synth.LayerSpec("i4cb_d1b4", N=20, K=384, d=1, b=4, Br=4, Bc=96, int8=2), False),
+    (vq_synth.LayerSpec("i4cb_d4b8", N=16, K=1280, d=4, b=8, Br=16, Bc=640, int8=2), True),
+    (vq_synth.LayerSpec("i4cb_d4b8_tile", N=96, K=2560, d=4, b=8, Br=32, Bc=512, int8=2), True),   # tile decode kernel
+    (vq_synth.LayerSpec("i4cb_d1b4_tile", N=40, K=512, d=1, b=4, Br=8, Bc=128, int8=2), True),
+    (vq_synth.LayerSpec("i4cb_d2b5_4x256", N=212, K=1280, d=2, b=5, Br=4, Bc=256, int8=2), True),
+    (vq_synth.LayerSpec("i4cb_d1b2_1x128", N=50, K=1152, d=1, b=2, Br=1, Bc=128, int8=2), True),
+    (vq_synth.LayerSpec("i4cb_d1b1_2x64", N=34, K=384, d=1, b=1, Br=2, Bc=64, int8=2), True),
 ]
 
 
-@pytest.mark.parametrize("spec", INT4_CODEBOOK_CASES, ids=lambda s: s.name)
-def test_int4_codebooks_with_group_scales(spec):
+@pytest.mark.parametrize("spec,tuned", INT4_CODEBOOK_CASES, ids=lambda v: v.name if hasattr(v, "name") else None)
+def test_int4_codebooks_with_group_scales(spec, tuned):
     """INT4 codebooks decoded with a scale per row and group of 128 columns (Sec. 4.2): bit-exact
-    decode, mat-vec within the tolerance, through the format-generic kernels; VQ_IMPL_TUNED must refuse
-    these shapes (it takes this codebook type for the 2-D 5/6-bit tall-block formats only, tested below)."""
+    decode, mat-vec within the tolerance through the format-generic kernel and through whatever the
+    library picks; VQ_IMPL_TUNED runs the pair-table kernel (entries in the tables as exact fp16 integers,
+    every looked-up pair multiplied by its row-group scale) on the shapes it takes and refuses the others."""
     _check_layer(spec, seed=55, batches=(1, 5, 16), impls=[vq.VQ_IMPL_GENERIC, vq.VQ_IMPL_AUTO])
+    if tuned:
+        _check_layer(spec, seed=56, batches=(1, 8, 9), impls=[vq.VQ_IMPL_TUNED], decode=False)
+        return
     L = draw(spec, 55)
     dev = DeviceLayer(spec, L)
     with pytest.raises(vq.VQError) as err:

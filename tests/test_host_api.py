@@ -199,7 +199,8 @@ def test_grouped_call_argument_errors_and_launch_counts():
     # small blocks / index widths only the pair-table kernel takes: 2-D 5-bit 4x256, 1-D 2-bit 1x256, 4-D 8-bit 128x256
     pair = [vq.VQFormat(6144, 4096, 2, 5, 4, 256, vq.VQ_CB_INT8_SCALED), vq.VQFormat(6144, 4096, 1, 2, 1, 256, vq.VQ_CB_INT8_SCALED),
             vq.VQFormat(6144, 4096, 4, 8, 128, 256, vq.VQ_CB_FP16)]
-    i4 = vq.VQFormat(6144, 4096, 2, 5, 4, 256, vq.VQ_CB_INT4_G128)   # INT4 codebooks on small blocks: generic kernel, member by member
+    i4 = vq.VQFormat(6142, 4096, 2, 5, 37, 256, vq.VQ_CB_INT4_G128)   # INT4 codebooks on 37-row blocks: generic kernel, member by member
+    pair.append(vq.VQFormat(6144, 4096, 2, 5, 4, 256, vq.VQ_CB_INT4_G128))
     for batch in (1, 4, 16):
         assert vq.vq_grouped_kernel_launches(row4, 3, batch) == 1
         assert vq.vq_grouped_kernel_launches(blk6, 3, batch) == 1
