@@ -38,7 +38,7 @@ namespace {
 
 using namespace dev;
 
-constexpr int kMaxWarps = 8;   // per CTA; three CTAs of that size fit an SM's registers
+constexpr int kMaxWarps = 8;   // per CTA; four CTAs of that size fit an SM's registers at batch <= 8 (64 per thread), three above
 constexpr int kChunkSteps = 8;   // steps per staged chunk of the index stream
 constexpr int kStages = 2;
 constexpr int kBuildGroup = 4;   // table words per lane whose loads are in flight together
@@ -62,16 +62,15 @@ struct WarpTabArgs {
   const __half* X;
   long long stride;
   int K, batch;
-  int d, b, entries, cb_int8;
+  int d, b, cb_int8;              // b: log2 of the entries of a block's codebook (a 4-D codebook counts as a 2-D one of 512)
   int cb_int4;                    // 4-bit entries (tables hold them as exact fp16 integers) + a scale per row and 128 columns
   int Br, br_shift;               // br_shift: log2(Br) when Br < 16
   int bsteps;                     // 64-column steps per codebook block (Bc / 64)
   int blocks_per_row;
   int steps_total, steps_per_warp;
-  int tbl_words;                  // words of one warp's tables (tables << EB)
+  int tbl_words;                  // words of one warp's tables
   int tbl_bytes;                  // the same in bytes, rounded up to 16
   int warp_bytes;                 // shared memory of one warp: tables, then kStages chunk stages
-  int red_off;                    // byte offset of the reduction buffer in shared memory (it reuses the warps' regions)
 };
 
 __device__ __forceinline__ uint32_t mul_f16x2(uint32_t a, uint32_t b) {
@@ -385,7 +384,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
   __syncthreads();   // the reduction buffer lies over the warps' tables and stages
 
   // K parts of the warps meet in shared memory; thread i then owns output (batch row i / 16, row i % 16).
-  float* red = reinterpret_cast<float*>(smem + a.red_off);
+  float* red = reinterpret_cast<float*>(smem);   // over the warps' tables and stages, which are no longer needed
 #pragma unroll
   for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
@@ -510,7 +509,6 @@ vq_status launch_gemm_warptab_group(const StreamCall& call, cudaStream_t s) {
   // (a 4-D codebook of 256 entries lies in memory like a 2-D one of 512: the table build treats it as such)
   a.d = quad_format(g) ? 2 : g.d;
   a.b = quad_format(g) ? 9 : g.b;
-  a.entries = quad_format(g) ? 512 : g.entries;
   a.cb_int8 = g.cb_int8;
   a.cb_int4 = g.cb_int4;
   a.Br = g.Br;
@@ -523,7 +521,6 @@ vq_status launch_gemm_warptab_group(const StreamCall& call, cudaStream_t s) {
   a.tbl_bytes = (a.tbl_words * 4 + 15) / 16 * 16;
   const int tbl_align = region_align(table_bits(g));
   a.warp_bytes = (a.tbl_bytes + kStages * stage_bytes(eb) + tbl_align - 1) / tbl_align * tbl_align;
-  a.red_off = 0;
   int sms = 0;
   if (device_sms(&sms) != VQ_OK) return VQ_ERR_CUDA;
   switch (eb) {
