@@ -225,6 +225,10 @@ PAIR_TABLE_CASES = [
     vq_synth.LayerSpec("pt_d4b8_128x256_i8", N=256, K=1024, d=4, b=8, Br=128, Bc=256, int8=True),
     vq_synth.LayerSpec("pt_d4b8_16x64", N=48, K=704, d=4, b=8, Br=16, Bc=64, int8=False, cb_sigma=0.015),
     vq_synth.LayerSpec("pt_d4b8_8x128_i8", N=40, K=640, d=4, b=8, Br=8, Bc=128, int8=True),
+    # degenerate shapes: one row, one step, one block spanning K, the largest table set a warp may hold
+    vq_synth.LayerSpec("pt_one_row_one_step", N=1, K=64, d=2, b=5, Br=1, Bc=64, int8=True),
+    vq_synth.LayerSpec("pt_17_rows", N=17, K=128, d=1, b=3, Br=1, Bc=64, int8=False),
+    vq_synth.LayerSpec("pt_block_spans_k", N=5, K=4096, d=2, b=6, Br=1, Bc=4096, int8=True),
 ]
 
 
