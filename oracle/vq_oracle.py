@@ -183,6 +183,63 @@ def gemm(f: Fmt, idx, cb, scale, X, rows=None, threads: int = 1):
     return Y, A
 
 
+# ---- block-wise data normalisation (App. on blockwise data normalization) ---------------------------
+# The quantizer divides every sub-row of `block_cols` columns by a scale before clustering and stores the
+# scale as a 4-bit integer on a log2 grid; the decoder multiplies the looked-up values by the inverse.
+# What the decoder needs is, per codebook block, the 16 values the 4-bit code can stand for: a table
+# lut[blk][16] (binary16) and a code per (row, sub-row).  The grid itself (norm_lut_log2 below) belongs
+# to the quantizer; its printed formula is garbled in the paper, the reading taken is
+#   value(s) = 2^(a*s + z),  s = 0..15,  a = step of the group, z = floating-point offset,
+# rounded once to binary16.
+def norm_lut_log2(a: float, z: float) -> np.ndarray:
+    """The 16 scales of one group on the log2 grid: float16 [16]."""
+    return np.array([2.0 ** (a * s + z) for s in range(16)], dtype=np.float64).astype(np.float16)
+
+
+def norm_code_row_bytes(K: int, block_cols: int) -> int:
+    """Bytes of one row of 4-bit codes (two per byte, low nibble first)."""
+    return (K // block_cols + 1) // 2
+
+
+def norm_factors(f: Fmt, codes, lut, block_cols: int) -> np.ndarray:
+    """F[n][k] (float64) = lut[blk(n, k)][code(n, k // block_cols)]; blk ordered as the codebooks are."""
+    assert f.Bc % block_cols == 0 and block_cols % f.d == 0
+    codes = np.ascontiguousarray(codes, dtype=np.uint8).reshape(f.N, norm_code_row_bytes(f.K, block_cols))
+    lut = _u16(lut).view(np.float16).astype(np.float64).reshape(f.n_blocks, 16)
+    F = np.empty((f.N, f.K), np.float64)
+    for n in range(f.N):
+        for j in range(f.K // block_cols):
+            byte = int(codes[n, j // 2])
+            code = (byte >> 4) if (j % 2) else (byte & 15)
+            k0 = j * block_cols
+            blk = (n // f.Br) * (f.K // f.Bc) + k0 // f.Bc
+            F[n, k0:k0 + block_cols] = lut[blk, code]
+    return F
+
+
+def normalized_decode(f: Fmt, idx, cb, scale, codes, lut, block_cols: int):
+    """(W exact float64, W16 uint16): the decoded weight times its sub-row's scale; the product of at most
+    three short significands (30 bits) is exact in float64 and rounded once to binary16."""
+    We, _ = decode(f, idx, cb, scale, exact=True, half=False)
+    Wn = We * norm_factors(f, codes, lut, block_cols)
+    return Wn, Wn.astype(np.float16).view(np.uint16)
+
+
+def normalized_gemm(f: Fmt, idx, cb, scale, codes, lut, block_cols: int, X, rows=None):
+    """Y[m][r], A[m][r] (float64, k ascending) on the normalised weights."""
+    Wn, _ = normalized_decode(f, idx, cb, scale, codes, lut, block_cols)
+    if rows is not None:
+        Wn = Wn[np.asarray(rows)]
+    Xd = _u16(np.atleast_2d(X)).view(np.float16).astype(np.float64)
+    Y = np.empty((Xd.shape[0], Wn.shape[0]), np.float64)
+    A = np.empty_like(Y)
+    for m in range(Xd.shape[0]):
+        P = Wn * Xd[m][None, :]
+        Y[m] = np.cumsum(P, axis=1)[:, -1]      # left to right over k
+        A[m] = np.abs(P).sum(axis=1)
+    return Y, A
+
+
 def dense_gemm(W: np.ndarray, X) -> np.ndarray:
     W = np.ascontiguousarray(W, dtype=np.float64)
     X = _u16(np.atleast_2d(X))

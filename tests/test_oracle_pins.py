@@ -555,3 +555,62 @@ def test_int4_codebook_with_group_scales_hand_values():
     Y, A = orc.gemm(f, idx, cb, scale, x)
     assert np.allclose(Y[0], W @ x.astype(np.float64), rtol=1e-14, atol=0)
 
+
+
+# ---- block-wise normalisation at decode (App. on blockwise data normalization) ------------------------
+def test_norm_lut_log2_hand_values():
+    """2^(a*s + z): a = 1, z = -3 gives the powers of two 1/8 .. 4096 exactly; a = 0.5 puts sqrt(2) at s = 1,
+    whose nearest binary16 is 1.4140625 (0x3DA8: 1.4140625 < 1.41421356 < 1.415039, nearer the lower)."""
+    lut = orc.norm_lut_log2(1.0, -3.0)
+    assert lut.dtype == np.float16 and [float(v) for v in lut] == [2.0 ** (s - 3) for s in range(16)]
+    half = orc.norm_lut_log2(0.5, 0.0)
+    assert float(half[0]) == 1.0 and float(half[2]) == 2.0 and float(half[4]) == 4.0
+    assert half.view(np.uint16)[1] == 0x3DA8 and float(half[1]) == 1.4140625
+    assert float(orc.norm_lut_log2(0.0, 0.0)[7]) == 1.0                      # zero step: unit scaling whatever the code
+
+
+def test_normalized_decode_hand_built():
+    """2 x 8 weights, 2-D entries, 1-bit indices, one codebook for the whole matrix, sub-rows of 4 columns:
+    every number below is written by hand."""
+    f = orc.Fmt(N=2, K=8, d=2, b=1, Br=2, Bc=8, int8=False)
+    cb = np.array([[1.0, 2.0], [-3.0, 0.5]], np.float16)                       # entry 0 = (1, 2), entry 1 = (-3, 0.5)
+    I = np.array([[0, 1, 1, 0], [1, 1, 0, 0]], np.int32)                       # 4 indices per row
+    idx = orc.pack(f, I)
+    lut = np.zeros((1, 16), np.float16)
+    lut[0, 0], lut[0, 3], lut[0, 9], lut[0, 15] = 1.0, 0.5, 4.0, 0.25
+    # codes: row 0 -> sub-rows (3, 9) = byte 0x93; row 1 -> (15, 0) = byte 0x0F   (low nibble = first sub-row)
+    codes = np.array([[0x93], [0x0F]], np.uint8)
+    assert orc.norm_code_row_bytes(8, 4) == 1
+    W, W16 = orc.normalized_decode(f, idx, cb, None, codes, lut, 4)
+    expect = np.array([[0.5, 1.0, -1.5, 0.25, -12.0, 2.0, 4.0, 8.0],
+                       [-0.75, 0.125, -0.75, 0.125, 1.0, 2.0, 1.0, 2.0]])
+    assert np.array_equal(W, expect)
+    assert np.array_equal(W16.view(np.float16).astype(np.float64), expect)
+    x = np.array([[1, 1, 1, 1, 1, 1, 1, 1], [2, 0, 0, 0, 0, 0, 0, -1]], np.float16)
+    Y, A = orc.normalized_gemm(f, idx, cb, None, codes, lut, 4, x)
+    assert Y.tolist() == [[2.25, 4.75], [-7.0, -3.5]]
+    assert A.tolist() == [[29.25, 7.75], [9.0, 3.5]]
+
+
+def test_normalized_decode_int8_rounds_once_and_unit_lut_is_plain_decode():
+    """int8 codebook: w = fp16(scale * c * norm), one rounding of the exact product: scale 0.0999755859375
+    (0x2E66 = 819/8192), c = 127, norm 1.4140625 (= 181/128): exact 819 * 127 * 181 / 2^20 = 18826353 / 1048576
+    = 17.9542..., between the binary16 neighbours 17.953125 and 17.96875 and nearer the first.  With every
+    table entry 1.0 the result is the plain decode."""
+    f = orc.Fmt(N=1, K=2, d=1, b=1, Br=1, Bc=2, int8=True)
+    cb = np.array([127, -128], np.int8)
+    scale = np.array([0x2E66], np.uint16)
+    idx = orc.pack(f, np.array([[0, 1]], np.int32))
+    lut = np.full((1, 16), 1.4140625, np.float16)
+    W, W16 = orc.normalized_decode(f, idx, cb, scale, np.array([[5]], np.uint8), lut, 2)
+    assert Fraction(float(W[0, 0])) == Fraction(18826353, 1048576)
+    assert Fraction(float(W[0, 1])) == Fraction(819 * -128 * 181, 1048576)
+    assert float(W16.view(np.float16)[0, 0]) == 17.953125
+    spec = vq_synth.LayerSpec("n", N=6, K=32, d=2, b=3, Br=3, Bc=16, int8=True)
+    fo = orc.Fmt(spec.N, spec.K, spec.d, spec.b, spec.Br, spec.Bc, spec.int8)
+    L = vq_synth.make_layer(spec, fo.stride, 3)
+    ones = np.ones((fo.n_blocks, 16), np.float16)
+    codes = vq_synth.random_bytes(1, 2, spec.N * orc.norm_code_row_bytes(spec.K, 8)).reshape(spec.N, -1)
+    _, plain = orc.decode(fo, L.idx, L.cb, L.scale, exact=False)
+    _, normed = orc.normalized_decode(fo, L.idx, L.cb, L.scale, codes, ones, 8)
+    assert np.array_equal(plain, normed)
