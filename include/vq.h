@@ -286,6 +286,35 @@ size_t vq_int4g128_workspace_bytes(int32_t n_rows, int batch);
 vq_status vq_assign_indices(const vq_format* fmt, const void* d_W, const void* d_cb,
                             const void* d_scale, const void* d_hdiag, void* d_idx, void* stream);
 
+/* Block-wise data normalisation applied at the decode step (paper appendix "Blockwise data
+ * normalization": every sub-row of a codebook group is divided by a scale before clustering, the scale is
+ * stored as a 4-bit integer on a log2 grid, and the inverse scaling is applied when the weights are decoded).
+ * Layout fixed by this library (the paper's formula for the grid is garbled and it fixes no layout):
+ *   norm_block_cols : columns per sub-row (the paper names 16, 32, 64); divides block_cols, multiple of vq_dim.
+ *   d_norm_codes    : device, one 4-bit code per row and sub-row, two per byte, low nibble = lower sub-row;
+ *                     rows start every vq_norm_info().code_row_bytes = ceil(K / norm_block_cols / 2) bytes.
+ *   d_norm_lut      : device binary16 [blocks][16], blocks ordered as the codebooks: the 16 scales a code of
+ *                     that codebook block can stand for (on the paper's grid: 2^(a * code + z) with the
+ *                     group's step a and offset z; the decoder needs the values only).
+ *   w[n][k] = value decoded as without normalisation * d_norm_lut[blk(n, k)][code(n, k / norm_block_cols)].
+ * vq_decode_weights_normalized writes binary16(w), the exact product rounded once; vq_gemm_small_batch_normalized
+ * computes Y[m][n] = sum_k w[n][k] X[m][k] (fp32 accumulation, one rounding), batch 1..16.  Both run in
+ * format-generic kernels (every valid format; no tuned variant, no workspace, plain stream-order launches).
+ * Errors: as vq_decode_weights / vq_gemm_small_batch (without WORKSPACE); NULL for a missing code or table
+ * pointer; SHAPE for a norm_block_cols that does not divide block_cols or is not a multiple of vq_dim. */
+typedef struct {
+  size_t code_row_bytes;   /* bytes between rows of d_norm_codes                    */
+  size_t codes_bytes;      /* n_rows * code_row_bytes                                */
+  size_t lut_bytes;        /* blocks * 16 * 2                                        */
+} vq_norm_info_t;
+vq_status vq_norm_info(const vq_format* fmt, int norm_block_cols, vq_norm_info_t* out);
+vq_status vq_decode_weights_normalized(const vq_format* fmt, const void* d_idx, const void* d_cb, const void* d_scale,
+                                       const void* d_norm_codes, const void* d_norm_lut, int norm_block_cols, void* d_W,
+                                       void* stream);
+vq_status vq_gemm_small_batch_normalized(const vq_format* fmt, const void* d_idx, const void* d_cb, const void* d_scale,
+                                         const void* d_norm_codes, const void* d_norm_lut, int norm_block_cols, const void* d_X,
+                                         void* d_Y, int batch, void* stream);
+
 /* Uniformly quantized weights expanded to binary16: the yard-sticks of the transfer + decode
  * experiment (paper App. B: time to move and unpack a layer stored as FP16, INT8, INT4 or VQ),
  * timed beside vq_decode_weights.  w = s * q (Sec. 2.1), exact product rounded once to binary16.

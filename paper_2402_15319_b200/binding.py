@@ -77,6 +77,10 @@ _SIGNATURES = {
     "vq_workspace_bytes": (ctypes.c_size_t, [ctypes.c_void_p, ctypes.c_int]),
     "vq_workspace_bytes_host": (ctypes.c_size_t, [ctypes.c_void_p, ctypes.c_int]),
     "vq_decode_weights": (ctypes.c_int, [ctypes.c_void_p] * 6),
+    "vq_norm_info": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]),
+    "vq_decode_weights_normalized": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]),
+    "vq_gemm_small_batch_normalized": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
+                                                       ctypes.c_int, ctypes.c_void_p]),
     "vq_gemv": (ctypes.c_int, [ctypes.c_void_p] * 7 + [ctypes.c_size_t, ctypes.c_void_p]),
     "vq_gemm_small_batch": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
     "vq_gemm_small_batch_impl": (ctypes.c_int, [ctypes.c_void_p] * 6 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_int]),
@@ -163,6 +167,34 @@ def vq_decode_weights(fmt: VQFormat, d_idx, d_cb, d_scale, d_W, stream=None) -> 
     c = fmt.c()
     _check(load().vq_decode_weights(ctypes.byref(c), _ptr(d_idx), _ptr(d_cb), _ptr(d_scale), _ptr(d_W),
                                     _stream(stream)), "vq_decode_weights")
+
+
+class _CNormInfo(ctypes.Structure):
+    _fields_ = [("code_row_bytes", ctypes.c_size_t), ("codes_bytes", ctypes.c_size_t), ("lut_bytes", ctypes.c_size_t)]
+
+
+def vq_norm_info(fmt: VQFormat, norm_block_cols: int):
+    """(code_row_bytes, codes_bytes, lut_bytes) of the block-wise normalisation buffers."""
+    c = fmt.c()
+    out = _CNormInfo()
+    _check(load().vq_norm_info(ctypes.byref(c), int(norm_block_cols), ctypes.byref(out)), "vq_norm_info")
+    return int(out.code_row_bytes), int(out.codes_bytes), int(out.lut_bytes)
+
+
+def vq_decode_weights_normalized(fmt: VQFormat, d_idx, d_cb, d_scale, d_norm_codes, d_norm_lut, norm_block_cols: int, d_W,
+                                 stream=None) -> None:
+    c = fmt.c()
+    _check(load().vq_decode_weights_normalized(ctypes.byref(c), _ptr(d_idx), _ptr(d_cb), _ptr(d_scale), _ptr(d_norm_codes),
+                                               _ptr(d_norm_lut), int(norm_block_cols), _ptr(d_W), _stream(stream)),
+           "vq_decode_weights_normalized")
+
+
+def vq_gemm_small_batch_normalized(fmt: VQFormat, d_idx, d_cb, d_scale, d_norm_codes, d_norm_lut, norm_block_cols: int, d_X, d_Y,
+                                   batch: int, stream=None) -> None:
+    c = fmt.c()
+    _check(load().vq_gemm_small_batch_normalized(ctypes.byref(c), _ptr(d_idx), _ptr(d_cb), _ptr(d_scale), _ptr(d_norm_codes),
+                                                 _ptr(d_norm_lut), int(norm_block_cols), _ptr(d_X), _ptr(d_Y), int(batch),
+                                                 _stream(stream)), "vq_gemm_small_batch_normalized")
 
 
 def vq_gemv(fmt: VQFormat, d_idx, d_cb, d_scale, d_x, d_y, d_ws, stream=None) -> None:

@@ -256,6 +256,56 @@ vq_status vq_gemm_small_batch_grouped(const vq_format* fmt, const vq_group_membe
   return VQ_OK;
 }
 
+// Sub-rows of norm_block_cols columns: they tile a codebook block's columns and hold whole VQ vectors.
+static vq_status check_norm(const vq_format* fmt, const void* d_codes, const void* d_lut, int norm_block_cols) {
+  if (!d_codes || !d_lut) return VQ_ERR_NULL;
+  if (norm_block_cols <= 0 || fmt->block_cols % norm_block_cols || norm_block_cols % fmt->vq_dim) return VQ_ERR_SHAPE;
+  if (!aligned16(d_codes) || !aligned16(d_lut)) return VQ_ERR_ALIGN;
+  return VQ_OK;
+}
+
+vq_status vq_norm_info(const vq_format* fmt, int norm_block_cols, vq_norm_info_t* out) {
+  if (!out) return VQ_ERR_NULL;
+  Geometry g;
+  vq_status st = make_geometry(fmt, &g);
+  if (st != VQ_OK) return st;
+  if (norm_block_cols <= 0 || g.Bc % norm_block_cols || norm_block_cols % g.d) return VQ_ERR_SHAPE;
+  out->code_row_bytes = (g.K / norm_block_cols + 1) / 2;
+  out->codes_bytes = static_cast<size_t>(g.N) * out->code_row_bytes;
+  out->lut_bytes = static_cast<size_t>(g.N / g.Br) * g.blocks_per_row * 16 * sizeof(uint16_t);
+  return VQ_OK;
+}
+
+vq_status vq_decode_weights_normalized(const vq_format* fmt, const void* d_idx, const void* d_cb, const void* d_scale,
+                                       const void* d_norm_codes, const void* d_norm_lut, int norm_block_cols, void* d_W,
+                                       void* stream) {
+  Geometry g;
+  LayerPtrs p;
+  vq_status st = check_layer(fmt, d_idx, d_cb, d_scale, &g, &p);
+  if (st != VQ_OK) return st;
+  st = check_norm(fmt, d_norm_codes, d_norm_lut, norm_block_cols);
+  if (st != VQ_OK) return st;
+  if (!d_W) return VQ_ERR_NULL;
+  if (!aligned16(d_W)) return VQ_ERR_ALIGN;
+  return launch_decode_norm(g, p, d_norm_codes, d_norm_lut, norm_block_cols, static_cast<__half*>(d_W), static_cast<cudaStream_t>(stream));
+}
+
+vq_status vq_gemm_small_batch_normalized(const vq_format* fmt, const void* d_idx, const void* d_cb, const void* d_scale,
+                                         const void* d_norm_codes, const void* d_norm_lut, int norm_block_cols, const void* d_X,
+                                         void* d_Y, int batch, void* stream) {
+  Geometry g;
+  LayerPtrs p;
+  vq_status st = check_layer(fmt, d_idx, d_cb, d_scale, &g, &p);
+  if (st != VQ_OK) return st;
+  st = check_norm(fmt, d_norm_codes, d_norm_lut, norm_block_cols);
+  if (st != VQ_OK) return st;
+  if (batch < 1 || batch > 16) return VQ_ERR_BATCH;
+  if (!d_X || !d_Y) return VQ_ERR_NULL;
+  if (!aligned16(d_X) || !aligned16(d_Y)) return VQ_ERR_ALIGN;
+  return launch_gemm_norm(g, p, d_norm_codes, d_norm_lut, norm_block_cols, static_cast<const __half*>(d_X), static_cast<__half*>(d_Y),
+                          batch, static_cast<cudaStream_t>(stream));
+}
+
 vq_status vq_gemm_small_batch(const vq_format* fmt, const void* d_idx, const void* d_cb,
                               const void* d_scale, const void* d_X, void* d_Y, int batch,
                               void* d_ws, size_t ws_bytes, void* stream) {

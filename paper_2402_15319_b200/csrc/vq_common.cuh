@@ -84,6 +84,12 @@ vq_status launch_gemm_warptab_group(const StreamCall& call, cudaStream_t s);
 bool warptab_covers(const Geometry& g);
 vq_status launch_int4g128_rowcb(int N, int K, const uint8_t* q, const __half* scale, const __half* X, __half* Y, int batch,
                                 cudaStream_t s);
+// Block-wise normalisation at decode (format-generic kernels): codes = 4-bit code per row and sub-row of
+// block_cols columns, lut = 16 binary16 scales per codebook block.
+vq_status launch_decode_norm(const Geometry& g, const LayerPtrs& p, const void* codes, const void* lut, int block_cols,
+                             __half* W, cudaStream_t s);
+vq_status launch_gemm_norm(const Geometry& g, const LayerPtrs& p, const void* codes, const void* lut, int block_cols,
+                           const __half* X, __half* Y, int batch, cudaStream_t s);
 vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s);
 // E-step: nearest centroid under diagonal weights, packed into the index stream `idx` (output).
 vq_status launch_assign(const Geometry& g, const LayerPtrs& p, const __half* W, const float* hdiag, uint8_t* idx,

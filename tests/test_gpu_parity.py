@@ -611,6 +611,62 @@ def test_int4_codebooks_in_the_tall_block_kernel(spec):
     _check_layer(spec, seed=77, batches=(1, 3, 8, 16), impls=[vq.VQ_IMPL_TUNED, vq.VQ_IMPL_AUTO, vq.VQ_IMPL_GENERIC], decode=True)
 
 
+# ---- block-wise normalisation applied at decode ---------------------------------------------------------
+NORM_CASES = [
+    # (layer, columns per sub-row): the paper's sub-row sizes 16 / 32 / 64 and others, every codebook type,
+    # every d, ragged index groups, an odd number of sub-rows per row (a half-used last code byte)
+    (vq_synth.LayerSpec("nm_d2b6_i8", N=96, K=768, d=2, b=6, Br=32, Bc=256, int8=True), 32),
+    (vq_synth.LayerSpec("nm_d2b5_4x256_i8", N=52, K=1280, d=2, b=5, Br=4, Bc=256, int8=True), 64),
+    (vq_synth.LayerSpec("nm_d1b3_f16", N=37, K=208, d=1, b=3, Br=1, Bc=16, int8=False), 16),
+    (vq_synth.LayerSpec("nm_d4b8_f16", N=64, K=1536, d=4, b=8, Br=16, Bc=512, int8=False, cb_sigma=0.015), 16),
+    (vq_synth.LayerSpec("nm_d2b4_row_i8", N=40, K=2048, d=2, b=4, Br=1, Bc=2048, int8=True), 2048),
+    (vq_synth.LayerSpec("nm_d2b3_i4cb", N=64, K=1024, d=2, b=3, Br=32, Bc=256, int8=2), 32),
+    (vq_synth.LayerSpec("nm_d2b7_odd", N=9, K=36, d=2, b=7, Br=3, Bc=12, int8=False), 4),
+]
+
+
+@pytest.mark.parametrize("spec,nbc", NORM_CASES, ids=lambda v: v.name if hasattr(v, "name") else None)
+def test_normalized_decode_and_gemm(spec, nbc):
+    """vq_decode_weights_normalized bit-exact and vq_gemm_small_batch_normalized within the tolerance, against
+    the oracle's decoded value times the scale selected by the sub-row's 4-bit code."""
+    import torch
+    f = oracle_fmt(spec)
+    L = draw(spec, 71)
+    codes, lut = vq_synth.make_norm(spec, nbc, 72)
+    dev = DeviceLayer(spec, L)
+    row_bytes, codes_bytes, lut_bytes = vq.vq_norm_info(dev.fmt, nbc)
+    assert codes.shape == (spec.N, row_bytes) and codes.nbytes == codes_bytes and lut.nbytes == lut_bytes
+    d_codes, d_lut = torch.from_numpy(codes).cuda(), torch.from_numpy(lut).cuda()
+    dW, raw = guarded((spec.N, spec.K), torch.float16, "cuda")
+    vq.vq_decode_weights_normalized(dev.fmt, dev.idx, dev.cb, dev.scale, d_codes, d_lut, nbc, dW)
+    torch.cuda.synchronize()
+    assert_guards_intact(raw, spec.name)
+    _, W16 = orc.normalized_decode(f, L.idx, L.cb, L.scale, codes, lut, nbc)
+    assert np.array_equal(dW.cpu().numpy().view(np.uint16), W16), f"{spec.name}: normalised decode not bit-exact"
+    for batch in (1, 3, 8, 16):
+        X = vq_synth.make_x(spec, 73, batch)
+        dY, rawy = guarded((batch, spec.N), torch.float16, "cuda")
+        vq.vq_gemm_small_batch_normalized(dev.fmt, dev.idx, dev.cb, dev.scale, d_codes, d_lut, nbc, torch.from_numpy(X).cuda(), dY, batch)
+        torch.cuda.synchronize()
+        assert_guards_intact(rawy, spec.name)
+        Y, A = orc.normalized_gemm(f, L.idx, L.cb, L.scale, codes, lut, nbc, X)
+        assert_outputs_close(dY.cpu().numpy(), Y, A, f"{spec.name} normalised batch={batch}")
+
+
+def test_normalized_with_unit_table_equals_plain_entry_points():
+    """A table of ones switches the normalisation off: the decode equals vq_decode_weights bit for bit."""
+    import torch
+    spec = vq_synth.LayerSpec("nm_unit", N=128, K=512, d=2, b=6, Br=128, Bc=128, int8=False)
+    L = draw(spec, 5)
+    dev = DeviceLayer(spec, L)
+    codes, _ = vq_synth.make_norm(spec, 32, 6)
+    ones = torch.ones((spec.n_blocks, 16), dtype=torch.float16, device="cuda")
+    dW = torch.empty((spec.N, spec.K), dtype=torch.float16, device="cuda")
+    vq.vq_decode_weights_normalized(dev.fmt, dev.idx, dev.cb, dev.scale, torch.from_numpy(codes).cuda(), ones, 32, dW)
+    torch.cuda.synchronize()
+    assert np.array_equal(dW.cpu().numpy().view(np.uint16), dev.decode().view(np.uint16))
+
+
 @pytest.mark.parametrize("pinned", [True, False], ids=["pinned", "pageable"])
 def test_grouped_host_buffer_entry_point(pinned):
     """vq_gemm_small_batch_grouped_host: activations from host memory once for the group, every member's

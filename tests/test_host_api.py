@@ -231,3 +231,29 @@ def test_grouped_host_call_argument_errors():
     arr[1].n_rows = 8
     arr[0].d_Y = None
     assert call() == 1
+
+
+def test_normalized_entry_points_argument_errors_and_sizes():
+    """Block-wise normalisation: buffer sizes on the host, and every argument error before any launch."""
+    lib = vq.load()
+    fmt = vq.VQFormat(12, 256, 2, 5, 4, 128, vq.VQ_CB_INT8_SCALED)
+    assert vq.vq_norm_info(fmt, 32) == (4, 48, 3 * 2 * 16 * 2)            # 8 sub-rows -> 4 bytes per row; 6 blocks
+    assert vq.vq_norm_info(fmt, 128)[0] == 1                               # 2 sub-rows per row
+    assert vq.vq_norm_info(vq.VQFormat(3, 48, 1, 3, 1, 48, vq.VQ_CB_FP16), 16) == (2, 6, 3 * 16 * 2)   # 3 codes -> 2 bytes
+    c = fmt.c()
+
+    def dec(codes=FAKE, lut=FAKE, nbc=32, W=FAKE, scale=FAKE):
+        return lib.vq_decode_weights_normalized(ctypes.byref(c), FAKE, FAKE, scale, codes, lut, nbc, W, None)
+
+    def gemm(codes=FAKE, lut=FAKE, nbc=32, X=FAKE, Y=FAKE, batch=1):
+        return lib.vq_gemm_small_batch_normalized(ctypes.byref(c), FAKE, FAKE, FAKE, codes, lut, nbc, X, Y, batch, None)
+
+    assert dec(codes=None) == 1 and dec(lut=None) == 1 and dec(W=None) == 1 and dec(scale=None) == 1
+    assert dec(nbc=0) == 3 and dec(nbc=48) == 3 and dec(nbc=256) == 3       # must divide block_cols = 128
+    assert lib.vq_decode_weights_normalized(ctypes.byref(vq.VQFormat(12, 256, 4, 8, 4, 128, vq.VQ_CB_INT8_SCALED).c()),
+                                            FAKE, FAKE, FAKE, FAKE, FAKE, 2, FAKE, None) == 3            # not a multiple of vq_dim
+    assert dec(codes=ODD) == 4 and dec(lut=ODD) == 4 and dec(W=ODD) == 4
+    assert gemm(codes=None) == 1 and gemm(X=None) == 1 and gemm(Y=None) == 1
+    assert gemm(batch=0) == 6 and gemm(batch=17) == 6 and gemm(nbc=5) == 3 and gemm(X=ODD) == 4
+    out = ctypes.c_void_p(0)
+    assert lib.vq_norm_info(ctypes.byref(c), 32, None) == 1 and lib.vq_norm_info(ctypes.byref(c), 3, FAKE) == 3

@@ -112,6 +112,17 @@ def make_layer(spec: LayerSpec, stride: int, seed: int, layer_id: int = 0) -> La
     return Layer(spec, stride, idx, cb, scale)
 
 
+def make_norm(spec: LayerSpec, block_cols: int, seed: int, layer_id: int = 0):
+    """Block-wise normalisation inputs of one layer: uniform random 4-bit codes per row and sub-row of
+    `block_cols` columns (uint8 [N][ceil(K / block_cols / 2)], two codes per byte) and, per codebook block,
+    16 scales drawn uniformly from [0.25, 4) as float16 (the decoder treats the table as opaque values)."""
+    s0 = 16 * layer_id
+    row_bytes = (spec.K // block_cols + 1) // 2
+    codes = random_bytes(seed, s0 + 10, spec.N * row_bytes).reshape(spec.N, row_bytes)
+    lut = (0.25 + 3.75 * uniform01(seed, s0 + 11, spec.n_blocks * 16)).astype(np.float16).reshape(spec.n_blocks, 16)
+    return codes, lut
+
+
 def make_x(spec: LayerSpec, seed: int, batch: int, layer_id: int = 0) -> np.ndarray:
     """Activations X[batch][K] ~ N(0,1) as float16."""
     return normal(seed, 16 * layer_id + 4, batch * spec.K).astype(np.float16).reshape(batch, spec.K)
