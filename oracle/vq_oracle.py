@@ -190,7 +190,8 @@ def gemm(f: Fmt, idx, cb, scale, X, rows=None, threads: int = 1):
 # lut[blk][16] (binary16) and a code per (row, sub-row).  The grid itself (norm_lut_log2 below) belongs
 # to the quantizer; its printed formula is garbled in the paper, the reading taken is
 #   value(s) = 2^(a*s + z),  s = 0..15,  a = step of the group, z = floating-point offset,
-# rounded once to binary16.
+# rounded once to binary16.  norm_lut_log2 is "parity unpinned" as to the paper's intent (pinned by
+# mathematics only); the decode functions below take the table as given and are pinned by hand values.
 def norm_lut_log2(a: float, z: float) -> np.ndarray:
     """The 16 scales of one group on the log2 grid: float16 [16]."""
     return np.array([2.0 ** (a * s + z) for s in range(16)], dtype=np.float64).astype(np.float16)
