@@ -302,6 +302,10 @@ vq_status vq_gemm_small_batch_normalized(const vq_format* fmt, const void* d_idx
   if (batch < 1 || batch > 16) return VQ_ERR_BATCH;
   if (!d_X || !d_Y) return VQ_ERR_NULL;
   if (!aligned16(d_X) || !aligned16(d_Y)) return VQ_ERR_ALIGN;
+  // the pair-table kernel where it takes the format and the sub-row size, else the format-generic kernel
+  st = launch_gemm_warptab_norm(g, p, d_norm_codes, d_norm_lut, norm_block_cols, static_cast<const __half*>(d_X),
+                                static_cast<__half*>(d_Y), batch, static_cast<cudaStream_t>(stream));
+  if (st != VQ_ERR_UNSUPPORTED) return st;
   return launch_gemm_norm(g, p, d_norm_codes, d_norm_lut, norm_block_cols, static_cast<const __half*>(d_X), static_cast<__half*>(d_Y),
                           batch, static_cast<cudaStream_t>(stream));
 }

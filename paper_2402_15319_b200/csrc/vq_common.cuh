@@ -82,6 +82,9 @@ vq_status launch_gemm_warptab(const Geometry& g, const LayerPtrs& p, const __hal
 // ... over several layers of one format and K in one launch (rows per layer in call.N; call.ws is not used)
 vq_status launch_gemm_warptab_group(const StreamCall& call, cudaStream_t s);
 bool warptab_covers(const Geometry& g);
+// ... with block-wise normalisation (one layer; sub-rows of a power of two >= 16 columns; fp16 / int8 codebooks)
+vq_status launch_gemm_warptab_norm(const Geometry& g, const LayerPtrs& p, const void* norm_codes, const void* norm_lut,
+                                   int norm_block_cols, const __half* X, __half* Y, int batch, cudaStream_t s);
 vq_status launch_int4g128_rowcb(int N, int K, const uint8_t* q, const __half* scale, const __half* X, __half* Y, int batch,
                                 cudaStream_t s);
 // Block-wise normalisation at decode (format-generic kernels): codes = 4-bit code per row and sub-row of

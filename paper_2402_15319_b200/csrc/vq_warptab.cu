@@ -1,4 +1,4 @@
-// warptab_kernel<EB, NB, QUAD, I4>: formats with SMALL codebook blocks (1, 2, 4, 8 rows, or any multiple of 16
+// warptab_kernel<EB, NB, QUAD, I4, NORM>: formats with SMALL codebook blocks (1, 2, 4, 8 rows, or any multiple of 16
 // rows) and any index width the other tuned families do not take: 2-D indices of 1..8 bits, 1-D indices
 // of 1..4 bits; fp16, scaled-int8 or int4 codebooks; block columns and K multiples of 64.  These are the
 // remaining rows of the paper's configuration table (App. on VQ configurations: 1-D 2-bit 1x256 and
@@ -68,8 +68,14 @@ struct WarpTabArgs {
   int bsteps;                     // 64-column steps per codebook block (Bc / 64)
   int blocks_per_row;
   int steps_total, steps_per_warp;
+  // block-wise normalisation (NORM kernels; single layer): 4-bit code per row and sub-row of 1 << norm_shift
+  // columns, 16 binary16 scales per codebook block
+  const uint8_t* norm_codes;
+  const __half* norm_lut;
+  int norm_shift, norm_row_bytes;
+  int norm_off;                   // byte offset, in a warp's region, of its copy of the 16 scales of each of its tables
   int tbl_words;                  // words of one warp's tables
-  int tbl_bytes;                  // the same in bytes, rounded up to 16
+  int tbl_bytes;                  // bytes in front of the stages: tables (+ the normalisation scales), rounded up to 16
   int warp_bytes;                 // shared memory of one warp: tables, then kStages chunk stages
 };
 
@@ -123,7 +129,7 @@ __device__ __forceinline__ void load_bits(uint32_t base, int sh, bool two, bool 
   hi = __funnelshift_r(w1, w2, sh);
 }
 
-template <int EB, int NB, bool QUAD, bool I4>
+template <int EB, int NB, bool QUAD, bool I4, bool NORM>
 __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kernel(const WarpTabArgs a) {
   static_assert(!QUAD || EB == 4, "4-D entries: one 8-bit index per 4 columns = 4 stream bytes per lane and step");
   constexpr int TB = QUAD ? 9 : EB;   // log2 of the words of one table
@@ -241,6 +247,14 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
         }
       }
     }
+    if constexpr (NORM) {   // the 16 scales of each table's codebook block
+      __half* nl = reinterpret_cast<__half*>(mine + a.norm_off);
+      for (int i = lane; i < (a.tbl_words >> TB) * 16; i += 32) {
+        const uint32_t blk = static_cast<uint32_t>(min(brow0 + (i >> 4), block_rows - 1)) * static_cast<uint32_t>(a.blocks_per_row) +
+                             static_cast<uint32_t>(col_blk);
+        nl[i] = __ldg(a.norm_lut + blk * 16 + (i & 15));
+      }
+    }
   };
 
   // Chunk c of this warp (steps s_begin + 8c ..) into stage c % kStages: 2 * EB pieces of 16 bytes per row,
@@ -292,6 +306,11 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
     xn[nb][1] = ldg128_nc(xp[nb] + 8);
   }
 
+  // normalisation: code rows of rows g and g + 8, and where the scales of their tables' blocks are staged
+  const uint8_t* const ncA = a.norm_codes + static_cast<long long>(rA) * a.norm_row_bytes;
+  const uint8_t* const ncB = a.norm_codes + static_cast<long long>(rB) * a.norm_row_bytes;
+  const uint32_t nlA = smem_u32(mine) + a.norm_off + (((tA - smem_u32(tbl)) >> (TB + 2)) << 5);
+  const uint32_t nlB = smem_u32(mine) + a.norm_off + (((tB - smem_u32(tbl)) >> (TB + 2)) << 5);
   // INT4 codebooks: the scales of rows g and g + 8, one per group of 128 columns
   const __half* const scA = seg_scale + static_cast<long long>(rA) * (a.K / 128);
   const __half* const scB = seg_scale + static_cast<long long>(rB) * (a.K / 128);
@@ -351,6 +370,21 @@ __global__ void __launch_bounds__(kMaxWarps * 32, NB == 1 ? 4 : 3) warptab_kerne
         VQ_WT_PAIR(0) VQ_WT_PAIR(1) VQ_WT_PAIR(2) VQ_WT_PAIR(3)
         VQ_WT_PAIR(4) VQ_WT_PAIR(5) VQ_WT_PAIR(6) VQ_WT_PAIR(7)
 #undef VQ_WT_PAIR
+      }
+      if constexpr (NORM) {   // every pair times the scale its sub-row's 4-bit code selects (a lane's 16 columns lie in one sub-row)
+        const int j = (s * 64 + t * 16) >> a.norm_shift;
+        const uint32_t cA = (static_cast<uint32_t>(__ldg(ncA + (j >> 1))) >> (4 * (j & 1))) & 15u;
+        const uint32_t cB = (static_cast<uint32_t>(__ldg(ncB + (j >> 1))) >> (4 * (j & 1))) & 15u;
+        uint32_t fA, fB;
+        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(fA) : "r"(nlA + 2 * cA) : "memory");
+        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(fB) : "r"(nlB + 2 * cB) : "memory");
+        fA |= fA << 16;
+        fB |= fB << 16;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          wa[q] = mul_f16x2(wa[q], fA);
+          wb[q] = mul_f16x2(wb[q], fB);
+        }
       }
       if constexpr (I4) {   // w = fp16(scale of the row's group of 128 columns * c): the value vq_decode_weights writes
         const int grp = s >> 1;   // a step's 64 columns lie inside one group
@@ -423,7 +457,7 @@ constexpr size_t kSmemPerSm = 228 * 1024;   // shared memory of an SM; every res
 
 // Picks the K split, finishes the arguments and launches.  The dynamic shared-memory limit is raised and the
 // kernel's register count read once per device and instantiation.
-template <int EB, int NB, bool QUAD, bool I4>
+template <int EB, int NB, bool QUAD, bool I4, bool NORM>
 vq_status launch_one(WarpTabArgs a, long long tiles, int sms, cudaStream_t s) {
   constexpr int TB = QUAD ? 9 : EB;
   static int regs_of[kMaxDevices] = {};
@@ -432,9 +466,9 @@ vq_status launch_one(WarpTabArgs a, long long tiles, int sms, cudaStream_t s) {
   int regs = __atomic_load_n(&regs_of[dev], __ATOMIC_ACQUIRE);
   if (!regs) {
     cudaFuncAttributes fa;
-    if (cudaFuncSetAttribute(warptab_kernel<EB, NB, QUAD, I4>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemLimit)) !=
+    if (cudaFuncSetAttribute(warptab_kernel<EB, NB, QUAD, I4, NORM>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemLimit)) !=
             cudaSuccess ||
-        cudaFuncGetAttributes(&fa, warptab_kernel<EB, NB, QUAD, I4>) != cudaSuccess || fa.numRegs < 1)
+        cudaFuncGetAttributes(&fa, warptab_kernel<EB, NB, QUAD, I4, NORM>) != cudaSuccess || fa.numRegs < 1)
       return VQ_ERR_CUDA;
     regs = fa.numRegs;
     __atomic_store_n(&regs_of[dev], regs, __ATOMIC_RELEASE);
@@ -460,14 +494,16 @@ vq_status launch_one(WarpTabArgs a, long long tiles, int sms, cudaStream_t s) {
   // A plain launch, in stream order.  (With programmatic dependent launch the next launch's CTAs take the
   // SM slots this grid leaves free and stay where they land: two such layers back to back then run with
   // 3 CTAs on some SMs and 1 on others; measured 31.5 against 23.2 us on 4096 x 14336.)
-  warptab_kernel<EB, NB, QUAD, I4><<<static_cast<unsigned>(tiles), static_cast<unsigned>(wk) * 32u, smem_bytes, s>>>(a);
+  warptab_kernel<EB, NB, QUAD, I4, NORM><<<static_cast<unsigned>(tiles), static_cast<unsigned>(wk) * 32u, smem_bytes, s>>>(a);
   return check_launch();
 }
 
 template <int EB, bool QUAD = false>
 vq_status launch_eb(const WarpTabArgs& a, int nb, long long tiles, int sms, cudaStream_t s) {
-  if (a.cb_int4) return nb == 1 ? launch_one<EB, 1, QUAD, true>(a, tiles, sms, s) : launch_one<EB, 2, QUAD, true>(a, tiles, sms, s);
-  return nb == 1 ? launch_one<EB, 1, QUAD, false>(a, tiles, sms, s) : launch_one<EB, 2, QUAD, false>(a, tiles, sms, s);
+  if (a.norm_codes)   // (normalisation with INT4 codebooks stays in the format-generic kernel)
+    return nb == 1 ? launch_one<EB, 1, QUAD, false, true>(a, tiles, sms, s) : launch_one<EB, 2, QUAD, false, true>(a, tiles, sms, s);
+  if (a.cb_int4) return nb == 1 ? launch_one<EB, 1, QUAD, true, false>(a, tiles, sms, s) : launch_one<EB, 2, QUAD, true, false>(a, tiles, sms, s);
+  return nb == 1 ? launch_one<EB, 1, QUAD, false, false>(a, tiles, sms, s) : launch_one<EB, 2, QUAD, false, false>(a, tiles, sms, s);
 }
 
 }  // namespace
@@ -481,9 +517,18 @@ bool warptab_covers(const Geometry& g) {
   return (tables_per_tile(g) << table_bits(g)) <= 1024;
 }
 
-vq_status launch_gemm_warptab_group(const StreamCall& call, cudaStream_t s) {
+namespace {
+// norm_codes == nullptr: no normalisation.  With it: one layer, sub-rows of a power of two of at least 16 columns
+// (a lane's 16 columns of a step then lie inside one sub-row), fp16 or int8 codebooks.
+vq_status launch_impl(const StreamCall& call, const void* norm_codes, const void* norm_lut, int norm_block_cols, cudaStream_t s) {
   const Geometry& g = call.g;
   if (!warptab_covers(g) || call.n_seg < 1 || call.n_seg > kMaxSegments) return VQ_ERR_UNSUPPORTED;
+  int norm_shift = -1;
+  if (norm_codes) {
+    for (int sh = 4; sh < 31; ++sh)
+      if ((1 << sh) == norm_block_cols) norm_shift = sh;
+    if (norm_shift < 0 || g.cb_int4 || call.n_seg != 1) return VQ_ERR_UNSUPPORTED;
+  }
   const int eb = pair_bits(g);
   const int nb = call.batch <= 8 ? 1 : 2;
   WarpTabArgs a = {};
@@ -519,6 +564,14 @@ vq_status launch_gemm_warptab_group(const StreamCall& call, cudaStream_t s) {
   a.tbl_words = tables_per_tile(g) << table_bits(g);
   // per warp: tables + chunk stages; the reduction buffer (nb * 512 bytes per warp) reuses that space
   a.tbl_bytes = (a.tbl_words * 4 + 15) / 16 * 16;
+  if (norm_codes) {
+    a.norm_codes = static_cast<const uint8_t*>(norm_codes);
+    a.norm_lut = static_cast<const __half*>(norm_lut);
+    a.norm_shift = norm_shift;
+    a.norm_row_bytes = (g.K / norm_block_cols + 1) / 2;
+    a.norm_off = a.tbl_bytes;
+    a.tbl_bytes += tables_per_tile(g) * 32;   // 16 binary16 scales per table
+  }
   const int tbl_align = region_align(table_bits(g));
   a.warp_bytes = (a.tbl_bytes + kStages * stage_bytes(eb) + tbl_align - 1) / tbl_align * tbl_align;
   int sms = 0;
@@ -533,6 +586,25 @@ vq_status launch_gemm_warptab_group(const StreamCall& call, cudaStream_t s) {
     case 7: return launch_eb<7>(a, nb, tiles, sms, s);
     default: return launch_eb<8>(a, nb, tiles, sms, s);
   }
+}
+}  // namespace
+
+vq_status launch_gemm_warptab_group(const StreamCall& call, cudaStream_t s) { return launch_impl(call, nullptr, nullptr, 0, s); }
+
+vq_status launch_gemm_warptab_norm(const Geometry& g, const LayerPtrs& p, const void* norm_codes, const void* norm_lut,
+                                   int norm_block_cols, const __half* X, __half* Y, int batch, cudaStream_t s) {
+  if (!norm_codes || !norm_lut) return VQ_ERR_UNSUPPORTED;
+  StreamCall call = {};
+  call.g = g;
+  call.n_seg = 1;
+  call.idx[0] = p.idx;
+  call.cb[0] = p.cb;
+  call.scale[0] = p.scale;
+  call.Y[0] = Y;
+  call.N[0] = g.N;
+  call.X = X;
+  call.batch = batch;
+  return launch_impl(call, norm_codes, norm_lut, norm_block_cols, s);
 }
 
 vq_status launch_gemm_warptab(const Geometry& g, const LayerPtrs& p, const __half* X, __half* Y, int batch,

@@ -653,6 +653,26 @@ def test_normalized_decode_and_gemm(spec, nbc):
         assert_outputs_close(dY.cpu().numpy(), Y, A, f"{spec.name} normalised batch={batch}")
 
 
+def test_normalized_gemm_layer_size():
+    """A 2048 x 4096 layer in the deployed 2-D 6-bit format with 32-column sub-rows (the pair-table kernel
+    with the normalisation multiply, in the launch shape a layer of that size gets): every output row."""
+    import torch
+    spec = vq_synth.LayerSpec("nm_layer", N=2048, K=4096, d=2, b=6, Br=32, Bc=256, int8=True)
+    f = oracle_fmt(spec)
+    L = draw(spec, 81)
+    codes, lut = vq_synth.make_norm(spec, 32, 82)
+    dev = DeviceLayer(spec, L)
+    d_codes, d_lut = torch.from_numpy(codes).cuda(), torch.from_numpy(lut).cuda()
+    for batch in (1, 9):
+        X = vq_synth.make_x(spec, 83, batch)
+        dY, rawy = guarded((batch, spec.N), torch.float16, "cuda")
+        vq.vq_gemm_small_batch_normalized(dev.fmt, dev.idx, dev.cb, dev.scale, d_codes, d_lut, 32, torch.from_numpy(X).cuda(), dY, batch)
+        torch.cuda.synchronize()
+        assert_guards_intact(rawy, spec.name)
+        Y, A = orc.normalized_gemm(f, L.idx, L.cb, L.scale, codes, lut, 32, X)
+        assert_outputs_close(dY.cpu().numpy(), Y, A, f"{spec.name} batch={batch}")
+
+
 def test_normalized_with_unit_table_equals_plain_entry_points():
     """A table of ones switches the normalisation off: the decode equals vq_decode_weights bit for bit."""
     import torch
