@@ -301,7 +301,9 @@ vq_status vq_assign_indices(const vq_format* fmt, const void* d_W, const void* d
  * computes Y[m][n] = sum_k w[n][k] X[m][k] (fp32 accumulation, one rounding), batch 1..16.  Every valid
  * format is taken (format-generic kernels; no workspace, plain stream-order launches); the product runs in
  * the tuned pair-table kernel when the format is one of its (see vq_impl), the codebooks are fp16 or int8
- * and norm_block_cols is a power of two of at least 16 (weights then enter the sum as binary16 values).
+ * and norm_block_cols is a power of two of at least 16 (weights then enter the sum as binary16 values);
+ * the decode runs in the tile kernel of vq_decode_weights for the formats that one takes and power-of-two
+ * sub-rows of at least 8 columns, bit-identical to the format-generic kernel.
  * Errors: as vq_decode_weights / vq_gemm_small_batch (without WORKSPACE); NULL for a missing code or table
  * pointer; SHAPE for a norm_block_cols that does not divide block_cols or is not a multiple of vq_dim. */
 typedef struct {

@@ -287,6 +287,9 @@ vq_status vq_decode_weights_normalized(const vq_format* fmt, const void* d_idx, 
   if (st != VQ_OK) return st;
   if (!d_W) return VQ_ERR_NULL;
   if (!aligned16(d_W)) return VQ_ERR_ALIGN;
+  // the tile kernel where it takes the format and the sub-row size, else the format-generic kernel
+  st = launch_decode_tuned(g, p, static_cast<__half*>(d_W), static_cast<cudaStream_t>(stream), d_norm_codes, d_norm_lut, norm_block_cols);
+  if (st != VQ_ERR_UNSUPPORTED) return st;
   return launch_decode_norm(g, p, d_norm_codes, d_norm_lut, norm_block_cols, static_cast<__half*>(d_W), static_cast<cudaStream_t>(stream));
 }
 

@@ -93,7 +93,8 @@ vq_status launch_decode_norm(const Geometry& g, const LayerPtrs& p, const void* 
                              __half* W, cudaStream_t s);
 vq_status launch_gemm_norm(const Geometry& g, const LayerPtrs& p, const void* codes, const void* lut, int block_cols,
                            const __half* X, __half* Y, int batch, cudaStream_t s);
-vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s);
+vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s, const void* norm_codes = nullptr,
+                              const void* norm_lut = nullptr, int norm_block_cols = 0);
 // E-step: nearest centroid under diagonal weights, packed into the index stream `idx` (output).
 vq_status launch_assign(const Geometry& g, const LayerPtrs& p, const __half* W, const float* hdiag, uint8_t* idx,
                         cudaStream_t s);

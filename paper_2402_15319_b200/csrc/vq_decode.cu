@@ -36,6 +36,11 @@ struct DecodeArgs {
   const void* cb;
   const __half* scale;
   const __half* row_scale;   // int4 codebooks: [N][K/128] scales applied after the look-up, else null
+  // block-wise normalisation (null codes: off): a 4-bit code per row and sub-row of 1 << norm_shift columns
+  // (at least 8: a lane's 8 columns lie in one sub-row) selects one of the 16 scales of the codebook block
+  const uint8_t* norm_codes;
+  const __half* norm_lut;
+  int norm_shift, norm_row_bytes;
   __half* W;
   long long stride;
   int N, K, b, Br, Bc, entries, blocks_per_row;
@@ -102,6 +107,8 @@ __global__ void __launch_bounds__(32 * kWarps) decode_tile_kernel(const DecodeAr
         v = __int2half_rn(nib >= 8 ? nib - 16 : nib);
       } else if (a.scale == nullptr) {
         v = __ldg(static_cast<const __half*>(a.cb) + blk * table_halves + within);
+      } else if (a.norm_codes != nullptr) {   // normalised int8: entry kept unscaled (exact), block and sub-row scales applied together later
+        v = __int2half_rn(static_cast<int>(__ldg(static_cast<const int8_t*>(a.cb) + blk * table_halves + within)));
       } else {
         const float c = static_cast<float>(__ldg(static_cast<const int8_t*>(a.cb) + blk * table_halves + within));
         v = __float2half_rn(__half2float(__ldg(a.scale + blk)) * c);   // exact fp32 product, one rounding
@@ -132,7 +139,36 @@ __global__ void __launch_bounds__(32 * kWarps) decode_tile_kernel(const DecodeAr
       const uint32_t v = __funnelshift_r(w0, w1, sh) & vmask;
       const __half* tab = row_tabs + ((seg * 256 + lane_cols) >> a.bc_shift) * table_halves;
       uint4 out = lookup8<D>(tab, v, a.b, emask);
-      if (a.row_scale != nullptr) {   // the lane's 8 columns lie in one group of 128: exact fp32 product, one rounding
+      if (a.norm_codes != nullptr) {
+        // w = binary16(value * scale of the sub-row), the exact product rounded once.  The factor p collects the
+        // sub-row's scale and, for int8 / int4 codebooks, the block's / row group's scale: exact in fp32 (22 bits).
+        // fp16 entries: p * entry has 22 significand bits, exact in fp32; integer entries: up to 30 bits, formed in fp64.
+        const int col = col0 + seg * 256 + lane_cols;
+        const long long blk = static_cast<long long>(n / a.Br) * a.blocks_per_row + (col >> a.bc_shift);
+        const int j = col >> a.norm_shift;
+        const uint32_t code = (static_cast<uint32_t>(__ldg(a.norm_codes + static_cast<long long>(n) * a.norm_row_bytes + (j >> 1))) >> (4 * (j & 1))) & 15u;
+        float pf = __half2float(__ldg(a.norm_lut + blk * 16 + code));
+        uint32_t* o32 = reinterpret_cast<uint32_t*>(&out);
+        if (a.row_scale == nullptr && a.scale == nullptr) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const __half2 hv = *reinterpret_cast<const __half2*>(&o32[q]);
+            const __half2 r = __halves2half2(__float2half_rn(pf * __low2float(hv)), __float2half_rn(pf * __high2float(hv)));
+            o32[q] = *reinterpret_cast<const uint32_t*>(&r);
+          }
+        } else {
+          pf *= a.row_scale != nullptr ? __half2float(__ldg(a.row_scale + static_cast<long long>(n) * (a.K / 128) + col / 128))
+                                       : __half2float(__ldg(a.scale + blk));
+          const double pd = static_cast<double>(pf);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const __half2 hv = *reinterpret_cast<const __half2*>(&o32[q]);
+            const __half2 r = __halves2half2(__double2half(pd * static_cast<double>(__low2float(hv))),
+                                             __double2half(pd * static_cast<double>(__high2float(hv))));
+            o32[q] = *reinterpret_cast<const uint32_t*>(&r);
+          }
+        }
+      } else if (a.row_scale != nullptr) {   // the lane's 8 columns lie in one group of 128: exact fp32 product, one rounding
         const float sc = __half2float(__ldg(a.row_scale + static_cast<long long>(n) * (a.K / 128) + (col0 + seg * 256 + lane_cols) / 128));
         uint32_t* o32 = reinterpret_cast<uint32_t*>(&out);
 #pragma unroll
@@ -161,9 +197,22 @@ __global__ void __launch_bounds__(32 * kWarps) decode_tile_kernel(const DecodeAr
 // Formats the tile kernel covers: K a multiple of 256, at most 32 index bits per lane and segment
 // (8 b / d <= 32), block columns a power of two >= 8 that divide or are divided by the tile's columns,
 // block rows that divide or are divided by 32, tables of the tile within 96 KB of shared memory.
-vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s) {
+// With norm_codes: block-wise normalisation, sub-rows of a power of two of at least 8 columns.
+vq_status launch_decode_tuned(const Geometry& g, const LayerPtrs& p, __half* W, cudaStream_t s, const void* norm_codes,
+                              const void* norm_lut, int norm_block_cols) {
   if (g.K % 256 || (8 * g.b) % g.d || 8 * g.b / g.d > 32 || g.Bc % 8) return VQ_ERR_UNSUPPORTED;
   DecodeArgs a;
+  a.norm_codes = static_cast<const uint8_t*>(norm_codes);
+  a.norm_lut = static_cast<const __half*>(norm_lut);
+  a.norm_shift = 0;
+  a.norm_row_bytes = 0;
+  if (norm_codes) {
+    a.norm_shift = -1;
+    for (int sft = 3; sft < 31; ++sft)
+      if ((1 << sft) == norm_block_cols) a.norm_shift = sft;
+    if (a.norm_shift < 0 || !norm_lut) return VQ_ERR_UNSUPPORTED;
+    a.norm_row_bytes = (g.K / norm_block_cols + 1) / 2;
+  }
   a.tile_cols = g.K < kTileCols ? g.K : kTileCols;
   a.bc_shift = -1;
   for (int sft = 3; sft < 31; ++sft)
