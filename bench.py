@@ -612,6 +612,44 @@ def time_assign(device, torch, vq, cfg_name: str = "cfg3", N: int = 11008, K: in
             "alu_frac": ops / us * 1e6 / peak, "sqnr_db_random_codebook": sqnr}
 
 
+def time_normalized(device, torch, vq, N: int = 14336, K: int = 4096, block_cols: int = 32, copies: int = 6, reps: int = 5):
+    """Block-wise normalisation applied at decode (paper appendix on blockwise data normalization) on a
+    gate_proj-shaped layer of the deployed format (2-D, 6-bit, int8 codebook per 32x256 block): batch-1 product and
+    weight materialisation, each over `copies` device copies of the layer (cold cache), beside the same calls
+    without normalisation."""
+    spec = vq_synth.LayerSpec("norm", N, K, 2, 6, 32, 256, True)
+    fmt = vq.VQFormat(N, K, 2, 6, 32, 256, vq.VQ_CB_INT8_SCALED)
+    info = vq.vq_pack_info(fmt)
+    L = vq_synth.make_layer(spec, info.row_stride_bytes, 31, 0)
+    codes, lut = vq_synth.make_norm(spec, block_cols, 32)
+    dev = [tuple(torch.from_numpy(a).to(device) for a in (L.idx, L.cb, L.scale, codes, lut)) for _ in range(copies)]
+    X = torch.from_numpy(vq_synth.make_x(spec, 33, 1)).to(device)
+    Y = torch.empty((1, N), dtype=torch.float16, device=device)
+    W = torch.empty((N, K), dtype=torch.float16, device=device)
+    ws = torch.zeros(vq.vq_workspace_bytes(fmt, 1), dtype=torch.uint8, device=device)
+
+    def timed(call):
+        call(0)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for r in range(reps):
+            for c in range(copies):
+                call(c)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (reps * copies)
+
+    nbytes = info.total_bytes + codes.nbytes + lut.nbytes + 2 * (N + K)
+    g_us = timed(lambda c: vq.vq_gemm_small_batch_normalized(fmt, *dev[c], block_cols, X, Y, 1))
+    p_us = timed(lambda c: vq.vq_gemm_small_batch(fmt, dev[c][0], dev[c][1], dev[c][2], X, Y, 1, ws))
+    d_us = timed(lambda c: vq.vq_decode_weights_normalized(fmt, *dev[c], block_cols, W))
+    q_us = timed(lambda c: vq.vq_decode_weights(fmt, dev[c][0], dev[c][1], dev[c][2], W))
+    return {"layer": f"{N}x{K}", "format": "d=2 b=6 32x256 int8", "norm_block_cols": block_cols,
+            "gemm_b1_us": g_us, "gemm_b1_GBps": nbytes / g_us / 1e3, "gemm_b1_plain_us": p_us,
+            "decode_us": d_us, "decode_plain_us": q_us}
+
+
 def time_decode(ds, reps: int = 3):
     """vq_decode_weights on the largest layer of the set: (us, GB/s over indices + codebooks + fp16 output)."""
     torch, vq = ds.torch, ds.vq
@@ -791,6 +829,7 @@ def run_ours(args):
         if args.all_configs:
             line["transfer_decode"] = time_transfer_decode(dev, torch, vq)
             line["assign"] = time_assign(dev, torch, vq)
+            line["normalized"] = time_normalized(dev, torch, vq)
     if rank == 0:
         print(json.dumps(line))
     if dist:
